@@ -1,0 +1,264 @@
+// CPU oracle for the AdaPT precision-switch search (PushDown inner body).
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, single-threaded
+// restatement of the paper's definitions that the GPU library is checked
+// against.  It shares no source, header, table or helper with the CUDA path
+// and must never be reached from a product call.
+//
+// What each function follows:
+//   quantize    - signed fixed-point <WL,FL> (Sec. 2.1 "Fixed-Point
+//                 Quantization"; Sec. 3.2 "Precision Levels", the SR(x) rule)
+//   range/bins  - discretisation "via binning" at resolution r (Sec. 3.3,
+//                 the EDF equation), read as r equal-width bins on [min,max]
+//   kld         - discrete Kullback-Leibler divergence KL(P||Q), P the
+//                 quantized tensor, Q the float tensor (Sec. 3.3, Eq. dkld)
+//   select      - "smallest quantization s.t. KL = 0" (Sec. 3.3; Algorithm 3)
+//   sparsity    - share of non-zero elements (Sec. 3.4 "Inducing Sparsity")
+//
+// The paper gives no bit-level rules; the readings taken (saturation,
+// ties-to-even, the stochastic-rounding hash, bin arithmetic, the KLD
+// summation form, candidate order) are listed in the design notes of the
+// repository.  All of them are pinned only by the tests of this oracle
+// against hand-worked values, exact rational brute force, closed forms and
+// library routines; the counter hash has no outside definition at all
+// (parity unpinned beyond its stored vectors and statistics).
+//
+// Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
+
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+namespace {
+
+constexpr int kRoundNearestEven = 0;
+constexpr int kRoundStochastic = 1;
+
+// Counter hash (seed, layer, element index) -> 24 uniform bits.
+// The paper only says "a random number P" (Sec. 3.2); this mixer is the
+// build's own definition: golden-ratio / sqrt(2) / sqrt(3) odd constants,
+// three xor-shift-multiply rounds, top 24 bits.
+inline uint32_t hash24(uint64_t seed, uint64_t layer, uint64_t index) {
+  const uint64_t c1 = 0x9E3779B97F4A7C15ull;
+  const uint64_t c2 = 0x6A09E667F3BCC909ull;
+  const uint64_t c3 = 0xBB67AE8584CAA73Bull;
+  uint64_t z = seed ^ ((layer + 1ull) * c1);
+  z += index * c2;
+  z ^= z >> 32;
+  z *= c1;
+  z ^= z >> 29;
+  z *= c3;
+  z ^= z >> 32;
+  return static_cast<uint32_t>(z >> 40);
+}
+
+// Rounded, unsaturated integer value of x * 2^FL, kept as a float.
+// RNE: nearest, ties to even.  Stochastic (Sec. 3.2, SR(x)): floor, plus one
+// when P < (distance above the floor, in quanta); P = k24 * 2^-24 in [0,1).
+inline float round_scaled(float x, int fl, int round_mode, uint32_t k24) {
+  const float y = x * std::ldexp(1.0f, fl);  // exact power-of-two scaling
+  if (round_mode == kRoundNearestEven) {
+    return std::nearbyintf(y);  // default rounding mode: ties to even
+  }
+  const float f = std::floor(y);
+  const float frac = y - f;  // one fp32 subtraction
+  const float p = static_cast<float>(k24) * std::ldexp(1.0f, -24);  // exact
+  return (p < frac) ? f + 1.0f : f;
+}
+
+// Two's-complement saturation to WL bits (Sec. 2.1: results must lie within
+// the representable boundaries).
+inline int32_t saturate(float r, int wl) {
+  const float top = std::ldexp(1.0f, wl - 1);  // 2^(WL-1)
+  if (r >= top) return static_cast<int32_t>((int64_t(1) << (wl - 1)) - 1);
+  if (r <= -top) return static_cast<int32_t>(-(int64_t(1) << (wl - 1)));
+  return static_cast<int32_t>(r);  // integral and in range: exact
+}
+
+inline float dequantize(int32_t code, int fl) {
+  return static_cast<float>(code) * std::ldexp(1.0f, -fl);
+}
+
+// Shared-bin index of value v for bins on [lo,hi] (Sec. 3.3, EDF at
+// resolution r = n_bins).  Every operation is one IEEE fp32 operation.
+inline int bin_index(float v, float lo, float hi, int n_bins) {
+  const float w = hi - lo;
+  const float scale = (w == 0.0f) ? 0.0f : static_cast<float>(n_bins) / w;
+  const float t = v - lo;
+  const float u = t * scale;
+  float bf = std::floor(u);
+  bf = std::fmax(bf, 0.0f);  // fmax returns the non-NaN operand
+  bf = std::fmin(bf, static_cast<float>(n_bins - 1));
+  return static_cast<int>(bf);
+}
+
+}  // namespace
+
+extern "C" {
+
+// ---- element-level entry points (used by the pins) -------------------------
+
+uint32_t adapt_oracle_hash24(uint64_t seed, uint64_t layer, uint64_t index) {
+  return hash24(seed, layer, index);
+}
+
+int32_t adapt_oracle_quantize_one(float x, int wl, int fl, int round_mode,
+                                  uint32_t k24) {
+  return saturate(round_scaled(x, fl, round_mode, k24), wl);
+}
+
+float adapt_oracle_dequantize_one(int32_t code, int fl) {
+  return dequantize(code, fl);
+}
+
+int adapt_oracle_bin_index(float v, float lo, float hi, int n_bins) {
+  return bin_index(v, lo, hi, n_bins);
+}
+
+// ---- tensor-level steps -----------------------------------------------------
+
+// Quantize(L, <WL,FL>) (Algorithm 1, the re-quantisation step; Algorithm 3,
+// the Quantize call).  codes_out / xhat_out may be null.
+void adapt_oracle_quantize(const float* x, int64_t n, int wl, int fl,
+                           int round_mode, uint64_t seed, uint64_t layer,
+                           int32_t* codes_out, float* xhat_out) {
+  for (int64_t i = 0; i < n; ++i) {
+    const uint32_t k =
+        (round_mode == kRoundStochastic) ? hash24(seed, layer, uint64_t(i)) : 0u;
+    const int32_t c = saturate(round_scaled(x[i], fl, round_mode, k), wl);
+    if (codes_out) codes_out[i] = c;
+    if (xhat_out) xhat_out[i] = dequantize(c, fl);
+  }
+}
+
+// min / max of the float tensor; returns 1 if any element is NaN or Inf.
+int adapt_oracle_range(const float* x, int64_t n, float* lo_out, float* hi_out) {
+  float lo = std::numeric_limits<float>::infinity();
+  float hi = -std::numeric_limits<float>::infinity();
+  int nonfinite = 0;
+  for (int64_t i = 0; i < n; ++i) {
+    if (!std::isfinite(x[i])) nonfinite = 1;
+    if (x[i] < lo) lo = x[i];
+    if (x[i] > hi) hi = x[i];
+  }
+  if (n == 0) { lo = 0.0f; hi = 0.0f; }
+  *lo_out = lo;
+  *hi_out = hi;
+  return nonfinite;
+}
+
+// Histogram of v[0..n) over n_bins shared bins on [lo,hi]; hist is zeroed here.
+void adapt_oracle_histogram(const float* v, int64_t n, float lo, float hi,
+                            int n_bins, uint64_t* hist) {
+  for (int b = 0; b < n_bins; ++b) hist[b] = 0;
+  for (int64_t i = 0; i < n; ++i) hist[bin_index(v[i], lo, hi, n_bins)] += 1;
+}
+
+// KL(P||Q) from integer bin counts (Eq. dkld), P = quantized, Q = float.
+// Both histograms count the same N elements (equal totals are a precondition).
+// With p_b/N and q_b/N the bin masses, p*log(p/q) = p*log1p((p-q)/q); the
+// count difference is formed exactly in integers so that histograms that
+// differ by a few counts in well-filled bins keep their accuracy.  alpha is
+// an optional pseudo-count added to every bin of both histograms.  A bin with
+// p_b + alpha > 0 and q_b + alpha = 0 makes the divergence +infinity.
+// log_base = 2 gives bits (the paper's "number of bits lost").
+double adapt_oracle_kld(const uint64_t* p_hist, const uint64_t* q_hist,
+                        int n_bins, double alpha, double log_base) {
+  double total = 0.0;
+  for (int b = 0; b < n_bins; ++b) total += static_cast<double>(p_hist[b]);
+  const double n_eff = total + alpha * n_bins;
+  if (n_eff <= 0.0) return 0.0;
+  double sum = 0.0;
+  for (int b = 0; b < n_bins; ++b) {
+    const double p = static_cast<double>(p_hist[b]) + alpha;
+    const double q = static_cast<double>(q_hist[b]) + alpha;
+    if (p <= 0.0) continue;
+    if (q <= 0.0) return std::numeric_limits<double>::infinity();
+    const int64_t diff =
+        static_cast<int64_t>(p_hist[b]) - static_cast<int64_t>(q_hist[b]);
+    sum += p * std::log1p(static_cast<double>(diff) / q);
+  }
+  const double kld = sum / (n_eff * std::log(log_base));
+  return kld > 0.0 ? kld : 0.0;
+}
+
+// Lowest <WL,FL> whose divergence is <= eps (Sec. 3.3; Algorithm 3).
+// Candidates are compared in (WL, FL) lexicographic order whatever their
+// order in the arrays.  If none meets eps the candidate of minimal divergence
+// is returned (first in that order among ties; if every divergence is +inf,
+// the last in that order).  out = {wl, fl, grid index, flags}; flag bit 0 =
+// "met eps".
+void adapt_oracle_select(const double* kld, const int32_t* wl, const int32_t* fl,
+                         int n_cand, double eps, int32_t* out) {
+  auto before = [&](int a, int b) {  // a strictly before b in (WL,FL) order
+    if (wl[a] != wl[b]) return wl[a] < wl[b];
+    if (fl[a] != fl[b]) return fl[a] < fl[b];
+    return a < b;
+  };
+  int best_ok = -1, best_min = -1, last = -1;
+  for (int c = 0; c < n_cand; ++c) {
+    if (last < 0 || before(last, c)) last = c;
+    if (kld[c] <= eps && (best_ok < 0 || before(c, best_ok))) best_ok = c;
+    if (std::isfinite(kld[c])) {
+      if (best_min < 0 || kld[c] < kld[best_min] ||
+          (kld[c] == kld[best_min] && before(c, best_min)))
+        best_min = c;
+    }
+  }
+  int pick = best_ok >= 0 ? best_ok : (best_min >= 0 ? best_min : last);
+  out[0] = pick >= 0 ? wl[pick] : 0;
+  out[1] = pick >= 0 ? fl[pick] : 0;
+  out[2] = pick;
+  out[3] = best_ok >= 0 ? 1 : 0;
+}
+
+// The whole search for one layer, one candidate at a time, in the order the
+// paper's PushDown body takes them: Quantize -> (zero count) -> EDF of both
+// tensors over shared bins -> KL -> choice.  No shortcut of any kind.
+//   kld_out   double[n_cand]
+//   zeros_out int64[n_cand]   count of zero codes (sparsity = 1 - zeros/n)
+//   best_out  int32[4]        {wl, fl, grid index, flags}; flag bit 1 = the
+//                             tensor's range is degenerate (max == min or n==0)
+//   hist_out  uint64[(n_cand+1)*n_bins] or null; slot 0 = float histogram
+//   range_out float[2] or null
+// Returns 1 if the tensor holds a NaN or Inf (outputs then unspecified).
+int adapt_oracle_precision_search(const float* x, int64_t n, uint64_t layer,
+                                  const int32_t* wl, const int32_t* fl,
+                                  int n_cand, int n_bins, int round_mode,
+                                  uint64_t seed, double eps, double alpha,
+                                  double log_base, double* kld_out,
+                                  int64_t* zeros_out, int32_t* best_out,
+                                  uint64_t* hist_out, float* range_out) {
+  float lo, hi;
+  const int nonfinite = adapt_oracle_range(x, n, &lo, &hi);
+  if (range_out) { range_out[0] = lo; range_out[1] = hi; }
+  if (nonfinite) return 1;
+
+  std::vector<uint64_t> q_hist(n_bins), p_hist(n_bins);
+  std::vector<int32_t> codes(static_cast<size_t>(n));
+  std::vector<float> xhat(static_cast<size_t>(n));
+
+  adapt_oracle_histogram(x, n, lo, hi, n_bins, q_hist.data());
+  if (hist_out) std::memcpy(hist_out, q_hist.data(), sizeof(uint64_t) * n_bins);
+
+  for (int c = 0; c < n_cand; ++c) {
+    adapt_oracle_quantize(x, n, wl[c], fl[c], round_mode, seed, layer,
+                          codes.data(), xhat.data());
+    int64_t zeros = 0;
+    for (int64_t i = 0; i < n; ++i) zeros += (codes[i] == 0);
+    zeros_out[c] = zeros;
+    adapt_oracle_histogram(xhat.data(), n, lo, hi, n_bins, p_hist.data());
+    if (hist_out)
+      std::memcpy(hist_out + size_t(c + 1) * n_bins, p_hist.data(),
+                  sizeof(uint64_t) * n_bins);
+    kld_out[c] = adapt_oracle_kld(p_hist.data(), q_hist.data(), n_bins, alpha,
+                                  log_base);
+  }
+  adapt_oracle_select(kld_out, wl, fl, n_cand, eps, best_out);
+  if (n == 0 || hi == lo) best_out[3] |= 2;
+  return 0;
+}
+
+}  // extern "C"
