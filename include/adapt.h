@@ -1,0 +1,184 @@
+/* adapt.h - C ABI of the B200 precision-switch search library (libadapt_b200.so).
+ *
+ * The library implements the data-parallel body of AdaPT's PushDown operation
+ * (Sec. 3.3 "The PushDown Operation"; Algorithm 3), evaluated for a whole grid
+ * of candidate fixed-point formats at once, plus the stand-alone Quantize step
+ * (Algorithm 1, the per-layer re-quantisation loop).
+ *
+ * Conventions that hold for every entry point unless its comment says otherwise
+ *  - Pointers marked DEVICE are CUDA device pointers on the current device and
+ *    stay owned by the caller; pointers marked HOST are ordinary host memory,
+ *    read (or written) before the call returns.
+ *  - Calls enqueue their kernels on a CUDA stream (the legacy default stream
+ *    for the entry points without a stream argument) and return without
+ *    waiting; outputs are valid once that stream has been synchronised.
+ *  - The return value is an adapt_status.  Errors that the host can see (null
+ *    pointers, sizes or formats out of range, workspace too small) return
+ *    before anything is launched and write nothing.  Errors in the data
+ *    (NaN/Inf elements, |x| >= 2^64) cannot be seen by the host without a
+ *    device round trip: they are reported per layer in best_out's flag word,
+ *    the other outputs of that layer are then unspecified (but in bounds).
+ *    Nothing traps on the device and no C++ exception crosses this boundary.
+ *  - Formats: 2 <= WL <= 32, 0 <= FL <= WL-1 (Sec. 2.1: a WL-bit signed word
+ *    with FL fractional bits; value = code * 2^-FL, code in
+ *    [-2^(WL-1), 2^(WL-1)-1]).  Values outside the range saturate.
+ *  - Limits: fewer than 2^32 elements per layer; 1 <= n_bins <= 65536;
+ *    1 <= n_cand <= 65535; 1 <= n_layers <= 65535.
+ */
+#ifndef ADAPT_B200_H_
+#define ADAPT_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  ADAPT_OK = 0,
+  ADAPT_ERR_INVALID_ARG = 1, /* null pointer, bad size, bad <WL,FL>, bad mode   */
+  ADAPT_ERR_NONFINITE = 2,   /* (host-side entry points only) NaN/Inf in input  */
+  ADAPT_ERR_RANGE = 3,       /* (host-side entry points only) |x| >= 2^64       */
+  ADAPT_ERR_CUDA = 4,        /* a CUDA runtime call failed                      */
+  ADAPT_ERR_WORKSPACE = 5    /* caller-supplied workspace is too small          */
+} adapt_status;
+
+/* Rounding of x * 2^FL to an integer (Sec. 3.2 "Precision Levels").
+ * RNE: round to nearest, ties to even.
+ * STOCHASTIC: the SR(x) rule - floor, plus one when P < fractional position,
+ * with P = k / 2^24 drawn per element from a counter hash of
+ * (seed, layer, element index); all candidates of one element share its P. */
+enum { ADAPT_ROUND_RNE = 0, ADAPT_ROUND_STOCHASTIC = 1 };
+
+/* Flag bits of best_out[l*4 + 3]. */
+enum {
+  ADAPT_FLAG_MET_EPS = 1,    /* the returned candidate has KLD <= eps           */
+  ADAPT_FLAG_DEGENERATE = 2, /* max == min (or empty layer): one bin, KLD == 0  */
+  ADAPT_FLAG_NONFINITE = 4,  /* layer holds NaN/Inf: its outputs are unspecified */
+  ADAPT_FLAG_RANGE = 8       /* layer holds |x| >= 2^64: outputs unspecified     */
+};
+
+/* Candidate formats. HOST arrays of n_cand entries each, in any order. */
+typedef struct adapt_grid {
+  int32_t n_cand;
+  const int32_t* wl;
+  const int32_t* fl;
+} adapt_grid;
+
+/* Options of the _ex / _host search calls.  Zero-initialise, then set fields;
+ * log_base == 0 means 2 (bits). */
+typedef struct adapt_search_opts {
+  int32_t round_mode;     /* ADAPT_ROUND_*                                      */
+  int32_t layer_base;     /* hash layer id of tensors[l] is layer_base + l      */
+  uint64_t seed;          /* stochastic rounding seed                           */
+  double eps;             /* accept a candidate when KLD <= eps (default 0)     */
+  double pseudo_count;    /* added to every bin of both histograms (default 0)  */
+  double log_base;        /* base of the logarithm; 0 -> 2                      */
+  void* stream;           /* cudaStream_t; NULL = legacy default stream         */
+  void* workspace;        /* DEVICE scratch, 256-byte aligned, or NULL to use a
+                             library-owned buffer that grows on demand          */
+  size_t workspace_bytes; /* size of workspace                                  */
+  uint32_t* hist_out;     /* DEVICE, optional: uint32[n_layers][n_cand+1][n_bins],
+                             slot 0 = histogram of the float tensor, slot c+1 =
+                             histogram of candidate c's dequantized tensor      */
+  float* range_out;       /* DEVICE, optional: float[n_layers][2] = {min, max}  */
+} adapt_search_opts;
+
+/* Library version string, e.g. "adapt-b200 0.1". Never NULL. */
+const char* adapt_version(void);
+
+/* Static English text for an adapt_status value. Never NULL. */
+const char* adapt_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread's most recent failing
+ * call ("" if none). Valid until the next call from any thread. */
+const char* adapt_last_error(void);
+
+/* Quantize(L, <WL,FL>) - Algorithm 1 (re-quantisation of each layer after the
+ * update) and Algorithm 3 (the Quantize call inside PushDown); format and
+ * rounding as in Sec. 2.1 / Sec. 3.2.
+ *   x         DEVICE fp32[n], any 4-byte alignment
+ *   codes_out DEVICE int32[n]: saturated two's-complement codes
+ *   seed      used only by ADAPT_ROUND_STOCHASTIC; hash layer id is 0
+ * n == 0 is legal and launches nothing. */
+int adapt_quantize(const float* x, int64_t n, int wl, int fl, int round_mode,
+                   uint64_t seed, int32_t* codes_out);
+
+/* As adapt_quantize with a hash layer id, an output width and a stream.
+ *   code_bits 8, 16 or 32: codes_out is int8/int16/int32[n]; WL must fit.
+ *   stream    cudaStream_t or NULL */
+int adapt_quantize_ex(const float* x, int64_t n, int wl, int fl, int round_mode,
+                      uint64_t seed, int32_t layer, int code_bits,
+                      void* codes_out, void* stream);
+
+/* Quantize at a format that is still on the device: `selected` is DEVICE
+ * int32[4] as written by a search into best_out + 4*l ({wl, fl, index, flags}).
+ * This is Algorithm 1's Quantize(L[l], Q[l].quant) directly after the switch,
+ * without a host round trip.  codes_out is DEVICE int32[n]. */
+int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected,
+                            int round_mode, uint64_t seed, int32_t layer,
+                            int32_t* codes_out, void* stream);
+
+/* Bytes of DEVICE workspace the search needs for these sizes (0 on invalid
+ * arguments).  lens is a HOST array. */
+size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers,
+                                    const adapt_grid* wl_fl_grid, int n_bins);
+
+/* The precision-switch search - the body of PushDown (Sec. 3.3; Algorithm 3)
+ * for every candidate of the grid and every layer in one batched pass:
+ * quantize each element to each <WL,FL>, count zero codes (the sparsity of
+ * Sec. 3.4), histogram the float tensor and every candidate's dequantized
+ * tensor over n_bins shared equal-width bins on the float tensor's [min,max]
+ * (the EDF of Sec. 3.3 at resolution n_bins), take KL(P||Q) in bits with P the
+ * candidate and Q the float histogram (the discrete KL equation), and pick the
+ * lowest <WL,FL> (by WL, then FL) whose divergence is 0; if none is, the
+ * candidate of least divergence.  Round-to-nearest-even, eps = 0.
+ *   tensors   HOST array of n_layers DEVICE pointers, fp32, 4-byte aligned
+ *   lens      HOST array of n_layers element counts (0 allowed)
+ *   kld_out   DEVICE double[n_layers][n_cand]   (+inf where a filled P bin
+ *             meets an empty Q bin)
+ *   zeros_out DEVICE int64[n_layers][n_cand]    zero codes per candidate
+ *   best_out  DEVICE int32[n_layers][4]         {wl, fl, grid index, flags}
+ * Scratch comes from a library-owned device buffer that is allocated (and
+ * grown) inside the call when needed; use the _ex call to supply your own. */
+int adapt_precision_search(const float* const* tensors, const int64_t* lens,
+                           int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                           double* kld_out, int64_t* zeros_out, int32_t* best_out);
+
+/* As adapt_precision_search, with options (rounding mode and seed, eps,
+ * pseudo-count, log base, stream, caller workspace, optional histogram and
+ * range outputs).  opts may be NULL (= all defaults). */
+int adapt_precision_search_ex(const float* const* tensors, const int64_t* lens,
+                              int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                              double* kld_out, int64_t* zeros_out, int32_t* best_out,
+                              const adapt_search_opts* opts);
+
+/* Host-buffer form of the search: tensors[l] and the three outputs are HOST
+ * memory (pinned memory makes the copies asynchronous and fast).  The call
+ * copies the layers to a library-owned device buffer, runs the search,
+ * copies the results back and synchronises the stream before returning, so
+ * data errors are returned as ADAPT_ERR_NONFINITE / ADAPT_ERR_RANGE.
+ * opts->workspace, hist_out and range_out must be NULL/0 here. */
+int adapt_precision_search_host(const float* const* tensors, const int64_t* lens,
+                                int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                                double* kld_out, int64_t* zeros_out, int32_t* best_out,
+                                const adapt_search_opts* opts);
+
+/* Host-buffer form of adapt_quantize_ex: x and codes_out are HOST memory;
+ * synchronous. */
+int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mode,
+                        uint64_t seed, int32_t layer, int code_bits, void* codes_out);
+
+/* Number of kernels the library has launched since it was loaded (all
+ * devices, all entry points). */
+uint64_t adapt_kernel_launch_count(void);
+
+/* Frees every library-owned device and pinned buffer of the current device's
+ * caches.  Safe to call at any time no library work is in flight. */
+int adapt_release(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAPT_B200_H_ */

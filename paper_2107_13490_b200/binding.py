@@ -1,0 +1,280 @@
+"""ctypes binding of libadapt_b200.so: the same entry points as include/adapt.h,
+argument marshalling only.  Tensors are torch CUDA tensors (device memory and
+streams come from torch); every computation runs in the library's kernels.
+
+The library must have been built (``python -m paper_2107_13490_b200.build``);
+there is no fallback: a missing library raises at the first call.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libadapt_b200.so")
+
+ROUND_RNE = 0
+ROUND_STOCHASTIC = 1
+FLAG_MET_EPS, FLAG_DEGENERATE, FLAG_NONFINITE, FLAG_RANGE = 1, 2, 4, 8
+OK, ERR_INVALID_ARG, ERR_NONFINITE, ERR_RANGE, ERR_CUDA, ERR_WORKSPACE = range(6)
+
+EXPORTS = (
+    "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
+    "adapt_quantize_ex", "adapt_quantize_selected", "adapt_search_workspace_bytes",
+    "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
+    "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_release",
+)
+
+
+class AdaptGrid(C.Structure):
+    _fields_ = [("n_cand", C.c_int32), ("wl", C.POINTER(C.c_int32)), ("fl", C.POINTER(C.c_int32))]
+
+
+class AdaptSearchOpts(C.Structure):
+    _fields_ = [("round_mode", C.c_int32), ("layer_base", C.c_int32), ("seed", C.c_uint64),
+                ("eps", C.c_double), ("pseudo_count", C.c_double), ("log_base", C.c_double),
+                ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("hist_out", C.c_void_p), ("range_out", C.c_void_p)]
+
+
+class AdaptError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        L = lib()
+        msg = L.adapt_status_string(status).decode()
+        detail = L.adapt_last_error().decode() if status == ERR_CUDA else ""
+        super().__init__(f"{where}: {msg}" + (f" ({detail})" if detail else ""))
+
+
+_lib = None
+
+
+def lib():
+    """Loads the shared library (once). Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2107_13490_b200.build` "
+                "(there is no CPU fallback)")
+        L = C.CDLL(LIB_PATH)
+        L.adapt_version.restype = C.c_char_p
+        L.adapt_status_string.restype = C.c_char_p
+        L.adapt_status_string.argtypes = [C.c_int]
+        L.adapt_last_error.restype = C.c_char_p
+        L.adapt_quantize.restype = C.c_int
+        L.adapt_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_uint64,
+                                     C.c_void_p]
+        L.adapt_quantize_ex.restype = C.c_int
+        L.adapt_quantize_ex.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_uint64,
+                                        C.c_int32, C.c_int, C.c_void_p, C.c_void_p]
+        L.adapt_quantize_selected.restype = C.c_int
+        L.adapt_quantize_selected.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_uint64,
+                                              C.c_int32, C.c_void_p, C.c_void_p]
+        L.adapt_search_workspace_bytes.restype = C.c_size_t
+        L.adapt_search_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int]
+        search_args = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int, C.c_void_p,
+                       C.c_void_p, C.c_void_p]
+        L.adapt_precision_search.restype = C.c_int
+        L.adapt_precision_search.argtypes = search_args
+        L.adapt_precision_search_ex.restype = C.c_int
+        L.adapt_precision_search_ex.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
+        L.adapt_precision_search_host.restype = C.c_int
+        L.adapt_precision_search_host.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
+        L.adapt_quantize_host.restype = C.c_int
+        L.adapt_quantize_host.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                          C.c_uint64, C.c_int32, C.c_int, C.c_void_p]
+        L.adapt_kernel_launch_count.restype = C.c_uint64
+        L.adapt_release.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise AdaptError(status, where)
+
+
+class Grid:
+    """Host-side candidate grid: keeps the numpy arrays alive for the C struct."""
+
+    def __init__(self, wl: Sequence[int], fl: Sequence[int]):
+        self.wl = np.ascontiguousarray(wl, dtype=np.int32)
+        self.fl = np.ascontiguousarray(fl, dtype=np.int32)
+        assert self.wl.shape == self.fl.shape and self.wl.ndim == 1
+        self.c = AdaptGrid(int(self.wl.size), self.wl.ctypes.data_as(C.POINTER(C.c_int32)),
+                           self.fl.ctypes.data_as(C.POINTER(C.c_int32)))
+
+    def __len__(self):
+        return int(self.wl.size)
+
+
+def _stream_handle(stream) -> Optional[int]:
+    if stream is None:
+        return int(torch.cuda.current_stream().cuda_stream) or None
+    return int(stream.cuda_stream) or None
+
+
+_CODE_DTYPES = {8: torch.int8, 16: torch.int16, 32: torch.int32}
+
+
+def adapt_version() -> str:
+    return lib().adapt_version().decode()
+
+
+def adapt_kernel_launch_count() -> int:
+    return int(lib().adapt_kernel_launch_count())
+
+
+def adapt_release() -> None:
+    _check(lib().adapt_release(), "adapt_release")
+
+
+def adapt_quantize(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                   codes_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """adapt_quantize of adapt.h (int32 codes, hash layer 0, legacy default stream)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    if codes_out is None:
+        codes_out = torch.empty(x.numel(), dtype=torch.int32, device=x.device)
+    assert codes_out.dtype == torch.int32 and codes_out.numel() == x.numel()
+    torch.cuda.current_stream().synchronize()  # the named call runs on the legacy default stream
+    _check(lib().adapt_quantize(x.data_ptr(), x.numel(), wl, fl, round_mode, seed,
+                                codes_out.data_ptr()), "adapt_quantize")
+    return codes_out
+
+
+def adapt_quantize_ex(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                      layer: int = 0, code_bits: int = 32, codes_out: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    if codes_out is None:
+        codes_out = torch.empty(x.numel(), dtype=_CODE_DTYPES.get(code_bits, torch.int32),
+                                device=x.device)
+    _check(lib().adapt_quantize_ex(x.data_ptr(), x.numel(), wl, fl, round_mode, seed, layer,
+                                   code_bits, codes_out.data_ptr(), _stream_handle(stream)),
+           "adapt_quantize_ex")
+    return codes_out
+
+
+def adapt_quantize_selected(x: torch.Tensor, selected: torch.Tensor, round_mode: int = ROUND_RNE,
+                            seed: int = 0, layer: int = 0,
+                            codes_out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    assert selected.is_cuda and selected.dtype == torch.int32 and selected.numel() >= 2
+    if codes_out is None:
+        codes_out = torch.empty(x.numel(), dtype=torch.int32, device=x.device)
+    _check(lib().adapt_quantize_selected(x.data_ptr(), x.numel(), selected.data_ptr(), round_mode,
+                                         seed, layer, codes_out.data_ptr(), _stream_handle(stream)),
+           "adapt_quantize_selected")
+    return codes_out
+
+
+def adapt_search_workspace_bytes(lens: Sequence[int], grid: Grid, n_bins: int) -> int:
+    ln = np.ascontiguousarray(lens, dtype=np.int64)
+    return int(lib().adapt_search_workspace_bytes(ln.ctypes.data, int(ln.size), C.byref(grid.c),
+                                                  n_bins))
+
+
+class SearchResult:
+    """Device outputs of one search call (torch tensors on the input device)."""
+
+    def __init__(self, kld, zeros, best, hist=None, value_range=None):
+        self.kld, self.zeros, self.best, self.hist, self.range = kld, zeros, best, hist, value_range
+
+
+def _marshal_tensors(tensors):
+    ptrs = np.zeros(len(tensors), dtype=np.uint64)
+    lens = np.zeros(len(tensors), dtype=np.int64)
+    for i, t in enumerate(tensors):
+        assert t.dtype == torch.float32 and t.is_contiguous()
+        ptrs[i] = t.data_ptr()
+        lens[i] = t.numel()
+    return ptrs, lens
+
+
+def adapt_precision_search(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                           out: Optional[SearchResult] = None) -> SearchResult:
+    """adapt_precision_search of adapt.h (RNE, eps 0, bits, legacy default stream)."""
+    dev = tensors[0].device
+    assert all(t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(grid)
+    if out is None:
+        out = SearchResult(torch.empty((L, Cn), dtype=torch.float64, device=dev),
+                           torch.empty((L, Cn), dtype=torch.int64, device=dev),
+                           torch.empty((L, 4), dtype=torch.int32, device=dev))
+    torch.cuda.current_stream().synchronize()
+    _check(lib().adapt_precision_search(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
+                                        n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
+                                        out.best.data_ptr()), "adapt_precision_search")
+    return out
+
+
+def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                              round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                              eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
+                              stream=None, workspace: Optional[torch.Tensor] = None,
+                              want_hist: bool = False, want_range: bool = False,
+                              out: Optional[SearchResult] = None) -> SearchResult:
+    dev = tensors[0].device
+    assert all(t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(grid)
+    if out is None:
+        out = SearchResult(
+            torch.empty((L, Cn), dtype=torch.float64, device=dev),
+            torch.empty((L, Cn), dtype=torch.int64, device=dev),
+            torch.empty((L, 4), dtype=torch.int32, device=dev),
+            torch.empty((L, Cn + 1, n_bins), dtype=torch.int32, device=dev) if want_hist else None,
+            torch.empty((L, 2), dtype=torch.float32, device=dev) if want_range else None)
+    o = AdaptSearchOpts()
+    o.round_mode, o.layer_base, o.seed = round_mode, layer_base, seed
+    o.eps, o.pseudo_count, o.log_base = eps, pseudo_count, log_base
+    o.stream = _stream_handle(stream)
+    if workspace is not None:
+        o.workspace, o.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    o.hist_out = out.hist.data_ptr() if out.hist is not None else None
+    o.range_out = out.range.data_ptr() if out.range is not None else None
+    _check(lib().adapt_precision_search_ex(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
+                                           n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
+                                           out.best.data_ptr(), C.byref(o)),
+           "adapt_precision_search_ex")
+    return out
+
+
+def adapt_precision_search_host(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                                round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                                eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
+                                out: Optional[SearchResult] = None) -> SearchResult:
+    """Host-buffer form: ``tensors`` and the outputs are CPU tensors (pinned for speed)."""
+    assert all(not t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(grid)
+    if out is None:
+        out = SearchResult(torch.empty((L, Cn), dtype=torch.float64),
+                           torch.empty((L, Cn), dtype=torch.int64),
+                           torch.empty((L, 4), dtype=torch.int32))
+    o = AdaptSearchOpts()
+    o.round_mode, o.layer_base, o.seed = round_mode, layer_base, seed
+    o.eps, o.pseudo_count, o.log_base = eps, pseudo_count, log_base
+    o.stream = _stream_handle(None)
+    _check(lib().adapt_precision_search_host(ptrs.ctypes.data, lens.ctypes.data, L,
+                                             C.byref(grid.c), n_bins, out.kld.data_ptr(),
+                                             out.zeros.data_ptr(), out.best.data_ptr(),
+                                             C.byref(o)), "adapt_precision_search_host")
+    return out
+
+
+def adapt_quantize_host(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROUND_RNE,
+                        seed: int = 0, layer: int = 0, code_bits: int = 32,
+                        codes_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    assert (not x.is_cuda) and x.dtype == torch.float32 and x.is_contiguous()
+    if codes_out is None:
+        codes_out = torch.empty(x.numel(), dtype=_CODE_DTYPES.get(code_bits, torch.int32))
+    _check(lib().adapt_quantize_host(x.data_ptr(), x.numel(), wl, fl, round_mode, seed, layer,
+                                     code_bits, codes_out.data_ptr()), "adapt_quantize_host")
+    return codes_out

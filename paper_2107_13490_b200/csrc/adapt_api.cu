@@ -1,0 +1,538 @@
+// C-ABI entry points of libadapt_b200.so: argument checks, workspace layout,
+// kernel launches.  Declarations and argument contracts live in adapt.h.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <numeric>
+#include <vector>
+
+#include "../../include/adapt.h"
+#include "common.cuh"
+#include "k_kld_select.cuh"
+#include "k_quantize.cuh"
+#include "k_range.cuh"
+#include "k_search_direct.cuh"
+
+namespace {
+
+using namespace adapt;
+
+std::mutex g_mutex;                     // serialises calls that touch library-owned state
+std::atomic<uint64_t> g_launches{0};
+char g_last_error[512] = "";
+
+int cuda_fail(cudaError_t e, const char* what) {
+  std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+  return ADAPT_ERR_CUDA;
+}
+#define ADAPT_CUDA(call)                                     \
+  do {                                                       \
+    cudaError_t e_ = (call);                                 \
+    if (e_ != cudaSuccess) return cuda_fail(e_, #call);      \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- per-device caches --------------------------------------------------------
+
+constexpr int kMaxDevices = 64;
+constexpr int kRingSlots = 4;
+
+struct PinnedSlot {
+  void* host = nullptr;
+  size_t bytes = 0;
+  cudaEvent_t done = nullptr;
+};
+
+struct DeviceCache {
+  bool props_ready = false;
+  int sm_count = 0;
+  int max_smem_optin = 0;
+  void* workspace = nullptr;   size_t workspace_bytes = 0;
+  void* stage_in = nullptr;    size_t stage_in_bytes = 0;    // host-form calls: inputs
+  void* stage_out = nullptr;   size_t stage_out_bytes = 0;   // host-form calls: outputs
+  PinnedSlot ring[kRingSlots];
+  int ring_next = 0;
+};
+
+DeviceCache g_cache[kMaxDevices];
+
+int current_cache(DeviceCache** out) {
+  int dev = 0;
+  ADAPT_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "device index %d not supported", dev);
+    return ADAPT_ERR_CUDA;
+  }
+  DeviceCache& c = g_cache[dev];
+  if (!c.props_ready) {
+    ADAPT_CUDA(cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    ADAPT_CUDA(cudaDeviceGetAttribute(&c.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    c.props_ready = true;
+  }
+  *out = &c;
+  return ADAPT_OK;
+}
+
+int grow_device(void** ptr, size_t* have, size_t need) {
+  if (*have >= need) return ADAPT_OK;
+  if (*ptr) { ADAPT_CUDA(cudaFree(*ptr)); *ptr = nullptr; *have = 0; }
+  ADAPT_CUDA(cudaMalloc(ptr, need));
+  *have = need;
+  return ADAPT_OK;
+}
+
+// A pinned host slot whose previous upload has finished.
+int acquire_slot(DeviceCache& c, size_t bytes, PinnedSlot** out) {
+  PinnedSlot& s = c.ring[c.ring_next];
+  c.ring_next = (c.ring_next + 1) % kRingSlots;
+  if (!s.done) ADAPT_CUDA(cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming));
+  ADAPT_CUDA(cudaEventSynchronize(s.done));
+  if (s.bytes < bytes) {
+    if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }
+    size_t want = align_up(std::max<size_t>(bytes, 16384), 4096);
+    ADAPT_CUDA(cudaMallocHost(&s.host, want));
+    s.bytes = want;
+  }
+  *out = &s;
+  return ADAPT_OK;
+}
+
+// ---- search plan ----------------------------------------------------------------
+
+struct Plan {
+  int n_layers = 0, n_cand = 0, n_fl = 0, n_bins = 0;
+  long long n_tiles = 0;
+  std::vector<int> fl_list, slot, order;
+  // byte offsets inside the workspace
+  size_t off_layers = 0, off_wl = 0, off_fl = 0, off_slot = 0, off_order = 0, off_fl_list = 0,
+         off_state = 0, blob_bytes = 0;
+  size_t off_zeros = 0, off_q = 0, off_u = 0, accum_bytes = 0;
+  size_t total = 0;
+};
+
+constexpr int kMaxBins = 16384;
+
+bool valid_format(int wl, int fl) { return wl >= 2 && wl <= 32 && fl >= 0 && fl < wl; }
+
+// Validates sizes and fills the layout.  Returns false on invalid arguments.
+bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_bins, Plan* p) {
+  if (!lens || !grid || !grid->wl || !grid->fl) return false;
+  if (n_layers < 1 || n_layers > 65535) return false;
+  if (grid->n_cand < 1 || grid->n_cand > 65535) return false;
+  if (n_bins < 1 || n_bins > kMaxBins) return false;
+  for (int c = 0; c < grid->n_cand; ++c)
+    if (!valid_format(grid->wl[c], grid->fl[c])) return false;
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    if (lens[l] < 0 || lens[l] >= (1ll << 32)) return false;
+    tiles += (lens[l] + 3 + kTile - 1) / kTile;  // upper bound, misalignment included
+  }
+  (void)tiles;
+  p->n_layers = n_layers; p->n_cand = grid->n_cand; p->n_bins = n_bins;
+
+  bool seen[kMaxFl] = {false};
+  for (int c = 0; c < grid->n_cand; ++c) seen[grid->fl[c]] = true;
+  int slot_of[kMaxFl];
+  p->fl_list.clear();
+  for (int f = 0; f < kMaxFl; ++f)
+    if (seen[f]) { slot_of[f] = static_cast<int>(p->fl_list.size()); p->fl_list.push_back(f); }
+  p->n_fl = static_cast<int>(p->fl_list.size());
+  p->slot.resize(grid->n_cand);
+  for (int c = 0; c < grid->n_cand; ++c) p->slot[c] = slot_of[grid->fl[c]];
+  p->order.resize(grid->n_cand);
+  std::iota(p->order.begin(), p->order.end(), 0);
+  std::stable_sort(p->order.begin(), p->order.end(), [&](int a, int b) {
+    if (grid->wl[a] != grid->wl[b]) return grid->wl[a] < grid->wl[b];
+    return grid->fl[a] < grid->fl[b];
+  });
+
+  const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_fl;
+  size_t o = 0;
+  p->off_layers = o;  o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
+  p->off_wl = o;      o = align_up(o + sizeof(int) * C, 16);
+  p->off_fl = o;      o = align_up(o + sizeof(int) * C, 16);
+  p->off_slot = o;    o = align_up(o + sizeof(int) * C, 16);
+  p->off_order = o;   o = align_up(o + sizeof(int) * C, 16);
+  p->off_fl_list = o; o = align_up(o + sizeof(int) * F, 16);
+  p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
+  p->blob_bytes = o;
+  p->off_zeros = o;   o = align_up(o + sizeof(unsigned long long) * L * F, 256);
+  p->off_q = o;       o = align_up(o + sizeof(unsigned) * L * B, 256);
+  p->off_u = o;       o = align_up(o + sizeof(unsigned) * L * F * B, 256);
+  p->accum_bytes = o - p->off_zeros;
+  p->total = o;
+  return true;
+}
+
+}  // namespace
+
+// ---- search driver ----------------------------------------------------------------
+
+namespace {
+
+struct SearchArgs {
+  const float* const* tensors;  // host array of device pointers
+  const int64_t* lens;
+  int n_layers;
+  const adapt_grid* grid;
+  int n_bins;
+  double* kld_out;
+  int64_t* zeros_out;
+  int32_t* best_out;
+  adapt_search_opts opts;
+};
+
+adapt_search_opts default_opts() {
+  adapt_search_opts o;
+  std::memset(&o, 0, sizeof(o));
+  return o;
+}
+
+// Enqueues the whole search on opts.stream.  Caller holds g_mutex.
+int run_search(DeviceCache& dc, const SearchArgs& a) {
+  const adapt_search_opts& o = a.opts;
+  if (!a.tensors || !a.kld_out || !a.zeros_out || !a.best_out) return ADAPT_ERR_INVALID_ARG;
+  if (o.round_mode != ADAPT_ROUND_RNE && o.round_mode != ADAPT_ROUND_STOCHASTIC)
+    return ADAPT_ERR_INVALID_ARG;
+  if (!(o.eps >= 0.0) || !(o.pseudo_count >= 0.0)) return ADAPT_ERR_INVALID_ARG;
+  const double base = (o.log_base == 0.0) ? 2.0 : o.log_base;
+  if (!(base > 0.0) || base == 1.0 || !std::isfinite(base)) return ADAPT_ERR_INVALID_ARG;
+
+  Plan plan;
+  if (!make_plan(a.lens, a.n_layers, a.grid, a.n_bins, &plan)) return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < a.n_layers; ++l) {
+    if (a.lens[l] > 0 && !a.tensors[l]) return ADAPT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(a.tensors[l]) & 3u) return ADAPT_ERR_INVALID_ARG;
+  }
+
+  char* ws = nullptr;
+  if (o.workspace) {
+    if (reinterpret_cast<uintptr_t>(o.workspace) & 255u) return ADAPT_ERR_INVALID_ARG;
+    if (o.workspace_bytes < plan.total) return ADAPT_ERR_WORKSPACE;
+    ws = static_cast<char*>(o.workspace);
+  } else {
+    int rc = grow_device(&dc.workspace, &dc.workspace_bytes, plan.total);
+    if (rc != ADAPT_OK) return rc;
+    ws = static_cast<char*>(dc.workspace);
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
+
+  // host image of the descriptor block
+  PinnedSlot* slot = nullptr;
+  int rc = acquire_slot(dc, plan.blob_bytes, &slot);
+  if (rc != ADAPT_OK) return rc;
+  char* h = static_cast<char*>(slot->host);
+  std::memset(h, 0, plan.blob_bytes);
+  LayerDesc* hl = reinterpret_cast<LayerDesc*>(h + plan.off_layers);
+  long long tiles = 0;
+  for (int l = 0; l < a.n_layers; ++l) {
+    const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(a.tensors[l]) >> 2) & 3u);
+    hl[l].ptr = a.tensors[l];
+    hl[l].n = a.lens[l];
+    hl[l].tile_begin = tiles;
+    hl[l].mis = a.lens[l] > 0 ? mis : 0;
+    hl[l].layer_id = o.layer_base + l;
+    if (a.lens[l] > 0) tiles += (a.lens[l] + mis + kTile - 1) / kTile;
+  }
+  hl[a.n_layers].ptr = nullptr;
+  hl[a.n_layers].n = 0;
+  hl[a.n_layers].tile_begin = tiles;
+  plan.n_tiles = tiles;
+  std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_order, plan.order.data(), sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_fl_list, plan.fl_list.data(), sizeof(int) * plan.n_fl);
+  LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+
+  ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
+  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  ADAPT_CUDA(cudaMemsetAsync(ws + plan.off_zeros, 0, plan.accum_bytes, stream));
+
+  const LayerDesc* d_layers = reinterpret_cast<const LayerDesc*>(ws + plan.off_layers);
+  LayerState* d_state = reinterpret_cast<LayerState*>(ws + plan.off_state);
+  unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + plan.off_zeros);
+  unsigned* d_q = reinterpret_cast<unsigned*>(ws + plan.off_q);
+  unsigned* d_u = reinterpret_cast<unsigned*>(ws + plan.off_u);
+
+  // K1: range scan
+  if (tiles > 0) {
+    const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc.sm_count));
+    range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(d_layers, a.n_layers, tiles, d_state);
+    ADAPT_CUDA(cudaGetLastError());
+    ++g_launches;
+  }
+  range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
+      d_layers, a.n_layers, a.n_bins, d_state, o.range_out);
+  ADAPT_CUDA(cudaGetLastError());
+  ++g_launches;
+
+  // K2: fused quantize / zero count / histograms
+  if (tiles > 0) {
+    SearchParams sp;
+    sp.layers = d_layers; sp.state = d_state;
+    sp.fl_list = reinterpret_cast<const int*>(ws + plan.off_fl_list);
+    sp.n_layers = a.n_layers; sp.n_fl = plan.n_fl; sp.n_bins = a.n_bins; sp.n_tiles = tiles;
+    sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed;
+    const size_t per_hist = sizeof(unsigned) * a.n_bins;
+    const size_t budget = 100 * 1024;
+    int fg = static_cast<int>(budget / per_hist) - 1;
+    fg = std::max(1, std::min(fg, plan.n_fl));
+    sp.fl_per_group = fg;
+    const int groups = (plan.n_fl + fg - 1) / fg;
+    const size_t smem = per_hist * (fg + 1);
+    if (smem + 1024 > static_cast<size_t>(dc.max_smem_optin)) return ADAPT_ERR_INVALID_ARG;
+    auto kern = (o.round_mode == ADAPT_ROUND_STOCHASTIC) ? search_direct_kernel<true>
+                                                         : search_direct_kernel<false>;
+    ADAPT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(smem)));
+    const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
+    dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)),
+              groups);
+    kern<<<grid, kSearchThreads, smem, stream>>>(sp);
+    ADAPT_CUDA(cudaGetLastError());
+    ++g_launches;
+  }
+
+  // K3: divergence per (layer, candidate), then selection per layer
+  KldParams kp;
+  kp.layers = d_layers; kp.state = d_state;
+  kp.cand_wl = reinterpret_cast<const int*>(ws + plan.off_wl);
+  kp.cand_fl = reinterpret_cast<const int*>(ws + plan.off_fl);
+  kp.cand_slot = reinterpret_cast<const int*>(ws + plan.off_slot);
+  kp.cand_order = reinterpret_cast<const int*>(ws + plan.off_order);
+  kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_fl; kp.n_bins = a.n_bins;
+  kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
+  kp.alpha = o.pseudo_count; kp.inv_ln_base = 1.0 / std::log(base); kp.eps = o.eps;
+  kp.kld_out = a.kld_out; kp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
+  kp.best_out = a.best_out; kp.hist_out = o.hist_out;
+  kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(kp);
+  ADAPT_CUDA(cudaGetLastError());
+  ++g_launches;
+  select_kernel<<<a.n_layers, 32, 0, stream>>>(kp);
+  ADAPT_CUDA(cudaGetLastError());
+  ++g_launches;
+  return ADAPT_OK;
+}
+
+template <typename T>
+int launch_quantize_t(const QuantParams& qp, bool stochastic, bool vec, int grid, cudaStream_t s) {
+  if (stochastic) {
+    if (vec) quantize_kernel<T, true, true><<<grid, kQuantThreads, 0, s>>>(qp);
+    else quantize_kernel<T, true, false><<<grid, kQuantThreads, 0, s>>>(qp);
+  } else {
+    if (vec) quantize_kernel<T, false, true><<<grid, kQuantThreads, 0, s>>>(qp);
+    else quantize_kernel<T, false, false><<<grid, kQuantThreads, 0, s>>>(qp);
+  }
+  ADAPT_CUDA(cudaGetLastError());
+  ++g_launches;
+  return ADAPT_OK;
+}
+
+int run_quantize(const float* x, int64_t n, int wl, int fl, const int32_t* selected,
+                 int round_mode, uint64_t seed, int32_t layer, int code_bits, void* codes_out,
+                 void* stream) {
+  if (n < 0) return ADAPT_ERR_INVALID_ARG;
+  if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
+    return ADAPT_ERR_INVALID_ARG;
+  if (code_bits != 8 && code_bits != 16 && code_bits != 32) return ADAPT_ERR_INVALID_ARG;
+  if (!selected && (!valid_format(wl, fl) || wl > code_bits)) return ADAPT_ERR_INVALID_ARG;
+  if (n == 0) return ADAPT_OK;
+  if (!x || !codes_out) return ADAPT_ERR_INVALID_ARG;
+  const int ob = code_bits / 8;
+  if ((reinterpret_cast<uintptr_t>(x) & 3u) || (reinterpret_cast<uintptr_t>(codes_out) & (ob - 1)))
+    return ADAPT_ERR_INVALID_ARG;
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+
+  QuantParams qp;
+  qp.x = x; qp.out = codes_out; qp.n = n; qp.wl = wl; qp.fl = fl; qp.selected = selected;
+  qp.seed = seed; qp.layer_id = layer;
+  const bool vec = !(reinterpret_cast<uintptr_t>(x) & 15u) &&
+                   !(reinterpret_cast<uintptr_t>(codes_out) & (4 * ob - 1));
+  const long long work = vec ? std::max<long long>(1, n / 4) : n;
+  const long long want = (work + kQuantThreads - 1) / kQuantThreads;
+  const int grid = static_cast<int>(std::min<long long>(want, 16ll * dc->sm_count));
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const bool st = round_mode == ADAPT_ROUND_STOCHASTIC;
+  if (code_bits == 8) return launch_quantize_t<int8_t>(qp, st, vec, grid, s);
+  if (code_bits == 16) return launch_quantize_t<int16_t>(qp, st, vec, grid, s);
+  return launch_quantize_t<int32_t>(qp, st, vec, grid, s);
+}
+
+}  // namespace
+
+// ---- exported entry points ---------------------------------------------------------
+
+extern "C" {
+
+const char* adapt_version(void) { return "adapt-b200 0.1"; }
+
+const char* adapt_status_string(int status) {
+  switch (status) {
+    case ADAPT_OK: return "ok";
+    case ADAPT_ERR_INVALID_ARG: return "invalid argument";
+    case ADAPT_ERR_NONFINITE: return "input holds NaN or Inf";
+    case ADAPT_ERR_RANGE: return "input holds |x| >= 2^64";
+    case ADAPT_ERR_CUDA: return "CUDA runtime error";
+    case ADAPT_ERR_WORKSPACE: return "workspace too small";
+    default: return "unknown status";
+  }
+}
+
+const char* adapt_last_error(void) { return g_last_error; }
+
+uint64_t adapt_kernel_launch_count(void) { return g_launches.load(); }
+
+int adapt_quantize(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
+                   int32_t* codes_out) {
+  return run_quantize(x, n, wl, fl, nullptr, round_mode, seed, 0, 32, codes_out, nullptr);
+}
+
+int adapt_quantize_ex(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
+                      int32_t layer, int code_bits, void* codes_out, void* stream) {
+  return run_quantize(x, n, wl, fl, nullptr, round_mode, seed, layer, code_bits, codes_out, stream);
+}
+
+int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected, int round_mode,
+                            uint64_t seed, int32_t layer, int32_t* codes_out, void* stream) {
+  if (!selected) return ADAPT_ERR_INVALID_ARG;
+  return run_quantize(x, n, 0, 0, selected, round_mode, seed, layer, 32, codes_out, stream);
+}
+
+size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers, const adapt_grid* grid,
+                                    int n_bins) {
+  Plan plan;
+  if (!make_plan(lens, n_layers, grid, n_bins, &plan)) return 0;
+  return plan.total;
+}
+
+int adapt_precision_search_ex(const float* const* tensors, const int64_t* lens, int n_layers,
+                              const adapt_grid* grid, int n_bins, double* kld_out,
+                              int64_t* zeros_out, int32_t* best_out,
+                              const adapt_search_opts* opts) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  SearchArgs a{tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
+               opts ? *opts : default_opts()};
+  return run_search(*dc, a);
+}
+
+int adapt_precision_search(const float* const* tensors, const int64_t* lens, int n_layers,
+                           const adapt_grid* grid, int n_bins, double* kld_out,
+                           int64_t* zeros_out, int32_t* best_out) {
+  return adapt_precision_search_ex(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out,
+                                   best_out, nullptr);
+}
+
+int adapt_precision_search_host(const float* const* tensors, const int64_t* lens, int n_layers,
+                                const adapt_grid* grid, int n_bins, double* kld_out,
+                                int64_t* zeros_out, int32_t* best_out,
+                                const adapt_search_opts* opts) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  adapt_search_opts o = opts ? *opts : default_opts();
+  if (o.workspace || o.workspace_bytes || o.hist_out || o.range_out) return ADAPT_ERR_INVALID_ARG;
+  if (!tensors || !kld_out || !zeros_out || !best_out) return ADAPT_ERR_INVALID_ARG;
+  Plan plan;
+  if (!make_plan(lens, n_layers, grid, n_bins, &plan)) return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (lens[l] > 0 && !tensors[l]) return ADAPT_ERR_INVALID_ARG;
+
+  // device copies of the layers, 256-byte aligned each
+  std::vector<size_t> off(n_layers);
+  size_t in_bytes = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    off[l] = in_bytes;
+    in_bytes = align_up(in_bytes + sizeof(float) * static_cast<size_t>(lens[l]), 256);
+  }
+  const size_t C = plan.n_cand, L = n_layers;
+  const size_t kld_bytes = align_up(sizeof(double) * L * C, 256);
+  const size_t zeros_bytes = align_up(sizeof(int64_t) * L * C, 256);
+  const size_t best_bytes = align_up(sizeof(int32_t) * 4 * L, 256);
+  rc = grow_device(&dc->stage_in, &dc->stage_in_bytes, std::max<size_t>(in_bytes, 256));
+  if (rc != ADAPT_OK) return rc;
+  rc = grow_device(&dc->stage_out, &dc->stage_out_bytes, kld_bytes + zeros_bytes + best_bytes);
+  if (rc != ADAPT_OK) return rc;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
+  std::vector<const float*> dptr(n_layers);
+  for (int l = 0; l < n_layers; ++l) {
+    dptr[l] = reinterpret_cast<const float*>(static_cast<char*>(dc->stage_in) + off[l]);
+    if (lens[l] > 0)
+      ADAPT_CUDA(cudaMemcpyAsync(const_cast<float*>(dptr[l]), tensors[l],
+                                 sizeof(float) * static_cast<size_t>(lens[l]),
+                                 cudaMemcpyHostToDevice, stream));
+  }
+  char* so = static_cast<char*>(dc->stage_out);
+  SearchArgs a{dptr.data(), lens, n_layers, grid, n_bins, reinterpret_cast<double*>(so),
+               reinterpret_cast<int64_t*>(so + kld_bytes),
+               reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes), o};
+  rc = run_search(*dc, a);
+  if (rc != ADAPT_OK) return rc;
+  ADAPT_CUDA(cudaMemcpyAsync(kld_out, a.kld_out, sizeof(double) * L * C, cudaMemcpyDeviceToHost, stream));
+  ADAPT_CUDA(cudaMemcpyAsync(zeros_out, a.zeros_out, sizeof(int64_t) * L * C, cudaMemcpyDeviceToHost, stream));
+  ADAPT_CUDA(cudaMemcpyAsync(best_out, a.best_out, sizeof(int32_t) * 4 * L, cudaMemcpyDeviceToHost, stream));
+  ADAPT_CUDA(cudaStreamSynchronize(stream));
+  int status = ADAPT_OK;
+  for (int l = 0; l < n_layers; ++l) {
+    if (best_out[4 * l + 3] & ADAPT_FLAG_NONFINITE) return ADAPT_ERR_NONFINITE;
+    if (best_out[4 * l + 3] & ADAPT_FLAG_RANGE) status = ADAPT_ERR_RANGE;
+  }
+  return status;
+}
+
+int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
+                        int32_t layer, int code_bits, void* codes_out) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (n < 0 || (code_bits != 8 && code_bits != 16 && code_bits != 32)) return ADAPT_ERR_INVALID_ARG;
+  if (!valid_format(wl, fl) || wl > code_bits) return ADAPT_ERR_INVALID_ARG;
+  if (n == 0) return ADAPT_OK;
+  if (!x || !codes_out) return ADAPT_ERR_INVALID_ARG;
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  const size_t in_bytes = sizeof(float) * static_cast<size_t>(n);
+  const size_t out_bytes = static_cast<size_t>(code_bits / 8) * static_cast<size_t>(n);
+  rc = grow_device(&dc->stage_in, &dc->stage_in_bytes, in_bytes);
+  if (rc != ADAPT_OK) return rc;
+  rc = grow_device(&dc->stage_out, &dc->stage_out_bytes, out_bytes);
+  if (rc != ADAPT_OK) return rc;
+  ADAPT_CUDA(cudaMemcpyAsync(dc->stage_in, x, in_bytes, cudaMemcpyHostToDevice, nullptr));
+  rc = run_quantize(static_cast<const float*>(dc->stage_in), n, wl, fl, nullptr, round_mode, seed,
+                    layer, code_bits, dc->stage_out, nullptr);
+  if (rc != ADAPT_OK) return rc;
+  ADAPT_CUDA(cudaMemcpyAsync(codes_out, dc->stage_out, out_bytes, cudaMemcpyDeviceToHost, nullptr));
+  ADAPT_CUDA(cudaStreamSynchronize(nullptr));
+  return ADAPT_OK;
+}
+
+int adapt_release(void) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  ADAPT_CUDA(cudaDeviceSynchronize());
+  if (dc->workspace) { ADAPT_CUDA(cudaFree(dc->workspace)); dc->workspace = nullptr; dc->workspace_bytes = 0; }
+  if (dc->stage_in) { ADAPT_CUDA(cudaFree(dc->stage_in)); dc->stage_in = nullptr; dc->stage_in_bytes = 0; }
+  if (dc->stage_out) { ADAPT_CUDA(cudaFree(dc->stage_out)); dc->stage_out = nullptr; dc->stage_out_bytes = 0; }
+  for (PinnedSlot& s : dc->ring) {
+    if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }
+    if (s.done) { ADAPT_CUDA(cudaEventDestroy(s.done)); s.done = nullptr; }
+  }
+  return ADAPT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,170 @@
+// K3: batched divergence and selection over all (layer, candidate) pairs.
+//
+// kld_kernel: one CTA per (candidate, layer).  Folds the layer's unsaturated
+// per-FL histogram into the candidate's histogram (both tails collapse into
+// the bins of the two saturation values), then sums the discrete
+// Kullback-Leibler divergence KL(P||Q) (Sec. 3.3), P = candidate, Q = float
+// tensor, in double precision.  With integer counts p, q that share the total
+// N, the term (p/N) log((p/N)/(q/N)) is evaluated as p * log1p((p - q)/q) / N:
+// the difference is exact in integers, so histograms that differ by a few
+// counts in well-filled bins do not lose their divergence to cancellation.
+//
+// select_kernel: one warp per layer; the lowest <WL,FL> (WL first, then FL)
+// with KLD <= eps, else the candidate of least divergence (Algorithm 3).
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+#include "k_range.cuh"
+
+namespace adapt {
+
+constexpr int kKldThreads = 256;
+
+struct KldParams {
+  const LayerDesc* layers;
+  const LayerState* state;
+  const int* cand_wl;          // [n_cand]
+  const int* cand_fl;          // [n_cand]
+  const int* cand_slot;        // [n_cand] index of the candidate's FL in the distinct-FL list
+  const int* cand_order;       // [n_cand] candidate indices sorted by (WL, FL, index)
+  int n_layers, n_cand, n_fl, n_bins;
+  const unsigned* q_hist;      // [n_layers][n_bins]
+  const unsigned* u_hist;      // [n_layers][n_fl][n_bins]
+  const unsigned long long* zeros;  // [n_layers][n_fl]
+  double alpha;                // pseudo-count
+  double inv_ln_base;          // 1 / ln(log base)
+  double eps;
+  double* kld_out;             // [n_layers][n_cand]
+  long long* zeros_out;        // [n_layers][n_cand]
+  int* best_out;               // [n_layers][4]
+  unsigned* hist_out;          // optional [n_layers][n_cand + 1][n_bins]
+};
+
+__device__ __forceinline__ double block_sum(double v, double* s_buf) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  const int w = threadIdx.x >> 5;
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_buf[w] = v;
+  __syncthreads();
+  double t = 0.0;
+  for (int i = 0; i < kKldThreads / 32; ++i) t += s_buf[i];
+  return t;
+}
+
+__global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
+  __shared__ double s_buf[kKldThreads / 32];
+  __shared__ int s_inf;
+  const int c = blockIdx.x, l = blockIdx.y;
+  const int B = p.n_bins;
+  const LayerState S = p.state[l];
+  const long long n = p.layers[l].n;
+  const size_t out = static_cast<size_t>(l) * p.n_cand + c;
+  const int wl = p.cand_wl[c], fl = p.cand_fl[c], slot = p.cand_slot[c];
+
+  if (S.flags & (kFlagNonfinite | kFlagRange)) {
+    if (threadIdx.x == 0) {
+      p.kld_out[out] = __longlong_as_double(0x7ff8000000000000ll);  // NaN: unspecified output
+      p.zeros_out[out] = 0;
+    }
+    return;
+  }
+
+  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + slot) * B;
+  const unsigned* Q = p.q_hist + static_cast<size_t>(l) * B;
+
+  // bins of the two saturation values of <WL,FL>
+  const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
+  const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
+  const int bh = bin_of(dequantize(hi_code, fl), S.lo, S.scale, S.bmax);
+  const int bl = bin_of(dequantize(lo_code, fl), S.lo, S.scale, S.bmax);
+
+  // tail masses that fold into bl and bh
+  double lo_mass = 0.0, hi_mass = 0.0;
+  for (int b = threadIdx.x; b < B; b += kKldThreads) {
+    unsigned u = U[b];
+    if (b <= bl) lo_mass += u;
+    if (b >= bh) hi_mass += u;
+  }
+  lo_mass = block_sum(lo_mass, s_buf);
+  hi_mass = block_sum(hi_mass, s_buf);
+  if (threadIdx.x == 0) s_inf = 0;
+  __syncthreads();
+
+  unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * B
+                           : nullptr;
+  unsigned* H0 = (p.hist_out && c == 0)
+                     ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * B : nullptr;
+  double sum = 0.0;
+  bool inf = false;
+  for (int b = threadIdx.x; b < B; b += kKldThreads) {
+    long long pc;
+    if (bl == bh) pc = (b == bl) ? n : 0;
+    else if (b < bl || b > bh) pc = 0;
+    else if (b == bl) pc = static_cast<long long>(lo_mass);
+    else if (b == bh) pc = static_cast<long long>(hi_mass);
+    else pc = U[b];
+    const long long qc = Q[b];
+    if (H) H[b] = static_cast<unsigned>(pc);
+    if (H0) H0[b] = static_cast<unsigned>(qc);
+    const double pa = static_cast<double>(pc) + p.alpha;
+    const double qa = static_cast<double>(qc) + p.alpha;
+    if (pa > 0.0) {
+      if (qa <= 0.0) inf = true;
+      else sum += pa * log1p(static_cast<double>(pc - qc) / qa);
+    }
+  }
+  if (inf) s_inf = 1;
+  sum = block_sum(sum, s_buf);
+  if (threadIdx.x == 0) {
+    const double n_eff = static_cast<double>(n) + p.alpha * B;
+    double k;
+    if (n_eff <= 0.0) k = 0.0;
+    else if (s_inf) k = __longlong_as_double(0x7ff0000000000000ll);
+    else { k = sum * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
+    p.kld_out[out] = k;
+    p.zeros_out[out] = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + slot]);
+  }
+}
+
+// lexicographic minimum over (key, position): smaller key wins, then earlier position
+__device__ __forceinline__ void arg_min_merge(double& k, int& pos, double k2, int pos2) {
+  if (pos2 >= 0 && (pos < 0 || k2 < k || (k2 == k && pos2 < pos))) { k = k2; pos = pos2; }
+}
+
+__global__ void select_kernel(const KldParams p) {
+  const int l = blockIdx.x;
+  const int lane = threadIdx.x;  // one warp
+  const LayerState S = p.state[l];
+  const double* kld = p.kld_out + static_cast<size_t>(l) * p.n_cand;
+
+  int first_ok = 0x7fffffff;  // position (in candidate order) of the first KLD <= eps
+  double min_k = 0.0;
+  int min_pos = -1;           // position of the least finite divergence
+  for (int pos = lane; pos < p.n_cand; pos += 32) {
+    const double k = kld[p.cand_order[pos]];
+    if (k <= p.eps) first_ok = min(first_ok, pos);
+    if (k < __longlong_as_double(0x7ff0000000000000ll)) arg_min_merge(min_k, min_pos, k, pos);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    first_ok = min(first_ok, __shfl_xor_sync(0xffffffffu, first_ok, o));
+    double k2 = __shfl_xor_sync(0xffffffffu, min_k, o);
+    int pos2 = __shfl_xor_sync(0xffffffffu, min_pos, o);
+    arg_min_merge(min_k, min_pos, k2, pos2);
+  }
+  if (lane == 0) {
+    unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
+    int pos;
+    if (first_ok != 0x7fffffff) { pos = first_ok; flags |= 1u; }
+    else if (min_pos >= 0) pos = min_pos;
+    else pos = p.n_cand - 1;
+    const int c = p.cand_order[pos];
+    int* o = p.best_out + 4 * l;
+    o[0] = p.cand_wl[c]; o[1] = p.cand_fl[c]; o[2] = c; o[3] = static_cast<int>(flags);
+  }
+}
+
+}  // namespace adapt

@@ -1,0 +1,74 @@
+// K4: stand-alone Quantize(L, <WL,FL>) writing int8 / int16 / int32 codes
+// (Algorithm 1, the re-quantisation of each layer; Sec. 2.1 / 3.2).
+// Streaming: 4 bytes read and 1/2/4 bytes written per element.
+#pragma once
+
+#include "common.cuh"
+
+namespace adapt {
+
+constexpr int kQuantThreads = 256;
+
+template <typename T> struct Pack4;
+template <> struct Pack4<int8_t>  { using type = char4;  };
+template <> struct Pack4<int16_t> { using type = short4; };
+template <> struct Pack4<int32_t> { using type = int4;   };
+
+struct QuantParams {
+  const float* x;
+  void* out;
+  long long n;
+  int wl, fl;
+  const int* selected;  // optional device {wl, fl, ...}: overrides wl/fl
+  unsigned long long seed;
+  int layer_id;
+};
+
+template <bool kStochastic>
+__device__ __forceinline__ int quantize_one(float x, float two_fl, int wl, unsigned long long seed,
+                                            int layer_id, long long i) {
+  float pr = 0.0f;
+  if (kStochastic) {
+    unsigned h = hash24(seed, static_cast<unsigned long long>(layer_id),
+                        static_cast<unsigned long long>(i));
+    pr = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);
+  }
+  return saturate_code(round_scaled<kStochastic>(x, two_fl, pr), wl);
+}
+
+// kVec: x is 16-byte aligned and out is aligned for a 4-element store; each
+// thread then handles whole quads, the last (n % 4) elements go through the
+// scalar tail.  Otherwise every element takes the scalar path.
+template <typename T, bool kStochastic, bool kVec>
+__global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const QuantParams p) {
+  int wl = p.wl, fl = p.fl;
+  if (p.selected) { wl = p.selected[0]; fl = p.selected[1]; }
+  if (wl < 2 || wl > 32 || fl < 0 || fl >= wl) return;  // never true for validated input
+  const float two_fl = pow2f(fl);
+  T* out = static_cast<T*>(p.out);
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (kVec) {
+    using P4 = typename Pack4<T>::type;
+    const long long nq = p.n >> 2;
+    const float4* x4 = reinterpret_cast<const float4*>(p.x);
+    P4* o4 = reinterpret_cast<P4*>(out);
+    for (long long q = tid; q < nq; q += stride) {
+      const float4 v = __ldcs(x4 + q);
+      P4 c;
+      c.x = static_cast<T>(quantize_one<kStochastic>(v.x, two_fl, wl, p.seed, p.layer_id, 4 * q + 0));
+      c.y = static_cast<T>(quantize_one<kStochastic>(v.y, two_fl, wl, p.seed, p.layer_id, 4 * q + 1));
+      c.z = static_cast<T>(quantize_one<kStochastic>(v.z, two_fl, wl, p.seed, p.layer_id, 4 * q + 2));
+      c.w = static_cast<T>(quantize_one<kStochastic>(v.w, two_fl, wl, p.seed, p.layer_id, 4 * q + 3));
+      __stcs(o4 + q, c);
+    }
+    for (long long i = (nq << 2) + tid; i < p.n; i += stride)
+      out[i] = static_cast<T>(quantize_one<kStochastic>(p.x[i], two_fl, wl, p.seed, p.layer_id, i));
+  } else {
+    for (long long i = tid; i < p.n; i += stride)
+      out[i] = static_cast<T>(quantize_one<kStochastic>(__ldcs(p.x + i), two_fl, wl, p.seed,
+                                                        p.layer_id, i));
+  }
+}
+
+}  // namespace adapt

@@ -1,0 +1,105 @@
+// K1: per-layer range scan (min, max, non-finite / out-of-range flags) over all
+// layers in one launch, and the small finalisation kernel that turns the
+// result into the bin origin and scale shared by all histograms of the layer
+// (Sec. 3.3: binning at resolution r on the float tensor's own range).
+#pragma once
+
+#include "common.cuh"
+
+namespace adapt {
+
+constexpr int kTile = 4096;          // elements per tile (in aligned indexing)
+constexpr int kRangeThreads = 256;
+
+constexpr unsigned kFlagDegenerate = 2u;
+constexpr unsigned kFlagNonfinite = 4u;
+constexpr unsigned kFlagRange = 8u;
+
+__global__ void __launch_bounds__(kRangeThreads)
+range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long n_tiles,
+                  LayerState* __restrict__ state) {
+  // contiguous slice of the global tile list for this CTA
+  const long long per = (n_tiles + gridDim.x - 1) / gridDim.x;
+  long long t = per * blockIdx.x;
+  const long long t_end = min(n_tiles, t + per);
+  if (t >= t_end) return;
+
+  __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
+  int l = layer_of_tile(layers, n_layers, t);
+
+  while (t < t_end) {
+    const LayerDesc L = layers[l];
+    const long long layer_tiles_end = min(t_end, layers[l + 1].tile_begin);
+    const float* base = L.ptr - L.mis;
+    const long long jbeg = L.mis, jend = L.mis + L.n;
+
+    float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
+    unsigned flags = 0;
+    for (; t < layer_tiles_end; ++t) {
+      const long long j_tile = (t - L.tile_begin) * kTile;
+#pragma unroll
+      for (int q = 0; q < kTile / 4 / kRangeThreads; ++q) {
+        const long long j0 = j_tile + 4ll * (q * kRangeThreads + threadIdx.x);
+        if (j0 >= jend) continue;
+        float v[4];
+        unsigned m = load_quad(base, j0, jbeg, jend, v);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (m & (1u << k)) {
+            float a = fabsf(v[k]);
+            // NaN fails both compares; Inf is caught by the first
+            if (!(a <= 3.402823466e38f)) flags |= kFlagNonfinite;
+            else if (a >= 18446744073709551616.0f) flags |= kFlagRange;
+            vmin = fminf(vmin, v[k]);
+            vmax = fmaxf(vmax, v[k]);
+          }
+        }
+      }
+    }
+    // -0.0 and +0.0 are the same value: canonicalise before taking keys
+    unsigned kmin = float_key(__fadd_rn(vmin, 0.0f));
+    unsigned kmax = float_key(__fadd_rn(vmax, 0.0f));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+      flags |= __shfl_xor_sync(0xffffffffu, flags, o);
+    }
+    const int w = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int i = 1; i < kRangeThreads / 32; ++i) {
+        kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
+      }
+      atomicMin(&state[l].min_key, kmin);
+      atomicMax(&state[l].max_key, kmax);
+      if (flags) atomicOr(&state[l].flags, flags);
+    }
+    __syncthreads();
+    ++l;
+    while (l < n_layers && layers[l + 1].tile_begin <= t) ++l;  // skip empty layers
+  }
+}
+
+// One thread per layer: decode min/max, derive the bin scale and flags.
+__global__ void range_finalize_kernel(const LayerDesc* __restrict__ layers, int n_layers,
+                                      int n_bins, LayerState* __restrict__ state,
+                                      float* __restrict__ range_out) {
+  int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_layers) return;
+  LayerState s = state[l];
+  float lo = 0.0f, hi = 0.0f;
+  if (layers[l].n > 0 && !(s.flags & kFlagNonfinite)) {
+    lo = key_float(s.min_key);
+    hi = key_float(s.max_key);
+  }
+  float w = __fsub_rn(hi, lo);
+  float scale = (w == 0.0f) ? 0.0f : __fdiv_rn(static_cast<float>(n_bins), w);
+  if (layers[l].n == 0 || hi == lo) s.flags |= kFlagDegenerate;
+  s.lo = lo; s.hi = hi; s.scale = scale; s.bmax = static_cast<float>(n_bins - 1);
+  state[l] = s;
+  if (range_out) { range_out[2 * l] = lo; range_out[2 * l + 1] = hi; }
+}
+
+}  // namespace adapt

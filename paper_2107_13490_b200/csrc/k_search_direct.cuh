@@ -1,0 +1,136 @@
+// K2 (direct form): fused multi-candidate quantize + zero count + privatised
+// shared-memory histograms, every fraction length evaluated explicitly.
+//
+// For one FL the rounded value round(x * 2^FL) is the same for every WL of the
+// grid - WL only clamps - and the bin function is monotone, so a candidate's
+// histogram is the unsaturated per-FL histogram with both tails folded into
+// the bins of the two saturation values.  This kernel therefore builds, per
+// layer, one unsaturated histogram U[FL] and one zero count Z[FL] for each
+// distinct FL of the grid plus the float histogram Q; the fold happens in the
+// divergence kernel.  (Quantize / EDF steps of Algorithm 3; Sec. 3.2, 3.3.)
+//
+// Handles both rounding modes.  When (distinct FLs + 1) * n_bins counters do
+// not fit in shared memory the FL list is cut into groups (blockIdx.y), each
+// group re-reading the tensor.
+#pragma once
+
+#include "common.cuh"
+#include "k_range.cuh"
+
+namespace adapt {
+
+constexpr int kSearchThreads = 256;
+
+struct SearchParams {
+  const LayerDesc* layers;
+  const LayerState* state;
+  const int* fl_list;          // distinct fraction lengths, ascending
+  int n_layers;
+  int n_fl;                    // number of distinct FLs
+  int fl_per_group;            // FLs handled by one blockIdx.y
+  int n_bins;
+  long long n_tiles;
+  unsigned* q_hist;            // [n_layers][n_bins]
+  unsigned* u_hist;            // [n_layers][n_fl][n_bins]
+  unsigned long long* zeros;   // [n_layers][n_fl]
+  unsigned long long seed;
+};
+
+template <bool kStochastic>
+__global__ void __launch_bounds__(kSearchThreads)
+search_direct_kernel(const SearchParams p) {
+  extern __shared__ unsigned s_hist[];  // [(fl_per_group + 1)][n_bins]
+  __shared__ float s_two[kMaxFl], s_inv[kMaxFl];
+  __shared__ unsigned s_zero[kMaxFl];
+
+  const int B = p.n_bins;
+  const int f0 = blockIdx.y * p.fl_per_group;
+  const int nf = min(p.fl_per_group, p.n_fl - f0);
+  const bool do_q = (blockIdx.y == 0);
+  const int lane = threadIdx.x & 31;
+
+  const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
+  long long t = per * blockIdx.x;
+  const long long t_end = min(p.n_tiles, t + per);
+  if (t >= t_end) return;
+
+  for (int i = threadIdx.x; i < (nf + 1) * B; i += blockDim.x) s_hist[i] = 0;
+  if (threadIdx.x < kMaxFl) {
+    s_zero[threadIdx.x] = 0;
+    if (threadIdx.x < nf) {
+      int fl = p.fl_list[f0 + threadIdx.x];
+      s_two[threadIdx.x] = pow2f(fl);
+      s_inv[threadIdx.x] = pow2f(-fl);
+    }
+  }
+  __syncthreads();
+
+  int l = layer_of_tile(p.layers, p.n_layers, t);
+  while (t < t_end) {
+    const LayerDesc L = p.layers[l];
+    const LayerState S = p.state[l];
+    const long long layer_tiles_end = min(t_end, p.layers[l + 1].tile_begin);
+    const float* base = L.ptr - L.mis;
+    const long long jbeg = L.mis, jend = L.mis + L.n;
+    const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
+
+    for (; t < layer_tiles_end; ++t) {
+      if (!layer_ok) continue;
+      const long long j_tile = (t - L.tile_begin) * kTile;
+      for (int q = 0; q < kTile / 4 / kSearchThreads; ++q) {
+        const long long j0 = j_tile + 4ll * (q * kSearchThreads + threadIdx.x);
+        float v[4];
+        unsigned m = 0;
+        if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
+        else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const bool valid = (m >> k) & 1u;
+          const float x = v[k];
+          if (valid && do_q) atomicAdd(&s_hist[bin_of(x, S.lo, S.scale, S.bmax)], 1u);
+          float pr = 0.0f;
+          if (kStochastic) {
+            unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
+                                static_cast<unsigned long long>(j0 + k - jbeg));
+            pr = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+          }
+          for (int f = 0; f < nf; ++f) {
+            float r = round_scaled<kStochastic>(x, s_two[f], pr);
+            float xq = __fmul_rn(r, s_inv[f]);
+            int b = bin_of(xq, S.lo, S.scale, S.bmax);
+            if (valid) atomicAdd(&s_hist[(f + 1) * B + b], 1u);
+            unsigned zm = __ballot_sync(0xffffffffu, valid && r == 0.0f);
+            if (lane == 0 && zm) atomicAdd(&s_zero[f], __popc(zm));
+          }
+        }
+      }
+    }
+    __syncthreads();
+    // flush this layer's private counts and clear them for the next layer
+    if (layer_ok) {
+      for (int i = threadIdx.x; i < (nf + 1) * B; i += blockDim.x) {
+        unsigned c = s_hist[i];
+        if (c) {
+          int slot = i / B, b = i - slot * B;
+          if (slot == 0) {
+            if (do_q) atomicAdd(&p.q_hist[static_cast<size_t>(l) * B + b], c);
+          } else {
+            atomicAdd(&p.u_hist[(static_cast<size_t>(l) * p.n_fl + f0 + slot - 1) * B + b], c);
+          }
+          s_hist[i] = 0;
+        }
+      }
+      if (threadIdx.x < nf) {
+        unsigned c = s_zero[threadIdx.x];
+        if (c) atomicAdd(&p.zeros[static_cast<size_t>(l) * p.n_fl + f0 + threadIdx.x],
+                         static_cast<unsigned long long>(c));
+        s_zero[threadIdx.x] = 0;
+      }
+    }
+    __syncthreads();
+    ++l;
+    while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
+  }
+}
+
+}  // namespace adapt

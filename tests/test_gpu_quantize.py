@@ -1,0 +1,101 @@
+"""GPU parity of the stand-alone Quantize kernel against the CPU oracle (bit-exact codes)."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2107_13490_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2107_13490_b200 import binding
+    binding.lib()
+    return binding
+
+
+def _specials():
+    return np.float32([0.0, -0.0, 0.5, -0.5, 1.5, 2.5, -2.5, 0.3, 1e-45, -1e-45, 2 ** -32, 3e9, -3e9,
+                       2 ** 31, -2 ** 31, 2 ** 30, 16777217.0, 8388607.5, -8388608.5, 0.49999997,
+                       127.5, -128.5, 32767.5, 1e30, -1e30, 2.0 ** 63, 0.9375])
+
+
+def test_single4k_every_candidate_both_modes(B):
+    import torch
+    w = W.WORKLOADS["single4k"]
+    x = np.concatenate([W.generate(w)[0], _specials()])
+    xd = torch.from_numpy(x).cuda()
+    wl, fl = w.grid()
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        for a, f in zip(wl.tolist(), fl.tolist()):
+            got = B.adapt_quantize(xd, a, f, mode, seed=7)
+            want, _ = O.quantize(x, a, f, mode, seed=7, layer=0)
+            assert np.array_equal(got.cpu().numpy(), want), (a, f, mode)
+
+
+@pytest.mark.parametrize("bits", [8, 16, 32])
+def test_code_widths_layers_and_alignment(B, bits):
+    import torch
+    rng = np.random.default_rng(bits)
+    dt = {8: np.int8, 16: np.int16, 32: np.int32}[bits]
+    for n in (0, 1, 3, 4, 5, 255, 1024, 4099, 100003):
+        for mis in (0, 1, 3):
+            x = np.concatenate([(rng.standard_normal(n) * 20).astype(np.float32)])
+            buf = torch.zeros(n + 4, dtype=torch.float32, device="cuda")
+            buf[mis:mis + n] = torch.from_numpy(x).cuda()
+            out = torch.full((n + 4,), -1, dtype=getattr(torch, f"int{bits}"), device="cuda")
+            for wl, fl in ((2, 0), (bits, bits // 2), (bits, bits - 1), (min(bits, 7), 3)):
+                for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+                    view = out[mis:mis + n]
+                    B.adapt_quantize_ex(buf[mis:mis + n], wl, fl, mode, seed=5, layer=3,
+                                        code_bits=bits, codes_out=view)
+                    torch.cuda.synchronize()
+                    want, _ = O.quantize(x, wl, fl, mode, seed=5, layer=3)
+                    assert np.array_equal(view.cpu().numpy(), want.astype(dt)), (n, mis, wl, fl, mode)
+                    # nothing is written outside [0, n)
+                    assert (out[:mis] == -1).all() and (out[mis + n:] == -1).all()
+
+
+def test_quantize_large_multi_wave(B):
+    import torch
+    w = W.scaled(W.WORKLOADS["stress_1g"], (1 << 24) + 3)
+    x = W.generate(w)[0]
+    xd = torch.from_numpy(x).cuda()
+    for wl, fl, mode in ((8, 4, O.ROUND_RNE), (16, 10, O.ROUND_STOCHASTIC), (32, 20, O.ROUND_RNE)):
+        got = B.adapt_quantize_ex(xd, wl, fl, mode, seed=3, layer=0, code_bits=32)
+        want, _ = O.quantize(x, wl, fl, mode, seed=3, layer=0)
+        assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_quantize_at_device_resident_selection(B):
+    import torch
+    rng = np.random.default_rng(1)
+    x = (rng.standard_normal(50001) * 0.4).astype(np.float32)
+    xd = torch.from_numpy(x).cuda()
+    wl, fl = W.candidate_grid(range(2, 17))
+    res = B.adapt_precision_search_ex([xd], B.Grid(wl, fl), 100)
+    got = B.adapt_quantize_selected(xd, res.best[0], O.ROUND_RNE)
+    torch.cuda.synchronize()
+    ora = O.precision_search_layer(x, wl, fl, 100)
+    want, _ = O.quantize(x, int(ora["best"][0]), int(ora["best"][1]))
+    assert np.array_equal(got.cpu().numpy(), want)
+
+
+def test_quantize_argument_errors_and_host_form(B):
+    import torch
+    x = torch.zeros(16, dtype=torch.float32, device="cuda")
+    for wl, fl, bits in ((1, 0, 32), (33, 0, 32), (8, 8, 32), (9, 0, 8), (17, 3, 16), (8, 4, 12)):
+        with pytest.raises(B.AdaptError) as e:
+            B.adapt_quantize_ex(x, wl, fl, code_bits=bits)
+        assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.AdaptError):
+        B.adapt_quantize_ex(x, 8, 4, round_mode=5)
+    rng = np.random.default_rng(4)
+    h = (rng.standard_normal(70001) * 3).astype(np.float32)
+    got = B.adapt_quantize_host(torch.from_numpy(h), 8, 3, O.ROUND_STOCHASTIC, seed=2, layer=1,
+                                code_bits=8)
+    want, _ = O.quantize(h, 8, 3, O.ROUND_STOCHASTIC, seed=2, layer=1)
+    assert np.array_equal(got.numpy(), want.astype(np.int8))

@@ -1,0 +1,206 @@
+"""GPU parity of the precision-switch search against the CPU oracle, through the
+C ABI: zero counts, histograms and the chosen <WL,FL> bit-exact, divergences to
+1e-5 relative (exactly where the oracle gives 0 or inf)."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2107_13490_b200 import workloads as W
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    assert torch.cuda.is_available()
+    from paper_2107_13490_b200 import binding
+    binding.lib()  # fails loudly when the CUDA library has not been built
+    return binding
+
+
+def test_single4k_all_candidates(B):
+    w = W.WORKLOADS["single4k"]
+    wl, fl = w.grid()
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, where="single4k")
+    # the named call (RNE, eps 0, bits) gives the same answer
+    import torch
+    dev = G.to_device(W.generate(w))
+    r = B.adapt_precision_search(dev, B.Grid(wl, fl), w.n_bins)
+    torch.cuda.synchronize()
+    ora = O.precision_search(W.generate(w), wl, fl, w.n_bins)
+    G.compare_search(r, ora, 1, "single4k named call")
+
+
+def test_resnet20_weights_grads_stochastic(B):
+    w = W.WORKLOADS["resnet20_weights_grads"]
+    wl, fl = w.grid()
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, round_mode=w.round_mode, seed=w.seed,
+                      where="resnet20")
+
+
+def test_alexnet_weights_full_grid(B):
+    w = W.WORKLOADS["alexnet_weights"]
+    wl, fl = w.grid()
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, where="alexnet")
+
+
+def test_resnet18_weights_acts_full_grid(B):
+    w = W.WORKLOADS["resnet18_weights_acts"]
+    wl, fl = w.grid()
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, where="resnet18")
+
+
+def test_stress_scaled_full_grid(B):
+    # same distribution, grid and bins as the 2^30 stress case, several hundred tiles, ragged tail
+    w = W.scaled(W.WORKLOADS["stress_1g"], (1 << 22) + 4099)
+    wl, fl = w.grid()
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, where="stress scaled")
+    G.run_and_compare(B, W.generate(w), wl, fl, w.n_bins, round_mode=O.ROUND_STOCHASTIC, seed=3,
+                      where="stress scaled SR")
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 31, 32, 33, 127, 1023, 1024, 1025, 4093, 4095, 4096,
+                               4097, 8191, 8193, 12289])
+def test_ragged_sizes_and_misaligned_pointers(B, n):
+    import torch
+    rng = np.random.default_rng(n)
+    wl, fl = W.candidate_grid([2, 3, 7, 12, 20, 32])
+    grid = B.Grid(wl, fl)
+    for mis in range(4):
+        buf = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+        x = (rng.standard_normal(n) * 0.3).astype(np.float32)
+        buf[mis:mis + n] = torch.from_numpy(x).cuda()
+        view = buf[mis:mis + n]
+        for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+            res = B.adapt_precision_search_ex([view], grid, 37, round_mode=mode, seed=11,
+                                              layer_base=2, want_hist=True, want_range=True)
+            torch.cuda.synchronize()
+            ora = O.precision_search([x], wl, fl, 37, mode, 11, 2, want_hist=True)
+            G.compare_search(res, ora, 1, f"n={n} mis={mis} mode={mode}", True, True)
+
+
+def test_many_layers_with_empty_and_degenerate_ones(B):
+    rng = np.random.default_rng(77)
+    xs = [np.zeros(0, np.float32),
+          (rng.standard_normal(5000) * 0.1).astype(np.float32),
+          np.full(300, 0.37, np.float32),                     # max == min
+          np.zeros(0, np.float32),
+          (-np.abs(rng.standard_normal(4096))).astype(np.float32),   # negative only
+          np.float32([1e-40, -1e-41, 3e-39, 0.0]),            # subnormals
+          np.float32([5.0]),
+          (rng.standard_normal(9000) * 1e4).astype(np.float32),      # saturates most formats
+          np.zeros(100, np.float32),
+          np.zeros(0, np.float32)]
+    wl, fl = W.candidate_grid(range(2, 33))
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        res, ora = G.run_and_compare(B, xs, wl, fl, 50, round_mode=mode, seed=5,
+                                     where=f"mixed layers mode={mode}")
+        best = res.best.cpu().numpy()
+        for l in (0, 2, 3, 6, 8, 9):
+            assert best[l][3] & B.FLAG_DEGENERATE
+        assert not (best[1][3] & B.FLAG_DEGENERATE)
+
+
+def test_options_eps_pseudocount_base_and_grid_order(B):
+    rng = np.random.default_rng(3)
+    xs = [(rng.laplace(0, 0.02, 20000)).astype(np.float32),
+          (rng.standard_normal(7777) * 0.5).astype(np.float32)]
+    wl, fl = W.candidate_grid([4, 6, 8, 10, 16])
+    perm = rng.permutation(wl.size)
+    wl_p = np.concatenate([wl[perm], wl[:5]])       # shuffled, with duplicates
+    fl_p = np.concatenate([fl[perm], fl[:5]])
+    G.run_and_compare(B, xs, wl_p, fl_p, 150, eps=1e-3, where="eps")
+    G.run_and_compare(B, xs, wl_p, fl_p, 150, pseudo_count=0.5, where="pseudo-count")
+    G.run_and_compare(B, xs, wl_p, fl_p, 150, log_base=float(np.e), where="nats")
+    G.run_and_compare(B, xs, wl_p, fl_p, 1, where="one bin")
+    G.run_and_compare(B, xs, [8], [4], 64, where="single candidate")
+    G.run_and_compare(B, xs, wl_p, fl_p, 16384, where="max bins")
+
+
+def test_on_grid_tensor_is_lossless(B):
+    rng = np.random.default_rng(40)
+    x = (rng.integers(-128, 128, 50000) * 2.0 ** -4).astype(np.float32)
+    wl, fl = W.candidate_grid(range(2, 17))
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        res, _ = G.run_and_compare(B, [x], wl, fl, 150, round_mode=mode, seed=9, where="on grid")
+        kld = res.kld.cpu().numpy()[0]
+        ok = (fl >= 4) & (wl - fl >= 4)
+        assert (kld[ok] == 0.0).all()
+        assert tuple(res.best.cpu().numpy()[0][:2]) <= (8, 4)
+
+
+def test_nonfinite_and_out_of_range_layers_are_flagged(B):
+    import torch
+    rng = np.random.default_rng(2)
+    good = (rng.standard_normal(6000)).astype(np.float32)
+    bad_nan = good.copy(); bad_nan[4097] = np.nan
+    bad_inf = good.copy(); bad_inf[17] = -np.inf
+    bad_big = good.copy(); bad_big[5000] = 3e19            # |x| >= 2^64
+    wl, fl = W.candidate_grid([4, 8])
+    grid = B.Grid(wl, fl)
+    dev = G.to_device([good, bad_nan, bad_inf, bad_big, good])
+    res = B.adapt_precision_search_ex(dev, grid, 64, want_hist=True)
+    torch.cuda.synchronize()
+    flags = res.best.cpu().numpy()[:, 3]
+    assert not flags[0] & (B.FLAG_NONFINITE | B.FLAG_RANGE)
+    assert flags[1] & B.FLAG_NONFINITE and flags[2] & B.FLAG_NONFINITE
+    assert flags[3] & B.FLAG_RANGE
+    ora = O.precision_search([good], wl, fl, 64, want_hist=True)
+    for l in (0, 4):   # the clean layers are unaffected by their neighbours
+        assert np.array_equal(res.zeros.cpu().numpy()[l], ora[0]["zeros"])
+        G.assert_kld_close(res.kld.cpu().numpy()[l], ora[0]["kld"])
+    assert O.value_range(bad_nan)[2] == 1 and O.value_range(bad_inf)[2] == 1
+    # the host-buffer form returns the data error as its status
+    with pytest.raises(B.AdaptError) as e:
+        B.adapt_precision_search_host([torch.from_numpy(bad_nan)], grid, 64)
+    assert e.value.status == B.ERR_NONFINITE
+    with pytest.raises(B.AdaptError) as e:
+        B.adapt_precision_search_host([torch.from_numpy(bad_big)], grid, 64)
+    assert e.value.status == B.ERR_RANGE
+
+
+def test_caller_workspace_and_argument_errors(B):
+    import torch
+    rng = np.random.default_rng(8)
+    x = (rng.standard_normal(10000) * 0.2).astype(np.float32)
+    wl, fl = W.candidate_grid([3, 9])
+    grid = B.Grid(wl, fl)
+    dev = G.to_device([x])
+    need = B.adapt_search_workspace_bytes([x.size], grid, 100)
+    assert need > 0
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    res = B.adapt_precision_search_ex(dev, grid, 100, workspace=ws, want_hist=True, want_range=True)
+    torch.cuda.synchronize()
+    G.compare_search(res, O.precision_search([x], wl, fl, 100, want_hist=True), 1, "workspace",
+                     True, True)
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.AdaptError) as e:
+        B.adapt_precision_search_ex(dev, grid, 100, workspace=small)
+    assert e.value.status == B.ERR_WORKSPACE
+    for bad_bins in (0, -3, 16385):
+        with pytest.raises(B.AdaptError) as e:
+            B.adapt_precision_search_ex(dev, grid, bad_bins)
+        assert e.value.status == B.ERR_INVALID_ARG
+    for bw, bf in (([1], [0]), ([33], [0]), ([8], [8]), ([8], [-1])):
+        with pytest.raises(B.AdaptError) as e:
+            B.adapt_precision_search_ex(dev, B.Grid(bw, bf), 10)
+        assert e.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.AdaptError):
+        B.adapt_precision_search_ex(dev, grid, 10, round_mode=7)
+    with pytest.raises(B.AdaptError):
+        B.adapt_precision_search_ex(dev, grid, 10, eps=-1.0)
+    assert B.adapt_search_workspace_bytes([-1], grid, 10) == 0
+
+
+def test_host_buffer_form_matches(B):
+    import torch
+    w = W.WORKLOADS["resnet20_weights_grads"]
+    xs = W.generate(w)[:6] + W.generate(w)[20:24]
+    wl, fl = w.grid()
+    host = [torch.from_numpy(x).pin_memory() for x in xs]
+    res = B.adapt_precision_search_host(host, B.Grid(wl, fl), w.n_bins, round_mode=w.round_mode,
+                                        seed=w.seed)
+    ora = O.precision_search(xs, wl, fl, w.n_bins, w.round_mode, w.seed, threads=G.host_threads())
+    G.compare_search(res, ora, len(xs), "host form")
