@@ -1,0 +1,355 @@
+#!/usr/bin/env python
+"""Benchmark of the precision-switch search on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+One step = one pass of the whole path over the workload: the batched search
+(range scan, fused multi-candidate quantize / zero count / histograms,
+divergence, selection) followed by the re-quantisation of every layer at its
+selected <WL,FL>.  Prints one JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "precision-search element-candidates/s"
+UNIT = "element-candidates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the search kernel from an ncu capture (bytes per element per launch),
+# valid only for the library version it was taken on; see profiles/.
+TRAFFIC_CAPTURE = {"version": None, "bytes_per_element": None}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="stress_1g")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-sample", type=int, default=1 << 21,
+                    help="elements of the workload the CPU baseline is timed on")
+    ap.add_argument("--elements", type=int, default=0,
+                    help="profiling aid: shrink a single-layer workload to this many elements")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def oracle_step(O, xs, wl, fl, w, eps=0.0):
+    """One pass of the path on the CPU oracle: search, then quantize at the selection."""
+    res = O.precision_search(xs, wl, fl, w.n_bins, w.round_mode, w.seed, 0, eps, threads=1)
+    for l, x in enumerate(xs):
+        if x.size:
+            O.quantize(x, int(res[l]["best"][0]), int(res[l]["best"][1]), w.round_mode, w.seed, l)
+    return res
+
+
+def cpu_sample(xs, n_sample):
+    """A bounded prefix sample of the workload: whole layers until the budget is used."""
+    out, left = [], n_sample
+    for x in xs:
+        if left <= 0:
+            break
+        out.append(x[:left])
+        left -= out[-1].size
+    return out
+
+
+def time_oracle(xs, wl, fl, w, n_sample):
+    from oracle import oracle as O
+    sample = cpu_sample(xs, n_sample)
+    units = sum(s.size for s in sample) * len(wl)
+    t0 = time.perf_counter()
+    oracle_step(O, sample, wl, fl, w)
+    dt = time.perf_counter() - t0
+    return {"value": units / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"first {sum(s.size for s in sample)} elements ({len(sample)} layer(s)) of "
+                      f"{w.name}, all {len(wl)} candidates, {w.n_bins} bins, one pass in {dt:.1f} s"}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on the machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import oracle as O
+    from paper_2107_13490_b200 import workloads as W
+    w = W.WORKLOADS[args.workload]
+    wl, fl = w.grid()
+    n_sample = min(w.numel, 1 << 18)
+    first = w.layers[0]
+    if first.numel > n_sample:   # generate only what the sample needs
+        xs = [W.generate_layer(W.LayerSpec(first.name, (n_sample,), first.dist, first.scale,
+                                           first.zero_frac, first.outlier_frac, first.outlier_gain),
+                               w.seed, 0)]
+    else:
+        xs = cpu_sample(W.generate(w), n_sample)
+    units = sum(x.size for x in xs) * len(wl)
+    for _ in range(args.warmup):
+        oracle_step(O, xs, wl, fl, w)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(O, xs, wl, fl, w)
+    dt = time.perf_counter() - t0
+    value = units * args.steps / dt
+    sample = f"first {sum(x.size for x in xs)} elements of {w.name} per step, all {len(wl)} candidates"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "elements": w.numel, "candidates": len(wl),
+                       "n_bins": w.n_bins, "round_mode": "rne" if w.round_mode == 0 else "stochastic",
+                       "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2107_13490_b200 import binding as B
+    from paper_2107_13490_b200 import sharding as S
+    from paper_2107_13490_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    rank, local_rank, world = S.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+
+    base = W.WORKLOADS[args.workload]
+    if args.elements:
+        base = W.scaled(base, args.elements)
+    w = S.rank_workload(base, rank)
+    wl, fl = w.grid()
+    grid = B.Grid(wl, fl)
+    n_cand = len(grid)
+
+    xs_np = W.generate(w)
+    pinned = [torch.from_numpy(x).pin_memory() for x in xs_np]
+    xs = [p.to(dev, non_blocking=True) for p in pinned]
+    codes = [torch.empty(x.numel(), dtype=torch.int32, device=dev) for x in xs]
+    lens = [x.numel() for x in xs]
+    total = sum(lens)
+    ws = torch.empty(B.adapt_search_workspace_bytes(lens, grid, w.n_bins), dtype=torch.uint8, device=dev)
+    out = B.SearchResult(torch.empty((len(xs), n_cand), dtype=torch.float64, device=dev),
+                         torch.empty((len(xs), n_cand), dtype=torch.int64, device=dev),
+                         torch.empty((len(xs), 4), dtype=torch.int32, device=dev))
+    torch.cuda.synchronize()
+
+    def step():
+        B.adapt_precision_search_ex(xs, grid, w.n_bins, round_mode=w.round_mode, seed=w.seed,
+                                    workspace=ws, out=out)
+        for l, x in enumerate(xs):
+            if lens[l]:
+                B.adapt_quantize_selected(x, out.best[l], w.round_mode, w.seed, l, codes_out=codes[l])
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+
+    # ---- device-resident timing -------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    S.barrier()
+    torch.cuda.synchronize()
+    B.adapt_kernel_times(reset=True)
+    B.adapt_kernel_timing(True)
+    launches0 = B.adapt_kernel_launch_count()
+    sampler.start()
+    fits_l2 = 4 * total <= 2 * 126e6
+    if not fits_l2:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        secs = e0.elapsed_time(e1) * 1e-3
+    else:
+        # inputs could stay in L2 from one step to the next: flush it between steps,
+        # outside the per-step events
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(args.steps)]
+        for a, b in evs:
+            flush.zero_()
+            a.record()
+            step()
+            b.record()
+        torch.cuda.synchronize()
+        secs = sum(a.elapsed_time(b) for a, b in evs) * 1e-3
+        del flush
+    S.barrier()
+    clocks = sampler.stop()
+    launches = B.adapt_kernel_launch_count() - launches0
+    B.adapt_kernel_timing(False)
+    ktimes = B.adapt_kernel_times(reset=True)
+    units = float(total) * n_cand * args.steps
+    value, secs_max = S.job_throughput(units, secs, dev)
+
+    # ---- roofline of the dominant kernel (the fused search kernel) ----------------
+    peak, peak_kind = measured_peak_gbs()
+    ms_search, n_search = ktimes["search"]
+    algo_bytes = 4.0 * total     # one fp32 read of every element per launch
+    achieved = algo_bytes / (ms_search / n_search * 1e-3) / 1e9 if n_search else None
+    traffic = None
+    if TRAFFIC_CAPTURE["version"] == B.adapt_version() and TRAFFIC_CAPTURE["bytes_per_element"]:
+        traffic = TRAFFIC_CAPTURE["bytes_per_element"] * total
+    roofline = {"bound": "hbm", "kernel": "search (fused quantize/zero-count/histograms)",
+                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                "algorithmic_bytes_per_launch": algo_bytes,
+                "avg_launch_ms": ms_search / n_search if n_search else None}
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
+               for k, v in ktimes.items() if v[1]}
+
+    # ---- end to end through the host-buffer entry points ---------------------------
+    e2e = None
+    if not args.no_e2e:
+        host_out = B.SearchResult(torch.empty((len(xs), n_cand), dtype=torch.float64).pin_memory(),
+                                  torch.empty((len(xs), n_cand), dtype=torch.int64).pin_memory(),
+                                  torch.empty((len(xs), 4), dtype=torch.int32).pin_memory())
+        host_codes = [torch.empty(n, dtype=torch.int32).pin_memory() for n in lens]
+
+        def e2e_step():
+            B.adapt_precision_search_host(pinned, grid, w.n_bins, round_mode=w.round_mode,
+                                          seed=w.seed, out=host_out)
+            best = host_out.best.numpy()
+            for l, p in enumerate(pinned):
+                if lens[l]:
+                    B.adapt_quantize_host(p, int(best[l][0]), int(best[l][1]), w.round_mode, w.seed,
+                                          l, 32, codes_out=host_codes[l])
+
+        e2e_step()
+        S.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        S.barrier()
+        e2e_value, _ = S.job_throughput(float(total) * n_cand * args.e2e_steps, dt, dev)
+        res_bytes = len(xs) * (n_cand * 16 + 16)
+        e2e = {"value": e2e_value, "unit": UNIT, "steps": args.e2e_steps,
+               "ms_per_step": dt / args.e2e_steps * 1e3,
+               "h2d_bytes_per_step": 8 * total, "d2h_bytes_per_step": res_bytes + 4 * total,
+               "api": "adapt_precision_search_host + adapt_quantize_host (pinned host buffers)"}
+        del host_codes
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = time_oracle(xs_np, wl, fl, w, args.cpu_sample)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(args.warmup, 3),
+                "ms_per_step": secs_max / args.steps * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": base.name, "description": base.description,
+                           "elements_per_gpu": total, "layers": len(xs), "candidates": n_cand,
+                           "n_bins": w.n_bins,
+                           "round_mode": "rne" if w.round_mode == 0 else "stochastic",
+                           "step": "adapt_precision_search_ex + adapt_quantize_selected per layer",
+                           "l2": "inputs exceed L2" if not fits_l2 else
+                                 "L2 flushed (512 MiB write) between timed steps",
+                           "parallelism": f"independent layer sets x{world}, no collective"},
+                "hbm_gbs_whole_step": (8.0 * total + 8.0 * total) * args.steps / secs_max / 1e9 * world,
+                "roofline": roofline, "kernels": kernels, "e2e": e2e,
+                "cpu_baseline": cpu_baseline, "gpu_launches": int(launches), "clocks": clocks,
+                "library": B.adapt_version()}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

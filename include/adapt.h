@@ -22,7 +22,7 @@
  *  - Formats: 2 <= WL <= 32, 0 <= FL <= WL-1 (Sec. 2.1: a WL-bit signed word
  *    with FL fractional bits; value = code * 2^-FL, code in
  *    [-2^(WL-1), 2^(WL-1)-1]).  Values outside the range saturate.
- *  - Limits: fewer than 2^32 elements per layer; 1 <= n_bins <= 65536;
+ *  - Limits: fewer than 2^32 elements per layer; 1 <= n_bins <= 16384;
  *    1 <= n_cand <= 65535; 1 <= n_layers <= 65535.
  */
 #ifndef ADAPT_B200_H_
@@ -141,7 +141,9 @@ size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers,
  *   zeros_out DEVICE int64[n_layers][n_cand]    zero codes per candidate
  *   best_out  DEVICE int32[n_layers][4]         {wl, fl, grid index, flags}
  * Scratch comes from a library-owned device buffer that is allocated (and
- * grown) inside the call when needed; use the _ex call to supply your own. */
+ * grown) inside the call when needed and is shared by every call that does
+ * not bring its own: such calls must not overlap on the device (issue them on
+ * one stream).  Use the _ex call to supply your own workspace. */
 int adapt_precision_search(const float* const* tensors, const int64_t* lens,
                            int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
                            double* kld_out, int64_t* zeros_out, int32_t* best_out);
@@ -173,6 +175,27 @@ int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mod
 /* Number of kernels the library has launched since it was loaded (all
  * devices, all entry points). */
 uint64_t adapt_kernel_launch_count(void);
+
+/* Kernel kinds for the timing calls below. */
+enum {
+  ADAPT_KERNEL_RANGE = 0,          /* range scan                               */
+  ADAPT_KERNEL_RANGE_FINALIZE = 1, /* per-layer bin origin / scale             */
+  ADAPT_KERNEL_SEARCH = 2,         /* fused quantize / zero count / histograms */
+  ADAPT_KERNEL_KLD = 3,            /* divergence per (layer, candidate)        */
+  ADAPT_KERNEL_SELECT = 4,         /* lowest <WL,FL> per layer                 */
+  ADAPT_KERNEL_QUANTIZE = 5,       /* stand-alone quantize                     */
+  ADAPT_KERNEL_KINDS = 6
+};
+
+/* Switches per-kernel device timing on (non-zero) or off.  While on, every
+ * launch is bracketed by two CUDA events on the stream it is launched on. */
+int adapt_kernel_timing(int enable);
+
+/* Waits for the timed launches recorded so far and returns, per kernel kind,
+ * the accumulated device time in milliseconds and the number of launches.
+ *   ms_out, launches_out  HOST arrays of ADAPT_KERNEL_KINDS entries (or NULL)
+ *   reset                 non-zero clears the accumulators after reading */
+int adapt_kernel_times(double* ms_out, uint64_t* launches_out, int reset);
 
 /* Frees every library-owned device and pinned buffer of the current device's
  * caches.  Safe to call at any time no library work is in flight. */

@@ -26,8 +26,10 @@ EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_search_workspace_bytes",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
-    "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_release",
+    "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
+    "adapt_kernel_times", "adapt_release",
 )
+KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize")
 
 
 class AdaptGrid(C.Structure):
@@ -90,6 +92,10 @@ def lib():
                                           C.c_uint64, C.c_int32, C.c_int, C.c_void_p]
         L.adapt_kernel_launch_count.restype = C.c_uint64
         L.adapt_release.restype = C.c_int
+        L.adapt_kernel_timing.restype = C.c_int
+        L.adapt_kernel_timing.argtypes = [C.c_int]
+        L.adapt_kernel_times.restype = C.c_int
+        L.adapt_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
         _lib = L
     return _lib
 
@@ -128,6 +134,19 @@ def adapt_version() -> str:
 
 def adapt_kernel_launch_count() -> int:
     return int(lib().adapt_kernel_launch_count())
+
+
+def adapt_kernel_timing(enable: bool) -> None:
+    _check(lib().adapt_kernel_timing(1 if enable else 0), "adapt_kernel_timing")
+
+
+def adapt_kernel_times(reset: bool = False):
+    """Returns {kind: (milliseconds, launches)} accumulated while timing was on."""
+    ms = np.zeros(len(KERNEL_KINDS), dtype=np.float64)
+    cnt = np.zeros(len(KERNEL_KINDS), dtype=np.uint64)
+    _check(lib().adapt_kernel_times(ms.ctypes.data, cnt.ctypes.data, 1 if reset else 0),
+           "adapt_kernel_times")
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
 
 
 def adapt_release() -> None:

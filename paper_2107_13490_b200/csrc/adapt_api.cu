@@ -26,6 +26,42 @@ std::mutex g_mutex;                     // serialises calls that touch library-o
 std::atomic<uint64_t> g_launches{0};
 char g_last_error[512] = "";
 
+// Optional per-kernel device timing: events around each launch, on its stream.
+struct TimedLaunch { int kind; cudaEvent_t start, stop; };
+std::atomic<bool> g_timing{false};
+std::mutex g_timing_mutex;
+std::vector<TimedLaunch> g_pending;
+std::vector<cudaEvent_t> g_event_pool;
+double g_kind_ms[ADAPT_KERNEL_KINDS] = {0};
+uint64_t g_kind_launches[ADAPT_KERNEL_KINDS] = {0};
+
+cudaEvent_t pooled_event() {
+  if (!g_event_pool.empty()) { cudaEvent_t e = g_event_pool.back(); g_event_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  cudaEventCreate(&e);
+  return e;
+}
+
+// Brackets one kernel launch; counts it, and times it when timing is on.
+struct LaunchScope {
+  int kind; cudaStream_t stream; cudaEvent_t start = nullptr;
+  LaunchScope(int k, cudaStream_t s) : kind(k), stream(s) {
+    if (g_timing.load()) {
+      std::lock_guard<std::mutex> l(g_timing_mutex);
+      start = pooled_event();
+      if (start) cudaEventRecord(start, stream);
+    }
+  }
+  ~LaunchScope() {
+    ++g_launches;
+    if (start) {
+      std::lock_guard<std::mutex> l(g_timing_mutex);
+      cudaEvent_t stop = pooled_event();
+      if (stop) { cudaEventRecord(stop, stream); g_pending.push_back({kind, start, stop}); }
+    }
+  }
+};
+
 int cuda_fail(cudaError_t e, const char* what) {
   std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
   return ADAPT_ERR_CUDA;
@@ -265,14 +301,16 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   // K1: range scan
   if (tiles > 0) {
     const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc.sm_count));
+    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
     range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(d_layers, a.n_layers, tiles, d_state);
     ADAPT_CUDA(cudaGetLastError());
-    ++g_launches;
   }
-  range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
-      d_layers, a.n_layers, a.n_bins, d_state, o.range_out);
-  ADAPT_CUDA(cudaGetLastError());
-  ++g_launches;
+  {
+    LaunchScope ls(ADAPT_KERNEL_RANGE_FINALIZE, stream);
+    range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
+        d_layers, a.n_layers, a.n_bins, d_state, o.range_out);
+    ADAPT_CUDA(cudaGetLastError());
+  }
 
   // K2: fused quantize / zero count / histograms
   if (tiles > 0) {
@@ -296,9 +334,9 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
     dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)),
               groups);
+    LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
     kern<<<grid, kSearchThreads, smem, stream>>>(sp);
     ADAPT_CUDA(cudaGetLastError());
-    ++g_launches;
   }
 
   // K3: divergence per (layer, candidate), then selection per layer
@@ -313,17 +351,22 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.alpha = o.pseudo_count; kp.inv_ln_base = 1.0 / std::log(base); kp.eps = o.eps;
   kp.kld_out = a.kld_out; kp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
   kp.best_out = a.best_out; kp.hist_out = o.hist_out;
-  kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(kp);
-  ADAPT_CUDA(cudaGetLastError());
-  ++g_launches;
-  select_kernel<<<a.n_layers, 32, 0, stream>>>(kp);
-  ADAPT_CUDA(cudaGetLastError());
-  ++g_launches;
+  {
+    LaunchScope ls(ADAPT_KERNEL_KLD, stream);
+    kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(kp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_SELECT, stream);
+    select_kernel<<<a.n_layers, 32, 0, stream>>>(kp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
   return ADAPT_OK;
 }
 
 template <typename T>
 int launch_quantize_t(const QuantParams& qp, bool stochastic, bool vec, int grid, cudaStream_t s) {
+  LaunchScope ls(ADAPT_KERNEL_QUANTIZE, s);
   if (stochastic) {
     if (vec) quantize_kernel<T, true, true><<<grid, kQuantThreads, 0, s>>>(qp);
     else quantize_kernel<T, true, false><<<grid, kQuantThreads, 0, s>>>(qp);
@@ -332,7 +375,6 @@ int launch_quantize_t(const QuantParams& qp, bool stochastic, bool vec, int grid
     else quantize_kernel<T, false, false><<<grid, kQuantThreads, 0, s>>>(qp);
   }
   ADAPT_CUDA(cudaGetLastError());
-  ++g_launches;
   return ADAPT_OK;
 }
 
@@ -391,6 +433,31 @@ const char* adapt_status_string(int status) {
 const char* adapt_last_error(void) { return g_last_error; }
 
 uint64_t adapt_kernel_launch_count(void) { return g_launches.load(); }
+
+int adapt_kernel_timing(int enable) {
+  g_timing.store(enable != 0);
+  return ADAPT_OK;
+}
+
+int adapt_kernel_times(double* ms_out, uint64_t* launches_out, int reset) {
+  std::lock_guard<std::mutex> l(g_timing_mutex);
+  for (const TimedLaunch& t : g_pending) {
+    ADAPT_CUDA(cudaEventSynchronize(t.stop));
+    float ms = 0.0f;
+    ADAPT_CUDA(cudaEventElapsedTime(&ms, t.start, t.stop));
+    g_kind_ms[t.kind] += ms;
+    g_kind_launches[t.kind] += 1;
+    g_event_pool.push_back(t.start);
+    g_event_pool.push_back(t.stop);
+  }
+  g_pending.clear();
+  for (int k = 0; k < ADAPT_KERNEL_KINDS; ++k) {
+    if (ms_out) ms_out[k] = g_kind_ms[k];
+    if (launches_out) launches_out[k] = g_kind_launches[k];
+    if (reset) { g_kind_ms[k] = 0.0; g_kind_launches[k] = 0; }
+  }
+  return ADAPT_OK;
+}
 
 int adapt_quantize(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
                    int32_t* codes_out) {
