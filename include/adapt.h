@@ -83,7 +83,15 @@ typedef struct adapt_search_opts {
                              slot 0 = histogram of the float tensor, slot c+1 =
                              histogram of candidate c's dequantized tensor      */
   float* range_out;       /* DEVICE, optional: float[n_layers][2] = {min, max}  */
+  int32_t algorithm;      /* ADAPT_ALGO_*: which form of the fused kernel runs  */
 } adapt_search_opts;
+
+/* Forms of the fused quantize / zero-count / histogram kernel.  Both give the
+ * same results bit for bit.  AUTO: the keyed form for round-to-nearest-even
+ * layers of at least 32768 elements with n_bins <= 8192, the direct form for
+ * the rest.  KEYED: the keyed form for every layer it can serve (RNE,
+ * n_bins <= 8192).  DIRECT: the direct form everywhere. */
+enum { ADAPT_ALGO_AUTO = 0, ADAPT_ALGO_KEYED = 1, ADAPT_ALGO_DIRECT = 2 };
 
 /* Library version string, e.g. "adapt-b200 0.1". Never NULL. */
 const char* adapt_version(void);
@@ -180,11 +188,16 @@ uint64_t adapt_kernel_launch_count(void);
 enum {
   ADAPT_KERNEL_RANGE = 0,          /* range scan                               */
   ADAPT_KERNEL_RANGE_FINALIZE = 1, /* per-layer bin origin / scale             */
-  ADAPT_KERNEL_SEARCH = 2,         /* fused quantize / zero count / histograms */
+  ADAPT_KERNEL_SEARCH = 2,         /* fused quantize / zero count / histograms,
+                                      keyed form (one pass, one atomic/element) */
   ADAPT_KERNEL_KLD = 3,            /* divergence per (layer, candidate)        */
   ADAPT_KERNEL_SELECT = 4,         /* lowest <WL,FL> per layer                 */
   ADAPT_KERNEL_QUANTIZE = 5,       /* stand-alone quantize                     */
-  ADAPT_KERNEL_KINDS = 6
+  ADAPT_KERNEL_PLAN = 6,           /* per-layer cell plan of the keyed form    */
+  ADAPT_KERNEL_EXPAND = 7,         /* cell counts -> per-level histograms      */
+  ADAPT_KERNEL_SEARCH_DIRECT = 8,  /* fused kernel, direct form (every FL
+                                      evaluated per element)                   */
+  ADAPT_KERNEL_KINDS = 9
 };
 
 /* Switches per-kernel device timing on (non-zero) or off.  While on, every

@@ -29,7 +29,9 @@ EXPORTS = (
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_release",
 )
-KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize")
+KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize", "plan",
+                "expand", "search_direct")
+ALGO_AUTO, ALGO_KEYED, ALGO_DIRECT = 0, 1, 2
 
 
 class AdaptGrid(C.Structure):
@@ -40,7 +42,7 @@ class AdaptSearchOpts(C.Structure):
     _fields_ = [("round_mode", C.c_int32), ("layer_base", C.c_int32), ("seed", C.c_uint64),
                 ("eps", C.c_double), ("pseudo_count", C.c_double), ("log_base", C.c_double),
                 ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("hist_out", C.c_void_p), ("range_out", C.c_void_p)]
+                ("hist_out", C.c_void_p), ("range_out", C.c_void_p), ("algorithm", C.c_int32)]
 
 
 class AdaptError(RuntimeError):
@@ -238,7 +240,8 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
                               eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
                               stream=None, workspace: Optional[torch.Tensor] = None,
                               want_hist: bool = False, want_range: bool = False,
-                              out: Optional[SearchResult] = None) -> SearchResult:
+                              out: Optional[SearchResult] = None,
+                              algorithm: int = ALGO_AUTO) -> SearchResult:
     dev = tensors[0].device
     assert all(t.is_cuda for t in tensors)
     ptrs, lens = _marshal_tensors(tensors)
@@ -258,6 +261,7 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
         o.workspace, o.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     o.hist_out = out.hist.data_ptr() if out.hist is not None else None
     o.range_out = out.range.data_ptr() if out.range is not None else None
+    o.algorithm = algorithm
     _check(lib().adapt_precision_search_ex(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
                                            n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
                                            out.best.data_ptr(), C.byref(o)),

@@ -13,10 +13,13 @@
 
 #include "../../include/adapt.h"
 #include "common.cuh"
+#include "k_expand.cuh"
 #include "k_kld_select.cuh"
+#include "k_plan.cuh"
 #include "k_quantize.cuh"
 #include "k_range.cuh"
 #include "k_search_direct.cuh"
+#include "k_search_keyed.cuh"
 
 namespace {
 
@@ -141,18 +144,27 @@ int acquire_slot(DeviceCache& c, size_t bytes, PinnedSlot** out) {
 
 // ---- search plan ----------------------------------------------------------------
 
+constexpr int kMaxBins = 16384;
+constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
+constexpr int kKeyedMaxBins = 8192;
+constexpr size_t kKeyedSmemBudget = 110 * 1024; // two CTAs per SM
+
 struct Plan {
-  int n_layers = 0, n_cand = 0, n_fl = 0, n_bins = 0;
-  long long n_tiles = 0;
-  std::vector<int> fl_list, slot, order;
-  // byte offsets inside the workspace
-  size_t off_layers = 0, off_wl = 0, off_fl = 0, off_slot = 0, off_order = 0, off_fl_list = 0,
-         off_state = 0, blob_bytes = 0;
-  size_t off_zeros = 0, off_q = 0, off_u = 0, accum_bytes = 0;
+  int n_layers = 0, n_cand = 0, n_levels = 0, n_bins = 0;
+  std::vector<int> slot, order;
+  // keyed-kernel shared-memory shape
+  int cell_cap = 0, d_levels = 0;
+  size_t keyed_smem = 0;
+  // byte offsets inside the workspace -- descriptor block (uploaded)
+  size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
+         off_order = 0, off_state = 0, blob_bytes = 0;
+  // written by kernels, not cleared
+  size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
+  // accumulators (cleared every call)
+  size_t off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0, off_stable = 0,
+         off_zclass = 0, off_nzero = 0, accum_begin = 0, accum_bytes = 0;
   size_t total = 0;
 };
-
-constexpr int kMaxBins = 16384;
 
 bool valid_format(int wl, int fl) { return wl >= 2 && wl <= 32 && fl >= 0 && fl < wl; }
 
@@ -162,25 +174,17 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   if (n_layers < 1 || n_layers > 65535) return false;
   if (grid->n_cand < 1 || grid->n_cand > 65535) return false;
   if (n_bins < 1 || n_bins > kMaxBins) return false;
-  for (int c = 0; c < grid->n_cand; ++c)
+  int fmax = 0;
+  for (int c = 0; c < grid->n_cand; ++c) {
     if (!valid_format(grid->wl[c], grid->fl[c])) return false;
-  long long tiles = 0;
-  for (int l = 0; l < n_layers; ++l) {
-    if (lens[l] < 0 || lens[l] >= (1ll << 32)) return false;
-    tiles += (lens[l] + 3 + kTile - 1) / kTile;  // upper bound, misalignment included
+    fmax = std::max(fmax, grid->fl[c]);
   }
-  (void)tiles;
+  for (int l = 0; l < n_layers; ++l)
+    if (lens[l] < 0 || lens[l] >= (1ll << 32)) return false;
   p->n_layers = n_layers; p->n_cand = grid->n_cand; p->n_bins = n_bins;
+  p->n_levels = fmax + 1;   // fraction lengths 0..fmax get a histogram each
 
-  bool seen[kMaxFl] = {false};
-  for (int c = 0; c < grid->n_cand; ++c) seen[grid->fl[c]] = true;
-  int slot_of[kMaxFl];
-  p->fl_list.clear();
-  for (int f = 0; f < kMaxFl; ++f)
-    if (seen[f]) { slot_of[f] = static_cast<int>(p->fl_list.size()); p->fl_list.push_back(f); }
-  p->n_fl = static_cast<int>(p->fl_list.size());
-  p->slot.resize(grid->n_cand);
-  for (int c = 0; c < grid->n_cand; ++c) p->slot[c] = slot_of[grid->fl[c]];
+  p->slot.assign(grid->fl, grid->fl + grid->n_cand);
   p->order.resize(grid->n_cand);
   std::iota(p->order.begin(), p->order.end(), 0);
   std::stable_sort(p->order.begin(), p->order.end(), [&](int a, int b) {
@@ -188,20 +192,43 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
     return grid->fl[a] < grid->fl[b];
   });
 
-  const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_fl;
+  // shared-memory shape of the keyed kernel: queue + Qe + a few correction levels + cells
+  const size_t hist = sizeof(unsigned) * n_bins;
+  const size_t queue = keyed_smem_bytes(0, 0, 0);
+  p->d_levels = static_cast<int>(std::min<size_t>(6, (32 * 1024) / hist));
+  p->d_levels = std::min(p->d_levels, p->n_levels);
+  if (n_bins <= kKeyedMaxBins) {
+    p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (1 + p->d_levels)) / 4);
+    p->cell_cap = std::min(p->cell_cap, 1 << 15);
+  } else {
+    p->cell_cap = 0;
+  }
+  p->keyed_smem = keyed_smem_bytes(p->cell_cap, n_bins, p->d_levels);
+
+  const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_levels, K = p->cell_cap;
   size_t o = 0;
   p->off_layers = o;  o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
+  p->off_keyed = o;   o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
+  p->off_direct = o;  o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
   p->off_wl = o;      o = align_up(o + sizeof(int) * C, 16);
   p->off_fl = o;      o = align_up(o + sizeof(int) * C, 16);
   p->off_slot = o;    o = align_up(o + sizeof(int) * C, 16);
   p->off_order = o;   o = align_up(o + sizeof(int) * C, 16);
-  p->off_fl_list = o; o = align_up(o + sizeof(int) * F, 16);
   p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
   p->blob_bytes = o;
+  p->off_plan = o;      o = align_up(o + sizeof(LayerPlan) * L, 256);
+  p->off_edges = o;     o = align_up(o + sizeof(float) * L * (B + 1), 256);
+  p->off_cell_init = o; o = align_up(o + sizeof(unsigned) * L * K, 256);
+  p->accum_begin = o;
   p->off_zeros = o;   o = align_up(o + sizeof(unsigned long long) * L * F, 256);
+  p->off_zclass = o;  o = align_up(o + sizeof(unsigned long long) * L * kZeroClasses, 256);
+  p->off_nzero = o;   o = align_up(o + sizeof(unsigned long long) * L, 256);
   p->off_q = o;       o = align_up(o + sizeof(unsigned) * L * B, 256);
+  p->off_qe = o;      o = align_up(o + sizeof(unsigned) * L * B, 256);
+  p->off_stable = o;  o = align_up(o + sizeof(unsigned) * L * B, 256);
+  p->off_cells = o;   o = align_up(o + sizeof(unsigned) * L * K, 256);
   p->off_u = o;       o = align_up(o + sizeof(unsigned) * L * F * B, 256);
-  p->accum_bytes = o - p->off_zeros;
+  p->accum_bytes = o - p->accum_begin;
   p->total = o;
   return true;
 }
@@ -228,6 +255,27 @@ adapt_search_opts default_opts() {
   adapt_search_opts o;
   std::memset(&o, 0, sizeof(o));
   return o;
+}
+
+// Fills a layer list (descriptors + sentinel) from the chosen layers; returns its tile count.
+long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchArgs& a) {
+  long long tiles = 0;
+  size_t k = 0;
+  for (int l : pick) {
+    const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(a.tensors[l]) >> 2) & 3u);
+    LayerDesc& d = out[k++];
+    d.ptr = a.tensors[l];
+    d.n = a.lens[l];
+    d.tile_begin = tiles;
+    d.mis = a.lens[l] > 0 ? mis : 0;
+    d.layer_id = a.opts.layer_base + l;
+    d.index = l;
+    d.pad_ = 0;
+    if (a.lens[l] > 0) tiles += (a.lens[l] + mis + kTile - 1) / kTile;
+  }
+  LayerDesc& s = out[k];
+  s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.pad_ = 0;
+  return tiles;
 }
 
 // Enqueues the whole search on opts.stream.  Caller holds g_mutex.
@@ -259,46 +307,57 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   }
   cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
 
+  // which kernel serves which layer
+  const bool keyed_possible = o.round_mode == ADAPT_ROUND_RNE && plan.cell_cap >= 1024 &&
+                              plan.keyed_smem + 2048 <= static_cast<size_t>(dc.max_smem_optin) &&
+                              (o.algorithm == ADAPT_ALGO_AUTO || o.algorithm == ADAPT_ALGO_KEYED);
+  if (o.algorithm != ADAPT_ALGO_AUTO && o.algorithm != ADAPT_ALGO_KEYED &&
+      o.algorithm != ADAPT_ALGO_DIRECT) return ADAPT_ERR_INVALID_ARG;
+  const long long keyed_min = (o.algorithm == ADAPT_ALGO_KEYED) ? 1 : kKeyedMinElements;
+  std::vector<int> all(a.n_layers), keyed, direct;
+  std::iota(all.begin(), all.end(), 0);
+  for (int l = 0; l < a.n_layers; ++l) {
+    if (keyed_possible && a.lens[l] >= keyed_min) keyed.push_back(l);
+    else direct.push_back(l);
+  }
+
   // host image of the descriptor block
   PinnedSlot* slot = nullptr;
   int rc = acquire_slot(dc, plan.blob_bytes, &slot);
   if (rc != ADAPT_OK) return rc;
   char* h = static_cast<char*>(slot->host);
   std::memset(h, 0, plan.blob_bytes);
-  LayerDesc* hl = reinterpret_cast<LayerDesc*>(h + plan.off_layers);
-  long long tiles = 0;
-  for (int l = 0; l < a.n_layers; ++l) {
-    const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(a.tensors[l]) >> 2) & 3u);
-    hl[l].ptr = a.tensors[l];
-    hl[l].n = a.lens[l];
-    hl[l].tile_begin = tiles;
-    hl[l].mis = a.lens[l] > 0 ? mis : 0;
-    hl[l].layer_id = o.layer_base + l;
-    if (a.lens[l] > 0) tiles += (a.lens[l] + mis + kTile - 1) / kTile;
-  }
-  hl[a.n_layers].ptr = nullptr;
-  hl[a.n_layers].n = 0;
-  hl[a.n_layers].tile_begin = tiles;
-  plan.n_tiles = tiles;
+  const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, a);
+  const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a);
+  const long long direct_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_direct), direct, a);
   std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_order, plan.order.data(), sizeof(int) * plan.n_cand);
-  std::memcpy(h + plan.off_fl_list, plan.fl_list.data(), sizeof(int) * plan.n_fl);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
   for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
-  ADAPT_CUDA(cudaMemsetAsync(ws + plan.off_zeros, 0, plan.accum_bytes, stream));
+  ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
 
   const LayerDesc* d_layers = reinterpret_cast<const LayerDesc*>(ws + plan.off_layers);
+  const LayerDesc* d_keyed = reinterpret_cast<const LayerDesc*>(ws + plan.off_keyed);
+  const LayerDesc* d_direct = reinterpret_cast<const LayerDesc*>(ws + plan.off_direct);
   LayerState* d_state = reinterpret_cast<LayerState*>(ws + plan.off_state);
+  LayerPlan* d_plan = reinterpret_cast<LayerPlan*>(ws + plan.off_plan);
+  float* d_edges = reinterpret_cast<float*>(ws + plan.off_edges);
+  unsigned* d_cell_init = reinterpret_cast<unsigned*>(ws + plan.off_cell_init);
   unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + plan.off_zeros);
+  unsigned long long* d_zclass = reinterpret_cast<unsigned long long*>(ws + plan.off_zclass);
+  unsigned long long* d_nzero = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
   unsigned* d_q = reinterpret_cast<unsigned*>(ws + plan.off_q);
+  unsigned* d_qe = reinterpret_cast<unsigned*>(ws + plan.off_qe);
+  unsigned* d_stable = reinterpret_cast<unsigned*>(ws + plan.off_stable);
+  unsigned* d_cells = reinterpret_cast<unsigned*>(ws + plan.off_cells);
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + plan.off_u);
 
-  // K1: range scan
+  // K1: range scan over every layer, then bin origin / scale per layer
   if (tiles > 0) {
     const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc.sm_count));
     LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
@@ -312,19 +371,62 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ADAPT_CUDA(cudaGetLastError());
   }
 
-  // K2: fused quantize / zero count / histograms
-  if (tiles > 0) {
+  // K2, keyed form: plan -> cell counting -> expansion
+  if (!keyed.empty() && keyed_tiles > 0) {
+    const int nk = static_cast<int>(keyed.size());
+    PlanParams pp;
+    pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
+    pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = a.n_bins; pp.cell_cap = plan.cell_cap;
+    {
+      LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
+      plan_kernel<<<nk, kPlanThreads, 0, stream>>>(pp);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+    KeyedParams kp;
+    kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
+    kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
+    kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
+    kp.n_zero = d_nzero; kp.n_bins = a.n_bins; kp.n_levels = plan.n_levels;
+    kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
+    ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(plan.keyed_smem)));
+    {
+      const int grid = static_cast<int>(std::min<long long>(keyed_tiles, 2ll * dc.sm_count));
+      LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
+      search_keyed_kernel<<<grid, kKeyedThreads, plan.keyed_smem, stream>>>(kp);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+    ExpandParams ep;
+    ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
+    ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
+    ep.stable_hist = d_stable; ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros;
+    ep.zero_class = d_zclass; ep.n_zero = d_nzero; ep.n_bins = a.n_bins;
+    ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
+    {
+      LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
+      expand_cells_kernel<<<dim3((plan.cell_cap + 255) / 256, nk), 256, 0, stream>>>(ep);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+    {
+      LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
+      combine_kernel<<<dim3((a.n_bins + 255) / 256, plan.n_levels + 1, nk), 256, 0, stream>>>(ep);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+  }
+
+  // K2, direct form: stochastic rounding, small layers, very large bin counts
+  if (!direct.empty() && direct_tiles > 0) {
     SearchParams sp;
-    sp.layers = d_layers; sp.state = d_state;
-    sp.fl_list = reinterpret_cast<const int*>(ws + plan.off_fl_list);
-    sp.n_layers = a.n_layers; sp.n_fl = plan.n_fl; sp.n_bins = a.n_bins; sp.n_tiles = tiles;
+    sp.layers = d_direct; sp.state = d_state;
+    sp.n_layers = static_cast<int>(direct.size()); sp.n_fl = plan.n_levels; sp.n_bins = a.n_bins;
+    sp.n_tiles = direct_tiles;
     sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed;
     const size_t per_hist = sizeof(unsigned) * a.n_bins;
     const size_t budget = 100 * 1024;
     int fg = static_cast<int>(budget / per_hist) - 1;
-    fg = std::max(1, std::min(fg, plan.n_fl));
+    fg = std::max(1, std::min(fg, plan.n_levels));
     sp.fl_per_group = fg;
-    const int groups = (plan.n_fl + fg - 1) / fg;
+    const int groups = (plan.n_levels + fg - 1) / fg;
     const size_t smem = per_hist * (fg + 1);
     if (smem + 1024 > static_cast<size_t>(dc.max_smem_optin)) return ADAPT_ERR_INVALID_ARG;
     auto kern = (o.round_mode == ADAPT_ROUND_STOCHASTIC) ? search_direct_kernel<true>
@@ -332,9 +434,9 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ADAPT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(smem)));
     const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
-    dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)),
+    dim3 grid(static_cast<unsigned>(std::min<long long>(direct_tiles, 1ll * ctas_per_sm * dc.sm_count)),
               groups);
-    LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
+    LaunchScope ls(ADAPT_KERNEL_SEARCH_DIRECT, stream);
     kern<<<grid, kSearchThreads, smem, stream>>>(sp);
     ADAPT_CUDA(cudaGetLastError());
   }
@@ -346,7 +448,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.cand_fl = reinterpret_cast<const int*>(ws + plan.off_fl);
   kp.cand_slot = reinterpret_cast<const int*>(ws + plan.off_slot);
   kp.cand_order = reinterpret_cast<const int*>(ws + plan.off_order);
-  kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_fl; kp.n_bins = a.n_bins;
+  kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_levels; kp.n_bins = a.n_bins;
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = o.pseudo_count; kp.inv_ln_base = 1.0 / std::log(base); kp.eps = o.eps;
   kp.kld_out = a.kld_out; kp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);

@@ -20,6 +20,8 @@ struct LayerDesc {
   long long tile_begin;  // index of the layer's first tile in the global tile list
   int mis;               // elements between the 16-byte boundary below ptr and ptr (0..3)
   int layer_id;          // hash layer id
+  int index;             // position in the caller's tensor list (addresses state and outputs)
+  int pad_;
 };
 
 // Per-layer state produced on the device by the range scan.

@@ -72,9 +72,9 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
       for (int i = 1; i < kRangeThreads / 32; ++i) {
         kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
       }
-      atomicMin(&state[l].min_key, kmin);
-      atomicMax(&state[l].max_key, kmax);
-      if (flags) atomicOr(&state[l].flags, flags);
+      atomicMin(&state[L.index].min_key, kmin);
+      atomicMax(&state[L.index].max_key, kmax);
+      if (flags) atomicOr(&state[L.index].flags, flags);
     }
     __syncthreads();
     ++l;

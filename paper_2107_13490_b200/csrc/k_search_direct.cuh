@@ -6,10 +6,11 @@
 // histogram is the unsaturated per-FL histogram with both tails folded into
 // the bins of the two saturation values.  This kernel therefore builds, per
 // layer, one unsaturated histogram U[FL] and one zero count Z[FL] for each
-// distinct FL of the grid plus the float histogram Q; the fold happens in the
-// divergence kernel.  (Quantize / EDF steps of Algorithm 3; Sec. 3.2, 3.3.)
+// FL from 0 to the grid's largest, plus the float histogram Q; the fold happens
+// in the divergence kernel.  (Quantize / EDF steps of Algorithm 3; Sec. 3.2, 3.3.)
 //
-// Handles both rounding modes.  When (distinct FLs + 1) * n_bins counters do
+// Handles both rounding modes; it serves stochastic rounding, small layers and
+// very large bin counts, the keyed kernel the rest.  When (FLs + 1) * n_bins counters do
 // not fit in shared memory the FL list is cut into groups (blockIdx.y), each
 // group re-reading the tensor.
 #pragma once
@@ -24,9 +25,8 @@ constexpr int kSearchThreads = 256;
 struct SearchParams {
   const LayerDesc* layers;
   const LayerState* state;
-  const int* fl_list;          // distinct fraction lengths, ascending
   int n_layers;
-  int n_fl;                    // number of distinct FLs
+  int n_fl;                    // fraction lengths 0..n_fl-1 are evaluated
   int fl_per_group;            // FLs handled by one blockIdx.y
   int n_bins;
   long long n_tiles;
@@ -58,7 +58,7 @@ search_direct_kernel(const SearchParams p) {
   if (threadIdx.x < kMaxFl) {
     s_zero[threadIdx.x] = 0;
     if (threadIdx.x < nf) {
-      int fl = p.fl_list[f0 + threadIdx.x];
+      int fl = f0 + threadIdx.x;
       s_two[threadIdx.x] = pow2f(fl);
       s_inv[threadIdx.x] = pow2f(-fl);
     }
@@ -68,7 +68,8 @@ search_direct_kernel(const SearchParams p) {
   int l = layer_of_tile(p.layers, p.n_layers, t);
   while (t < t_end) {
     const LayerDesc L = p.layers[l];
-    const LayerState S = p.state[l];
+    const int gl = L.index;
+    const LayerState S = p.state[gl];
     const long long layer_tiles_end = min(t_end, p.layers[l + 1].tile_begin);
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
@@ -113,16 +114,16 @@ search_direct_kernel(const SearchParams p) {
         if (c) {
           int slot = i / B, b = i - slot * B;
           if (slot == 0) {
-            if (do_q) atomicAdd(&p.q_hist[static_cast<size_t>(l) * B + b], c);
+            if (do_q) atomicAdd(&p.q_hist[static_cast<size_t>(gl) * B + b], c);
           } else {
-            atomicAdd(&p.u_hist[(static_cast<size_t>(l) * p.n_fl + f0 + slot - 1) * B + b], c);
+            atomicAdd(&p.u_hist[(static_cast<size_t>(gl) * p.n_fl + f0 + slot - 1) * B + b], c);
           }
           s_hist[i] = 0;
         }
       }
       if (threadIdx.x < nf) {
         unsigned c = s_zero[threadIdx.x];
-        if (c) atomicAdd(&p.zeros[static_cast<size_t>(l) * p.n_fl + f0 + threadIdx.x],
+        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_fl + f0 + threadIdx.x],
                          static_cast<unsigned long long>(c));
         s_zero[threadIdx.x] = 0;
       }

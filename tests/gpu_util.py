@@ -54,18 +54,27 @@ def compare_search(res, oracle_results, n_layers, where="", check_hist=False, ch
             assert rng[l][0] == o["range"][0] and rng[l][1] == o["range"][1], f"{tag}: range"
 
 
+ALGORITHMS = (0, 1, 2)   # auto, keyed wherever it can serve, direct everywhere
+
+
 def run_and_compare(B, tensors_np, wl, fl, n_bins, round_mode=0, seed=0, layer_base=0, eps=0.0,
-                    pseudo_count=0.0, log_base=0.0, check_hist=True, threads=None, where=""):
-    """B = the binding module. Returns (gpu result, oracle results)."""
+                    pseudo_count=0.0, log_base=0.0, check_hist=True, threads=None, where="",
+                    algorithms=ALGORITHMS):
+    """B = the binding module.  Runs the library once per kernel form and compares each
+    run with one oracle run.  Returns (last gpu result, oracle results)."""
     import torch
     grid = B.Grid(wl, fl)
     dev = to_device(tensors_np)
-    res = B.adapt_precision_search_ex(dev, grid, n_bins, round_mode=round_mode, seed=seed,
-                                      layer_base=layer_base, eps=eps, pseudo_count=pseudo_count,
-                                      log_base=log_base, want_hist=check_hist, want_range=True)
-    torch.cuda.synchronize()
     ora = O.precision_search(tensors_np, wl, fl, n_bins, round_mode, seed, layer_base, eps,
                              pseudo_count, 2.0 if log_base == 0.0 else log_base,
                              want_hist=check_hist, threads=threads or host_threads())
-    compare_search(res, ora, len(tensors_np), where, check_hist=check_hist, check_range=True)
+    res = None
+    for algo in algorithms:
+        res = B.adapt_precision_search_ex(dev, grid, n_bins, round_mode=round_mode, seed=seed,
+                                          layer_base=layer_base, eps=eps,
+                                          pseudo_count=pseudo_count, log_base=log_base,
+                                          want_hist=check_hist, want_range=True, algorithm=algo)
+        torch.cuda.synchronize()
+        compare_search(res, ora, len(tensors_np), f"{where} [algorithm {algo}]",
+                       check_hist=check_hist, check_range=True)
     return res, ora

@@ -74,11 +74,13 @@ def test_ragged_sizes_and_misaligned_pointers(B, n):
         buf[mis:mis + n] = torch.from_numpy(x).cuda()
         view = buf[mis:mis + n]
         for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
-            res = B.adapt_precision_search_ex([view], grid, 37, round_mode=mode, seed=11,
-                                              layer_base=2, want_hist=True, want_range=True)
-            torch.cuda.synchronize()
             ora = O.precision_search([x], wl, fl, 37, mode, 11, 2, want_hist=True)
-            G.compare_search(res, ora, 1, f"n={n} mis={mis} mode={mode}", True, True)
+            for algo in G.ALGORITHMS:
+                res = B.adapt_precision_search_ex([view], grid, 37, round_mode=mode, seed=11,
+                                                  layer_base=2, want_hist=True, want_range=True,
+                                                  algorithm=algo)
+                torch.cuda.synchronize()
+                G.compare_search(res, ora, 1, f"n={n} mis={mis} mode={mode} algo={algo}", True, True)
 
 
 def test_many_layers_with_empty_and_degenerate_ones(B):
@@ -117,6 +119,44 @@ def test_options_eps_pseudocount_base_and_grid_order(B):
     G.run_and_compare(B, xs, wl_p, fl_p, 1, where="one bin")
     G.run_and_compare(B, xs, [8], [4], 64, where="single candidate")
     G.run_and_compare(B, xs, wl_p, fl_p, 16384, where="max bins")
+
+
+def test_adversarial_value_patterns(B):
+    """Inputs built to sit on the places where the keyed kernel's shortcuts could
+    go wrong: bin edges, cell boundaries, rounding ties, powers of two around zero,
+    subnormals, ranges far from zero, very wide and very narrow ranges."""
+    rng = np.random.default_rng(123)
+    n = 40000
+    cases = {}
+    base = (rng.standard_normal(n) * 0.25).astype(np.float32)
+    # values on and next to the exact bin edges of a 100-bin histogram of `base`
+    lo, hi = base.min(), base.max()
+    edges = (lo + (hi - lo) * np.arange(1, 100, dtype=np.float32) / np.float32(100)).astype(np.float32)
+    near = np.concatenate([edges, np.nextafter(edges, np.float32(np.inf)),
+                           np.nextafter(edges, np.float32(-np.inf))])
+    cases["bin_edges"] = np.concatenate([base, np.tile(near, 20)]).astype(np.float32)
+    # multiples of 2^-k: every element is a tie at some coarser level
+    cases["ties"] = (rng.integers(-4000, 4000, n) * 2.0 ** -9 + 2.0 ** -10).astype(np.float32)
+    cases["on_grid_mixed"] = np.where(rng.random(n) < 0.5, np.round(base * 1024) / 1024, base).astype(np.float32)
+    # powers of two and their neighbours around zero (zero-count ties), subnormals, exact zeros
+    p2 = np.float32(2.0) ** np.arange(-40, 2, dtype=np.float32)
+    p2 = np.concatenate([p2, -p2, np.nextafter(p2, np.float32(0)), np.nextafter(p2, np.float32(4)),
+                         np.float32([0.0, -0.0, 1e-45, -1e-45, 1e-39])])
+    cases["pow2_near_zero"] = np.concatenate([np.tile(p2, 100), base[:5000] * np.float32(1e-3)]).astype(np.float32)
+    cases["half_zero"] = np.maximum(rng.standard_normal(n), 0).astype(np.float32)
+    cases["far_from_zero"] = (1000.0 + rng.random(n) * 0.01).astype(np.float32)
+    cases["far_negative"] = (-123456.0 - rng.random(n) * 64).astype(np.float32)
+    cases["wide"] = (rng.standard_normal(n) * 1e6).astype(np.float32)
+    cases["very_wide"] = (rng.standard_normal(n) * 1e15).astype(np.float32)
+    cases["tiny"] = (rng.standard_normal(n) * 1e-9).astype(np.float32)
+    cases["narrow_offset"] = (0.75 + rng.integers(0, 50, n) * 2.0 ** -24).astype(np.float32)
+    cases["two_values"] = np.where(rng.random(n) < 0.3, 0.1, -0.7).astype(np.float32)
+    cases["integers"] = rng.integers(-300, 300, n).astype(np.float32)
+    wl, fl = W.candidate_grid(range(2, 33))
+    for name, x in cases.items():
+        for n_bins in (100, 2048):
+            G.run_and_compare(B, [x], wl, fl, n_bins, where=f"{name} B={n_bins}",
+                              algorithms=(1, 2))
 
 
 def test_on_grid_tensor_is_lossless(B):
