@@ -147,7 +147,7 @@ int acquire_slot(DeviceCache& c, size_t bytes, PinnedSlot** out) {
 constexpr int kMaxBins = 16384;
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
 constexpr int kKeyedMaxBins = 8192;
-constexpr size_t kKeyedSmemBudget = 110 * 1024; // two CTAs per SM
+constexpr size_t kKeyedSmemBudget = 224 * 1024; // one CTA per SM owns its shared memory
 
 struct Plan {
   int n_layers = 0, n_cand = 0, n_levels = 0, n_bins = 0;
@@ -199,7 +199,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->d_levels = std::min(p->d_levels, p->n_levels);
   if (n_bins <= kKeyedMaxBins) {
     p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (1 + p->d_levels)) / 4);
-    p->cell_cap = std::min(p->cell_cap, 1 << 15);
+    p->cell_cap = std::min(p->cell_cap, 1 << 16);
   } else {
     p->cell_cap = 0;
   }
@@ -258,7 +258,8 @@ adapt_search_opts default_opts() {
 }
 
 // Fills a layer list (descriptors + sentinel) from the chosen layers; returns its tile count.
-long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchArgs& a) {
+long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchArgs& a,
+                    int tile) {
   long long tiles = 0;
   size_t k = 0;
   for (int l : pick) {
@@ -271,7 +272,7 @@ long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchAr
     d.layer_id = a.opts.layer_base + l;
     d.index = l;
     d.pad_ = 0;
-    if (a.lens[l] > 0) tiles += (a.lens[l] + mis + kTile - 1) / kTile;
+    if (a.lens[l] > 0) tiles += (a.lens[l] + mis + tile - 1) / tile;
   }
   LayerDesc& s = out[k];
   s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.pad_ = 0;
@@ -327,9 +328,9 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   if (rc != ADAPT_OK) return rc;
   char* h = static_cast<char*>(slot->host);
   std::memset(h, 0, plan.blob_bytes);
-  const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, a);
-  const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a);
-  const long long direct_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_direct), direct, a);
+  const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, a, kTile);
+  const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a, kKeyedTile);
+  const long long direct_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_direct), direct, a, kTile);
   std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
@@ -377,6 +378,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     PlanParams pp;
     pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
     pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = a.n_bins; pp.cell_cap = plan.cell_cap;
+    pp.cell_target = std::min(plan.cell_cap, std::max(2048, 24 * a.n_bins));
     {
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
       plan_kernel<<<nk, kPlanThreads, 0, stream>>>(pp);
@@ -386,12 +388,12 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
     kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
-    kp.n_zero = d_nzero; kp.n_bins = a.n_bins; kp.n_levels = plan.n_levels;
+    kp.n_bins = a.n_bins; kp.n_levels = plan.n_levels;
     kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(plan.keyed_smem)));
     {
-      const int grid = static_cast<int>(std::min<long long>(keyed_tiles, 2ll * dc.sm_count));
+      const int grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
       LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
       search_keyed_kernel<<<grid, kKeyedThreads, plan.keyed_smem, stream>>>(kp);
       ADAPT_CUDA(cudaGetLastError());
@@ -400,7 +402,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
     ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
     ep.stable_hist = d_stable; ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros;
-    ep.zero_class = d_zclass; ep.n_zero = d_nzero; ep.n_bins = a.n_bins;
+    ep.zero_class = d_zclass; ep.cell_total = d_nzero; ep.n_bins = a.n_bins;
     ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
     {
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);

@@ -9,7 +9,8 @@
 // combine_kernel: one thread per (bin, level, layer) adds the base terms to
 // the correction counts already sitting in U: stable + edge-element histogram
 // for fine levels, the exact zeros at the bin of 0, and builds Q and the zero
-// counts of the fine levels from the zero classes.
+// counts of the fine levels from the zero classes.  The exact zeros are the
+// elements no cell counted.
 #pragma once
 
 #include "common.cuh"
@@ -31,7 +32,7 @@ struct ExpandParams {
   unsigned* u_hist;            // [layer][n_levels][n_bins]
   unsigned long long* zeros;   // [layer][n_levels]
   const unsigned long long* zero_class;  // [layer][kZeroClasses]
-  const unsigned long long* n_zero;      // [layer]
+  unsigned long long* cell_total;        // [layer] sum of the cell counts = non-zero elements
   int n_bins, n_levels, cell_cap;
 };
 
@@ -41,8 +42,12 @@ __global__ void __launch_bounds__(256) expand_cells_kernel(const ExpandParams p)
   const LayerPlan P = p.plan[l];
   if (!P.keyed) return;
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= P.cells) return;
-  const unsigned m = p.cell_count[static_cast<size_t>(l) * p.cell_cap + c];
+  const unsigned m = (c < P.cells) ? p.cell_count[static_cast<size_t>(l) * p.cell_cap + c] : 0u;
+  // the layer's non-zero elements = sum of all its cell counts
+  unsigned long long wsum = m;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
+  if ((threadIdx.x & 31) == 0 && wsum) atomicAdd(&p.cell_total[l], wsum);
   if (m == 0) return;
   const LayerState S = p.state[l];
   const int B = p.n_bins;
@@ -75,7 +80,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const ExpandParams p) {
   const int B = p.n_bins;
   if (b >= B) return;
   const LayerState S = p.state[l];
-  const unsigned nz = static_cast<unsigned>(p.n_zero[l]);
+  const unsigned nz = static_cast<unsigned>(static_cast<unsigned long long>(L.n) - p.cell_total[l]);
   const int bz = bin_of(0.0f, S.lo, S.scale, S.bmax);
   const unsigned base = p.stable_hist[static_cast<size_t>(l) * B + b] +
                         p.qe_hist[static_cast<size_t>(l) * B + b];

@@ -48,7 +48,8 @@ struct PlanParams {
   float* edges;              // [all layers][n_bins + 1]
   unsigned* cell_init;       // [all layers][cell_cap]
   int n_bins;
-  int cell_cap;
+  int cell_cap;              // table entries per layer (memory stride)
+  int cell_target;           // most cells a layer may use (<= cell_cap)
 };
 
 __device__ __forceinline__ long long floor_scaled(float v, int g) {
@@ -72,12 +73,12 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     for (; g > -100; --g) {
       // products up to 2^64 * 2^32 overflow long long: skip levels that cannot fit anyway
       double span = ldexp(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
-      if (span >= static_cast<double>(p.cell_cap)) continue;
+      if (span >= static_cast<double>(p.cell_target)) continue;
       if (fabs(ldexp(static_cast<double>(S.hi), g)) > 9.0e18 ||
           fabs(ldexp(static_cast<double>(S.lo), g)) > 9.0e18) continue;
       c0 = floor_scaled(S.lo, g);
       c1 = floor_scaled(S.hi, g);
-      if (c1 - c0 + 1 <= p.cell_cap) break;
+      if (c1 - c0 + 1 <= p.cell_target) break;
     }
     P.g = g; P.c0 = c0; P.cells = static_cast<int>(c1 - c0 + 1);
     P.fs = g > 0 ? g : 0;

@@ -4,20 +4,24 @@
 //
 // Per element x != 0:   c = floor(x * 2^G) - c0;  old = atomicAdd(cell[c], 1)
 // The returned word carries the cell's marks in its two top bits:
-//   bit 30 (cell -1 / 0): add the element to the class counter "highest level
-//          at which it still rounds to zero";
-//   bit 31 (edge cell), or x exactly on the level-G grid: the element is pushed
-//          to a per-warp queue; queues are drained 32 entries at a time by the
-//          whole warp (dense lanes):
+//   bit 30 (cell -1 / 0): the element is added to the class counter "highest
+//          level at which it still rounds to zero";
+//   bit 31 (edge cell), or x exactly on the level-G grid: the element goes to a
+//          per-warp queue that the warp drains 32 entries at a time:
 //            edge entry: b0 = bin(x) into the edge-element histogram Qe, then
 //              only the fine levels f whose half quantum can reach one of the
 //              bin's edges are evaluated; a level is recorded only if its bin
 //              differs from b0 (-1 at b0, +1 at the new bin);
 //            on-grid entry: the one coarse level at which x is a rounding tie
 //              that goes down is corrected (the cell table assumes "up").
-// Exact zeros are only counted (warp ballot).  Everything else about the
-// element - the float histogram, all coarse levels, all fine levels of
-// interior cells - is derived from the cell counts by the expand kernels.
+// Exact zeros touch nothing (their number is the layer size minus the sum of
+// the cell counts).  Everything else about an element - the float histogram,
+// all coarse levels, all fine levels of interior cells - is derived from the
+// cell counts by the expand kernels.
+//
+// One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
+// for its cell table; each thread keeps 16 elements (four 128-bit loads) in
+// flight per tile.
 #pragma once
 
 #include "common.cuh"
@@ -26,13 +30,15 @@
 
 namespace adapt {
 
-constexpr int kKeyedThreads = 512;
+constexpr int kKeyedThreads = 1024;
 constexpr int kKeyedWarps = kKeyedThreads / 32;
-constexpr int kQueueCap = 64;       // per-warp queue entries (drained at >= 32)
-constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..31 (32 = all)
+constexpr int kKeyedQuads = 4;                                  // 128-bit loads per thread per tile
+constexpr int kKeyedTile = kKeyedThreads * kKeyedQuads * 4;     // 16384 elements
+constexpr int kQueueCap = 128;      // per-warp queue entries; a full queue handles entries inline
+constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..32
 
 struct KeyedParams {
-  const LayerDesc* layers;     // keyed layer list (+ sentinel)
+  const LayerDesc* layers;     // keyed layer list (+ sentinel), tiles of kKeyedTile elements
   int n_layers;
   long long n_tiles;
   const LayerState* state;     // by LayerDesc::index
@@ -40,57 +46,56 @@ struct KeyedParams {
   const float* edges;          // [layer][n_bins + 1]
   const unsigned* cell_init;   // [layer][cell_cap]
   unsigned* cell_count;        // [layer][cell_cap]      global cell counts
-  unsigned* qe_hist;           // [layer][n_bins]        float histogram of queue "edge" elements
+  unsigned* qe_hist;           // [layer][n_bins]        float histogram of the edge elements
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
   unsigned long long* zeros;   // [layer][n_levels]      receives tie corrections
   unsigned long long* zero_class;  // [layer][kZeroClasses]
-  unsigned long long* n_zero;  // [layer]                exact zeros
   int n_bins;
   int n_levels;                // levels 0..n_levels-1 are wanted
   int cell_cap;
   int d_levels;                // fine levels whose corrections are kept in shared memory
 };
 
-// shared memory carve-up (dynamic): cells | qe | d | queue_x | queue_tag
-struct KeyedSmem {
-  unsigned* cells;   // [cell_cap]
-  unsigned* qe;      // [n_bins]
-  int* d;            // [d_levels][n_bins]
-  float* qx;         // [warps][kQueueCap]
-  unsigned* qtag;    // [warps][kQueueCap]   bit 31 edge, bit 30 on-grid, low bits cell index
-};
-
 __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int d_levels) {
   return sizeof(unsigned) * (static_cast<size_t>(cell_cap) + n_bins +
                              static_cast<size_t>(d_levels) * n_bins) +
-         (sizeof(float) + sizeof(unsigned)) * kKeyedWarps * kQueueCap;
+         sizeof(float) * kKeyedWarps * kQueueCap;
 }
 
+// Everything the special-element handler needs about the current layer.
 struct LayerCtx {
-  LayerState S;
-  LayerPlan P;
-  const float* E;
-  unsigned* u_hist;            // this layer's [n_levels][n_bins]
-  unsigned long long* zeros;   // this layer's [n_levels]
+  float lo, scale, bmax;       // bin function
+  float two_g, c0f;            // cell function (general form)
+  long long c0;
+  int g, fs;
+  const float* E;              // exact bin edges [n_bins + 1]
+  const unsigned* cells;       // shared cell table (marks in the two top bits)
+  unsigned* qe;                // shared [n_bins]
+  int* d;                      // shared [d_levels][n_bins]
+  unsigned* u_hist;            // global, this layer's [n_levels][n_bins]
+  unsigned long long* zeros;   // global, this layer's [n_levels]
   int n_bins, n_levels, d_levels;
 };
 
-// Processes one queue entry (all 32 lanes call this; `live` masks real entries).
-__device__ __forceinline__ void drain_entry(const LayerCtx& c, const KeyedSmem& sm, bool live,
-                                            float x, unsigned tag) {
+// Handles one queued element (x != 0, finite).  No warp-level primitive inside:
+// any subset of lanes may call it.
+__device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   const int B = c.n_bins;
-  // ---- on-grid entry: fix the single coarse tie level ----------------------
-  if (live && (tag & 0x40000000u)) {
-    const long long cc = c.P.c0 + static_cast<long long>(tag & 0x3FFFFFFFu);
+  const float z = __fmul_rn(x, c.two_g);
+  const float cf = floorf(z);
+  const int idx = __float2int_rz(__fsub_rn(cf, c.c0f));
+  // ---- x on the level-G grid: fix the single coarse level at which it is a tie --
+  if (z == cf) {
+    const long long cc = c.c0 + idx;
     if (cc != 0) {
       const int tz = __ffsll(cc) - 1;          // lowest set bit
-      const int ft = c.P.g - 1 - tz;           // the level at which x is a tie
+      const int ft = c.g - 1 - tz;             // the level at which x is a tie
       if (ft >= 0 && ft < c.n_levels) {
         const long long a = cc >> (tz + 1);    // floor(x * 2^ft)
         if ((a & 1ll) == 0) {                  // tie goes down to a; the table counted a + 1
           const float s = pow2f(-ft);
-          const int b_up = bin_of(__fmul_rn(__ll2float_rn(a + 1), s), c.S.lo, c.S.scale, c.S.bmax);
-          const int b_dn = bin_of(__fmul_rn(__ll2float_rn(a), s), c.S.lo, c.S.scale, c.S.bmax);
+          const int b_up = bin_of(__fmul_rn(__ll2float_rn(a + 1), s), c.lo, c.scale, c.bmax);
+          const int b_dn = bin_of(__fmul_rn(__ll2float_rn(a), s), c.lo, c.scale, c.bmax);
           unsigned* U = c.u_hist + static_cast<size_t>(ft) * B;
           if (b_up != b_dn) { atomicAdd(&U[b_up], 0xFFFFFFFFu); atomicAdd(&U[b_dn], 1u); }
           if (a + 1 == 0) atomicAdd(&c.zeros[ft], 0xFFFFFFFFFFFFFFFFull);
@@ -99,57 +104,138 @@ __device__ __forceinline__ void drain_entry(const LayerCtx& c, const KeyedSmem& 
       }
     }
   }
-  // ---- edge entry: float bin, then the fine levels that can still move ------
-  const bool edge = live && (tag & 0x80000000u);
-  int b0 = 0, f_end = 0;
-  if (edge) {
-    b0 = bin_of(x, c.S.lo, c.S.scale, c.S.bmax);
-    atomicAdd(&sm.qe[b0], 1u);
-    // distance to the bin's two edges, rounded down: safe once 2^-(f+1) < margin
-    const float dl = __fsub_rd(x, __ldg(c.E + b0));
-    const float dh = __fsub_rd(__ldg(c.E + b0 + 1), x);
-    const float m = fminf(dl, dh);
-    int f_safe = 32;
-    if (m > 0.0f) f_safe = 126 - static_cast<int>((__float_as_uint(m) - 1u) >> 23);
-    f_end = min(f_safe, c.n_levels);
-  }
-  for (int f = c.P.fs;; ++f) {
-    const bool act = edge && f < f_end;
-    if (!__any_sync(0xffffffffu, act)) break;
-    if (act) {
-      const float r = rintf(__fmul_rn(x, pow2f(f)));
-      const int b = bin_of(__fmul_rn(r, pow2f(-f)), c.S.lo, c.S.scale, c.S.bmax);
-      if (b != b0) {
-        const int j = f - c.P.fs;
-        if (j < c.d_levels) {
-          atomicAdd(&sm.d[j * B + b], 1);
-          atomicAdd(&sm.d[j * B + b0], -1);
-        } else {
-          unsigned* U = c.u_hist + static_cast<size_t>(f) * B;
-          atomicAdd(&U[b], 1u);
-          atomicAdd(&U[b0], 0xFFFFFFFFu);
-        }
-      }
+  // ---- edge cell: float bin, then the fine levels that can still move ------------
+  if (!(c.cells[idx] & kCellEdge)) return;
+  const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
+  atomicAdd(&c.qe[b0], 1u);
+  const float e_lo = __ldg(c.E + b0), e_hi = __ldg(c.E + b0 + 1);
+  // distance to the bin's two edges, rounded down: a level is safe once 2^-(f+1) < margin
+  const float m = fminf(__fsub_rd(x, e_lo), __fsub_rd(e_hi, x));
+  int f_end = 32;
+  if (m > 0.0f) f_end = 126 - static_cast<int>((__float_as_uint(m) - 1u) >> 23);
+  f_end = min(f_end, c.n_levels);
+  for (int f = c.fs; f < f_end; ++f) {
+    const float r = rintf(__fmul_rn(x, pow2f(f)));
+    const float v = __fmul_rn(r, pow2f(-f));
+    if (v >= e_lo && v < e_hi) continue;       // still in b0 (edges are exact)
+    const int b = bin_of(v, c.lo, c.scale, c.bmax);
+    const int j = f - c.fs;
+    if (j < c.d_levels) {
+      atomicAdd(&c.d[j * B + b], 1);
+      atomicAdd(&c.d[j * B + b0], -1);
+    } else {
+      unsigned* U = c.u_hist + static_cast<size_t>(f) * B;
+      atomicAdd(&U[b], 1u);
+      atomicAdd(&U[b0], 0xFFFFFFFFu);
     }
   }
 }
 
-__global__ void __launch_bounds__(kKeyedThreads, 2) search_keyed_kernel(const KeyedParams p) {
+// Adds a near-zero element (cells -1 / 0) to its zero class.
+__device__ __forceinline__ void count_zero_class(unsigned* s_zclass, float x) {
+  // highest level k at which x still rounds to zero: |x| <= 2^-(k+1)
+  const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
+  int kz = 125 - static_cast<int>((ax - 1u) >> 23);
+  kz = max(-1, min(kz, 32));
+  atomicAdd(&s_zclass[kz + 1], 1u);
+}
+
+// Cell index of x.  Fast form: |cell indices| < 2^22, so adding the magic
+// constant 1.5 * 2^23 - c0 with round-down leaves floor(x * 2^G) - c0 in the
+// low mantissa bits; x is on the grid exactly when round-up gives the same.
+template <bool kFast>
+__device__ __forceinline__ int cell_index(float x, float two_g, float magic, float c0f,
+                                          bool* on_grid) {
+  if (kFast) {
+    const float rd = __fmaf_rd(x, two_g, magic);
+    const float ru = __fmaf_ru(x, two_g, magic);
+    *on_grid = (rd == ru);
+    return __float_as_int(rd) - 0x4B400000;
+  }
+  const float z = __fmul_rn(x, two_g);
+  const float cf = floorf(z);
+  *on_grid = (z == cf);
+  return __float2int_rz(__fsub_rn(cf, c0f));
+}
+
+template <bool kFast, bool kFull>
+__device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, unsigned* s_zclass,
+                                           float* queue, unsigned* qcount, float two_g, float c0f,
+                                           float magic, const float* base, long long j_tile,
+                                           long long jbeg, long long jend) {
+  float v[kKeyedQuads][4];
+  unsigned vm[kKeyedQuads];
+#pragma unroll
+  for (int q = 0; q < kKeyedQuads; ++q) {
+    const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
+    if (kFull) {
+      const float4 t = __ldcs(reinterpret_cast<const float4*>(base + j0));
+      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
+      vm[q] = 0xFu;
+    } else {
+      vm[q] = 0;
+      v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
+      if (j0 < jend) vm[q] = load_quad(base, j0, jbeg, jend, v[q]);
+    }
+  }
+  // per quad: phase A, four atomics in flight; phase B, marked cells and on-grid elements
+#pragma unroll
+  for (int q = 0; q < kKeyedQuads; ++q) {
+    unsigned old[4];
+    unsigned grid_mask = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float x = v[q][k];
+      bool on_grid;
+      const int idx = cell_index<kFast>(x, two_g, magic, c0f, &on_grid);
+      const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
+      old[k] = 0;
+      if (nz) old[k] = atomicAdd(&cells[idx], 1u);
+      if (nz && on_grid) grid_mask |= 1u << k;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const unsigned o = old[k];
+      const bool on_grid = (grid_mask >> k) & 1u;
+      if (o >= kCellNearZero || on_grid) {
+        const float x = v[q][k];
+        if (o & kCellNearZero) count_zero_class(s_zclass, x);
+        if ((o & kCellEdge) || on_grid) {
+          const unsigned pos = atomicAdd(qcount, 1u);
+          if (pos < kQueueCap) queue[pos] = x;
+          else handle_special(c, x);          // queue full: do it now
+        }
+      }
+    }
+  }
+  // drain full groups of 32 queued elements (dense lanes)
+  __syncwarp();
+  unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
+  __syncwarp();
+  if (n >= 32u) {
+    const int lane = threadIdx.x & 31;
+    const unsigned groups = n >> 5;
+    for (unsigned gq = 0; gq < groups; ++gq) handle_special(c, queue[n - 32u * (gq + 1) + lane]);
+    __syncwarp();
+    if (lane == 0) *qcount = n & 31u;
+    __syncwarp();
+  }
+}
+
+__global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const KeyedParams p) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ unsigned s_zclass[kZeroClasses];
-  __shared__ unsigned s_nzero;
+  __shared__ unsigned s_qcount[kKeyedWarps];
+  __shared__ LayerCtx s_ctx;
 
-  KeyedSmem sm;
-  sm.cells = reinterpret_cast<unsigned*>(s_raw);
-  sm.qe = sm.cells + p.cell_cap;
-  sm.d = reinterpret_cast<int*>(sm.qe + p.n_bins);
-  sm.qx = reinterpret_cast<float*>(sm.d + static_cast<size_t>(p.d_levels) * p.n_bins);
-  sm.qtag = reinterpret_cast<unsigned*>(sm.qx + kKeyedWarps * kQueueCap);
+  unsigned* cells = reinterpret_cast<unsigned*>(s_raw);
+  unsigned* qe = cells + p.cell_cap;
+  int* dtab = reinterpret_cast<int*>(qe + p.n_bins);
+  float* queues = reinterpret_cast<float*>(dtab + static_cast<size_t>(p.d_levels) * p.n_bins);
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned lt_mask = (1u << lane) - 1u;
-  float* qx = sm.qx + warp * kQueueCap;
-  unsigned* qtag = sm.qtag + warp * kQueueCap;
+  float* queue = queues + warp * kQueueCap;
+  unsigned* qcount = &s_qcount[warp];
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
@@ -160,113 +246,78 @@ __global__ void __launch_bounds__(kKeyedThreads, 2) search_keyed_kernel(const Ke
   while (t < t_end) {
     const LayerDesc L = p.layers[li];
     const int l = L.index;
-    LayerCtx c;
-    c.S = p.state[l];
-    c.P = p.plan[l];
-    c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
-    c.u_hist = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
-    c.zeros = p.zeros + static_cast<size_t>(l) * p.n_levels;
-    c.n_bins = p.n_bins; c.n_levels = p.n_levels; c.d_levels = p.d_levels;
+    const LayerState S = p.state[l];
+    const LayerPlan P = p.plan[l];
+    if (threadIdx.x == 0) {
+      LayerCtx c;
+      c.lo = S.lo; c.scale = S.scale; c.bmax = S.bmax;
+      c.two_g = P.two_g; c.c0f = P.c0f; c.c0 = P.c0; c.g = P.g; c.fs = P.fs;
+      c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
+      c.cells = cells; c.qe = qe; c.d = dtab;
+      c.u_hist = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
+      c.zeros = p.zeros + static_cast<size_t>(l) * p.n_levels;
+      c.n_bins = p.n_bins; c.n_levels = p.n_levels; c.d_levels = p.d_levels;
+      s_ctx = c;
+    }
+    const LayerCtx& c = s_ctx;   // read only after the barrier below
+    unsigned* const layer_u = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
     const long long layer_tiles_end = min(t_end, p.layers[li + 1].tile_begin);
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
-    const bool ok = c.P.keyed != 0;
+    const bool ok = P.keyed != 0;
+    // fast cell index when every cell index stays below 2^22 in magnitude
+    const bool fast = (P.c0 > -(1ll << 22)) && (P.c0 + P.cells < (1ll << 22));
+    const float magic = 12582912.0f - static_cast<float>(P.c0);
 
-    // ---- per-layer set-up of the private tables --------------------------------
+    // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
       const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-      for (int i = threadIdx.x; i < c.P.cells; i += kKeyedThreads) sm.cells[i] = __ldg(init + i);
-      for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) sm.qe[i] = 0;
+      for (int i = threadIdx.x; i < P.cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
+      for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
-      if (threadIdx.x == 0) s_nzero = 0;
+      if (lane == 0) *qcount = 0;
     }
     __syncthreads();
-    int qn = 0;             // this warp's queue fill (uniform across the warp)
-    unsigned n_zero = 0;    // exact zeros seen by this warp (lane 0's copy is used)
 
     for (; t < layer_tiles_end; ++t) {
       if (!ok) continue;
-      const long long j_tile = (t - L.tile_begin) * kTile;
-      float v[kTile / 4 / kKeyedThreads][4];
-      unsigned vm[kTile / 4 / kKeyedThreads];
-#pragma unroll
-      for (int q = 0; q < kTile / 4 / kKeyedThreads; ++q) {
-        const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
-        vm[q] = 0;
-        v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
-        if (j0 < jend) vm[q] = load_quad(base, j0, jbeg, jend, v[q]);
-      }
-#pragma unroll
-      for (int q = 0; q < kTile / 4 / kKeyedThreads; ++q) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float x = v[q][k];
-          const bool valid = (vm[q] >> k) & 1u;
-          const bool nz = valid && (x != 0.0f);
-          n_zero += __popc(__ballot_sync(0xffffffffu, valid && !nz));
-          const float z = __fmul_rn(x, c.P.two_g);
-          const float cf = floorf(z);
-          const int idx = __float2int_rz(__fsub_rn(cf, c.P.c0f));
-          unsigned old = 0;
-          if (nz) old = atomicAdd(&sm.cells[idx], 1u);
-          if (old & kCellNearZero) {
-            // highest level at which x still rounds to zero: |x| <= 2^-(k+1)
-            const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
-            int kz = 125 - static_cast<int>((ax - 1u) >> 23);
-            kz = max(-1, min(kz, 32));
-            atomicAdd(&s_zclass[kz + 1], 1u);
-          }
-          const bool on_grid = nz && (z == cf);
-          const bool push = nz && ((old & kCellEdge) || on_grid);
-          const unsigned pm = __ballot_sync(0xffffffffu, push);
-          if (pm) {
-            if (push) {
-              const int pos = qn + __popc(pm & lt_mask);
-              qx[pos] = x;
-              qtag[pos] = (old & kCellEdge) | (on_grid ? 0x40000000u : 0u) |
-                          static_cast<unsigned>(idx);
-            }
-            qn += __popc(pm);
-            __syncwarp();
-            if (qn >= 32) {
-              qn -= 32;
-              drain_entry(c, sm, true, qx[qn + lane], qtag[qn + lane]);
-              __syncwarp();
-            }
-          }
-        }
+      const long long j_tile = (t - L.tile_begin) * kKeyedTile;
+      const bool full = (j_tile >= jbeg) && (j_tile + kKeyedTile <= jend);
+      if (fast) {
+        if (full) keyed_tile<true, true>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
+        else keyed_tile<true, false>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
+      } else {
+        if (full) keyed_tile<false, true>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
+        else keyed_tile<false, false>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
       }
     }
-    // ---- drain what is left in the queue ------------------------------------------
+    // ---- what is left in the queues ----------------------------------------------
     if (ok) {
       __syncwarp();
-      if (qn > 0) {
-        const bool live = lane < qn;
-        drain_entry(c, sm, live, live ? qx[lane] : 0.0f, live ? qtag[lane] : 0u);
-      }
-      if (lane == 0 && n_zero) atomicAdd(&s_nzero, n_zero);
+      const unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
+      if (static_cast<unsigned>(lane) < n) handle_special(c, queue[lane]);
     }
     __syncthreads();
 
     // ---- flush the private tables into the layer's global ones -----------------------
     if (ok) {
       unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
-      for (int i = threadIdx.x; i < c.P.cells; i += kKeyedThreads) {
-        const unsigned n = sm.cells[i] & kCellCountMask;
+      for (int i = threadIdx.x; i < P.cells; i += kKeyedThreads) {
+        const unsigned n = cells[i] & kCellCountMask;
         if (n) atomicAdd(&gc[i], n);
       }
       unsigned* gq = p.qe_hist + static_cast<size_t>(l) * p.n_bins;
       for (int i = threadIdx.x; i < p.n_bins; i += kKeyedThreads) {
-        const unsigned n = sm.qe[i];
+        const unsigned n = qe[i];
         if (n) atomicAdd(&gq[i], n);
       }
       for (int i = threadIdx.x; i < p.n_bins * p.d_levels; i += kKeyedThreads) {
-        const int dv = sm.d[i];
+        const int dv = dtab[i];
         if (dv) {
           const int j = i / p.n_bins, b = i - j * p.n_bins;
-          const int f = c.P.fs + j;
+          const int f = P.fs + j;
           if (f < p.n_levels)
-            atomicAdd(&c.u_hist[static_cast<size_t>(f) * p.n_bins + b], static_cast<unsigned>(dv));
+            atomicAdd(&layer_u[static_cast<size_t>(f) * p.n_bins + b], static_cast<unsigned>(dv));
         }
       }
       if (threadIdx.x < kZeroClasses) {
@@ -274,7 +325,6 @@ __global__ void __launch_bounds__(kKeyedThreads, 2) search_keyed_kernel(const Ke
         if (n) atomicAdd(&p.zero_class[static_cast<size_t>(l) * kZeroClasses + threadIdx.x],
                          static_cast<unsigned long long>(n));
       }
-      if (threadIdx.x == 0 && s_nzero) atomicAdd(&p.n_zero[l], static_cast<unsigned long long>(s_nzero));
     }
     __syncthreads();
     ++li;
