@@ -161,7 +161,7 @@ struct Plan {
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
   // accumulators (cleared every call)
-  size_t off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0, off_stable = 0,
+  size_t off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
          off_zclass = 0, off_nzero = 0, accum_begin = 0, accum_bytes = 0;
   size_t total = 0;
 };
@@ -198,7 +198,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->d_levels = static_cast<int>(std::min<size_t>(6, (32 * 1024) / hist));
   p->d_levels = std::min(p->d_levels, p->n_levels);
   if (n_bins <= kKeyedMaxBins) {
-    p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (1 + p->d_levels)) / 4);
+    p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (1 + p->d_levels)) / 4) - 64;
     p->cell_cap = std::min(p->cell_cap, 1 << 16);
   } else {
     p->cell_cap = 0;
@@ -224,8 +224,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_zclass = o;  o = align_up(o + sizeof(unsigned long long) * L * kZeroClasses, 256);
   p->off_nzero = o;   o = align_up(o + sizeof(unsigned long long) * L, 256);
   p->off_q = o;       o = align_up(o + sizeof(unsigned) * L * B, 256);
-  p->off_qe = o;      o = align_up(o + sizeof(unsigned) * L * B, 256);
-  p->off_stable = o;  o = align_up(o + sizeof(unsigned) * L * B, 256);
+  p->off_qe = o;      o = align_up(o + sizeof(unsigned) * L * B * 2, 256);
   p->off_cells = o;   o = align_up(o + sizeof(unsigned) * L * K, 256);
   p->off_u = o;       o = align_up(o + sizeof(unsigned) * L * F * B, 256);
   p->accum_bytes = o - p->accum_begin;
@@ -351,10 +350,8 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   unsigned* d_cell_init = reinterpret_cast<unsigned*>(ws + plan.off_cell_init);
   unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + plan.off_zeros);
   unsigned long long* d_zclass = reinterpret_cast<unsigned long long*>(ws + plan.off_zclass);
-  unsigned long long* d_nzero = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
   unsigned* d_q = reinterpret_cast<unsigned*>(ws + plan.off_q);
   unsigned* d_qe = reinterpret_cast<unsigned*>(ws + plan.off_qe);
-  unsigned* d_stable = reinterpret_cast<unsigned*>(ws + plan.off_stable);
   unsigned* d_cells = reinterpret_cast<unsigned*>(ws + plan.off_cells);
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + plan.off_u);
 
@@ -378,7 +375,9 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     PlanParams pp;
     pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
     pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = a.n_bins; pp.cell_cap = plan.cell_cap;
-    pp.cell_target = std::min(plan.cell_cap, std::max(2048, 24 * a.n_bins));
+    pp.fine_ratio = ADAPT_FINE_RATIO;
+    const int keyed_grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
+    pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
     {
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
       plan_kernel<<<nk, kPlanThreads, 0, stream>>>(pp);
@@ -393,7 +392,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(plan.keyed_smem)));
     {
-      const int grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
+      const int grid = keyed_grid;
       LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
       search_keyed_kernel<<<grid, kKeyedThreads, plan.keyed_smem, stream>>>(kp);
       ADAPT_CUDA(cudaGetLastError());
@@ -401,17 +400,12 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ExpandParams ep;
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
     ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
-    ep.stable_hist = d_stable; ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros;
-    ep.zero_class = d_zclass; ep.cell_total = d_nzero; ep.n_bins = a.n_bins;
-    ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
+    ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
+    ep.n_bins = a.n_bins; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
     {
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      expand_cells_kernel<<<dim3((plan.cell_cap + 255) / 256, nk), 256, 0, stream>>>(ep);
-      ADAPT_CUDA(cudaGetLastError());
-    }
-    {
-      LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      combine_kernel<<<dim3((a.n_bins + 255) / 256, plan.n_levels + 1, nk), 256, 0, stream>>>(ep);
+      expand_kernel<<<dim3(plan.n_levels + 1, nk), kExpandThreads, sizeof(unsigned) * a.n_bins,
+                      stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
   }

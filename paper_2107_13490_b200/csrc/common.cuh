@@ -30,6 +30,7 @@ struct LayerState {
   unsigned max_key;  // ... of the maximum
   unsigned flags;    // ADAPT_FLAG_NONFINITE / ADAPT_FLAG_RANGE / ADAPT_FLAG_DEGENERATE
   float lo, hi, scale, bmax;
+  float abs_sum;     // sum of |x| (any summation order; only steers table shapes, never results)
 };
 
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).

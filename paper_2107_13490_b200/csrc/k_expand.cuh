@@ -1,16 +1,19 @@
 // Expansion of the keyed kernel's cell counts into the per-level histograms.
 //
-// expand_cells_kernel: one thread per (cell, layer).  A cell's count feeds
-//   * the "stable" histogram (interior cells only): these elements fall in the
-//     cell's bin in the float histogram and at every fine level f >= G;
-//   * every coarse level f < G: the rounded value rint(x * 2^f) of any element
-//     of the cell is a + (rem >= half), with c = a * 2^d + rem, d = G - f
-//     (ties that go down were fixed up element by element in the keyed kernel).
-// combine_kernel: one thread per (bin, level, layer) adds the base terms to
-// the correction counts already sitting in U: stable + edge-element histogram
-// for fine levels, the exact zeros at the bin of 0, and builds Q and the zero
-// counts of the fine levels from the zero classes.  The exact zeros are the
-// elements no cell counted.
+// One CTA per (level, layer); level n_levels stands for the float histogram Q.
+// The CTA walks the layer's cells (both segments) and adds each cell's count to
+// a shared-memory histogram of its level:
+//   * float histogram and fine levels (f >= the segment's G), interior cells
+//     only: the cell's own bin (elements of edge cells were binned one by one
+//     by the keyed kernel into the segment's edge-element histogram, which is
+//     added here, and their level-by-level moves already sit in U);
+//   * coarse levels (f < G), every cell: the rounded value rint(x * 2^f) of any
+//     element of the cell is a + (rem >= half), with c = a * 2^d + rem,
+//     d = G - f (ties that go down were fixed up element by element);
+// then the exact zeros (layer size minus all cell counts) at the bin of 0, and
+// for the zero counts the cells that round to 0 plus, at fine levels of the
+// main segment, the zero classes.  The result is added to the corrections
+// already in U; no global atomics.
 #pragma once
 
 #include "common.cuh"
@@ -19,6 +22,8 @@
 
 namespace adapt {
 
+constexpr int kExpandThreads = 512;
+
 struct ExpandParams {
   const LayerDesc* layers;     // keyed layer list
   int n_layers;
@@ -26,74 +31,83 @@ struct ExpandParams {
   const LayerPlan* plan;
   const unsigned* cell_init;   // [layer][cell_cap]
   const unsigned* cell_count;  // [layer][cell_cap]
-  const unsigned* qe_hist;     // [layer][n_bins]
-  unsigned* stable_hist;       // [layer][n_bins]
+  const unsigned* qe_hist;     // [layer][2][n_bins]
   unsigned* q_hist;            // [layer][n_bins]
   unsigned* u_hist;            // [layer][n_levels][n_bins]
   unsigned long long* zeros;   // [layer][n_levels]
   const unsigned long long* zero_class;  // [layer][kZeroClasses]
-  unsigned long long* cell_total;        // [layer] sum of the cell counts = non-zero elements
   int n_bins, n_levels, cell_cap;
 };
 
-__global__ void __launch_bounds__(256) expand_cells_kernel(const ExpandParams p) {
+__global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandParams p) {
+  extern __shared__ unsigned s_hist[];          // [n_bins]
+  __shared__ unsigned long long s_total, s_zero;
   const LayerDesc L = p.layers[blockIdx.y];
   const int l = L.index;
   const LayerPlan P = p.plan[l];
   if (!P.keyed) return;
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  const unsigned m = (c < P.cells) ? p.cell_count[static_cast<size_t>(l) * p.cell_cap + c] : 0u;
-  // the layer's non-zero elements = sum of all its cell counts
-  unsigned long long wsum = m;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, o);
-  if ((threadIdx.x & 31) == 0 && wsum) atomicAdd(&p.cell_total[l], wsum);
-  if (m == 0) return;
   const LayerState S = p.state[l];
   const int B = p.n_bins;
-  const long long cc = P.c0 + c;
-  if (!(p.cell_init[static_cast<size_t>(l) * p.cell_cap + c] & kCellEdge)) {
-    const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -P.g));
-    atomicAdd(&p.stable_hist[static_cast<size_t>(l) * B + bin_of(lf, S.lo, S.scale, S.bmax)], m);
-  }
-  unsigned* U = p.u_hist + static_cast<size_t>(l) * p.n_levels * B;
-  const int coarse_end = min(P.g, p.n_levels);
-  for (int f = 0; f < coarse_end; ++f) {
-    const int d = P.g - f;                       // 1..32
-    const long long a = cc >> d;                 // floor(c / 2^d)
-    const long long rem = cc - (a << d);
-    const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
-    const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
-    atomicAdd(&U[static_cast<size_t>(f) * B + bin_of(v, S.lo, S.scale, S.bmax)], m);
-    if (r == 0) atomicAdd(&p.zeros[static_cast<size_t>(l) * p.n_levels + f],
-                          static_cast<unsigned long long>(m));
-  }
-}
+  const int f = blockIdx.x;                     // level, or n_levels for the float histogram
+  const bool is_q = (f == p.n_levels);
 
-__global__ void __launch_bounds__(256) combine_kernel(const ExpandParams p) {
-  const LayerDesc L = p.layers[blockIdx.z];
-  const int l = L.index;
-  const LayerPlan P = p.plan[l];
-  if (!P.keyed) return;
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  const int f = blockIdx.y;                      // level, or n_levels for the float histogram
-  const int B = p.n_bins;
-  if (b >= B) return;
-  const LayerState S = p.state[l];
-  const unsigned nz = static_cast<unsigned>(static_cast<unsigned long long>(L.n) - p.cell_total[l]);
-  const int bz = bin_of(0.0f, S.lo, S.scale, S.bmax);
-  const unsigned base = p.stable_hist[static_cast<size_t>(l) * B + b] +
-                        p.qe_hist[static_cast<size_t>(l) * B + b];
-  const unsigned zero_here = (b == bz) ? nz : 0u;
-  if (f == p.n_levels) {
-    p.q_hist[static_cast<size_t>(l) * B + b] = base + zero_here;
-    return;
+  for (int b = threadIdx.x; b < B; b += kExpandThreads) s_hist[b] = 0;
+  if (threadIdx.x == 0) { s_total = 0; s_zero = 0; }
+  __syncthreads();
+
+  const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
+  const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
+  unsigned long long total = 0, zero = 0;
+  for (int i = threadIdx.x; i < P.total_cells; i += kExpandThreads) {
+    const unsigned m = count[i];
+    if (m == 0) continue;
+    total += m;
+    const int s = (P.seg[1].cells > 0 && i >= P.seg[1].offset) ? 1 : 0;
+    const SegPlan& sp = P.seg[s];
+    const long long cc = sp.c0 + (i - sp.offset);
+    if (is_q || f >= sp.g) {
+      if (!(init[i] & kCellEdge)) {
+        const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
+        atomicAdd(&s_hist[bin_of(lf, S.lo, S.scale, S.bmax)], m);
+      }
+    } else {
+      const int d = sp.g - f;                      // 1..32
+      const long long a = cc >> d;                 // floor(c / 2^d)
+      const long long rem = cc - (a << d);
+      const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
+      const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
+      atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+      if (r == 0) zero += m;
+    }
   }
-  unsigned* u = p.u_hist + (static_cast<size_t>(l) * p.n_levels + f) * B + b;
-  *u = *u + (f >= P.fs ? base : 0u) + zero_here;
-  if (b == 0) {
-    unsigned long long z = nz;
-    if (f >= P.fs) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    total += __shfl_xor_sync(0xffffffffu, total, o);
+    zero += __shfl_xor_sync(0xffffffffu, zero, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    if (total) atomicAdd(&s_total, total);
+    if (zero) atomicAdd(&s_zero, zero);
+  }
+  __syncthreads();
+
+  const unsigned n_zero = static_cast<unsigned>(static_cast<unsigned long long>(L.n) - s_total);
+  const int bz = bin_of(0.0f, S.lo, S.scale, S.bmax);
+  const unsigned* qe0 = p.qe_hist + static_cast<size_t>(l) * 2 * B;
+  const unsigned* qe1 = qe0 + B;
+  const bool fine0 = is_q || f >= P.seg[0].fs;
+  const bool fine1 = P.seg[1].cells > 0 && (is_q || f >= P.seg[1].fs);
+  unsigned* out = is_q ? p.q_hist + static_cast<size_t>(l) * B
+                       : p.u_hist + (static_cast<size_t>(l) * p.n_levels + f) * B;
+  for (int b = threadIdx.x; b < B; b += kExpandThreads) {
+    unsigned h = s_hist[b] + (b == bz ? n_zero : 0u);
+    if (fine0) h += qe0[b];
+    if (fine1) h += qe1[b];
+    out[b] = is_q ? h : out[b] + h;
+  }
+  if (!is_q && threadIdx.x == 0) {
+    unsigned long long z = s_zero + n_zero;
+    if (f >= P.seg[0].fs) {
       const unsigned long long* zc = p.zero_class + static_cast<size_t>(l) * kZeroClasses;
       for (int k = f; k <= 32; ++k) z += zc[k + 1];   // classes whose highest zero level >= f
     }

@@ -1,7 +1,6 @@
 // Per-layer plan of the keyed search kernel (round-to-nearest-even only).
 //
-// Idea.  Cut the value axis into cells of width 2^-G (G per layer, as fine as
-// the cell table that fits in shared memory allows).  An element x lies in
+// Idea.  Cut the value axis into cells of width 2^-G.  An element x lies in
 // cell c = floor(x * 2^G).  Then, exactly:
 //  * for every coarser level f < G the rounded value rint(x * 2^f) is a
 //    function of c alone (unless x sits exactly on the level-G grid AND on a
@@ -15,9 +14,19 @@
 //    fine levels looked at one by one, and among those only the levels whose
 //    half quantum 2^-(f+1) exceeds the element's distance to its bin's edges;
 //  * for f >= G an element rounds to zero only if it lies in cell -1 or 0.
-// This kernel chooses G, computes the exact bin edges (smallest float of each
-// bin, by bisection over the float order with the bin function itself), and
-// marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0.
+// The finer the cells, the fewer elements fall in edge cells or next to zero.
+// The table that holds the counts lives in shared memory, so its size is
+// fixed; to spend it where the elements are, a layer whose range contains
+// zero and whose mass sits in a small part of the range gets TWO segments:
+// a main segment of fine cells on [-R, R) (R a power of two, a multiple of the
+// mean magnitude found by the range scan) and an auxiliary segment of coarse
+// cells over the whole range for the few elements outside.  R only steers
+// speed: any R gives the same results.
+//
+// This kernel chooses the segments, computes the exact bin edges (smallest
+// float of each bin, by bisection over the float order with the bin function
+// itself), and marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0 of
+// the main segment.
 #pragma once
 
 #include "common.cuh"
@@ -30,14 +39,33 @@ constexpr unsigned kCellNearZero = 0x40000000u;
 constexpr unsigned kCellCountMask = 0x3FFFFFFFu;
 constexpr int kPlanThreads = 256;
 
-struct LayerPlan {
-  long long c0;   // cell index of the first cell: floor(lo * 2^G)
+// Tunables of the table shape (performance only).
+#ifndef ADAPT_CELL_BALANCE
+#define ADAPT_CELL_BALANCE 4    // cells ~ sqrt(balance * n_bins * elements one CTA sees of the layer)
+#endif
+#ifndef ADAPT_FINE_RATIO
+#define ADAPT_FINE_RATIO 512    // stop refining once a bin holds this many cells
+#endif
+
+struct SegPlan {
+  long long c0;   // cell index of the segment's first cell: floor(left end * 2^G)
   int g;          // cell level G (cells are 2^-G wide); may be negative
-  int cells;      // number of cells covering [lo, hi]
+  int cells;      // number of cells
   int fs;         // first fine level: max(G, 0)
-  float c0f;      // (float)c0 when it is exact, else unused
+  int offset;     // position of the segment's first cell in the layer's table
   float two_g;    // 2^G
-  int keyed;      // 1 if the layer goes through the keyed kernel
+  float c0f;      // (float)c0 (exact)
+  float magic;    // 1.5 * 2^23 - c0 + offset: x * 2^G + magic, rounded down, has the
+                  // table position in its low mantissa bits (fast layers only)
+  int pad_;
+};
+
+struct LayerPlan {
+  SegPlan seg[2];   // [0] main, [1] auxiliary (cells == 0 when unused)
+  float radius;     // elements with |x| < radius use the main segment (+inf: all of them)
+  int keyed;        // 1 if the layer goes through the keyed kernel
+  int fast;         // 1 if every cell index is below 2^22 in magnitude
+  int total_cells;  // seg[0].cells + seg[1].cells
 };
 
 struct PlanParams {
@@ -48,13 +76,41 @@ struct PlanParams {
   float* edges;              // [all layers][n_bins + 1]
   unsigned* cell_init;       // [all layers][cell_cap]
   int n_bins;
-  int cell_cap;              // table entries per layer (memory stride)
-  int cell_target;           // most cells a layer may use (<= cell_cap)
+  int cell_cap;              // table entries per layer (memory stride and upper limit)
+  int fine_ratio;            // stop refining once a bin holds this many cells
+  long long elems_per_cta;   // elements one CTA of the keyed kernel processes
 };
 
 __device__ __forceinline__ long long floor_scaled(float v, int g) {
-  // floor(v * 2^g) exactly: |v| < 2^64 and |g| <= 64 keep the product inside double
+  // floor(v * 2^g) exactly: the product stays inside double
   return static_cast<long long>(floor(ldexp(static_cast<double>(v), g)));
+}
+
+// Largest level G <= g_max such that the cells covering [lo, hi] number at most max_cells.
+__device__ inline void fit_segment(float lo, float hi, int max_cells, int g_max, SegPlan* s) {
+  int g = g_max;
+  long long c0 = 0, c1 = 0;
+  for (; g > -100; --g) {
+    const double span = ldexp(static_cast<double>(hi) - static_cast<double>(lo), g);
+    if (span >= static_cast<double>(max_cells)) continue;
+    if (fabs(ldexp(static_cast<double>(hi), g)) > 9.0e18 ||
+        fabs(ldexp(static_cast<double>(lo), g)) > 9.0e18) continue;
+    c0 = floor_scaled(lo, g);
+    c1 = floor_scaled(hi, g);
+    if (c1 - c0 + 1 <= max_cells) break;
+  }
+  s->g = g; s->c0 = c0; s->cells = static_cast<int>(c1 - c0 + 1);
+  s->fs = g > 0 ? g : 0;
+  s->two_g = pow2f(g);
+  s->c0f = static_cast<float>(c0);
+}
+
+// Level at which a bin of width bw holds about `ratio` cells (no need to go finer).
+__device__ inline int level_for_ratio(float lo, float hi, int n_bins, int ratio) {
+  const double bw = (static_cast<double>(hi) - static_cast<double>(lo)) / n_bins;
+  if (!(bw > 0.0)) return 32;
+  int g = static_cast<int>(ceil(log2(static_cast<double>(ratio) / bw)));
+  return max(-100, min(g, 32));
 }
 
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) {
@@ -67,23 +123,56 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   if (threadIdx.x == 0) {
     LayerPlan P;
     P.keyed = !(S.flags & (kFlagNonfinite | kFlagRange)) && L.n > 0;
-    int g = 32;
-    long long c0 = 0, c1 = 0;
-    // largest G <= 32 whose cells fit the table; the width shrinks by 2 per step
-    for (; g > -100; --g) {
-      // products up to 2^64 * 2^32 overflow long long: skip levels that cannot fit anyway
-      double span = ldexp(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
-      if (span >= static_cast<double>(p.cell_target)) continue;
-      if (fabs(ldexp(static_cast<double>(S.hi), g)) > 9.0e18 ||
-          fabs(ldexp(static_cast<double>(S.lo), g)) > 9.0e18) continue;
-      c0 = floor_scaled(S.lo, g);
-      c1 = floor_scaled(S.hi, g);
-      if (c1 - c0 + 1 <= p.cell_target) break;
+    P.radius = __int_as_float(0x7f800000);
+    P.seg[1].c0 = 0; P.seg[1].g = 0; P.seg[1].cells = 0; P.seg[1].fs = 0; P.seg[1].offset = 0;
+    P.seg[1].two_g = 1.0f; P.seg[1].c0f = 0.0f; P.seg[1].magic = 0.0f; P.seg[1].pad_ = 0;
+    P.seg[0].pad_ = 0;
+    const int g_want = level_for_ratio(S.lo, S.hi, B, p.fine_ratio);
+    // every CTA that meets the layer sets up and flushes its private table once (cost ~ cells),
+    // while the share of elements that need the slow path falls as n_bins / cells: the sum is
+    // least near cells = sqrt(k * n_bins * elements the CTA sees of the layer)
+    const double seen = static_cast<double>(min(L.n, p.elems_per_cta));
+    const long long want = static_cast<long long>(sqrt(ADAPT_CELL_BALANCE * static_cast<double>(B) * seen));
+    const int cap = static_cast<int>(min(static_cast<long long>(p.cell_cap), max(2048ll, want)));
+    fit_segment(S.lo, S.hi, cap, g_want, &P.seg[0]);
+    // two segments pay off when zero is inside the range, the single segment cannot reach
+    // the wanted fineness, and the mass sits within a small radius
+    const float amax = fmaxf(fabsf(S.lo), fabsf(S.hi));
+    const float mean = S.abs_sum / static_cast<float>(L.n > 0 ? L.n : 1);
+    if (P.keyed && S.lo <= 0.0f && S.hi >= 0.0f && P.seg[0].g < g_want && mean > 0.0f &&
+        mean < 3.0e38f) {
+      const int rexp = static_cast<int>(ceil(log2(static_cast<double>(mean) * 8.0)));
+      if (rexp > -100 && rexp < 100) {
+        const float r = pow2f(rexp);
+        if (r < 0.25f * amax) {
+          SegPlan aux, main;
+          fit_segment(S.lo, S.hi, cap / 4, g_want, &aux);
+          const float mlo = fmaxf(S.lo, -r), mhi = fminf(S.hi, r);
+          fit_segment(mlo, mhi, cap - aux.cells, g_want, &main);
+          // the auxiliary cells next to zero must stay empty: R at least two of them wide
+          if (main.g > P.seg[0].g + 1 && r > pow2f(-aux.g)) {
+            P.seg[0] = main; P.seg[1] = aux; P.radius = r;
+            P.seg[0].pad_ = 0; P.seg[1].pad_ = 0;
+          }
+        }
+      }
     }
-    P.g = g; P.c0 = c0; P.cells = static_cast<int>(c1 - c0 + 1);
-    P.fs = g > 0 ? g : 0;
-    P.c0f = static_cast<float>(c0);
-    P.two_g = pow2f(g);
+    P.seg[0].offset = 0;
+    P.seg[1].offset = P.seg[0].cells;
+    P.total_cells = P.seg[0].cells + P.seg[1].cells;
+    P.fast = 1;
+    for (int s = 0; s < 2; ++s) {
+      const SegPlan& sp = P.seg[s];
+      if (sp.c0 <= -(1ll << 22) || sp.c0 + sp.cells >= (1ll << 22)) P.fast = 0;
+    }
+    if (P.seg[1].cells > 0 && !P.fast) {   // cannot happen (zero is inside); stay safe
+      fit_segment(S.lo, S.hi, cap, g_want, &P.seg[0]);
+      P.seg[1].cells = 0; P.radius = __int_as_float(0x7f800000);
+      P.total_cells = P.seg[0].cells;
+    }
+    for (int s = 0; s < 2; ++s)
+      P.seg[s].magic = 12582912.0f - static_cast<float>(P.seg[s].c0) +
+                       static_cast<float>(P.seg[s].offset);
     s_plan = P;
     p.plan[l] = P;
   }
@@ -110,17 +199,18 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     E[b] = e;
   }
 
-  // cell marks
+  // cell marks, both segments
   unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-  for (int c = threadIdx.x; c < P.cells; c += kPlanThreads) {
-    const long long cc = P.c0 + c;
-    const double left = ldexp(static_cast<double>(cc), -P.g);
-    const double right = ldexp(static_cast<double>(cc + 1), -P.g);
-    const float lf = __double2float_rd(left), rf = __double2float_ru(right);
+  for (int i = threadIdx.x; i < P.total_cells; i += kPlanThreads) {
+    const int s = (i >= P.seg[1].offset && P.seg[1].cells > 0) ? 1 : 0;
+    const SegPlan& sp = P.seg[s];
+    const long long cc = sp.c0 + (i - sp.offset);
+    const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
+    const float rf = __double2float_ru(ldexp(static_cast<double>(cc + 1), -sp.g));
     unsigned mark = 0;
     if (bin_of(lf, S.lo, S.scale, S.bmax) != bin_of(rf, S.lo, S.scale, S.bmax)) mark |= kCellEdge;
-    if (cc == 0 || cc == -1) mark |= kCellNearZero;
-    init[c] = mark;
+    if (s == 0 && (cc == 0 || cc == -1)) mark |= kCellNearZero;
+    init[i] = mark;
   }
 }
 

@@ -25,6 +25,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
   if (t >= t_end) return;
 
   __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
+  __shared__ float s_abs[kRangeThreads / 32];
   int l = layer_of_tile(layers, n_layers, t);
 
   while (t < t_end) {
@@ -35,6 +36,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
 
     float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
     unsigned flags = 0;
+    float asum = 0.0f;
     for (; t < layer_tiles_end; ++t) {
       const long long j_tile = (t - L.tile_begin) * kTile;
 #pragma unroll
@@ -52,6 +54,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
             else if (a >= 18446744073709551616.0f) flags |= kFlagRange;
             vmin = fminf(vmin, v[k]);
             vmax = fmaxf(vmax, v[k]);
+            asum += a;
           }
         }
       }
@@ -64,17 +67,20 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
       kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
       kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
       flags |= __shfl_xor_sync(0xffffffffu, flags, o);
+      asum += __shfl_xor_sync(0xffffffffu, asum, o);
     }
     const int w = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; }
+    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; }
     __syncthreads();
     if (threadIdx.x == 0) {
       for (int i = 1; i < kRangeThreads / 32; ++i) {
         kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
+        asum += s_abs[i];
       }
       atomicMin(&state[L.index].min_key, kmin);
       atomicMax(&state[L.index].max_key, kmax);
       if (flags) atomicOr(&state[L.index].flags, flags);
+      if (asum == asum && asum < 3.0e38f) atomicAdd(&state[L.index].abs_sum, asum);
     }
     __syncthreads();
     ++l;

@@ -2,26 +2,26 @@
 // zero count + histograms with ONE shared-memory atomic per element on the
 // common path.  See k_plan.cuh for the cell decomposition this relies on.
 //
-// Per element x != 0:   c = floor(x * 2^G) - c0;  old = atomicAdd(cell[c], 1)
+// Per element x != 0:   pos = table position of x's cell;  old = atomicAdd(cell[pos], 1)
 // The returned word carries the cell's marks in its two top bits:
-//   bit 30 (cell -1 / 0): the element is added to the class counter "highest
-//          level at which it still rounds to zero";
-//   bit 31 (edge cell), or x exactly on the level-G grid: the element goes to a
+//   bit 30 (cell -1 / 0 of the main segment): the element is added to the class
+//          counter "highest level at which it still rounds to zero";
+//   bit 31 (edge cell), or x exactly on its segment's grid: the element goes to a
 //          per-warp queue that the warp drains 32 entries at a time:
-//            edge entry: b0 = bin(x) into the edge-element histogram Qe, then
-//              only the fine levels f whose half quantum can reach one of the
-//              bin's edges are evaluated; a level is recorded only if its bin
-//              differs from b0 (-1 at b0, +1 at the new bin);
+//            edge entry: b0 = bin(x) into the segment's edge-element histogram,
+//              then only the fine levels f whose half quantum can reach one of
+//              the bin's edges are evaluated; a level is recorded only if its
+//              bin differs from b0 (-1 at b0, +1 at the new bin);
 //            on-grid entry: the one coarse level at which x is a rounding tie
 //              that goes down is corrected (the cell table assumes "up").
-// Exact zeros touch nothing (their number is the layer size minus the sum of
-// the cell counts).  Everything else about an element - the float histogram,
-// all coarse levels, all fine levels of interior cells - is derived from the
-// cell counts by the expand kernels.
+// Exact zeros are sent to per-lane dummy slots (their number is the layer size
+// minus the sum of the cell counts).  Everything else about an element - the
+// float histogram, all coarse levels, all fine levels of interior cells - is
+// derived from the cell counts by the expand kernel.
 //
 // One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
-// for its cell table; each thread keeps 16 elements (four 128-bit loads) in
-// flight per tile.
+// for its tables; each thread keeps 16 elements (four 128-bit loads) in flight
+// per tile.
 #pragma once
 
 #include "common.cuh"
@@ -34,8 +34,9 @@ constexpr int kKeyedThreads = 1024;
 constexpr int kKeyedWarps = kKeyedThreads / 32;
 constexpr int kKeyedQuads = 4;                                  // 128-bit loads per thread per tile
 constexpr int kKeyedTile = kKeyedThreads * kKeyedQuads * 4;     // 16384 elements
-constexpr int kQueueCap = 128;      // per-warp queue entries; a full queue handles entries inline
+constexpr int kQueueCap = 96;       // per-warp queue entries; a full queue handles entries inline
 constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..32
+constexpr int kDummySlots = 32;     // where the atomics of exact zeros land (one per lane)
 
 struct KeyedParams {
   const LayerDesc* layers;     // keyed layer list (+ sentinel), tiles of kKeyedTile elements
@@ -46,56 +47,62 @@ struct KeyedParams {
   const float* edges;          // [layer][n_bins + 1]
   const unsigned* cell_init;   // [layer][cell_cap]
   unsigned* cell_count;        // [layer][cell_cap]      global cell counts
-  unsigned* qe_hist;           // [layer][n_bins]        float histogram of the edge elements
+  unsigned* qe_hist;           // [layer][2][n_bins]     float histogram of the edge elements, per segment
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
   unsigned long long* zeros;   // [layer][n_levels]      receives tie corrections
   unsigned long long* zero_class;  // [layer][kZeroClasses]
   int n_bins;
   int n_levels;                // levels 0..n_levels-1 are wanted
   int cell_cap;
-  int d_levels;                // fine levels whose corrections are kept in shared memory
+  int d_levels;                // fine levels of the main segment whose corrections stay in shared memory
 };
 
 __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int d_levels) {
-  return sizeof(unsigned) * (static_cast<size_t>(cell_cap) + n_bins +
+  return sizeof(unsigned) * (static_cast<size_t>(cell_cap) + kDummySlots + n_bins +
                              static_cast<size_t>(d_levels) * n_bins) +
          sizeof(float) * kKeyedWarps * kQueueCap;
 }
 
-// Everything the special-element handler needs about the current layer.
+// Everything the special-element handler needs about the current layer (in shared memory).
 struct LayerCtx {
   float lo, scale, bmax;       // bin function
-  float two_g, c0f;            // cell function (general form)
-  long long c0;
-  int g, fs;
+  float radius;
+  float two_g[2], c0f[2];      // cell function per segment (general form)
+  long long c0[2];
+  int g[2], fs[2], offset[2];
   const float* E;              // exact bin edges [n_bins + 1]
   const unsigned* cells;       // shared cell table (marks in the two top bits)
-  unsigned* qe;                // shared [n_bins]
+  unsigned* qe;                // shared [n_bins]: main segment's edge-element histogram
   int* d;                      // shared [d_levels][n_bins]
+  unsigned* qe_aux;            // global [n_bins]: auxiliary segment's edge-element histogram
   unsigned* u_hist;            // global, this layer's [n_levels][n_bins]
   unsigned long long* zeros;   // global, this layer's [n_levels]
   int n_bins, n_levels, d_levels;
+  float magic[2];
+  int keyed, fast, total_cells;
 };
 
 // Handles one queued element (x != 0, finite).  No warp-level primitive inside:
 // any subset of lanes may call it.
 __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   const int B = c.n_bins;
-  const float z = __fmul_rn(x, c.two_g);
+  const int s = (fabsf(x) < c.radius) ? 0 : 1;
+  const float z = __fmul_rn(x, c.two_g[s]);
   const float cf = floorf(z);
-  const int idx = __float2int_rz(__fsub_rn(cf, c.c0f));
-  // ---- x on the level-G grid: fix the single coarse level at which it is a tie --
+  const int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s]));   // cell index inside the segment
+  const int g = c.g[s];
+  // ---- x on the segment's grid: fix the single coarse level at which it is a tie ----
   if (z == cf) {
-    const long long cc = c.c0 + idx;
+    const long long cc = c.c0[s] + ci;
     if (cc != 0) {
       const int tz = __ffsll(cc) - 1;          // lowest set bit
-      const int ft = c.g - 1 - tz;             // the level at which x is a tie
+      const int ft = g - 1 - tz;               // the level at which x is a tie
       if (ft >= 0 && ft < c.n_levels) {
         const long long a = cc >> (tz + 1);    // floor(x * 2^ft)
         if ((a & 1ll) == 0) {                  // tie goes down to a; the table counted a + 1
-          const float s = pow2f(-ft);
-          const int b_up = bin_of(__fmul_rn(__ll2float_rn(a + 1), s), c.lo, c.scale, c.bmax);
-          const int b_dn = bin_of(__fmul_rn(__ll2float_rn(a), s), c.lo, c.scale, c.bmax);
+          const float sc = pow2f(-ft);
+          const int b_up = bin_of(__fmul_rn(__ll2float_rn(a + 1), sc), c.lo, c.scale, c.bmax);
+          const int b_dn = bin_of(__fmul_rn(__ll2float_rn(a), sc), c.lo, c.scale, c.bmax);
           unsigned* U = c.u_hist + static_cast<size_t>(ft) * B;
           if (b_up != b_dn) { atomicAdd(&U[b_up], 0xFFFFFFFFu); atomicAdd(&U[b_dn], 1u); }
           if (a + 1 == 0) atomicAdd(&c.zeros[ft], 0xFFFFFFFFFFFFFFFFull);
@@ -104,23 +111,24 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
       }
     }
   }
-  // ---- edge cell: float bin, then the fine levels that can still move ------------
-  if (!(c.cells[idx] & kCellEdge)) return;
+  // ---- edge cell: float bin, then the fine levels that can still move ----------------
+  if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
-  atomicAdd(&c.qe[b0], 1u);
+  if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
   const float e_lo = __ldg(c.E + b0), e_hi = __ldg(c.E + b0 + 1);
   // distance to the bin's two edges, rounded down: a level is safe once 2^-(f+1) < margin
   const float m = fminf(__fsub_rd(x, e_lo), __fsub_rd(e_hi, x));
   int f_end = 32;
   if (m > 0.0f) f_end = 126 - static_cast<int>((__float_as_uint(m) - 1u) >> 23);
   f_end = min(f_end, c.n_levels);
-  for (int f = c.fs; f < f_end; ++f) {
+  const int fs = c.fs[s];
+  for (int f = fs; f < f_end; ++f) {
     const float r = rintf(__fmul_rn(x, pow2f(f)));
     const float v = __fmul_rn(r, pow2f(-f));
     if (v >= e_lo && v < e_hi) continue;       // still in b0 (edges are exact)
     const int b = bin_of(v, c.lo, c.scale, c.bmax);
-    const int j = f - c.fs;
-    if (j < c.d_levels) {
+    const int j = f - fs;
+    if (s == 0 && j < c.d_levels) {
       atomicAdd(&c.d[j * B + b], 1);
       atomicAdd(&c.d[j * B + b0], -1);
     } else {
@@ -131,7 +139,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   }
 }
 
-// Adds a near-zero element (cells -1 / 0) to its zero class.
+// Adds a near-zero element (cells -1 / 0 of the main segment) to its zero class.
 __device__ __forceinline__ void count_zero_class(unsigned* s_zclass, float x) {
   // highest level k at which x still rounds to zero: |x| <= 2^-(k+1)
   const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
@@ -140,28 +148,37 @@ __device__ __forceinline__ void count_zero_class(unsigned* s_zclass, float x) {
   atomicAdd(&s_zclass[kz + 1], 1u);
 }
 
-// Cell index of x.  Fast form: |cell indices| < 2^22, so adding the magic
-// constant 1.5 * 2^23 - c0 with round-down leaves floor(x * 2^G) - c0 in the
-// low mantissa bits; x is on the grid exactly when round-up gives the same.
+// The constants one tile needs to place an element in the table.
+struct CellFn {
+  float radius;
+  float two_g0, magic0, c0f0;   // main segment
+  float two_g1, magic1;         // auxiliary segment (fast layers only)
+};
+
+// Table position of x.  Fast form: adding the segment's magic constant
+// (1.5 * 2^23 - c0 + offset) to x * 2^G with round-down leaves the position in
+// the low mantissa bits; x is on the grid exactly when round-up gives the same.
 template <bool kFast>
-__device__ __forceinline__ int cell_index(float x, float two_g, float magic, float c0f,
-                                          bool* on_grid) {
+__device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_grid) {
   if (kFast) {
-    const float rd = __fmaf_rd(x, two_g, magic);
-    const float ru = __fmaf_ru(x, two_g, magic);
+    const bool inner = fabsf(x) < f.radius;
+    const float s = inner ? f.two_g0 : f.two_g1;
+    const float mg = inner ? f.magic0 : f.magic1;
+    const float rd = __fmaf_rd(x, s, mg);
+    const float ru = __fmaf_ru(x, s, mg);
     *on_grid = (rd == ru);
     return __float_as_int(rd) - 0x4B400000;
   }
-  const float z = __fmul_rn(x, two_g);
+  const float z = __fmul_rn(x, f.two_g0);
   const float cf = floorf(z);
   *on_grid = (z == cf);
-  return __float2int_rz(__fsub_rn(cf, c0f));
+  return __float2int_rz(__fsub_rn(cf, f.c0f0));
 }
 
 template <bool kFast, bool kFull>
-__device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, unsigned* s_zclass,
-                                           float* queue, unsigned* qcount, float two_g, float c0f,
-                                           float magic, const float* base, long long j_tile,
+__device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                           unsigned* s_zclass, float* queue, unsigned* qcount,
+                                           const CellFn& fn, const float* base, long long j_tile,
                                            long long jbeg, long long jend) {
   float v[kKeyedQuads][4];
   unsigned vm[kKeyedQuads];
@@ -178,39 +195,43 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, u
       if (j0 < jend) vm[q] = load_quad(base, j0, jbeg, jend, v[q]);
     }
   }
-  // per quad: phase A, four atomics in flight; phase B, marked cells and on-grid elements
 #pragma unroll
   for (int q = 0; q < kKeyedQuads; ++q) {
+    // phase A (no branches): four atomics in flight; exact zeros go to a dummy slot
     unsigned old[4];
-    unsigned grid_mask = 0;
+    unsigned any = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float x = v[q][k];
       bool on_grid;
-      const int idx = cell_index<kFast>(x, two_g, magic, c0f, &on_grid);
+      int pos = cell_position<kFast>(x, fn, &on_grid);
       const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
-      old[k] = 0;
-      if (nz) old[k] = atomicAdd(&cells[idx], 1u);
-      if (nz && on_grid) grid_mask |= 1u << k;
+      pos = nz ? pos : dummy_pos;
+      unsigned o = atomicAdd(&cells[pos], 1u);
+      o = (nz && on_grid) ? (o | kCellEdge) : o;   // an on-grid element is queued like an edge one
+      old[k] = o;
+      any |= o;
     }
+    // phase B: marked cells and on-grid elements (rare)
+    if (any >= kCellNearZero) {
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const unsigned o = old[k];
-      const bool on_grid = (grid_mask >> k) & 1u;
-      if (o >= kCellNearZero || on_grid) {
-        const float x = v[q][k];
-        if (o & kCellNearZero) count_zero_class(s_zclass, x);
-        if ((o & kCellEdge) || on_grid) {
-          const unsigned pos = atomicAdd(qcount, 1u);
-          if (pos < kQueueCap) queue[pos] = x;
-          else handle_special(c, x);          // queue full: do it now
+      for (int k = 0; k < 4; ++k) {
+        const unsigned o = old[k];
+        if (o >= kCellNearZero) {
+          const float x = v[q][k];
+          if (o & kCellNearZero) count_zero_class(s_zclass, x);
+          if (o & kCellEdge) {
+            const unsigned pos = atomicAdd(qcount, 1u);
+            if (pos < kQueueCap) queue[pos] = x;
+            else handle_special(c, x);          // queue full: do it now
+          }
         }
       }
     }
   }
   // drain full groups of 32 queued elements (dense lanes)
   __syncwarp();
-  unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
+  const unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
   __syncwarp();
   if (n >= 32u) {
     const int lane = threadIdx.x & 31;
@@ -228,14 +249,15 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
   __shared__ unsigned s_qcount[kKeyedWarps];
   __shared__ LayerCtx s_ctx;
 
-  unsigned* cells = reinterpret_cast<unsigned*>(s_raw);
-  unsigned* qe = cells + p.cell_cap;
+  unsigned* cells = reinterpret_cast<unsigned*>(s_raw);          // [cell_cap + kDummySlots]
+  unsigned* qe = cells + p.cell_cap + kDummySlots;
   int* dtab = reinterpret_cast<int*>(qe + p.n_bins);
   float* queues = reinterpret_cast<float*>(dtab + static_cast<size_t>(p.d_levels) * p.n_bins);
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* queue = queues + warp * kQueueCap;
   unsigned* qcount = &s_qcount[warp];
+  const int dummy_pos = p.cell_cap + lane;
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
@@ -246,35 +268,47 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
   while (t < t_end) {
     const LayerDesc L = p.layers[li];
     const int l = L.index;
-    const LayerState S = p.state[l];
-    const LayerPlan P = p.plan[l];
+    unsigned* const layer_u = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
+    __syncthreads();             // the previous layer's users of s_ctx are done
     if (threadIdx.x == 0) {
+      const LayerState S = p.state[l];
+      const LayerPlan* P = p.plan + l;
       LayerCtx c;
-      c.lo = S.lo; c.scale = S.scale; c.bmax = S.bmax;
-      c.two_g = P.two_g; c.c0f = P.c0f; c.c0 = P.c0; c.g = P.g; c.fs = P.fs;
+      c.lo = S.lo; c.scale = S.scale; c.bmax = S.bmax; c.radius = P->radius;
+      c.two_g[0] = P->seg[0].two_g; c.c0f[0] = P->seg[0].c0f; c.c0[0] = P->seg[0].c0;
+      c.g[0] = P->seg[0].g; c.fs[0] = P->seg[0].fs; c.offset[0] = P->seg[0].offset;
+      c.two_g[1] = P->seg[1].two_g; c.c0f[1] = P->seg[1].c0f; c.c0[1] = P->seg[1].c0;
+      c.g[1] = P->seg[1].g; c.fs[1] = P->seg[1].fs; c.offset[1] = P->seg[1].offset;
+      c.magic[0] = P->seg[0].magic; c.magic[1] = P->seg[1].magic;
+      c.keyed = P->keyed; c.fast = P->fast; c.total_cells = P->total_cells;
       c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
       c.cells = cells; c.qe = qe; c.d = dtab;
-      c.u_hist = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
+      c.qe_aux = p.qe_hist + (static_cast<size_t>(l) * 2 + 1) * p.n_bins;
+      c.u_hist = layer_u;
       c.zeros = p.zeros + static_cast<size_t>(l) * p.n_levels;
       c.n_bins = p.n_bins; c.n_levels = p.n_levels; c.d_levels = p.d_levels;
       s_ctx = c;
     }
-    const LayerCtx& c = s_ctx;   // read only after the barrier below
-    unsigned* const layer_u = p.u_hist + static_cast<size_t>(l) * p.n_levels * p.n_bins;
+    __syncthreads();
+    const LayerCtx& c = s_ctx;
     const long long layer_tiles_end = min(t_end, p.layers[li + 1].tile_begin);
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
-    const bool ok = P.keyed != 0;
-    // fast cell index when every cell index stays below 2^22 in magnitude
-    const bool fast = (P.c0 > -(1ll << 22)) && (P.c0 + P.cells < (1ll << 22));
-    const float magic = 12582912.0f - static_cast<float>(P.c0);
+    const bool ok = c.keyed != 0;
+    const bool fast = c.fast != 0;
+    const int total_cells = c.total_cells;
+    CellFn fn;
+    fn.radius = c.radius;
+    fn.two_g0 = c.two_g[0]; fn.magic0 = c.magic[0]; fn.c0f0 = c.c0f[0];
+    fn.two_g1 = c.two_g[1]; fn.magic1 = c.magic[1];
 
     // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
       const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-      for (int i = threadIdx.x; i < P.cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
+      for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
       for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
+      if (threadIdx.x < kDummySlots) cells[p.cell_cap + threadIdx.x] = 0;
       if (lane == 0) *qcount = 0;
     }
     __syncthreads();
@@ -284,11 +318,11 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       const long long j_tile = (t - L.tile_begin) * kKeyedTile;
       const bool full = (j_tile >= jbeg) && (j_tile + kKeyedTile <= jend);
       if (fast) {
-        if (full) keyed_tile<true, true>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
-        else keyed_tile<true, false>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
+        if (full) keyed_tile<true, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
+        else keyed_tile<true, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
       } else {
-        if (full) keyed_tile<false, true>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
-        else keyed_tile<false, false>(c, cells, s_zclass, queue, qcount, P.two_g, P.c0f, magic, base, j_tile, jbeg, jend);
+        if (full) keyed_tile<false, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
+        else keyed_tile<false, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
       }
     }
     // ---- what is left in the queues ----------------------------------------------
@@ -302,11 +336,11 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     // ---- flush the private tables into the layer's global ones -----------------------
     if (ok) {
       unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
-      for (int i = threadIdx.x; i < P.cells; i += kKeyedThreads) {
+      for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) {
         const unsigned n = cells[i] & kCellCountMask;
         if (n) atomicAdd(&gc[i], n);
       }
-      unsigned* gq = p.qe_hist + static_cast<size_t>(l) * p.n_bins;
+      unsigned* gq = p.qe_hist + static_cast<size_t>(l) * 2 * p.n_bins;
       for (int i = threadIdx.x; i < p.n_bins; i += kKeyedThreads) {
         const unsigned n = qe[i];
         if (n) atomicAdd(&gq[i], n);
@@ -315,7 +349,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
         const int dv = dtab[i];
         if (dv) {
           const int j = i / p.n_bins, b = i - j * p.n_bins;
-          const int f = P.fs + j;
+          const int f = c.fs[0] + j;
           if (f < p.n_levels)
             atomicAdd(&layer_u[static_cast<size_t>(f) * p.n_bins + b], static_cast<unsigned>(dv));
         }
