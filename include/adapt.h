@@ -210,6 +210,50 @@ int adapt_kernel_timing(int enable);
  *   reset                 non-zero clears the accumulators after reading */
 int adapt_kernel_times(double* ms_out, uint64_t* launches_out, int reset);
 
+/* Limits of adapt_precision_search_static. */
+#define ADAPT_STATIC_MAX_LAYERS 8
+#define ADAPT_STATIC_MAX_BINS 512
+#define ADAPT_STATIC_MAX_CAND 1024
+
+/* The search for callers that must not allocate.  (The paper has no
+ * counterpart: this entry point exists for the way the library is embedded,
+ * not for the method.)
+ *
+ * Some hosts of this library cannot let it call cudaMalloc: a training process
+ * that has handed all device memory to its own pool, so that a late cudaMalloc
+ * fails or eats into that pool's head-room; a service with a fixed memory
+ * budget that is audited at start-up; a step loop in which the implicit
+ * device-wide synchronisation of cudaMalloc / cudaFree would stall every other
+ * stream.  The other search calls either grow a library-owned buffer or need a
+ * caller workspace sized by a query; this one needs neither.
+ *
+ * It computes exactly what adapt_precision_search computes (round-to-nearest-
+ * even, eps 0, bits; same argument meaning, same outputs, same flags), using
+ * the direct form of the fused kernel, with all scratch in one fixed array
+ * that is part of the library image: about 0.6 MB of device memory on every
+ * GPU that loads the library, held until the process exits.  It calls no
+ * cudaMalloc, cudaMallocHost, cudaFree or other allocating routine and creates
+ * no events or streams.
+ *
+ *   stream  cudaStream_t or NULL (legacy default stream); kernels and the two
+ *           small copies are enqueued there, results are valid after it syncs.
+ * Sizes beyond the fixed scratch - more than ADAPT_STATIC_MAX_LAYERS layers,
+ * ADAPT_STATIC_MAX_CAND candidates or ADAPT_STATIC_MAX_BINS bins - return
+ * ADAPT_ERR_WORKSPACE before anything is launched, with the limits spelled out
+ * in adapt_last_error().  Layer lengths are not limited (below 2^32 each).
+ *
+ * The first call on a device looks up the scratch array's device address
+ * (cudaGetSymbolAddress, with that device current) and keeps it; make that
+ * first call before any stream capture begins.
+ * Every call uses the same array and clears the parts that must start at zero,
+ * so calls that can overlap on the GPU (different streams, different host
+ * threads) race with each other: issue them on one stream or order them with
+ * events. */
+int adapt_precision_search_static(const float* const* tensors, const int64_t* lens,
+                                  int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                                  double* kld_out, int64_t* zeros_out, int32_t* best_out,
+                                  void* stream);
+
 /* Frees every library-owned device and pinned buffer of the current device's
  * caches.  Safe to call at any time no library work is in flight. */
 int adapt_release(void);

@@ -27,8 +27,9 @@ EXPORTS = (
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_search_workspace_bytes",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
-    "adapt_kernel_times", "adapt_release",
+    "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
 )
+STATIC_MAX_LAYERS, STATIC_MAX_BINS, STATIC_MAX_CAND = 8, 512, 1024
 KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize", "plan",
                 "expand", "search_direct")
 ALGO_AUTO, ALGO_KEYED, ALGO_DIRECT = 0, 1, 2
@@ -89,6 +90,8 @@ def lib():
         L.adapt_precision_search_ex.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
         L.adapt_precision_search_host.restype = C.c_int
         L.adapt_precision_search_host.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
+        L.adapt_precision_search_static.restype = C.c_int
+        L.adapt_precision_search_static.argtypes = search_args + [C.c_void_p]
         L.adapt_quantize_host.restype = C.c_int
         L.adapt_quantize_host.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int,
                                           C.c_uint64, C.c_int32, C.c_int, C.c_void_p]
@@ -232,6 +235,25 @@ def adapt_precision_search(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: 
     _check(lib().adapt_precision_search(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
                                         n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
                                         out.best.data_ptr()), "adapt_precision_search")
+    return out
+
+
+def adapt_precision_search_static(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                                  out: SearchResult, stream=None) -> SearchResult:
+    """adapt_precision_search_static of adapt.h: the search with all scratch in a fixed
+    array inside the library.  ``out`` must be passed in (this wrapper allocates nothing
+    on the device either); sizes beyond the STATIC_MAX_* limits raise ERR_WORKSPACE."""
+    assert all(t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    st = lib().adapt_precision_search_static(ptrs.ctypes.data, lens.ctypes.data, len(tensors),
+                                             C.byref(grid.c), n_bins, out.kld.data_ptr(),
+                                             out.zeros.data_ptr(), out.best.data_ptr(),
+                                             _stream_handle(stream))
+    if st == ERR_WORKSPACE:
+        err = AdaptError(st, "adapt_precision_search_static")
+        err.args = (err.args[0] + " (" + lib().adapt_last_error().decode() + ")",)
+        raise err
+    _check(st, "adapt_precision_search_static")
     return out
 
 

@@ -75,6 +75,13 @@ int cuda_fail(cudaError_t e, const char* what) {
     if (e_ != cudaSuccess) return cuda_fail(e_, #call);      \
   } while (0)
 
+// after a kernel launch: report which launch was refused
+#define ADAPT_LAUNCH_OK(what)                                \
+  do {                                                       \
+    cudaError_t e_ = cudaGetLastError();                     \
+    if (e_ != cudaSuccess) return cuda_fail(e_, what);       \
+  } while (0)
+
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // ---- per-device caches --------------------------------------------------------
@@ -681,6 +688,178 @@ int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mod
   if (rc != ADAPT_OK) return rc;
   ADAPT_CUDA(cudaMemcpyAsync(codes_out, dc->stage_out, out_bytes, cudaMemcpyDeviceToHost, nullptr));
   ADAPT_CUDA(cudaStreamSynchronize(nullptr));
+  return ADAPT_OK;
+}
+
+// ---- search without any allocation ------------------------------------------------
+//
+// Scratch of adapt_precision_search_static: one fixed device array, part of the library
+// image, so every GPU that loads the library holds it until the process exits.
+
+}  // extern "C"
+
+namespace {
+
+constexpr int kStaticMaxLayers = ADAPT_STATIC_MAX_LAYERS;
+constexpr int kStaticMaxBins = ADAPT_STATIC_MAX_BINS;
+constexpr int kStaticMaxCand = ADAPT_STATIC_MAX_CAND;
+
+// layout (bytes): descriptor block, then the accumulators that every call clears
+constexpr size_t kStLayers = 0;                                                   // LayerDesc[L + 1]
+constexpr size_t kStWl = kStLayers + 64 * (kStaticMaxLayers + 1);
+constexpr size_t kStFl = kStWl + 4 * kStaticMaxCand;
+constexpr size_t kStSlot = kStFl + 4 * kStaticMaxCand;
+constexpr size_t kStOrder = kStSlot + 4 * kStaticMaxCand;
+constexpr size_t kStState = kStOrder + 4 * kStaticMaxCand;                        // LayerState[L]
+constexpr size_t kStBlobEnd = kStState + 64 * kStaticMaxLayers;
+constexpr size_t kStZeros = (kStBlobEnd + 255) / 256 * 256;                       // u64[L][32]
+constexpr size_t kStQ = kStZeros + 8 * kStaticMaxLayers * kMaxFl;                 // u32[L][B]
+constexpr size_t kStU = kStQ + 4 * static_cast<size_t>(kStaticMaxLayers) * kStaticMaxBins;
+constexpr size_t kStEnd = kStU + 4 * static_cast<size_t>(kStaticMaxLayers) * kMaxFl * kStaticMaxBins;
+static_assert(sizeof(LayerDesc) <= 64 && sizeof(LayerState) <= 64, "descriptor slots too small");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStEnd];
+
+// The array's name is only a host-side handle; kernels need its device address, looked up
+// once per device (with that device current) and kept here.
+unsigned char* g_static_ptr[kMaxDevices] = {nullptr};
+unsigned char g_static_blob[kStBlobEnd];   // host image of the descriptor block (under g_mutex)
+
+int static_scratch_address(unsigned char** out) {
+  int dev = 0;
+  ADAPT_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) {
+    std::snprintf(g_last_error, sizeof(g_last_error), "device index %d not supported", dev);
+    return ADAPT_ERR_CUDA;
+  }
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    ADAPT_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+    g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+  }
+  *out = g_static_ptr[dev];
+  return ADAPT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int adapt_precision_search_static(const float* const* tensors, const int64_t* lens, int n_layers,
+                                  const adapt_grid* grid, int n_bins, double* kld_out,
+                                  int64_t* zeros_out, int32_t* best_out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!tensors || !lens || !grid || !grid->wl || !grid->fl || !kld_out || !zeros_out || !best_out)
+    return ADAPT_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > kStaticMaxLayers || grid->n_cand < 1 ||
+      grid->n_cand > kStaticMaxCand || n_bins < 1 || n_bins > kStaticMaxBins) {
+    std::snprintf(g_last_error, sizeof(g_last_error),
+                  "adapt_precision_search_static: sizes beyond the fixed scratch (at most %d layers, "
+                  "%d candidates, %d bins; got %d, %d, %d)", kStaticMaxLayers, kStaticMaxCand,
+                  kStaticMaxBins, n_layers, grid->n_cand, n_bins);
+    return ADAPT_ERR_WORKSPACE;
+  }
+  int fmax = 0;
+  for (int c = 0; c < grid->n_cand; ++c) {
+    if (!valid_format(grid->wl[c], grid->fl[c])) return ADAPT_ERR_INVALID_ARG;
+    fmax = std::max(fmax, grid->fl[c]);
+  }
+  for (int l = 0; l < n_layers; ++l) {
+    if (lens[l] < 0 || lens[l] >= (1ll << 32)) return ADAPT_ERR_INVALID_ARG;
+    if (lens[l] > 0 && !tensors[l]) return ADAPT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(tensors[l]) & 3u) return ADAPT_ERR_INVALID_ARG;
+  }
+  const int n_levels = fmax + 1, C = grid->n_cand;
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  unsigned char* ws = nullptr;
+  rc = static_scratch_address(&ws);
+  if (rc != ADAPT_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+
+  // descriptor block: layer list, candidates (slot = FL, order by (WL, FL, index)), fresh state
+  unsigned char* h = g_static_blob;
+  std::memset(h, 0, kStBlobEnd);
+  LayerDesc* hl = reinterpret_cast<LayerDesc*>(h + kStLayers);
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(tensors[l]) >> 2) & 3u);
+    hl[l].ptr = tensors[l]; hl[l].n = lens[l]; hl[l].tile_begin = tiles;
+    hl[l].mis = lens[l] > 0 ? mis : 0; hl[l].layer_id = l; hl[l].index = l;
+    if (lens[l] > 0) tiles += (lens[l] + mis + kTile - 1) / kTile;
+  }
+  hl[n_layers].tile_begin = tiles;
+  int* h_wl = reinterpret_cast<int*>(h + kStWl);
+  int* h_fl = reinterpret_cast<int*>(h + kStFl);
+  int* h_slot = reinterpret_cast<int*>(h + kStSlot);
+  int* h_order = reinterpret_cast<int*>(h + kStOrder);
+  for (int c = 0; c < C; ++c) { h_wl[c] = grid->wl[c]; h_fl[c] = grid->fl[c]; h_slot[c] = grid->fl[c]; h_order[c] = c; }
+  std::stable_sort(h_order, h_order + C, [&](int a, int b) {
+    if (grid->wl[a] != grid->wl[b]) return grid->wl[a] < grid->wl[b];
+    return grid->fl[a] < grid->fl[b];
+  });
+  LayerState* hs = reinterpret_cast<LayerState*>(h + kStState);
+  for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+
+  // the block is ordinary host memory: the copy is staged before the call returns
+  ADAPT_CUDA(cudaMemcpyAsync(ws, h, kStBlobEnd, cudaMemcpyHostToDevice, stream));
+  // the scratch keeps the previous call's counts: clear every accumulator
+  ADAPT_CUDA(cudaMemsetAsync(ws + kStZeros, 0, kStEnd - kStZeros, stream));
+
+  const LayerDesc* d_layers = reinterpret_cast<const LayerDesc*>(ws + kStLayers);
+  LayerState* d_state = reinterpret_cast<LayerState*>(ws + kStState);
+  unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + kStZeros);
+  unsigned* d_q = reinterpret_cast<unsigned*>(ws + kStQ);
+  unsigned* d_u = reinterpret_cast<unsigned*>(ws + kStU);
+
+  if (tiles > 0) {
+    const int g = static_cast<int>(std::min<long long>(tiles, 8ll * dc->sm_count));
+    range_scan_kernel<<<g, kRangeThreads, 0, stream>>>(d_layers, n_layers, tiles, d_state);
+    ADAPT_LAUNCH_OK("range scan launch");
+    ++g_launches;
+  }
+  range_finalize_kernel<<<1, 128, 0, stream>>>(d_layers, n_layers, n_bins, d_state, nullptr);
+  ADAPT_LAUNCH_OK("range finalize launch");
+  ++g_launches;
+  if (tiles > 0) {
+    SearchParams sp;
+    sp.layers = d_layers; sp.state = d_state; sp.n_layers = n_layers; sp.n_fl = n_levels;
+    sp.n_bins = n_bins; sp.n_tiles = tiles; sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros;
+    sp.seed = 0;
+    const size_t per_hist = sizeof(unsigned) * n_bins;
+    int fg = static_cast<int>((40 * 1024) / per_hist) - 1;   // stays under the 48 KB default limit
+    fg = std::max(1, std::min(fg, n_levels));
+    sp.fl_per_group = fg;
+    const int groups = (n_levels + fg - 1) / fg;
+    const size_t smem = per_hist * (fg + 1);
+    dim3 g(static_cast<unsigned>(std::min<long long>(tiles, 4ll * dc->sm_count)), groups);
+    // the other search calls leave their own dynamic shared-memory limit on this kernel
+    // (possibly a smaller one): state the one this launch needs (not an allocation)
+    ADAPT_CUDA(cudaFuncSetAttribute(search_direct_kernel<false>,
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(smem)));
+    search_direct_kernel<false><<<g, kSearchThreads, smem, stream>>>(sp);
+    ADAPT_LAUNCH_OK("direct search launch");
+    ++g_launches;
+  }
+  KldParams kp;
+  kp.layers = d_layers; kp.state = d_state;
+  kp.cand_wl = reinterpret_cast<const int*>(ws + kStWl);
+  kp.cand_fl = reinterpret_cast<const int*>(ws + kStFl);
+  kp.cand_slot = reinterpret_cast<const int*>(ws + kStSlot);
+  kp.cand_order = reinterpret_cast<const int*>(ws + kStOrder);
+  kp.n_layers = n_layers; kp.n_cand = C; kp.n_fl = n_levels; kp.n_bins = n_bins;
+  kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
+  kp.alpha = 0.0; kp.inv_ln_base = 1.0 / std::log(2.0); kp.eps = 0.0;
+  kp.kld_out = kld_out; kp.zeros_out = reinterpret_cast<long long*>(zeros_out);
+  kp.best_out = best_out; kp.hist_out = nullptr;
+  kld_kernel<<<dim3(C, n_layers), kKldThreads, 0, stream>>>(kp);
+  ADAPT_LAUNCH_OK("kld launch");
+  ++g_launches;
+  select_kernel<<<n_layers, 32, 0, stream>>>(kp);
+  ADAPT_LAUNCH_OK("select launch");
+  ++g_launches;
   return ADAPT_OK;
 }
 
