@@ -146,9 +146,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
         const float r = pow2f(rexp);
         if (r < 0.25f * amax) {
           SegPlan aux, main;
-          fit_segment(S.lo, S.hi, cap / 4, g_want, &aux);
+          // the main segment takes what it needs (up to three quarters), the rest is auxiliary
           const float mlo = fmaxf(S.lo, -r), mhi = fminf(S.hi, r);
-          fit_segment(mlo, mhi, cap - aux.cells, g_want, &main);
+          fit_segment(mlo, mhi, cap - cap / 4, g_want, &main);
+          fit_segment(S.lo, S.hi, cap - main.cells, g_want, &aux);
           // the auxiliary cells next to zero must stay empty: R at least two of them wide
           if (main.g > P.seg[0].g + 1 && r > pow2f(-aux.g)) {
             P.seg[0] = main; P.seg[1] = aux; P.radius = r;

@@ -20,8 +20,9 @@
 // derived from the cell counts by the expand kernel.
 //
 // One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
-// for its tables; each thread keeps 16 elements (four 128-bit loads) in flight
-// per tile.
+// for its tables; each thread handles 16 elements (four 128-bit loads) per tile
+// and refills a quad's registers with the next tile's quad as soon as the quad
+// has been used, so loads stay in flight while elements are processed.
 #pragma once
 
 #include "common.cuh"
@@ -175,21 +176,28 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_
   return __float2int_rz(__fsub_rn(cf, f.c0f0));
 }
 
+// One tile.  v holds this thread's elements of the tile when `loaded`; otherwise they are
+// fetched here (guarded loads when the tile is ragged).  As soon as a quad has been used its
+// registers are refilled with the same quad of the next tile (`next`, non-null only when that
+// tile is a full tile of the same layer), so loads stay in flight while elements are processed.
 template <bool kFast, bool kFull>
 __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, int dummy_pos,
                                            unsigned* s_zclass, float* queue, unsigned* qcount,
                                            const CellFn& fn, const float* base, long long j_tile,
-                                           long long jbeg, long long jend) {
-  float v[kKeyedQuads][4];
+                                           long long jbeg, long long jend,
+                                           float (&v)[kKeyedQuads][4], bool loaded,
+                                           const float4* src, const float4* next) {
   unsigned vm[kKeyedQuads];
 #pragma unroll
   for (int q = 0; q < kKeyedQuads; ++q) {
-    const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
-    if (kFull) {
-      const float4 t = __ldcs(reinterpret_cast<const float4*>(base + j0));
-      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
+    if (kFull) {      // src = this thread's first quad of the tile
+      if (!loaded) {
+        const float4 t = __ldcs(src + q * kKeyedThreads);
+        v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
+      }
       vm[q] = 0xFu;
     } else {
+      const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
       vm[q] = 0;
       v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
       if (j0 < jend) vm[q] = load_quad(base, j0, jbeg, jend, v[q]);
@@ -203,12 +211,25 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float x = v[q][k];
-      bool on_grid;
-      int pos = cell_position<kFast>(x, fn, &on_grid);
-      const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
-      pos = nz ? pos : dummy_pos;
-      unsigned o = atomicAdd(&cells[pos], 1u);
-      o = (nz && on_grid) ? (o | kCellEdge) : o;   // an on-grid element is queued like an edge one
+      unsigned o;
+      if (kFast && kFull) {
+        // both segments' products are formed (FMA pipe) and one is kept, instead of selecting
+        // scale and constant first (two selects on the narrower ALU pipe)
+        const bool inner = fabsf(x) < fn.radius;
+        const float rd = inner ? __fmaf_rd(x, fn.two_g0, fn.magic0) : __fmaf_rd(x, fn.two_g1, fn.magic1);
+        const float ru = inner ? __fmaf_ru(x, fn.two_g0, fn.magic0) : __fmaf_ru(x, fn.two_g1, fn.magic1);
+        const bool nz = (x != 0.0f);
+        const int pos = nz ? (__float_as_int(rd) - 0x4B400000) : dummy_pos;
+        o = atomicAdd(&cells[pos], 1u);
+        o = (nz && rd == ru) ? (o | kCellEdge) : o;
+      } else {
+        bool on_grid;
+        int pos = cell_position<kFast>(x, fn, &on_grid);
+        const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
+        pos = nz ? pos : dummy_pos;
+        o = atomicAdd(&cells[pos], 1u);
+        o = (nz && on_grid) ? (o | kCellEdge) : o;   // an on-grid element is queued like an edge one
+      }
       old[k] = o;
       any |= o;
     }
@@ -228,6 +249,11 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
         }
       }
     }
+    // this quad's registers are free: start the next tile's quad
+    if (kFull && next != nullptr) {
+      const float4 t = __ldcs(next + q * kKeyedThreads);
+      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
+    }
   }
   // drain full groups of 32 queued elements (dense lanes)
   __syncwarp();
@@ -241,6 +267,38 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
     if (lane == 0) *qcount = n & 31u;
     __syncwarp();
   }
+}
+
+// All tiles [k0, k1) of one layer that this CTA owns (k counts the layer's own tiles).  Only
+// the layer's first tile (when the tensor does not start on a 16-byte boundary) and its last
+// tile can be ragged; every tile between runs through a loop that carries one running pointer.
+template <bool kFast>
+__device__ __forceinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                              unsigned* s_zclass, float* queue, unsigned* qcount,
+                                              const CellFn& fn, const float* base, long long jbeg,
+                                              long long jend, int k0, int k1) {
+  float v[kKeyedQuads][4];
+  const int kf0 = max(k0, jbeg > 0 ? 1 : 0);
+  const int kf1 = min(k1, static_cast<int>(jend / kKeyedTile));
+  if (k0 < kf0)
+    keyed_tile<kFast, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base,
+                             static_cast<long long>(k0) * kKeyedTile, jbeg, jend, v, false, nullptr,
+                             nullptr);
+  if (kf0 < kf1) {
+    const float4* src = reinterpret_cast<const float4*>(base + static_cast<long long>(kf0) * kKeyedTile) +
+                        threadIdx.x;
+    bool loaded = false;
+    for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4) {
+      const float4* next = (k + 1 < kf1) ? src + kKeyedTile / 4 : nullptr;
+      keyed_tile<kFast, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, 0, 0, 0, v,
+                              loaded, src, next);
+      loaded = true;
+    }
+  }
+  for (int k = max(kf1, kf0); k < k1; ++k)
+    keyed_tile<kFast, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base,
+                             static_cast<long long>(k) * kKeyedTile, jbeg, jend, v, false, nullptr,
+                             nullptr);
 }
 
 __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const KeyedParams p) {
@@ -313,18 +371,12 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     }
     __syncthreads();
 
-    for (; t < layer_tiles_end; ++t) {
-      if (!ok) continue;
-      const long long j_tile = (t - L.tile_begin) * kKeyedTile;
-      const bool full = (j_tile >= jbeg) && (j_tile + kKeyedTile <= jend);
-      if (fast) {
-        if (full) keyed_tile<true, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
-        else keyed_tile<true, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
-      } else {
-        if (full) keyed_tile<false, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
-        else keyed_tile<false, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, j_tile, jbeg, jend);
-      }
+    if (ok) {
+      const int k0 = static_cast<int>(t - L.tile_begin), k1 = static_cast<int>(layer_tiles_end - L.tile_begin);
+      if (fast) keyed_segment<true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, jbeg, jend, k0, k1);
+      else keyed_segment<false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, jbeg, jend, k0, k1);
     }
+    t = layer_tiles_end;
     // ---- what is left in the queues ----------------------------------------------
     if (ok) {
       __syncwarp();
