@@ -4,10 +4,11 @@
 //
 // Per element x != 0:   pos = table position of x's cell;  old = atomicAdd(cell[pos], 1)
 // The returned word carries the cell's marks in its two top bits:
-//   bit 30 (cell -1 / 0 of the main segment): the element is added to the class
-//          counter "highest level at which it still rounds to zero";
-//   bit 31 (edge cell), or x exactly on its segment's grid: the element goes to a
-//          per-warp queue that the warp drains 32 entries at a time:
+//   bit 30 (cell -1 / 0 of the main segment), bit 31 (edge cell), or x exactly on its
+//          segment's grid: the element goes to a per-warp queue that the warp drains
+//          32 entries at a time:
+//            cell -1 / 0: the element is added to the class counter "highest level at
+//              which it still rounds to zero";
 //            edge entry: b0 = bin(x) into the segment's edge-element histogram,
 //              then only the fine levels f whose half quantum can reach one of
 //              the bin's edges are evaluated; a level is recorded only if its
@@ -35,7 +36,7 @@ constexpr int kKeyedThreads = 1024;
 constexpr int kKeyedWarps = kKeyedThreads / 32;
 constexpr int kKeyedQuads = 4;                                  // 128-bit loads per thread per tile
 constexpr int kKeyedTile = kKeyedThreads * kKeyedQuads * 4;     // 16384 elements
-constexpr int kQueueCap = 96;       // per-warp queue entries; a full queue handles entries inline
+constexpr int kQueueCap = 160;      // per-warp queue entries: under 32 left over + at most 128 from one quad
 constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..32
 constexpr int kDummySlots = 32;     // where the atomics of exact zeros land (one per lane)
 
@@ -78,6 +79,7 @@ struct LayerCtx {
   unsigned* qe_aux;            // global [n_bins]: auxiliary segment's edge-element histogram
   unsigned* u_hist;            // global, this layer's [n_levels][n_bins]
   unsigned long long* zeros;   // global, this layer's [n_levels]
+  unsigned* zclass;            // shared [kZeroClasses]
   int n_bins, n_levels, d_levels;
   float magic[2];
   int keyed, fast, total_cells;
@@ -92,9 +94,17 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   const float cf = floorf(z);
   const int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s]));   // cell index inside the segment
   const int g = c.g[s];
+  const long long cc = c.c0[s] + ci;
+  // ---- cells -1 / 0 of the main segment: the zero class of x --------------------------
+  if (s == 0 && (cc == 0 || cc == -1)) {
+    // highest level k at which x still rounds to zero: |x| <= 2^-(k+1)
+    const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
+    int kz = 125 - static_cast<int>((ax - 1u) >> 23);
+    kz = max(-1, min(kz, 32));
+    atomicAdd(&c.zclass[kz + 1], 1u);
+  }
   // ---- x on the segment's grid: fix the single coarse level at which it is a tie ----
   if (z == cf) {
-    const long long cc = c.c0[s] + ci;
     if (cc != 0) {
       const int tz = __ffsll(cc) - 1;          // lowest set bit
       const int ft = g - 1 - tz;               // the level at which x is a tie
@@ -140,15 +150,6 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   }
 }
 
-// Adds a near-zero element (cells -1 / 0 of the main segment) to its zero class.
-__device__ __forceinline__ void count_zero_class(unsigned* s_zclass, float x) {
-  // highest level k at which x still rounds to zero: |x| <= 2^-(k+1)
-  const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
-  int kz = 125 - static_cast<int>((ax - 1u) >> 23);
-  kz = max(-1, min(kz, 32));
-  atomicAdd(&s_zclass[kz + 1], 1u);
-}
-
 // The constants one tile needs to place an element in the table.
 struct CellFn {
   float radius;
@@ -182,7 +183,7 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_
 // tile is a full tile of the same layer), so loads stay in flight while elements are processed.
 template <bool kFast, bool kFull>
 __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                           unsigned* s_zclass, float* queue, unsigned* qcount,
+                                           float* queue, unsigned& qn,
                                            const CellFn& fn, const float* base, long long j_tile,
                                            long long jbeg, long long jend,
                                            float (&v)[kKeyedQuads][4], bool loaded,
@@ -233,20 +234,26 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
       old[k] = o;
       any |= o;
     }
-    // phase B: marked cells and on-grid elements (rare)
-    if (any >= kCellNearZero) {
+    // phase B (rare): elements of marked cells and on-grid elements join the warp's queue;
+    // the whole warp enters so that the queue position can stay in a register
+    if (__any_sync(0xffffffffu, any >= kCellNearZero)) {
+      const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const unsigned o = old[k];
-        if (o >= kCellNearZero) {
-          const float x = v[q][k];
-          if (o & kCellNearZero) count_zero_class(s_zclass, x);
-          if (o & kCellEdge) {
-            const unsigned pos = atomicAdd(qcount, 1u);
-            if (pos < kQueueCap) queue[pos] = x;
-            else handle_special(c, x);          // queue full: do it now
-          }
+        const bool push = old[k] >= kCellNearZero;
+        const unsigned pm = __ballot_sync(0xffffffffu, push);
+        if (pm) {
+          if (push) queue[qn + __popc(pm & lt)] = v[q][k];
+          qn += __popc(pm);
         }
+      }
+      if (qn >= 32u) {           // drain full groups of 32 (dense lanes)
+        __syncwarp();
+        do {
+          qn -= 32u;
+          handle_special(c, queue[qn + (threadIdx.x & 31)]);
+        } while (qn >= 32u);
+        __syncwarp();
       }
     }
     // this quad's registers are free: start the next tile's quad
@@ -255,18 +262,6 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
       v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
     }
   }
-  // drain full groups of 32 queued elements (dense lanes)
-  __syncwarp();
-  const unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
-  __syncwarp();
-  if (n >= 32u) {
-    const int lane = threadIdx.x & 31;
-    const unsigned groups = n >> 5;
-    for (unsigned gq = 0; gq < groups; ++gq) handle_special(c, queue[n - 32u * (gq + 1) + lane]);
-    __syncwarp();
-    if (lane == 0) *qcount = n & 31u;
-    __syncwarp();
-  }
 }
 
 // All tiles [k0, k1) of one layer that this CTA owns (k counts the layer's own tiles).  Only
@@ -274,14 +269,15 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
 // tile can be ragged; every tile between runs through a loop that carries one running pointer.
 template <bool kFast>
 __device__ __forceinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                              unsigned* s_zclass, float* queue, unsigned* qcount,
+                                              float* queue,
                                               const CellFn& fn, const float* base, long long jbeg,
                                               long long jend, int k0, int k1) {
   float v[kKeyedQuads][4];
+  unsigned qn = 0;             // entries in this warp's queue (same in every lane)
   const int kf0 = max(k0, jbeg > 0 ? 1 : 0);
   const int kf1 = min(k1, static_cast<int>(jend / kKeyedTile));
   if (k0 < kf0)
-    keyed_tile<kFast, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base,
+    keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
                              static_cast<long long>(k0) * kKeyedTile, jbeg, jend, v, false, nullptr,
                              nullptr);
   if (kf0 < kf1) {
@@ -290,21 +286,23 @@ __device__ __forceinline__ void keyed_segment(const LayerCtx& c, unsigned* cells
     bool loaded = false;
     for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4) {
       const float4* next = (k + 1 < kf1) ? src + kKeyedTile / 4 : nullptr;
-      keyed_tile<kFast, true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, 0, 0, 0, v,
+      keyed_tile<kFast, true>(c, cells, dummy_pos, queue, qn, fn, base, 0, 0, 0, v,
                               loaded, src, next);
       loaded = true;
     }
   }
   for (int k = max(kf1, kf0); k < k1; ++k)
-    keyed_tile<kFast, false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base,
+    keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
                              static_cast<long long>(k) * kKeyedTile, jbeg, jend, v, false, nullptr,
                              nullptr);
+  // what is left in the queue
+  __syncwarp();
+  if ((threadIdx.x & 31) < qn) handle_special(c, queue[threadIdx.x & 31]);
 }
 
 __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const KeyedParams p) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ unsigned s_zclass[kZeroClasses];
-  __shared__ unsigned s_qcount[kKeyedWarps];
   __shared__ LayerCtx s_ctx;
 
   unsigned* cells = reinterpret_cast<unsigned*>(s_raw);          // [cell_cap + kDummySlots]
@@ -314,7 +312,6 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* queue = queues + warp * kQueueCap;
-  unsigned* qcount = &s_qcount[warp];
   const int dummy_pos = p.cell_cap + lane;
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
@@ -340,7 +337,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.magic[0] = P->seg[0].magic; c.magic[1] = P->seg[1].magic;
       c.keyed = P->keyed; c.fast = P->fast; c.total_cells = P->total_cells;
       c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
-      c.cells = cells; c.qe = qe; c.d = dtab;
+      c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
       c.qe_aux = p.qe_hist + (static_cast<size_t>(l) * 2 + 1) * p.n_bins;
       c.u_hist = layer_u;
       c.zeros = p.zeros + static_cast<size_t>(l) * p.n_levels;
@@ -367,22 +364,15 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
       if (threadIdx.x < kDummySlots) cells[p.cell_cap + threadIdx.x] = 0;
-      if (lane == 0) *qcount = 0;
     }
     __syncthreads();
 
     if (ok) {
       const int k0 = static_cast<int>(t - L.tile_begin), k1 = static_cast<int>(layer_tiles_end - L.tile_begin);
-      if (fast) keyed_segment<true>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, jbeg, jend, k0, k1);
-      else keyed_segment<false>(c, cells, dummy_pos, s_zclass, queue, qcount, fn, base, jbeg, jend, k0, k1);
+      if (fast) keyed_segment<true>(c, cells, dummy_pos, queue, fn, base, jbeg, jend, k0, k1);
+      else keyed_segment<false>(c, cells, dummy_pos, queue, fn, base, jbeg, jend, k0, k1);
     }
     t = layer_tiles_end;
-    // ---- what is left in the queues ----------------------------------------------
-    if (ok) {
-      __syncwarp();
-      const unsigned n = min(*qcount, static_cast<unsigned>(kQueueCap));
-      if (static_cast<unsigned>(lane) < n) handle_special(c, queue[lane]);
-    }
     __syncthreads();
 
     // ---- flush the private tables into the layer's global ones -----------------------
