@@ -37,7 +37,7 @@ TRAFFIC_CAPTURE = {"version": None, "bytes_per_element": None}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="stress_1g")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -52,8 +52,10 @@ def parse_args():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples SM clocks and throttle reasons with nvidia-smi.  It is started before the
+    warm-up (nvidia-smi takes a moment to come up) and keeps only the samples whose
+    timestamps fall inside the timed region."""
+    Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -66,7 +68,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -75,11 +77,12 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t0: float, t1: float):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -87,15 +90,17 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for stamp, ln in self.lines:
+            if not (t0 <= stamp <= t1 + 0.06):     # a sample is read up to one period late
+                continue
             f = [t.strip() for t in ln.split(",")]
-            if len(f) < 9:
+            if len(f) < 10:
                 continue
             try:
-                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+                sm.append(float(f[2])); mx.append(float(f[3])); power.append(float(f[4]))
             except ValueError:
                 continue
-            for name, val in zip(names, f[5:9]):
+            for name, val in zip(names, f[6:10]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
@@ -226,22 +231,21 @@ def main():
     def step():
         B.adapt_precision_search_ex(xs, grid, w.n_bins, round_mode=w.round_mode, seed=w.seed,
                                     workspace=ws, out=out)
-        for l, x in enumerate(xs):
-            if lens[l]:
-                B.adapt_quantize_selected(x, out.best[l], w.round_mode, w.seed, l, codes_out=codes[l])
+        B.adapt_quantize_selected_batch(xs, out.best, w.round_mode, w.seed, 0, codes_out=codes)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
 
     # ---- device-resident timing -------------------------------------------------
-    sampler = ClockSampler(local_rank)
     S.barrier()
     torch.cuda.synchronize()
     B.adapt_kernel_times(reset=True)
     B.adapt_kernel_timing(True)
     launches0 = B.adapt_kernel_launch_count()
-    sampler.start()
+    t_region0 = time.time()
     fits_l2 = 4 * total <= 2 * 126e6
     if not fits_l2:
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -265,8 +269,9 @@ def main():
         torch.cuda.synchronize()
         secs = sum(a.elapsed_time(b) for a, b in evs) * 1e-3
         del flush
+    t_region1 = time.time()
     S.barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_region0, t_region1)
     launches = B.adapt_kernel_launch_count() - launches0
     B.adapt_kernel_timing(False)
     ktimes = B.adapt_kernel_times(reset=True)
@@ -336,7 +341,7 @@ def main():
                            "elements_per_gpu": total, "layers": len(xs), "candidates": n_cand,
                            "n_bins": w.n_bins,
                            "round_mode": "rne" if w.round_mode == 0 else "stochastic",
-                           "step": "adapt_precision_search_ex + adapt_quantize_selected per layer",
+                           "step": "adapt_precision_search_ex + adapt_quantize_selected_batch",
                            "l2": "inputs exceed L2" if not fits_l2 else
                                  "L2 flushed (512 MiB write) between timed steps",
                            "parallelism": f"independent layer sets x{world}, no collective"},

@@ -128,6 +128,22 @@ int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected,
                             int round_mode, uint64_t seed, int32_t layer,
                             int32_t* codes_out, void* stream);
 
+/* Batched form of adapt_quantize_selected: the whole re-quantisation loop of
+ * Algorithm 1 (for each layer l: Quantize(L[l], Q[l].quant)) in one launch,
+ * every layer at the <WL,FL> the search left for it on the device.
+ *   tensors   HOST array of n_layers DEVICE pointers (fp32, 4-byte aligned)
+ *   lens      HOST array of element counts (0 allowed)
+ *   best      DEVICE int32[n_layers][4], as written by a search
+ *   codes_out HOST array of n_layers DEVICE pointers, int32[lens[l]] each
+ *   hash layer id of tensors[l] is layer_base + l
+ * A layer whose selection is not a valid format is left untouched.  The layer
+ * table travels through a library-owned device buffer that is allocated (and
+ * grown) inside the call; calls that use it must not overlap on the device. */
+int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* lens,
+                                  int n_layers, const int32_t* best, int round_mode,
+                                  uint64_t seed, int32_t layer_base,
+                                  int32_t* const* codes_out, void* stream);
+
 /* Bytes of DEVICE workspace the search needs for these sizes (0 on invalid
  * arguments).  lens is a HOST array. */
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers,

@@ -24,7 +24,8 @@ OK, ERR_INVALID_ARG, ERR_NONFINITE, ERR_RANGE, ERR_CUDA, ERR_WORKSPACE = range(6
 
 EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
-    "adapt_quantize_ex", "adapt_quantize_selected", "adapt_search_workspace_bytes",
+    "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
+    "adapt_search_workspace_bytes",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
@@ -80,6 +81,10 @@ def lib():
         L.adapt_quantize_selected.restype = C.c_int
         L.adapt_quantize_selected.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int, C.c_uint64,
                                               C.c_int32, C.c_void_p, C.c_void_p]
+        L.adapt_quantize_selected_batch.restype = C.c_int
+        L.adapt_quantize_selected_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                                    C.c_int, C.c_uint64, C.c_int32, C.c_void_p,
+                                                    C.c_void_p]
         L.adapt_search_workspace_bytes.restype = C.c_size_t
         L.adapt_search_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int]
         search_args = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int, C.c_void_p,
@@ -194,6 +199,23 @@ def adapt_quantize_selected(x: torch.Tensor, selected: torch.Tensor, round_mode:
     _check(lib().adapt_quantize_selected(x.data_ptr(), x.numel(), selected.data_ptr(), round_mode,
                                          seed, layer, codes_out.data_ptr(), _stream_handle(stream)),
            "adapt_quantize_selected")
+    return codes_out
+
+
+def adapt_quantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.Tensor,
+                                  round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                                  codes_out: Optional[Sequence[torch.Tensor]] = None, stream=None):
+    """All layers at the <WL,FL> a search left in ``best`` (device int32[L][4]), one launch."""
+    assert best.is_cuda and best.dtype == torch.int32 and best.numel() >= 4 * len(tensors)
+    if codes_out is None:
+        codes_out = [torch.empty(t.numel(), dtype=torch.int32, device=t.device) for t in tensors]
+    ptrs, lens = _marshal_tensors(tensors)
+    outs = np.array([c.data_ptr() for c in codes_out], dtype=np.uint64)
+    assert all(c.dtype == torch.int32 and c.numel() == t.numel() for c, t in zip(codes_out, tensors))
+    _check(lib().adapt_quantize_selected_batch(ptrs.ctypes.data, lens.ctypes.data, len(tensors),
+                                               best.data_ptr(), round_mode, seed, layer_base,
+                                               outs.ctypes.data, _stream_handle(stream)),
+           "adapt_quantize_selected_batch")
     return codes_out
 
 

@@ -102,6 +102,7 @@ struct DeviceCache {
   void* workspace = nullptr;   size_t workspace_bytes = 0;
   void* stage_in = nullptr;    size_t stage_in_bytes = 0;    // host-form calls: inputs
   void* stage_out = nullptr;   size_t stage_out_bytes = 0;   // host-form calls: outputs
+  void* batch_tab = nullptr;   size_t batch_tab_bytes = 0;   // batched quantize: layer table
   PinnedSlot ring[kRingSlots];
   int ring_next = 0;
 };
@@ -158,13 +159,13 @@ constexpr size_t kKeyedSmemBudget = 224 * 1024; // one CTA per SM owns its share
 
 struct Plan {
   int n_layers = 0, n_cand = 0, n_levels = 0, n_bins = 0;
-  std::vector<int> slot, order;
+  std::vector<int> slot, order, by_fl, fl_begin;
   // keyed-kernel shared-memory shape
   int cell_cap = 0, d_levels = 0;
   size_t keyed_smem = 0;
   // byte offsets inside the workspace -- descriptor block (uploaded)
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
-         off_order = 0, off_state = 0, blob_bytes = 0;
+         off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_state = 0, blob_bytes = 0;
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
   // accumulators (cleared every call)
@@ -199,6 +200,14 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
     return grid->fl[a] < grid->fl[b];
   });
 
+  p->by_fl.resize(grid->n_cand);
+  std::iota(p->by_fl.begin(), p->by_fl.end(), 0);
+  std::stable_sort(p->by_fl.begin(), p->by_fl.end(),
+                   [&](int a, int b) { return grid->fl[a] < grid->fl[b]; });
+  p->fl_begin.assign(p->n_levels + 1, 0);
+  for (int c = 0; c < grid->n_cand; ++c) p->fl_begin[grid->fl[c] + 1] += 1;
+  for (int f = 0; f < p->n_levels; ++f) p->fl_begin[f + 1] += p->fl_begin[f];
+
   // shared-memory shape of the keyed kernel: queue + Qe + a few correction levels + cells
   const size_t hist = sizeof(unsigned) * n_bins;
   const size_t queue = keyed_smem_bytes(0, 0, 0);
@@ -221,6 +230,8 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_fl = o;      o = align_up(o + sizeof(int) * C, 16);
   p->off_slot = o;    o = align_up(o + sizeof(int) * C, 16);
   p->off_order = o;   o = align_up(o + sizeof(int) * C, 16);
+  p->off_by_fl = o;   o = align_up(o + sizeof(int) * C, 16);
+  p->off_fl_begin = o; o = align_up(o + sizeof(int) * (F + 1), 16);
   p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
   p->blob_bytes = o;
   p->off_plan = o;      o = align_up(o + sizeof(LayerPlan) * L, 256);
@@ -341,6 +352,8 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_order, plan.order.data(), sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_by_fl, plan.by_fl.data(), sizeof(int) * plan.n_cand);
+  std::memcpy(h + plan.off_fl_begin, plan.fl_begin.data(), sizeof(int) * (plan.n_levels + 1));
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
   for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
@@ -428,6 +441,10 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     const size_t budget = 100 * 1024;
     int fg = static_cast<int>(budget / per_hist) - 1;
     fg = std::max(1, std::min(fg, plan.n_levels));
+    // few tiles: spread the fraction lengths over more CTAs instead of looping over them in one
+    const long long want_groups = std::min<long long>(
+        plan.n_levels, std::max<long long>(1, (2ll * dc.sm_count + direct_tiles - 1) / direct_tiles));
+    fg = std::min<int>(fg, static_cast<int>((plan.n_levels + want_groups - 1) / want_groups));
     sp.fl_per_group = fg;
     const int groups = (plan.n_levels + fg - 1) / fg;
     const size_t smem = per_hist * (fg + 1);
@@ -451,6 +468,8 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.cand_fl = reinterpret_cast<const int*>(ws + plan.off_fl);
   kp.cand_slot = reinterpret_cast<const int*>(ws + plan.off_slot);
   kp.cand_order = reinterpret_cast<const int*>(ws + plan.off_order);
+  kp.cand_by_fl = reinterpret_cast<const int*>(ws + plan.off_by_fl);
+  kp.fl_begin = reinterpret_cast<const int*>(ws + plan.off_fl_begin);
   kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_levels; kp.n_bins = a.n_bins;
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = o.pseudo_count; kp.inv_ln_base = 1.0 / std::log(base); kp.eps = o.eps;
@@ -458,7 +477,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.best_out = a.best_out; kp.hist_out = o.hist_out;
   {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
-    kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(kp);
+    kld_kernel<<<dim3(plan.n_levels, a.n_layers), kKldThreads, 0, stream>>>(kp);
     ADAPT_CUDA(cudaGetLastError());
   }
   {
@@ -578,6 +597,53 @@ int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected, 
                             uint64_t seed, int32_t layer, int32_t* codes_out, void* stream) {
   if (!selected) return ADAPT_ERR_INVALID_ARG;
   return run_quantize(x, n, 0, 0, selected, round_mode, seed, layer, 32, codes_out, stream);
+}
+
+int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* lens, int n_layers,
+                                  const int32_t* best, int round_mode, uint64_t seed,
+                                  int32_t layer_base, int32_t* const* codes_out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!tensors || !lens || !best || !codes_out) return ADAPT_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > 65535) return ADAPT_ERR_INVALID_ARG;
+  if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
+    return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (lens[l] < 0) return ADAPT_ERR_INVALID_ARG;
+    if (lens[l] > 0 && (!tensors[l] || !codes_out[l])) return ADAPT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(tensors[l]) & 3u) || (reinterpret_cast<uintptr_t>(codes_out[l]) & 3u))
+      return ADAPT_ERR_INVALID_ARG;
+  }
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  const size_t bytes = sizeof(QuantLayer) * static_cast<size_t>(n_layers);
+  rc = grow_device(&dc->batch_tab, &dc->batch_tab_bytes, align_up(bytes, 4096));
+  if (rc != ADAPT_OK) return rc;
+  PinnedSlot* slot = nullptr;
+  rc = acquire_slot(*dc, bytes, &slot);
+  if (rc != ADAPT_OK) return rc;
+  QuantLayer* h = static_cast<QuantLayer*>(slot->host);
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    h[l].x = tensors[l]; h[l].out = codes_out[l]; h[l].n = lens[l]; h[l].tile_begin = tiles;
+    h[l].layer_id = layer_base + l;
+    h[l].vec = !(reinterpret_cast<uintptr_t>(tensors[l]) & 15u) &&
+               !(reinterpret_cast<uintptr_t>(codes_out[l]) & 15u);
+    tiles += (lens[l] + kQuantTile - 1) / kQuantTile;
+  }
+  if (tiles == 0) return ADAPT_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+  ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, h, bytes, cudaMemcpyHostToDevice, stream));
+  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  const int grid = static_cast<int>(std::min<long long>(tiles, 32ll * dc->sm_count));
+  const QuantLayer* d = static_cast<const QuantLayer*>(dc->batch_tab);
+  LaunchScope ls(ADAPT_KERNEL_QUANTIZE, stream);
+  if (round_mode == ADAPT_ROUND_STOCHASTIC)
+    quantize_batch_kernel<true><<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
+  else
+    quantize_batch_kernel<false><<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
+  ADAPT_CUDA(cudaGetLastError());
+  return ADAPT_OK;
 }
 
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers, const adapt_grid* grid,
@@ -710,7 +776,9 @@ constexpr size_t kStWl = kStLayers + 64 * (kStaticMaxLayers + 1);
 constexpr size_t kStFl = kStWl + 4 * kStaticMaxCand;
 constexpr size_t kStSlot = kStFl + 4 * kStaticMaxCand;
 constexpr size_t kStOrder = kStSlot + 4 * kStaticMaxCand;
-constexpr size_t kStState = kStOrder + 4 * kStaticMaxCand;                        // LayerState[L]
+constexpr size_t kStByFl = kStOrder + 4 * kStaticMaxCand;
+constexpr size_t kStFlBegin = kStByFl + 4 * kStaticMaxCand;                       // int[33]
+constexpr size_t kStState = kStFlBegin + 4 * 64;                                  // LayerState[L]
 constexpr size_t kStBlobEnd = kStState + 64 * kStaticMaxLayers;
 constexpr size_t kStZeros = (kStBlobEnd + 255) / 256 * 256;                       // u64[L][32]
 constexpr size_t kStQ = kStZeros + 8 * kStaticMaxLayers * kMaxFl;                 // u32[L][B]
@@ -799,6 +867,12 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
     if (grid->wl[a] != grid->wl[b]) return grid->wl[a] < grid->wl[b];
     return grid->fl[a] < grid->fl[b];
   });
+  int* h_by_fl = reinterpret_cast<int*>(h + kStByFl);
+  int* h_fl_begin = reinterpret_cast<int*>(h + kStFlBegin);
+  for (int c = 0; c < C; ++c) h_by_fl[c] = c;
+  std::stable_sort(h_by_fl, h_by_fl + C, [&](int a, int b) { return grid->fl[a] < grid->fl[b]; });
+  for (int c = 0; c < C; ++c) h_fl_begin[grid->fl[c] + 1] += 1;
+  for (int f = 0; f < n_levels; ++f) h_fl_begin[f + 1] += h_fl_begin[f];
   LayerState* hs = reinterpret_cast<LayerState*>(h + kStState);
   for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
@@ -849,12 +923,14 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   kp.cand_fl = reinterpret_cast<const int*>(ws + kStFl);
   kp.cand_slot = reinterpret_cast<const int*>(ws + kStSlot);
   kp.cand_order = reinterpret_cast<const int*>(ws + kStOrder);
+  kp.cand_by_fl = reinterpret_cast<const int*>(ws + kStByFl);
+  kp.fl_begin = reinterpret_cast<const int*>(ws + kStFlBegin);
   kp.n_layers = n_layers; kp.n_cand = C; kp.n_fl = n_levels; kp.n_bins = n_bins;
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = 0.0; kp.inv_ln_base = 1.0 / std::log(2.0); kp.eps = 0.0;
   kp.kld_out = kld_out; kp.zeros_out = reinterpret_cast<long long*>(zeros_out);
   kp.best_out = best_out; kp.hist_out = nullptr;
-  kld_kernel<<<dim3(C, n_layers), kKldThreads, 0, stream>>>(kp);
+  kld_kernel<<<dim3(n_levels, n_layers), kKldThreads, 0, stream>>>(kp);
   ADAPT_LAUNCH_OK("kld launch");
   ++g_launches;
   select_kernel<<<n_layers, 32, 0, stream>>>(kp);
@@ -872,6 +948,7 @@ int adapt_release(void) {
   if (dc->workspace) { ADAPT_CUDA(cudaFree(dc->workspace)); dc->workspace = nullptr; dc->workspace_bytes = 0; }
   if (dc->stage_in) { ADAPT_CUDA(cudaFree(dc->stage_in)); dc->stage_in = nullptr; dc->stage_in_bytes = 0; }
   if (dc->stage_out) { ADAPT_CUDA(cudaFree(dc->stage_out)); dc->stage_out = nullptr; dc->stage_out_bytes = 0; }
+  if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
   for (PinnedSlot& s : dc->ring) {
     if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }
     if (s.done) { ADAPT_CUDA(cudaEventDestroy(s.done)); s.done = nullptr; }

@@ -1,7 +1,7 @@
 // K3: batched divergence and selection over all (layer, candidate) pairs.
 //
-// kld_kernel: one CTA per (candidate, layer).  Folds the layer's unsaturated
-// per-FL histogram into the candidate's histogram (both tails collapse into
+// kld_kernel: one CTA per (fraction length, layer).  Folds the layer's unsaturated
+// per-FL histogram into each candidate's histogram (both tails collapse into
 // the bins of the two saturation values), then sums the discrete
 // Kullback-Leibler divergence KL(P||Q) (Sec. 3.3), P = candidate, Q = float
 // tensor, in double precision.  With integer counts p, q that share the total
@@ -29,6 +29,8 @@ struct KldParams {
   const int* cand_fl;          // [n_cand]
   const int* cand_slot;        // [n_cand] index of the candidate's FL in the distinct-FL list
   const int* cand_order;       // [n_cand] candidate indices sorted by (WL, FL, index)
+  const int* cand_by_fl;       // [n_cand] candidate indices grouped by FL
+  const int* fl_begin;         // [n_fl + 1] start of each FL's group in cand_by_fl
   int n_layers, n_cand, n_fl, n_bins;
   const unsigned* q_hist;      // [n_layers][n_bins]
   const unsigned* u_hist;      // [n_layers][n_fl][n_bins]
@@ -54,78 +56,109 @@ __device__ __forceinline__ double block_sum(double v, double* s_buf) {
   return t;
 }
 
+// One term of the divergence sum and whether it is infinite (a filled P bin over an empty Q bin).
+__device__ __forceinline__ double kld_term(long long pc, long long qc, double alpha, bool* inf) {
+  const double pa = static_cast<double>(pc) + alpha;
+  const double qa = static_cast<double>(qc) + alpha;
+  if (!(pa > 0.0)) return 0.0;
+  if (qa <= 0.0) { *inf = true; return 0.0; }
+  return pa * log1p(static_cast<double>(pc - qc) / qa);
+}
+
+// One CTA per (fraction length, layer).  The candidates of one FL differ only in where they
+// saturate; those whose two saturation values fall in the first and the last bin have exactly
+// the unsaturated histogram U[FL], so their divergence is computed once.  The others fold the
+// two tails of U[FL] into the bins of their saturation values and are summed one by one.
 __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   __shared__ double s_buf[kKldThreads / 32];
   __shared__ int s_inf;
-  const int c = blockIdx.x, l = blockIdx.y;
+  const int f = blockIdx.x, l = blockIdx.y;
+  const int c_begin = p.fl_begin[f], c_end = p.fl_begin[f + 1];
+  if (c_begin == c_end) return;
   const int B = p.n_bins;
   const LayerState S = p.state[l];
   const long long n = p.layers[l].n;
-  const size_t out = static_cast<size_t>(l) * p.n_cand + c;
-  const int wl = p.cand_wl[c], fl = p.cand_fl[c], slot = p.cand_slot[c];
 
   if (S.flags & (kFlagNonfinite | kFlagRange)) {
-    if (threadIdx.x == 0) {
+    for (int i = c_begin + threadIdx.x; i < c_end; i += kKldThreads) {
+      const size_t out = static_cast<size_t>(l) * p.n_cand + p.cand_by_fl[i];
       p.kld_out[out] = __longlong_as_double(0x7ff8000000000000ll);  // NaN: unspecified output
       p.zeros_out[out] = 0;
     }
     return;
   }
-
-  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + slot) * B;
+  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + f) * B;
   const unsigned* Q = p.q_hist + static_cast<size_t>(l) * B;
+  const double n_eff = static_cast<double>(n) + p.alpha * B;
+  const double inf_value = __longlong_as_double(0x7ff0000000000000ll);
+  const long long zero_count = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + f]);
 
-  // bins of the two saturation values of <WL,FL>
-  const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
-  const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
-  const int bh = bin_of(dequantize(hi_code, fl), S.lo, S.scale, S.bmax);
-  const int bl = bin_of(dequantize(lo_code, fl), S.lo, S.scale, S.bmax);
-
-  // tail masses that fold into bl and bh
-  double lo_mass = 0.0, hi_mass = 0.0;
-  for (int b = threadIdx.x; b < B; b += kKldThreads) {
-    unsigned u = U[b];
-    if (b <= bl) lo_mass += u;
-    if (b >= bh) hi_mass += u;
-  }
-  lo_mass = block_sum(lo_mass, s_buf);
-  hi_mass = block_sum(hi_mass, s_buf);
+  // divergence of the unsaturated histogram
   if (threadIdx.x == 0) s_inf = 0;
   __syncthreads();
-
-  unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * B
-                           : nullptr;
-  unsigned* H0 = (p.hist_out && c == 0)
-                     ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * B : nullptr;
   double sum = 0.0;
   bool inf = false;
-  for (int b = threadIdx.x; b < B; b += kKldThreads) {
-    long long pc;
-    if (bl == bh) pc = (b == bl) ? n : 0;
-    else if (b < bl || b > bh) pc = 0;
-    else if (b == bl) pc = static_cast<long long>(lo_mass);
-    else if (b == bh) pc = static_cast<long long>(hi_mass);
-    else pc = U[b];
-    const long long qc = Q[b];
-    if (H) H[b] = static_cast<unsigned>(pc);
-    if (H0) H0[b] = static_cast<unsigned>(qc);
-    const double pa = static_cast<double>(pc) + p.alpha;
-    const double qa = static_cast<double>(qc) + p.alpha;
-    if (pa > 0.0) {
-      if (qa <= 0.0) inf = true;
-      else sum += pa * log1p(static_cast<double>(pc - qc) / qa);
-    }
-  }
+  for (int b = threadIdx.x; b < B; b += kKldThreads) sum += kld_term(U[b], Q[b], p.alpha, &inf);
   if (inf) s_inf = 1;
   sum = block_sum(sum, s_buf);
-  if (threadIdx.x == 0) {
-    const double n_eff = static_cast<double>(n) + p.alpha * B;
+  double unsat;
+  if (n_eff <= 0.0) unsat = 0.0;
+  else if (s_inf) unsat = inf_value;
+  else { unsat = sum * p.inv_ln_base / n_eff; if (!(unsat > 0.0)) unsat = 0.0; }
+
+  for (int i = c_begin; i < c_end; ++i) {
+    const int c = p.cand_by_fl[i];
+    const int wl = p.cand_wl[c];
+    const size_t out = static_cast<size_t>(l) * p.n_cand + c;
+    // bins of the two saturation values of <WL,FL>
+    const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
+    const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
+    const int bh = bin_of(dequantize(hi_code, f), S.lo, S.scale, S.bmax);
+    const int bl = bin_of(dequantize(lo_code, f), S.lo, S.scale, S.bmax);
+    unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * B
+                             : nullptr;
+    unsigned* H0 = (p.hist_out && c == 0)
+                       ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * B : nullptr;
     double k;
-    if (n_eff <= 0.0) k = 0.0;
-    else if (s_inf) k = __longlong_as_double(0x7ff0000000000000ll);
-    else { k = sum * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
-    p.kld_out[out] = k;
-    p.zeros_out[out] = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + slot]);
+    if (bl == 0 && bh == B - 1 && B > 1 && !H) {
+      k = unsat;                     // nothing folds: the candidate's histogram is U[FL] itself
+    } else {
+      // tail masses that fold into bl and bh
+      double lo_mass = 0.0, hi_mass = 0.0;
+      for (int b = threadIdx.x; b < B; b += kKldThreads) {
+        const unsigned u = U[b];
+        if (b <= bl) lo_mass += u;
+        if (b >= bh) hi_mass += u;
+      }
+      lo_mass = block_sum(lo_mass, s_buf);
+      hi_mass = block_sum(hi_mass, s_buf);
+      if (threadIdx.x == 0) s_inf = 0;
+      __syncthreads();
+      sum = 0.0;
+      inf = false;
+      for (int b = threadIdx.x; b < B; b += kKldThreads) {
+        long long pc;
+        if (bl == bh) pc = (b == bl) ? n : 0;
+        else if (b < bl || b > bh) pc = 0;
+        else if (b == bl) pc = static_cast<long long>(lo_mass);
+        else if (b == bh) pc = static_cast<long long>(hi_mass);
+        else pc = U[b];
+        const long long qc = Q[b];
+        if (H) H[b] = static_cast<unsigned>(pc);
+        if (H0) H0[b] = static_cast<unsigned>(qc);
+        sum += kld_term(pc, qc, p.alpha, &inf);
+      }
+      if (inf) s_inf = 1;
+      sum = block_sum(sum, s_buf);
+      if (n_eff <= 0.0) k = 0.0;
+      else if (s_inf) k = inf_value;
+      else { k = sum * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
+      __syncthreads();               // s_inf is rewritten by the next candidate
+    }
+    if (threadIdx.x == 0) {
+      p.kld_out[out] = k;
+      p.zeros_out[out] = zero_count;
+    }
   }
 }
 

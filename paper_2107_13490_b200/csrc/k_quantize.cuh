@@ -71,4 +71,53 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const QuantPara
   }
 }
 
+// Batched form: every layer of a list is quantized at the <WL,FL> a search left on the
+// device for it, in one launch (Algorithm 1: for l in L: L^[l] = Quantize(L[l], Q[l].quant)).
+struct QuantLayer {
+  const float* x;
+  int* out;
+  long long n;
+  long long tile_begin;   // first tile of the layer in the launch's tile list (4096 elements each)
+  int layer_id;           // hash layer id
+  int vec;                // x is 16-byte aligned and out 16-byte aligned: 128-bit accesses
+};
+
+constexpr int kQuantTile = 4096;
+
+template <bool kStochastic>
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long long n_tiles,
+                      const int* __restrict__ best, unsigned long long seed) {
+  for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    int lo = 0, hi = n_layers - 1;                 // layer that owns tile t
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (layers[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
+    }
+    const QuantLayer L = layers[lo];
+    const int wl = best[4 * lo], fl = best[4 * lo + 1];
+    if (wl < 2 || wl > 32 || fl < 0 || fl >= wl) continue;   // layer without a valid selection
+    const float two_fl = pow2f(fl);
+    const long long i0 = (t - L.tile_begin) * kQuantTile;
+    const long long i1 = min(L.n, i0 + kQuantTile);
+    if (L.vec && i1 - i0 == kQuantTile) {
+      const float4* x4 = reinterpret_cast<const float4*>(L.x + i0);
+      int4* o4 = reinterpret_cast<int4*>(L.out + i0);
+      for (int q = threadIdx.x; q < kQuantTile / 4; q += kQuantThreads) {
+        const float4 v = __ldcs(x4 + q);
+        const long long i = i0 + 4ll * q;
+        int4 c;
+        c.x = quantize_one<kStochastic>(v.x, two_fl, wl, seed, L.layer_id, i + 0);
+        c.y = quantize_one<kStochastic>(v.y, two_fl, wl, seed, L.layer_id, i + 1);
+        c.z = quantize_one<kStochastic>(v.z, two_fl, wl, seed, L.layer_id, i + 2);
+        c.w = quantize_one<kStochastic>(v.w, two_fl, wl, seed, L.layer_id, i + 3);
+        __stcs(o4 + q, c);
+      }
+    } else {
+      for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads)
+        L.out[i] = quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i);
+    }
+  }
+}
+
 }  // namespace adapt

@@ -84,6 +84,30 @@ def test_quantize_at_device_resident_selection(B):
     assert np.array_equal(got.cpu().numpy(), want)
 
 
+def test_batched_quantize_at_device_resident_selections(B):
+    import torch
+    w = W.WORKLOADS["resnet20_weights_grads"]
+    xs = W.generate(w)
+    pick = [0, 3, 10, 19, 20, 25, 39]
+    wl, fl = w.grid()
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        bufs = []
+        for j, i in enumerate(pick):     # odd phases: some layers take the scalar path
+            b = torch.zeros(xs[i].size + 4, dtype=torch.float32, device="cuda")
+            b[j % 4:j % 4 + xs[i].size] = torch.from_numpy(xs[i]).cuda()
+            bufs.append(b[j % 4:j % 4 + xs[i].size])
+        bufs.append(torch.zeros(0, dtype=torch.float32, device="cuda"))       # an empty layer
+        res = B.adapt_precision_search_ex(bufs, B.Grid(wl, fl), w.n_bins, round_mode=mode, seed=7,
+                                          layer_base=2)
+        codes = B.adapt_quantize_selected_batch(bufs, res.best, mode, seed=7, layer_base=2)
+        torch.cuda.synchronize()
+        ora = O.precision_search([xs[i] for i in pick], wl, fl, w.n_bins, mode, 7, 2)
+        for j, i in enumerate(pick):
+            want, _ = O.quantize(xs[i], int(ora[j]["best"][0]), int(ora[j]["best"][1]), mode, 7, 2 + j)
+            assert np.array_equal(codes[j].cpu().numpy(), want), (mode, i)
+        assert codes[-1].numel() == 0
+
+
 def test_quantize_argument_errors_and_host_form(B):
     import torch
     x = torch.zeros(16, dtype=torch.float32, device="cuda")
