@@ -400,13 +400,15 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
     {
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
-      plan_kernel<<<nk, kPlanThreads, 0, stream>>>(pp);
+      const int plan_slices = std::max(1, std::min(16, (2 * dc.sm_count) / nk));
+      plan_kernel<<<dim3(nk, plan_slices), kPlanThreads, 0, stream>>>(pp);
       ADAPT_CUDA(cudaGetLastError());
     }
     KeyedParams kp;
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
     kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
+    kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
     kp.n_bins = a.n_bins; kp.n_levels = plan.n_levels;
     kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -421,11 +423,13 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
     ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
     ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
+    ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
     ep.n_bins = a.n_bins; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
     {
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      expand_kernel<<<dim3(plan.n_levels + 1, nk), kExpandThreads, sizeof(unsigned) * a.n_bins,
-                      stream>>>(ep);
+      const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / ((plan.n_levels + 1) * nk)));
+      expand_kernel<<<dim3(plan.n_levels + 1, nk, slices), kExpandThreads,
+                      sizeof(unsigned) * a.n_bins, stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
   }
@@ -477,7 +481,9 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.best_out = a.best_out; kp.hist_out = o.hist_out;
   {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
-    kld_kernel<<<dim3(plan.n_levels, a.n_layers), kKldThreads, 0, stream>>>(kp);
+    // enough CTAs to fill the GPU when there are few (FL, layer) pairs
+    const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / std::max(1, plan.n_levels * a.n_layers)));
+    kld_kernel<<<dim3(plan.n_levels, a.n_layers, slices), kKldThreads, 0, stream>>>(kp);
     ADAPT_CUDA(cudaGetLastError());
   }
   {
@@ -540,7 +546,7 @@ int run_quantize(const float* x, int64_t n, int wl, int fl, const int32_t* selec
 
 extern "C" {
 
-const char* adapt_version(void) { return "adapt-b200 0.1"; }
+const char* adapt_version(void) { return "adapt-b200 0.2"; }
 
 const char* adapt_status_string(int status) {
   switch (status) {

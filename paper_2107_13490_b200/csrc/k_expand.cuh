@@ -1,7 +1,7 @@
 // Expansion of the keyed kernel's cell counts into the per-level histograms.
 //
-// One CTA per (level, layer); level n_levels stands for the float histogram Q.
-// The CTA walks the layer's cells (both segments) and adds each cell's count to
+// One CTA (or a few, each with a slice of the cells) per (level, layer); level n_levels
+// stands for the float histogram Q.  The CTA walks its cells and adds each cell's count to
 // a shared-memory histogram of its level:
 //   * float histogram and fine levels (f >= the segment's G), interior cells
 //     only: the cell's own bin (elements of edge cells were binned one by one
@@ -13,7 +13,8 @@
 // then the exact zeros (layer size minus all cell counts) at the bin of 0, and
 // for the zero counts the cells that round to 0 plus, at fine levels of the
 // main segment, the zero classes.  The result is added to the corrections
-// already in U; no global atomics.
+// already in U.  When there are few (level, layer) pairs the cells are split over several
+// CTAs, each adding its part with one global atomic per non-empty bin.
 #pragma once
 
 #include "common.cuh"
@@ -36,12 +37,13 @@ struct ExpandParams {
   unsigned* u_hist;            // [layer][n_levels][n_bins]
   unsigned long long* zeros;   // [layer][n_levels]
   const unsigned long long* zero_class;  // [layer][kZeroClasses]
+  const unsigned long long* cell_total;  // [layer] non-zero elements (sum of all cell counts)
   int n_bins, n_levels, cell_cap;
 };
 
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandParams p) {
   extern __shared__ unsigned s_hist[];          // [n_bins]
-  __shared__ unsigned long long s_total, s_zero;
+  __shared__ unsigned long long s_zero;
   const LayerDesc L = p.layers[blockIdx.y];
   const int l = L.index;
   const LayerPlan P = p.plan[l];
@@ -52,16 +54,18 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   const bool is_q = (f == p.n_levels);
 
   for (int b = threadIdx.x; b < B; b += kExpandThreads) s_hist[b] = 0;
-  if (threadIdx.x == 0) { s_total = 0; s_zero = 0; }
+  if (threadIdx.x == 0) s_zero = 0;
   __syncthreads();
 
   const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
   const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-  unsigned long long total = 0, zero = 0;
-  for (int i = threadIdx.x; i < P.total_cells; i += kExpandThreads) {
+  unsigned long long zero = 0;
+  // the cells are shared by the gridDim.z CTAs of this (level, layer), a contiguous slice each
+  const int per_slice = (P.total_cells + gridDim.z - 1) / gridDim.z;
+  const int i_end = min(P.total_cells, static_cast<int>(blockIdx.z + 1) * per_slice);
+  for (int i = blockIdx.z * per_slice + threadIdx.x; i < i_end; i += kExpandThreads) {
     const unsigned m = count[i];
     if (m == 0) continue;
-    total += m;
     const int s = (P.seg[1].cells > 0 && i >= P.seg[1].offset) ? 1 : 0;
     const SegPlan& sp = P.seg[s];
     const long long cc = sp.c0 + (i - sp.offset);
@@ -81,37 +85,34 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
     }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    total += __shfl_xor_sync(0xffffffffu, total, o);
-    zero += __shfl_xor_sync(0xffffffffu, zero, o);
-  }
-  if ((threadIdx.x & 31) == 0) {
-    if (total) atomicAdd(&s_total, total);
-    if (zero) atomicAdd(&s_zero, zero);
-  }
+  for (int o = 16; o > 0; o >>= 1) zero += __shfl_xor_sync(0xffffffffu, zero, o);
+  if ((threadIdx.x & 31) == 0 && zero) atomicAdd(&s_zero, zero);
   __syncthreads();
 
-  const unsigned n_zero = static_cast<unsigned>(static_cast<unsigned long long>(L.n) - s_total);
+  // the first slice also adds what does not come from cells: exact zeros, edge elements, classes
+  const bool lead = (blockIdx.z == 0);
+  const unsigned n_zero =
+      lead ? static_cast<unsigned>(static_cast<unsigned long long>(L.n) - p.cell_total[l]) : 0u;
   const int bz = bin_of(0.0f, S.lo, S.scale, S.bmax);
   const unsigned* qe0 = p.qe_hist + static_cast<size_t>(l) * 2 * B;
   const unsigned* qe1 = qe0 + B;
-  const bool fine0 = is_q || f >= P.seg[0].fs;
-  const bool fine1 = P.seg[1].cells > 0 && (is_q || f >= P.seg[1].fs);
+  const bool fine0 = lead && (is_q || f >= P.seg[0].fs);
+  const bool fine1 = lead && P.seg[1].cells > 0 && (is_q || f >= P.seg[1].fs);
   unsigned* out = is_q ? p.q_hist + static_cast<size_t>(l) * B
                        : p.u_hist + (static_cast<size_t>(l) * p.n_levels + f) * B;
   for (int b = threadIdx.x; b < B; b += kExpandThreads) {
     unsigned h = s_hist[b] + (b == bz ? n_zero : 0u);
     if (fine0) h += qe0[b];
     if (fine1) h += qe1[b];
-    out[b] = is_q ? h : out[b] + h;
+    if (h) atomicAdd(&out[b], h);     // U holds the corrections, Q starts at zero
   }
   if (!is_q && threadIdx.x == 0) {
     unsigned long long z = s_zero + n_zero;
-    if (f >= P.seg[0].fs) {
+    if (lead && f >= P.seg[0].fs) {
       const unsigned long long* zc = p.zero_class + static_cast<size_t>(l) * kZeroClasses;
       for (int k = f; k <= 32; ++k) z += zc[k + 1];   // classes whose highest zero level >= f
     }
-    p.zeros[static_cast<size_t>(l) * p.n_levels + f] += z;
+    if (z) atomicAdd(&p.zeros[static_cast<size_t>(l) * p.n_levels + f], z);
   }
 }
 

@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   const long long n = p.layers[l].n;
 
   if (S.flags & (kFlagNonfinite | kFlagRange)) {
-    for (int i = c_begin + threadIdx.x; i < c_end; i += kKldThreads) {
+    for (int i = c_begin + blockIdx.z * kKldThreads + threadIdx.x; i < c_end;
+         i += kKldThreads * gridDim.z) {
       const size_t out = static_cast<size_t>(l) * p.n_cand + p.cand_by_fl[i];
       p.kld_out[out] = __longlong_as_double(0x7ff8000000000000ll);  // NaN: unspecified output
       p.zeros_out[out] = 0;
@@ -106,7 +107,8 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   else if (s_inf) unsat = inf_value;
   else { unsat = sum * p.inv_ln_base / n_eff; if (!(unsat > 0.0)) unsat = 0.0; }
 
-  for (int i = c_begin; i < c_end; ++i) {
+  // the FL's candidates are dealt round-robin to the gridDim.z CTAs that share this (FL, layer)
+  for (int i = c_begin + blockIdx.z; i < c_end; i += gridDim.z) {
     const int c = p.cand_by_fl[i];
     const int wl = p.cand_wl[c];
     const size_t out = static_cast<size_t>(l) * p.n_cand + c;

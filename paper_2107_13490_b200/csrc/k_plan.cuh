@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
       P.seg[s].magic = 12582912.0f - static_cast<float>(P.seg[s].c0) +
                        static_cast<float>(P.seg[s].offset);
     s_plan = P;
-    p.plan[l] = P;
+    if (blockIdx.y == 0) p.plan[l] = P;   // every CTA of the layer derives the same plan
   }
   __syncthreads();
   const LayerPlan P = s_plan;
@@ -184,7 +184,9 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   // exact lower edge of every bin: smallest float v with bin_of(v) >= b
   float* E = p.edges + static_cast<size_t>(l) * (B + 1);
   const unsigned klo = float_key(S.lo), khi = float_key(S.hi);
-  for (int b = threadIdx.x; b <= B; b += kPlanThreads) {
+  // the layer's CTAs (gridDim.y of them) share the edges and the cells
+  const int first = blockIdx.y * kPlanThreads + threadIdx.x, stride = kPlanThreads * gridDim.y;
+  for (int b = first; b <= B; b += stride) {
     float e;
     if (b == 0) e = __int_as_float(0xff800000);          // -inf: bin 0 takes everything below
     else if (b == B) e = __int_as_float(0x7f800000);     // +inf
@@ -202,7 +204,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
 
   // cell marks, both segments
   unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-  for (int i = threadIdx.x; i < P.total_cells; i += kPlanThreads) {
+  for (int i = first; i < P.total_cells; i += stride) {
     const int s = (i >= P.seg[1].offset && P.seg[1].cells > 0) ? 1 : 0;
     const SegPlan& sp = P.seg[s];
     const long long cc = sp.c0 + (i - sp.offset);

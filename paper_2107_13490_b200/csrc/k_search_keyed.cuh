@@ -53,6 +53,7 @@ struct KeyedParams {
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
   unsigned long long* zeros;   // [layer][n_levels]      receives tie corrections
   unsigned long long* zero_class;  // [layer][kZeroClasses]
+  unsigned long long* cell_total;  // [layer] sum of all cell counts = non-zero elements
   int n_bins;
   int n_levels;                // levels 0..n_levels-1 are wanted
   int cell_cap;
@@ -378,10 +379,15 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     // ---- flush the private tables into the layer's global ones -----------------------
     if (ok) {
       unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
+      unsigned long long counted = 0;
       for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) {
         const unsigned n = cells[i] & kCellCountMask;
         if (n) atomicAdd(&gc[i], n);
+        counted += n;
       }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) counted += __shfl_xor_sync(0xffffffffu, counted, o);
+      if (lane == 0 && counted) atomicAdd(&p.cell_total[l], counted);
       unsigned* gq = p.qe_hist + static_cast<size_t>(l) * 2 * p.n_bins;
       for (int i = threadIdx.x; i < p.n_bins; i += kKeyedThreads) {
         const unsigned n = qe[i];
