@@ -159,8 +159,19 @@ def run_reference(args):
     from paper_2107_13490_b200 import workloads as W
     w = W.WORKLOADS[args.workload]
     wl, fl = w.grid()
-    n_sample = min(w.numel, 1 << 18)
+    # size each step's sample so that the whole run (warm-up + steps) stays near two minutes:
+    # a short calibration pass gives the oracle's rate on this host
     first = w.layers[0]
+    probe_n = min(first.numel, 1 << 14)
+    probe = [W.generate_layer(W.LayerSpec(first.name, (probe_n,), first.dist, first.scale,
+                                          first.zero_frac, first.outlier_frac, first.outlier_gain),
+                              w.seed, 0)]
+    t0 = time.perf_counter()
+    oracle_step(O, probe, wl, fl, w)
+    rate = probe_n / max(time.perf_counter() - t0, 1e-6)          # elements per second, all candidates
+    budget_s = 120.0
+    n_sample = int(rate * budget_s / max(1, args.steps + args.warmup))
+    n_sample = max(1 << 12, min(n_sample, 1 << 18, w.numel))
     if first.numel > n_sample:   # generate only what the sample needs
         xs = [W.generate_layer(W.LayerSpec(first.name, (n_sample,), first.dist, first.scale,
                                            first.zero_frac, first.outlier_frac, first.outlier_gain),
