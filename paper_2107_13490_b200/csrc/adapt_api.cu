@@ -377,7 +377,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
 
   // K1: range scan over every layer, then bin origin / scale per layer
   if (tiles > 0) {
-    const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc.sm_count));
+    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc.sm_count));
     LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
     range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(d_layers, a.n_layers, tiles, d_state);
     ADAPT_CUDA(cudaGetLastError());
@@ -894,7 +894,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + kStU);
 
   if (tiles > 0) {
-    const int g = static_cast<int>(std::min<long long>(tiles, 8ll * dc->sm_count));
+    const int g = static_cast<int>(std::min<long long>(tiles, 16ll * dc->sm_count));
     range_scan_kernel<<<g, kRangeThreads, 0, stream>>>(d_layers, n_layers, tiles, d_state);
     ADAPT_LAUNCH_OK("range scan launch");
     ++g_launches;

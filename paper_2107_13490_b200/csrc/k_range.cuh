@@ -9,7 +9,7 @@
 namespace adapt {
 
 constexpr int kTile = 4096;          // elements per tile (in aligned indexing)
-constexpr int kRangeThreads = 256;
+constexpr int kRangeThreads = 128;   // 8 quads per thread per tile: loads first, then arithmetic
 
 constexpr unsigned kFlagDegenerate = 2u;
 constexpr unsigned kFlagNonfinite = 4u;
@@ -39,21 +39,37 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
     float asum = 0.0f;
     for (; t < layer_tiles_end; ++t) {
       const long long j_tile = (t - L.tile_begin) * kTile;
+      constexpr int kQ = kTile / 4 / kRangeThreads;
+      float v[kQ][4];
+      unsigned m[kQ];
+      if (j_tile >= jbeg && j_tile + kTile <= jend) {
+        // full tile: all loads first, then the arithmetic
 #pragma unroll
-      for (int q = 0; q < kTile / 4 / kRangeThreads; ++q) {
-        const long long j0 = j_tile + 4ll * (q * kRangeThreads + threadIdx.x);
-        if (j0 >= jend) continue;
-        float v[4];
-        unsigned m = load_quad(base, j0, jbeg, jend, v);
+        for (int q = 0; q < kQ; ++q) {
+          const float4 w4 = __ldg(reinterpret_cast<const float4*>(base + j_tile) + q * kRangeThreads + threadIdx.x);
+          v[q][0] = w4.x; v[q][1] = w4.y; v[q][2] = w4.z; v[q][3] = w4.w;
+          m[q] = 0xFu;
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < kQ; ++q) {
+          const long long j0 = j_tile + 4ll * (q * kRangeThreads + threadIdx.x);
+          m[q] = 0;
+          v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
+          if (j0 < jend) m[q] = load_quad(base, j0, jbeg, jend, v[q]);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < kQ; ++q) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          if (m & (1u << k)) {
-            float a = fabsf(v[k]);
+          if (m[q] & (1u << k)) {
+            float a = fabsf(v[q][k]);
             // NaN fails both compares; Inf is caught by the first
             if (!(a <= 3.402823466e38f)) flags |= kFlagNonfinite;
             else if (a >= 18446744073709551616.0f) flags |= kFlagRange;
-            vmin = fminf(vmin, v[k]);
-            vmax = fmaxf(vmax, v[k]);
+            vmin = fminf(vmin, v[q][k]);
+            vmax = fmaxf(vmax, v[q][k]);
             asum += a;
           }
         }
