@@ -21,9 +21,8 @@
 // derived from the cell counts by the expand kernel.
 //
 // One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
-// for its tables; each thread handles 16 elements (four 128-bit loads) per tile
-// and refills a quad's registers with the next tile's quad as soon as the quad
-// has been used, so loads stay in flight while elements are processed.
+// for its tables; each thread handles 16 elements (four 128-bit loads, issued
+// together) per tile.
 #pragma once
 
 #include "common.cuh"
@@ -178,25 +177,22 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_
   return __float2int_rz(__fsub_rn(cf, f.c0f0));
 }
 
-// One tile.  v holds this thread's elements of the tile when `loaded`; otherwise they are
-// fetched here (guarded loads when the tile is ragged).  As soon as a quad has been used its
-// registers are refilled with the same quad of the next tile (`next`, non-null only when that
-// tile is a full tile of the same layer), so loads stay in flight while elements are processed.
+// One tile: this thread's four quads are loaded first (guarded loads when the tile is ragged),
+// then processed quad by quad.  (Fetching the next tile ahead into the same registers was
+// measured and lost: under the 64-register cap it only bought spills.)
 template <bool kFast, bool kFull>
 __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, int dummy_pos,
                                            float* queue, unsigned& qn,
                                            const CellFn& fn, const float* base, long long j_tile,
                                            long long jbeg, long long jend,
-                                           float (&v)[kKeyedQuads][4], bool loaded,
-                                           const float4* src, const float4* next) {
+                                           const float4* src) {
+  float v[kKeyedQuads][4];
   unsigned vm[kKeyedQuads];
 #pragma unroll
   for (int q = 0; q < kKeyedQuads; ++q) {
     if (kFull) {      // src = this thread's first quad of the tile
-      if (!loaded) {
-        const float4 t = __ldcs(src + q * kKeyedThreads);
-        v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
-      }
+      const float4 t = __ldcs(src + q * kKeyedThreads);
+      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
       vm[q] = 0xFu;
     } else {
       const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
@@ -257,11 +253,6 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
         __syncwarp();
       }
     }
-    // this quad's registers are free: start the next tile's quad
-    if (kFull && next != nullptr) {
-      const float4 t = __ldcs(next + q * kKeyedThreads);
-      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
-    }
   }
 }
 
@@ -273,29 +264,21 @@ __device__ __forceinline__ void keyed_segment(const LayerCtx& c, unsigned* cells
                                               float* queue,
                                               const CellFn& fn, const float* base, long long jbeg,
                                               long long jend, int k0, int k1) {
-  float v[kKeyedQuads][4];
   unsigned qn = 0;             // entries in this warp's queue (same in every lane)
   const int kf0 = max(k0, jbeg > 0 ? 1 : 0);
   const int kf1 = min(k1, static_cast<int>(jend / kKeyedTile));
   if (k0 < kf0)
     keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
-                             static_cast<long long>(k0) * kKeyedTile, jbeg, jend, v, false, nullptr,
-                             nullptr);
+                             static_cast<long long>(k0) * kKeyedTile, jbeg, jend, nullptr);
   if (kf0 < kf1) {
     const float4* src = reinterpret_cast<const float4*>(base + static_cast<long long>(kf0) * kKeyedTile) +
                         threadIdx.x;
-    bool loaded = false;
-    for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4) {
-      const float4* next = (k + 1 < kf1) ? src + kKeyedTile / 4 : nullptr;
-      keyed_tile<kFast, true>(c, cells, dummy_pos, queue, qn, fn, base, 0, 0, 0, v,
-                              loaded, src, next);
-      loaded = true;
-    }
+    for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4)
+      keyed_tile<kFast, true>(c, cells, dummy_pos, queue, qn, fn, base, 0, 0, 0, src);
   }
   for (int k = max(kf1, kf0); k < k1; ++k)
     keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
-                             static_cast<long long>(k) * kKeyedTile, jbeg, jend, v, false, nullptr,
-                             nullptr);
+                             static_cast<long long>(k) * kKeyedTile, jbeg, jend, nullptr);
   // what is left in the queue
   __syncwarp();
   if ((threadIdx.x & 31) < qn) handle_special(c, queue[threadIdx.x & 31]);
