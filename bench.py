@@ -314,13 +314,8 @@ def main():
         host_codes = [torch.empty(n, dtype=torch.int32).pin_memory() for n in lens]
 
         def e2e_step():
-            B.adapt_precision_search_host(pinned, grid, w.n_bins, round_mode=w.round_mode,
-                                          seed=w.seed, out=host_out)
-            best = host_out.best.numpy()
-            for l, p in enumerate(pinned):
-                if lens[l]:
-                    B.adapt_quantize_host(p, int(best[l][0]), int(best[l][1]), w.round_mode, w.seed,
-                                          l, 32, codes_out=host_codes[l])
+            B.adapt_precision_switch_host(pinned, grid, w.n_bins, round_mode=w.round_mode,
+                                          seed=w.seed, out=host_out, codes_out=host_codes)
 
         e2e_step()
         S.barrier()
@@ -335,8 +330,8 @@ def main():
         res_bytes = len(xs) * (n_cand * 16 + 16)
         e2e = {"value": e2e_value, "unit": UNIT, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3,
-               "h2d_bytes_per_step": 8 * total, "d2h_bytes_per_step": res_bytes + 4 * total,
-               "api": "adapt_precision_search_host + adapt_quantize_host (pinned host buffers)"}
+               "h2d_bytes_per_step": 4 * total, "d2h_bytes_per_step": res_bytes + 4 * total,
+               "api": "adapt_precision_switch_host (pinned host buffers in, results and codes out)"}
         del host_codes
 
     cpu_baseline = None

@@ -191,6 +191,17 @@ int adapt_precision_search_host(const float* const* tensors, const int64_t* lens
                                 double* kld_out, int64_t* zeros_out, int32_t* best_out,
                                 const adapt_search_opts* opts);
 
+/* Host-buffer form of the whole switch step: the search as in
+ * adapt_precision_search_host, then Algorithm 1's re-quantisation of every
+ * layer at its selected <WL,FL>, from the same device copy of the layers (one
+ * upload serves both).
+ *   codes_out HOST array of n_layers HOST pointers, int32[lens[l]] each
+ * Everything else as adapt_precision_search_host; synchronous. */
+int adapt_precision_switch_host(const float* const* tensors, const int64_t* lens,
+                                int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                                double* kld_out, int64_t* zeros_out, int32_t* best_out,
+                                int32_t* const* codes_out, const adapt_search_opts* opts);
+
 /* Host-buffer form of adapt_quantize_ex: x and codes_out are HOST memory;
  * synchronous. */
 int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mode,

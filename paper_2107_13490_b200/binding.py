@@ -27,6 +27,7 @@ EXPORTS = (
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
     "adapt_search_workspace_bytes",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
+    "adapt_precision_switch_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
 )
@@ -95,6 +96,8 @@ def lib():
         L.adapt_precision_search_ex.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
         L.adapt_precision_search_host.restype = C.c_int
         L.adapt_precision_search_host.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
+        L.adapt_precision_switch_host.restype = C.c_int
+        L.adapt_precision_switch_host.argtypes = search_args + [C.c_void_p, C.POINTER(AdaptSearchOpts)]
         L.adapt_precision_search_static.restype = C.c_int
         L.adapt_precision_search_static.argtypes = search_args + [C.c_void_p]
         L.adapt_quantize_host.restype = C.c_int
@@ -334,6 +337,35 @@ def adapt_precision_search_host(tensors: Sequence[torch.Tensor], grid: Grid, n_b
                                              out.zeros.data_ptr(), out.best.data_ptr(),
                                              C.byref(o)), "adapt_precision_search_host")
     return out
+
+
+def adapt_precision_switch_host(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                                round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                                eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
+                                out: Optional[SearchResult] = None,
+                                codes_out: Optional[Sequence[torch.Tensor]] = None):
+    """Host-buffer search + quantization of every layer at its selected format.
+    Returns (SearchResult, list of CPU int32 code tensors)."""
+    assert all(not t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(grid)
+    if out is None:
+        out = SearchResult(torch.empty((L, Cn), dtype=torch.float64),
+                           torch.empty((L, Cn), dtype=torch.int64),
+                           torch.empty((L, 4), dtype=torch.int32))
+    if codes_out is None:
+        codes_out = [torch.empty(t.numel(), dtype=torch.int32) for t in tensors]
+    cptr = np.array([c.data_ptr() for c in codes_out], dtype=np.uint64)
+    o = AdaptSearchOpts()
+    o.round_mode, o.layer_base, o.seed = round_mode, layer_base, seed
+    o.eps, o.pseudo_count, o.log_base = eps, pseudo_count, log_base
+    o.stream = _stream_handle(None)
+    _check(lib().adapt_precision_switch_host(ptrs.ctypes.data, lens.ctypes.data, L,
+                                             C.byref(grid.c), n_bins, out.kld.data_ptr(),
+                                             out.zeros.data_ptr(), out.best.data_ptr(),
+                                             cptr.ctypes.data, C.byref(o)),
+           "adapt_precision_switch_host")
+    return out, codes_out
 
 
 def adapt_quantize_host(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROUND_RNE,

@@ -103,6 +103,7 @@ struct DeviceCache {
   void* stage_in = nullptr;    size_t stage_in_bytes = 0;    // host-form calls: inputs
   void* stage_out = nullptr;   size_t stage_out_bytes = 0;   // host-form calls: outputs
   void* batch_tab = nullptr;   size_t batch_tab_bytes = 0;   // batched quantize: layer table
+  void* stage_codes = nullptr; size_t stage_codes_bytes = 0; // host-form calls: codes
   PinnedSlot ring[kRingSlots];
   int ring_next = 0;
 };
@@ -605,10 +606,13 @@ int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected, 
   return run_quantize(x, n, 0, 0, selected, round_mode, seed, layer, 32, codes_out, stream);
 }
 
-int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* lens, int n_layers,
-                                  const int32_t* best, int round_mode, uint64_t seed,
-                                  int32_t layer_base, int32_t* const* codes_out, void* stream_handle) {
-  std::lock_guard<std::mutex> lock(g_mutex);
+}  // extern "C"
+
+namespace {
+// Body of adapt_quantize_selected_batch.  Caller holds g_mutex.
+int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_layers,
+                       const int32_t* best, int round_mode, uint64_t seed, int32_t layer_base,
+                       int32_t* const* codes_out, void* stream_handle) {
   if (!tensors || !lens || !best || !codes_out) return ADAPT_ERR_INVALID_ARG;
   if (n_layers < 1 || n_layers > 65535) return ADAPT_ERR_INVALID_ARG;
   if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
@@ -651,6 +655,17 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
   ADAPT_CUDA(cudaGetLastError());
   return ADAPT_OK;
 }
+}  // namespace
+
+extern "C" {
+
+int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* lens, int n_layers,
+                                  const int32_t* best, int round_mode, uint64_t seed,
+                                  int32_t layer_base, int32_t* const* codes_out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base, codes_out,
+                            stream_handle);
+}
 
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers, const adapt_grid* grid,
                                     int n_bins) {
@@ -679,10 +694,14 @@ int adapt_precision_search(const float* const* tensors, const int64_t* lens, int
                                    best_out, nullptr);
 }
 
-int adapt_precision_search_host(const float* const* tensors, const int64_t* lens, int n_layers,
-                                const adapt_grid* grid, int n_bins, double* kld_out,
-                                int64_t* zeros_out, int32_t* best_out,
-                                const adapt_search_opts* opts) {
+}  // extern "C"
+
+namespace {
+// Host-buffer search, optionally followed by the quantization of every layer at its selected
+// format from the same device copy (codes_out: HOST array of HOST int32 buffers, or null).
+int run_search_host(const float* const* tensors, const int64_t* lens, int n_layers,
+                    const adapt_grid* grid, int n_bins, double* kld_out, int64_t* zeros_out,
+                    int32_t* best_out, int32_t* const* codes_out, const adapt_search_opts* opts) {
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceCache* dc = nullptr;
   int rc = current_cache(&dc);
@@ -726,6 +745,23 @@ int adapt_precision_search_host(const float* const* tensors, const int64_t* lens
                reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes), o};
   rc = run_search(*dc, a);
   if (rc != ADAPT_OK) return rc;
+  if (codes_out) {
+    // codes of all layers in one more library-owned buffer, same offsets as the inputs
+    rc = grow_device(&dc->stage_codes, &dc->stage_codes_bytes, std::max<size_t>(in_bytes, 256));
+    if (rc != ADAPT_OK) return rc;
+    std::vector<int32_t*> dcodes(n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+      if (lens[l] > 0 && !codes_out[l]) return ADAPT_ERR_INVALID_ARG;
+      dcodes[l] = reinterpret_cast<int32_t*>(static_cast<char*>(dc->stage_codes) + off[l]);
+    }
+    rc = run_quantize_batch(dptr.data(), lens, n_layers, a.best_out, o.round_mode, o.seed,
+                            o.layer_base, dcodes.data(), o.stream);
+    if (rc != ADAPT_OK) return rc;
+    for (int l = 0; l < n_layers; ++l)
+      if (lens[l] > 0)
+        ADAPT_CUDA(cudaMemcpyAsync(codes_out[l], dcodes[l], sizeof(int32_t) * static_cast<size_t>(lens[l]),
+                                   cudaMemcpyDeviceToHost, stream));
+  }
   ADAPT_CUDA(cudaMemcpyAsync(kld_out, a.kld_out, sizeof(double) * L * C, cudaMemcpyDeviceToHost, stream));
   ADAPT_CUDA(cudaMemcpyAsync(zeros_out, a.zeros_out, sizeof(int64_t) * L * C, cudaMemcpyDeviceToHost, stream));
   ADAPT_CUDA(cudaMemcpyAsync(best_out, a.best_out, sizeof(int32_t) * 4 * L, cudaMemcpyDeviceToHost, stream));
@@ -736,6 +772,26 @@ int adapt_precision_search_host(const float* const* tensors, const int64_t* lens
     if (best_out[4 * l + 3] & ADAPT_FLAG_RANGE) status = ADAPT_ERR_RANGE;
   }
   return status;
+}
+}  // namespace
+
+extern "C" {
+
+int adapt_precision_search_host(const float* const* tensors, const int64_t* lens, int n_layers,
+                                const adapt_grid* grid, int n_bins, double* kld_out,
+                                int64_t* zeros_out, int32_t* best_out,
+                                const adapt_search_opts* opts) {
+  return run_search_host(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
+                         nullptr, opts);
+}
+
+int adapt_precision_switch_host(const float* const* tensors, const int64_t* lens, int n_layers,
+                                const adapt_grid* grid, int n_bins, double* kld_out,
+                                int64_t* zeros_out, int32_t* best_out, int32_t* const* codes_out,
+                                const adapt_search_opts* opts) {
+  if (!codes_out) return ADAPT_ERR_INVALID_ARG;
+  return run_search_host(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
+                         codes_out, opts);
 }
 
 int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
@@ -955,6 +1011,7 @@ int adapt_release(void) {
   if (dc->stage_in) { ADAPT_CUDA(cudaFree(dc->stage_in)); dc->stage_in = nullptr; dc->stage_in_bytes = 0; }
   if (dc->stage_out) { ADAPT_CUDA(cudaFree(dc->stage_out)); dc->stage_out = nullptr; dc->stage_out_bytes = 0; }
   if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
+  if (dc->stage_codes) { ADAPT_CUDA(cudaFree(dc->stage_codes)); dc->stage_codes = nullptr; dc->stage_codes_bytes = 0; }
   for (PinnedSlot& s : dc->ring) {
     if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }
     if (s.done) { ADAPT_CUDA(cudaEventDestroy(s.done)); s.done = nullptr; }

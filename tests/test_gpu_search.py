@@ -244,3 +244,10 @@ def test_host_buffer_form_matches(B):
                                         seed=w.seed)
     ora = O.precision_search(xs, wl, fl, w.n_bins, w.round_mode, w.seed, threads=G.host_threads())
     G.compare_search(res, ora, len(xs), "host form")
+    # search + re-quantisation of every layer from one upload
+    res2, codes = B.adapt_precision_switch_host(host, B.Grid(wl, fl), w.n_bins,
+                                                round_mode=w.round_mode, seed=w.seed)
+    G.compare_search(res2, ora, len(xs), "switch host form")
+    for l, x in enumerate(xs):
+        want, _ = O.quantize(x, int(ora[l]["best"][0]), int(ora[l]["best"][1]), w.round_mode, w.seed, l)
+        assert np.array_equal(codes[l].numpy(), want), l
