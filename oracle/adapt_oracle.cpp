@@ -14,6 +14,7 @@
 //                 quantized tensor, Q the float tensor (Sec. 3.3, Eq. dkld)
 //   select      - "smallest quantization s.t. KL = 0" (Sec. 3.3; Algorithm 3)
 //   sparsity    - share of non-zero elements (Sec. 3.4 "Inducing Sparsity")
+//   diversity   - gradient diversity of a layer's recent gradients (Sec. 3.3, PushUp)
 //
 // The paper gives no bit-level rules; the readings taken (saturation,
 // ties-to-even, the stochastic-rounding hash, bin arithmetic, the KLD
@@ -259,6 +260,37 @@ int adapt_oracle_precision_search(const float* x, int64_t n, uint64_t layer,
   adapt_oracle_select(kld_out, wl, fl, n_cand, eps, best_out);
   if (n == 0 || hi == lo) best_out[3] |= 2;
   return 0;
+}
+
+// ---- gradient diversity (PushUp's input) ---------------------------------------------
+
+// Gradient diversity of one layer over its last n_grads gradient tensors (Sec. 3.3, the
+// PushUp heuristic, Eq. ourgd / its log form):
+//   delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2 ,
+//   log form = log(delta_s) if 0 < delta_s < inf, else 1.
+// grads[k] points to n fp32 values; everything is accumulated in double, in index order.
+// out = {sum of norms, norm of the sum, delta_s, log form}.  0/0 gives NaN for delta_s
+// (log form 1); x/0 gives +inf (log form 1).
+void adapt_oracle_gradient_diversity(const float* const* grads, int n_grads, int64_t n,
+                                     double* out) {
+  double sum_norms = 0.0;
+  for (int k = 0; k < n_grads; ++k) {
+    double sq = 0.0;
+    for (int64_t i = 0; i < n; ++i) sq += static_cast<double>(grads[k][i]) * grads[k][i];
+    sum_norms += std::sqrt(sq);
+  }
+  double sq_sum = 0.0;
+  for (int64_t i = 0; i < n; ++i) {
+    double s = 0.0;
+    for (int k = 0; k < n_grads; ++k) s += grads[k][i];
+    sq_sum += s * s;
+  }
+  const double norm_sum = std::sqrt(sq_sum);
+  const double ds = sum_norms / norm_sum;
+  out[0] = sum_norms;
+  out[1] = norm_sum;
+  out[2] = ds;
+  out[3] = (ds > 0.0 && std::isfinite(ds)) ? std::log(ds) : 1.0;
 }
 
 }  // extern "C"

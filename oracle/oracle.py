@@ -73,6 +73,8 @@ def lib():
                 C.c_void_p, C.c_int64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                 C.c_int, C.c_uint64, C.c_double, C.c_double, C.c_double,
                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+            L.adapt_oracle_gradient_diversity.restype = None
+            L.adapt_oracle_gradient_diversity.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
             _lib = L
     return _lib
 
@@ -218,3 +220,15 @@ def precision_search(tensors, wl, fl, n_bins: int, round_mode: int = ROUND_RNE, 
         results.append({"kld": kl, "zeros": zeros, "best": best, "hist": hist, "range": rng,
                         "nonfinite": bad})
     return results
+
+
+def gradient_diversity(grads):
+    """grads: sequence of equally long fp32 arrays (one layer's recent gradients).
+    Returns float64[4] = {sum of norms, norm of the sum, delta_s, log form}."""
+    arrs = [_as_f32(g) for g in grads]
+    n = arrs[0].size if arrs else 0
+    assert all(a.size == n for a in arrs)
+    ptrs = (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+    out = np.zeros(4, dtype=np.float64)
+    lib().adapt_oracle_gradient_diversity(ptrs, len(arrs), n, out.ctypes.data)
+    return out
