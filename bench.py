@@ -46,6 +46,9 @@ def parse_args():
                     help="elements of the workload the CPU baseline is timed on")
     ap.add_argument("--elements", type=int, default=0,
                     help="profiling aid: shrink a single-layer workload to this many elements")
+    ap.add_argument("--path", default="search", choices=["search", "diversity"],
+                    help="search: the precision-switch search step (default); diversity: the "
+                         "gradient-diversity reduction that feeds PushUp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -202,10 +205,64 @@ def run_reference(args):
     return 0
 
 
+def run_diversity(args):
+    """Gradient-diversity reduction: one layer of 2^24 elements with 32 recent gradients
+    (2 GiB read per step), or --elements N."""
+    import torch
+    from paper_2107_13490_b200 import binding as B
+    from paper_2107_13490_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    n, k = (args.elements or (1 << 24)), 32
+    spec = W.LayerSpec("g", (n,), "laplace", 1e-4, zero_frac=0.05)
+    host = [W.generate_layer(spec, 7, j) for j in range(k)]
+    dev = [torch.from_numpy(g).cuda() for g in host]
+    out = torch.empty((1, 4), dtype=torch.float64, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        B.adapt_gradient_diversity([dev], out=out)
+    torch.cuda.synchronize()
+    B.adapt_kernel_times(reset=True)
+    B.adapt_kernel_timing(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        B.adapt_gradient_diversity([dev], out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    B.adapt_kernel_timing(False)
+    ms = e0.elapsed_time(e1) / args.steps
+    kt = B.adapt_kernel_times(reset=True)["diversity"]
+    peak, kind = measured_peak_gbs()
+    achieved = 4.0 * n * k / (kt[0] / args.steps * 1e-3) / 1e9
+    line = {"metric": "gradient-diversity element-gradients/s", "value": n * k / (ms * 1e-3),
+            "unit": "element-gradients/s", "n_gpus": 1, "steps": args.steps, "ms_per_step": ms,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"one layer, {n} elements, {k} Laplace(0,1e-4) gradients with 5% zeros",
+                       "l2": "inputs exceed L2" if 4 * n * k > 2 * 126e6 else "inputs may sit in L2"},
+            "roofline": {"bound": "hbm", "kernel": "diversity", "achieved": achieved, "peak": peak,
+                         "peak_kind": kind, "unit": "GB/s", "frac": achieved / peak, "traffic": None}}
+    if not args.no_cpu_baseline:
+        from oracle import oracle as O
+        m = min(n, 1 << 22)
+        t0 = time.perf_counter()
+        want = O.gradient_diversity([g[:m] for g in host])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": m * k / dt, "unit": "element-gradients/s", "cores": 1,
+                                "kind": "oracle", "sample": f"first {m} elements of each gradient"}
+        if m == n:
+            got = out.cpu().numpy()[0]
+            line["parity_rel_err"] = float(abs(got[2] - want[2]) / abs(want[2]))
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.path == "diversity":
+        return run_diversity(args)
 
     import torch
     from paper_2107_13490_b200 import binding as B

@@ -144,6 +144,22 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                                   uint64_t seed, int32_t layer_base,
                                   int32_t* const* codes_out, void* stream);
 
+/* Gradient diversity of each layer over its last n_grads gradient tensors -
+ * the quantity PushUp reads (Sec. 3.3, the gradient-diversity equation and its
+ * log form):  delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2, and
+ * log(delta_s) when 0 < delta_s < inf, else 1 (natural logarithm).
+ *   grads   HOST array of n_layers * n_grads DEVICE pointers, grads[l*n_grads+k]
+ *           = gradient k of layer l: fp32[lens[l]], 4-byte aligned
+ *   lens    HOST array of n_layers element counts
+ *   n_grads 1..256 gradient tensors per layer (the lookback)
+ *   out     DEVICE double[n_layers][4] = {sum of norms, norm of the sum,
+ *           delta_s, log form}; squares and sums are accumulated in double
+ * Pointer table and partial sums live in a library-owned device buffer that is
+ * allocated (and grown) inside the call; calls that use it must not overlap on
+ * the device. */
+int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
+                             int n_grads, double* out, void* stream);
+
 /* Bytes of DEVICE workspace the search needs for these sizes (0 on invalid
  * arguments).  lens is a HOST array. */
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers,
@@ -224,7 +240,8 @@ enum {
   ADAPT_KERNEL_EXPAND = 7,         /* cell counts -> per-level histograms      */
   ADAPT_KERNEL_SEARCH_DIRECT = 8,  /* fused kernel, direct form (every FL
                                       evaluated per element)                   */
-  ADAPT_KERNEL_KINDS = 9
+  ADAPT_KERNEL_DIVERSITY = 9,      /* gradient-diversity reduction              */
+  ADAPT_KERNEL_KINDS = 10
 };
 
 /* Switches per-kernel device timing on (non-zero) or off.  While on, every

@@ -25,7 +25,7 @@ OK, ERR_INVALID_ARG, ERR_NONFINITE, ERR_RANGE, ERR_CUDA, ERR_WORKSPACE = range(6
 EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
-    "adapt_search_workspace_bytes",
+    "adapt_search_workspace_bytes", "adapt_gradient_diversity",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_precision_switch_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
@@ -33,7 +33,7 @@ EXPORTS = (
 )
 STATIC_MAX_LAYERS, STATIC_MAX_BINS, STATIC_MAX_CAND = 8, 512, 1024
 KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize", "plan",
-                "expand", "search_direct")
+                "expand", "search_direct", "diversity")
 ALGO_AUTO, ALGO_KEYED, ALGO_DIRECT = 0, 1, 2
 
 
@@ -86,6 +86,9 @@ def lib():
         L.adapt_quantize_selected_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                                     C.c_int, C.c_uint64, C.c_int32, C.c_void_p,
                                                     C.c_void_p]
+        L.adapt_gradient_diversity.restype = C.c_int
+        L.adapt_gradient_diversity.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
+                                               C.c_void_p]
         L.adapt_search_workspace_bytes.restype = C.c_size_t
         L.adapt_search_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int]
         search_args = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int, C.c_void_p,
@@ -220,6 +223,27 @@ def adapt_quantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.T
                                                outs.ctypes.data, _stream_handle(stream)),
            "adapt_quantize_selected_batch")
     return codes_out
+
+
+def adapt_gradient_diversity(grads: Sequence[Sequence[torch.Tensor]],
+                             out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """grads[l][k] = gradient k of layer l (CUDA fp32, equal lengths within a layer).
+    Returns device float64[n_layers][4] = {sum of norms, norm of the sum, delta_s, log form}."""
+    n_layers, n_grads = len(grads), len(grads[0])
+    ptrs = np.zeros(n_layers * n_grads, dtype=np.uint64)
+    lens = np.zeros(n_layers, dtype=np.int64)
+    for l, gl in enumerate(grads):
+        assert len(gl) == n_grads
+        lens[l] = gl[0].numel()
+        for k, g in enumerate(gl):
+            assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous() and g.numel() == lens[l]
+            ptrs[l * n_grads + k] = g.data_ptr()
+    if out is None:
+        out = torch.empty((n_layers, 4), dtype=torch.float64, device=grads[0][0].device)
+    _check(lib().adapt_gradient_diversity(ptrs.ctypes.data, lens.ctypes.data, n_layers, n_grads,
+                                          out.data_ptr(), _stream_handle(stream)),
+           "adapt_gradient_diversity")
+    return out
 
 
 def adapt_search_workspace_bytes(lens: Sequence[int], grid: Grid, n_bins: int) -> int:

@@ -13,6 +13,7 @@
 
 #include "../../include/adapt.h"
 #include "common.cuh"
+#include "k_diversity.cuh"
 #include "k_expand.cuh"
 #include "k_kld_select.cuh"
 #include "k_plan.cuh"
@@ -104,6 +105,7 @@ struct DeviceCache {
   void* stage_out = nullptr;   size_t stage_out_bytes = 0;   // host-form calls: outputs
   void* batch_tab = nullptr;   size_t batch_tab_bytes = 0;   // batched quantize: layer table
   void* stage_codes = nullptr; size_t stage_codes_bytes = 0; // host-form calls: codes
+  void* div_buf = nullptr;     size_t div_buf_bytes = 0;     // gradient diversity: tables + sums
   PinnedSlot ring[kRingSlots];
   int ring_next = 0;
 };
@@ -667,6 +669,64 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                             stream_handle);
 }
 
+int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
+                             int n_grads, double* out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!grads || !lens || !out) return ADAPT_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > 65535 || n_grads < 1 || n_grads > kDivMaxGrads)
+    return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (lens[l] < 0) return ADAPT_ERR_INVALID_ARG;
+    for (int k = 0; k < n_grads; ++k) {
+      const float* g = grads[static_cast<size_t>(l) * n_grads + k];
+      if ((lens[l] > 0 && !g) || (reinterpret_cast<uintptr_t>(g) & 3u)) return ADAPT_ERR_INVALID_ARG;
+    }
+  }
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  const size_t L = n_layers, K = n_grads;
+  const size_t off_ptrs = align_up(sizeof(DivLayer) * (L + 1), 256);
+  const size_t blob = align_up(off_ptrs + sizeof(float*) * L * K, 256);
+  const size_t sums = sizeof(double) * L * (K + 1);
+  rc = grow_device(&dc->div_buf, &dc->div_buf_bytes, align_up(blob + sums, 4096));
+  if (rc != ADAPT_OK) return rc;
+  PinnedSlot* slot = nullptr;
+  rc = acquire_slot(*dc, blob, &slot);
+  if (rc != ADAPT_OK) return rc;
+  char* h = static_cast<char*>(slot->host);
+  DivLayer* hl = reinterpret_cast<DivLayer*>(h);
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    hl[l].n = lens[l]; hl[l].tile_begin = tiles;
+    tiles += (lens[l] + kDivTile - 1) / kDivTile;
+  }
+  hl[n_layers].n = 0; hl[n_layers].tile_begin = tiles;
+  std::memcpy(h + off_ptrs, grads, sizeof(float*) * L * K);
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+  char* d = static_cast<char*>(dc->div_buf);
+  ADAPT_CUDA(cudaMemcpyAsync(d, h, blob, cudaMemcpyHostToDevice, stream));
+  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  ADAPT_CUDA(cudaMemsetAsync(d + blob, 0, sums, stream));
+  DivParams dp;
+  dp.layers = reinterpret_cast<const DivLayer*>(d);
+  dp.grads = reinterpret_cast<const float* const*>(d + off_ptrs);
+  dp.sumsq = reinterpret_cast<double*>(d + blob);
+  dp.n_layers = n_layers; dp.n_grads = n_grads; dp.n_tiles = tiles;
+  if (tiles > 0) {
+    const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc->sm_count));
+    LaunchScope ls(ADAPT_KERNEL_DIVERSITY, stream);
+    diversity_kernel<<<grid, kDivThreads, 0, stream>>>(dp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_DIVERSITY, stream);
+    diversity_finalize_kernel<<<(n_layers + 127) / 128, 128, 0, stream>>>(dp.sumsq, n_layers, n_grads, out);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  return ADAPT_OK;
+}
+
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers, const adapt_grid* grid,
                                     int n_bins) {
   Plan plan;
@@ -1011,6 +1071,7 @@ int adapt_release(void) {
   if (dc->stage_in) { ADAPT_CUDA(cudaFree(dc->stage_in)); dc->stage_in = nullptr; dc->stage_in_bytes = 0; }
   if (dc->stage_out) { ADAPT_CUDA(cudaFree(dc->stage_out)); dc->stage_out = nullptr; dc->stage_out_bytes = 0; }
   if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
+  if (dc->div_buf) { ADAPT_CUDA(cudaFree(dc->div_buf)); dc->div_buf = nullptr; dc->div_buf_bytes = 0; }
   if (dc->stage_codes) { ADAPT_CUDA(cudaFree(dc->stage_codes)); dc->stage_codes = nullptr; dc->stage_codes_bytes = 0; }
   for (PinnedSlot& s : dc->ring) {
     if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }

@@ -1,0 +1,110 @@
+// Gradient diversity of each layer over its last K gradient tensors (Sec. 3.3, the PushUp
+// heuristic):  delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2 , log form = log(delta_s) if
+// 0 < delta_s < inf else 1.  A streaming reduction: every gradient element is read once
+// (4 B per element and tensor), squares and the element-wise sum are accumulated in double.
+#pragma once
+
+#include <math.h>
+
+#include "common.cuh"
+
+namespace adapt {
+
+constexpr int kDivThreads = 256;
+constexpr int kDivPerThread = 8;                        // elements per thread per tile
+constexpr int kDivTile = kDivThreads * kDivPerThread;   // 2048 elements
+constexpr int kDivMaxGrads = 256;                       // gradient tensors per layer
+
+struct DivLayer {
+  long long n;            // elements per gradient tensor
+  long long tile_begin;   // first tile of the layer in the launch's tile list
+};
+
+struct DivParams {
+  const DivLayer* layers;        // [n_layers + 1] (sentinel holds the tile total)
+  const float* const* grads;     // [n_layers][n_grads] device pointers
+  double* sumsq;                 // [n_layers][n_grads + 1]: per-gradient sums of squares, then
+                                 // the sum of squares of the element-wise sum
+  int n_layers, n_grads;
+  long long n_tiles;
+};
+
+__global__ void __launch_bounds__(kDivThreads) diversity_kernel(const DivParams p) {
+  __shared__ double s_sq[kDivMaxGrads + 1];
+  const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
+  long long t = per * blockIdx.x;
+  const long long t_end = min(p.n_tiles, t + per);
+  if (t >= t_end) return;
+  const int K = p.n_grads;
+  const int lane = threadIdx.x & 31;
+
+  int lo = 0, hi = p.n_layers - 1;          // layer that owns tile t
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (p.layers[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
+  }
+  int l = lo;
+  while (t < t_end) {
+    const DivLayer L = p.layers[l];
+    const long long layer_end = min(t_end, p.layers[l + 1].tile_begin);
+    const float* const* G = p.grads + static_cast<size_t>(l) * K;
+    for (int k = threadIdx.x; k <= K; k += kDivThreads) s_sq[k] = 0.0;
+    __syncthreads();
+    double sq_of_sum = 0.0;
+    for (; t < layer_end; ++t) {
+      const long long i0 = (t - L.tile_begin) * kDivTile + threadIdx.x;
+      double s[kDivPerThread];
+#pragma unroll
+      for (int j = 0; j < kDivPerThread; ++j) s[j] = 0.0;
+      for (int k = 0; k < K; ++k) {
+        const float* g = G[k];
+        float x[kDivPerThread];
+#pragma unroll
+        for (int j = 0; j < kDivPerThread; ++j) {
+          const long long i = i0 + static_cast<long long>(j) * kDivThreads;
+          x[j] = (i < L.n) ? __ldcs(g + i) : 0.0f;
+        }
+        double sq = 0.0;
+#pragma unroll
+        for (int j = 0; j < kDivPerThread; ++j) {
+          const double d = static_cast<double>(x[j]);
+          sq = fma(d, d, sq);
+          s[j] += d;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (lane == 0) atomicAdd(&s_sq[k], sq);
+      }
+#pragma unroll
+      for (int j = 0; j < kDivPerThread; ++j) sq_of_sum = fma(s[j], s[j], sq_of_sum);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq_of_sum += __shfl_xor_sync(0xffffffffu, sq_of_sum, o);
+    if (lane == 0) atomicAdd(&s_sq[K], sq_of_sum);
+    __syncthreads();
+    double* out = p.sumsq + static_cast<size_t>(l) * (K + 1);
+    for (int k = threadIdx.x; k <= K; k += kDivThreads)
+      if (s_sq[k] != 0.0) atomicAdd(&out[k], s_sq[k]);
+    __syncthreads();
+    ++l;
+    while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
+  }
+}
+
+// One thread per layer: norms from the sums of squares, then the two forms of the diversity.
+__global__ void diversity_finalize_kernel(const double* __restrict__ sumsq, int n_layers,
+                                          int n_grads, double* __restrict__ out) {
+  const int l = blockIdx.x * blockDim.x + threadIdx.x;
+  if (l >= n_layers) return;
+  const double* q = sumsq + static_cast<size_t>(l) * (n_grads + 1);
+  double sum_norms = 0.0;
+  for (int k = 0; k < n_grads; ++k) sum_norms += sqrt(q[k]);
+  const double norm_sum = sqrt(q[n_grads]);
+  const double ds = sum_norms / norm_sum;
+  out[4 * l + 0] = sum_norms;
+  out[4 * l + 1] = norm_sum;
+  out[4 * l + 2] = ds;
+  out[4 * l + 3] = (ds > 0.0 && ds < __longlong_as_double(0x7ff0000000000000ll)) ? log(ds) : 1.0;
+}
+
+}  // namespace adapt
