@@ -698,10 +698,12 @@ int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int
   DivLayer* hl = reinterpret_cast<DivLayer*>(h);
   long long tiles = 0;
   for (int l = 0; l < n_layers; ++l) {
-    hl[l].n = lens[l]; hl[l].tile_begin = tiles;
+    hl[l].n = lens[l]; hl[l].tile_begin = tiles; hl[l].vec = 1; hl[l].pad_ = 0;
+    for (int k = 0; k < n_grads; ++k)
+      if (reinterpret_cast<uintptr_t>(grads[static_cast<size_t>(l) * n_grads + k]) & 15u) hl[l].vec = 0;
     tiles += (lens[l] + kDivTile - 1) / kDivTile;
   }
-  hl[n_layers].n = 0; hl[n_layers].tile_begin = tiles;
+  hl[n_layers].n = 0; hl[n_layers].tile_begin = tiles; hl[n_layers].vec = 0; hl[n_layers].pad_ = 0;
   std::memcpy(h + off_ptrs, grads, sizeof(float*) * L * K);
   cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
   char* d = static_cast<char*>(dc->div_buf);
@@ -714,7 +716,7 @@ int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int
   dp.sumsq = reinterpret_cast<double*>(d + blob);
   dp.n_layers = n_layers; dp.n_grads = n_grads; dp.n_tiles = tiles;
   if (tiles > 0) {
-    const int grid = static_cast<int>(std::min<long long>(tiles, 8ll * dc->sm_count));
+    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc->sm_count));
     LaunchScope ls(ADAPT_KERNEL_DIVERSITY, stream);
     diversity_kernel<<<grid, kDivThreads, 0, stream>>>(dp);
     ADAPT_CUDA(cudaGetLastError());

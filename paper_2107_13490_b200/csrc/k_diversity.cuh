@@ -10,14 +10,16 @@
 
 namespace adapt {
 
-constexpr int kDivThreads = 256;
-constexpr int kDivPerThread = 8;                        // elements per thread per tile
+constexpr int kDivThreads = 128;
+constexpr int kDivPerThread = 16;                       // elements per thread per tile (4 quads)
 constexpr int kDivTile = kDivThreads * kDivPerThread;   // 2048 elements
 constexpr int kDivMaxGrads = 256;                       // gradient tensors per layer
 
 struct DivLayer {
   long long n;            // elements per gradient tensor
   long long tile_begin;   // first tile of the layer in the launch's tile list
+  int vec;                // every gradient pointer of the layer is 16-byte aligned
+  int pad_;
 };
 
 struct DivParams {
@@ -52,17 +54,28 @@ __global__ void __launch_bounds__(kDivThreads) diversity_kernel(const DivParams 
     __syncthreads();
     double sq_of_sum = 0.0;
     for (; t < layer_end; ++t) {
-      const long long i0 = (t - L.tile_begin) * kDivTile + threadIdx.x;
+      const long long tile_first = (t - L.tile_begin) * kDivTile;
+      const long long i0 = tile_first + threadIdx.x;
       double s[kDivPerThread];
 #pragma unroll
       for (int j = 0; j < kDivPerThread; ++j) s[j] = 0.0;
       for (int k = 0; k < K; ++k) {
         const float* g = G[k];
         float x[kDivPerThread];
+        // which elements a thread takes only has to be the same for every k of the tile
+        if (L.vec && tile_first + kDivTile <= L.n) {       // full tile, aligned: 128-bit loads
 #pragma unroll
-        for (int j = 0; j < kDivPerThread; ++j) {
-          const long long i = i0 + static_cast<long long>(j) * kDivThreads;
-          x[j] = (i < L.n) ? __ldcs(g + i) : 0.0f;
+          for (int q = 0; q < kDivPerThread / 4; ++q) {
+            const float4 v4 = __ldcs(reinterpret_cast<const float4*>(g + tile_first) +
+                                     q * kDivThreads + threadIdx.x);
+            x[4 * q] = v4.x; x[4 * q + 1] = v4.y; x[4 * q + 2] = v4.z; x[4 * q + 3] = v4.w;
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < kDivPerThread; ++j) {
+            const long long i = i0 + static_cast<long long>(j) * kDivThreads;
+            x[j] = (i < L.n) ? __ldcs(g + i) : 0.0f;
+          }
         }
         double sq = 0.0;
 #pragma unroll
