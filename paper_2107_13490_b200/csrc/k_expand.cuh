@@ -9,7 +9,7 @@
 //     added here, and their level-by-level moves already sit in U);
 //   * coarse levels (f < G), every cell: the rounded value rint(x * 2^f) of any
 //     element of the cell is a + (rem >= half), with c = a * 2^d + rem,
-//     d = G - f (ties that go down were fixed up element by element);
+//     d = G - f (grid points whose tie goes down were counted in the cell to their left);
 // then the exact zeros (layer size minus all cell counts) at the bin of 0, and
 // for the zero counts the cells that round to 0 plus, at fine levels of the
 // main segment, the zero classes.  The result is added to the corrections

@@ -3,10 +3,10 @@
 // Idea.  Cut the value axis into cells of width 2^-G.  An element x lies in
 // cell c = floor(x * 2^G).  Then, exactly:
 //  * for every coarser level f < G the rounded value rint(x * 2^f) is a
-//    function of c alone (unless x sits exactly on the level-G grid AND on a
-//    rounding tie of level f - at most one level per element, fixed up
-//    separately), so one count per cell yields the histograms of all coarse
-//    levels afterwards;
+//    function of c alone (an x exactly on the level-G grid is a rounding tie at
+//    one coarser level; it is counted in the cell to its left when that tie
+//    rounds down, which settles it), so one count per cell yields the
+//    histograms of all coarse levels afterwards;
 //  * for every finer level f >= G the rounded value stays inside the closed
 //    cell, so if the whole closed cell lies in one bin ("interior cell") the
 //    element falls in that bin at every fine level and in the float histogram;
@@ -54,7 +54,7 @@ struct SegPlan {
   int fs;         // first fine level: max(G, 0)
   int offset;     // position of the segment's first cell in the layer's table
   float two_g;    // 2^G
-  float c0f;      // (float)c0 (exact)
+  float c0f;      // (float)(c0 + 1) = floor(left end * 2^G), exact; c0 itself counts the spare cell
   float magic;    // 1.5 * 2^23 - c0 + offset: x * 2^G + magic, rounded down, has the
                   // table position in its low mantissa bits (fast layers only)
   int pad_;
@@ -92,17 +92,17 @@ __device__ inline void fit_segment(float lo, float hi, int max_cells, int g_max,
   long long c0 = 0, c1 = 0;
   for (; g > -100; --g) {
     const double span = ldexp(static_cast<double>(hi) - static_cast<double>(lo), g);
-    if (span >= static_cast<double>(max_cells)) continue;
+    if (span + 1.0 >= static_cast<double>(max_cells)) continue;
     if (fabs(ldexp(static_cast<double>(hi), g)) > 9.0e18 ||
         fabs(ldexp(static_cast<double>(lo), g)) > 9.0e18) continue;
-    c0 = floor_scaled(lo, g);
+    c0 = floor_scaled(lo, g) - 1;   // one spare cell on the left (grid points that go left)
     c1 = floor_scaled(hi, g);
     if (c1 - c0 + 1 <= max_cells) break;
   }
   s->g = g; s->c0 = c0; s->cells = static_cast<int>(c1 - c0 + 1);
   s->fs = g > 0 ? g : 0;
   s->two_g = pow2f(g);
-  s->c0f = static_cast<float>(c0);
+  s->c0f = static_cast<float>(c0 + 1);   // floor(lo * 2^G): exactly representable
 }
 
 // Level at which a bin of width bw holds about `ratio` cells (no need to go finer).

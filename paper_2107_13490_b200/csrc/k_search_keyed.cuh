@@ -4,17 +4,17 @@
 //
 // Per element x != 0:   pos = table position of x's cell;  old = atomicAdd(cell[pos], 1)
 // The returned word carries the cell's marks in its two top bits:
-//   bit 30 (cell -1 / 0 of the main segment), bit 31 (edge cell), or x exactly on its
-//          segment's grid: the element goes to a per-warp queue that the warp drains
-//          32 entries at a time:
+//   bit 30 (cell -1 / 0 of the main segment) or bit 31 (edge cell): the element goes to
+//          a per-warp queue that the warp drains 32 entries at a time:
 //            cell -1 / 0: the element is added to the class counter "highest level at
 //              which it still rounds to zero";
 //            edge entry: b0 = bin(x) into the segment's edge-element histogram,
 //              then only the fine levels f whose half quantum can reach one of
 //              the bin's edges are evaluated; a level is recorded only if its
-//              bin differs from b0 (-1 at b0, +1 at the new bin);
-//            on-grid entry: the one coarse level at which x is a rounding tie
-//              that goes down is corrected (the cell table assumes "up").
+//              bin differs from b0 (-1 at b0, +1 at the new bin).
+// An element exactly on the cell grid is counted in the cell to its left or right according to
+// the parity rule of grid_point_goes_left (its handler moves the count when it belongs left),
+// which makes every coarse rounding tie come out even.
 // Exact zeros are sent to per-lane dummy slots (their number is the layer size
 // minus the sum of the cell counts).  Everything else about an element - the
 // float histogram, all coarse levels, all fine levels of interior cells - is
@@ -50,7 +50,7 @@ struct KeyedParams {
   unsigned* cell_count;        // [layer][cell_cap]      global cell counts
   unsigned* qe_hist;           // [layer][2][n_bins]     float histogram of the edge elements, per segment
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
-  unsigned long long* zeros;   // [layer][n_levels]      receives tie corrections
+  unsigned long long* zeros;   // [layer][n_levels]
   unsigned long long* zero_class;  // [layer][kZeroClasses]
   unsigned long long* cell_total;  // [layer] sum of all cell counts = non-zero elements
   int n_bins;
@@ -73,7 +73,7 @@ struct LayerCtx {
   long long c0[2];
   int g[2], fs[2], offset[2];
   const float* E;              // exact bin edges [n_bins + 1]
-  const unsigned* cells;       // shared cell table (marks in the two top bits)
+  unsigned* cells;             // shared cell table (marks in the two top bits)
   unsigned* qe;                // shared [n_bins]: main segment's edge-element histogram
   int* d;                      // shared [d_levels][n_bins]
   unsigned* qe_aux;            // global [n_bins]: auxiliary segment's edge-element histogram
@@ -85,6 +85,18 @@ struct LayerCtx {
   int keyed, fast, total_cells;
 };
 
+// An element that sits exactly on its segment's grid (x * 2^G = p, an integer) is a rounding
+// tie at exactly one coarser level (the one whose half quantum is p's lowest set bit), where
+// it must go to the even neighbour a or a + 1, a = p >> (lowest set bit + 1).  The cell table
+// derives coarse levels from the cell index alone, and cell p rounds such a tie up while cell
+// p - 1 rounds it down; at every other level, and as closed intervals for the fine levels, both
+// cells serve p equally.  So the element is counted in cell p - 1 when a is even, in cell p
+// when a is odd: no correction is ever needed.  (Each segment has one spare cell on its left.)
+__device__ __forceinline__ int grid_point_goes_left(long long p) {
+  const long long low = p & -p;
+  return (p & (low << 1)) == 0 ? 1 : 0;
+}
+
 // Handles one queued element (x != 0, finite).  No warp-level primitive inside:
 // any subset of lanes may call it.
 __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
@@ -92,8 +104,13 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   const int s = (fabsf(x) < c.radius) ? 0 : 1;
   const float z = __fmul_rn(x, c.two_g[s]);
   const float cf = floorf(z);
-  const int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s]));   // cell index inside the segment
-  const int g = c.g[s];
+  int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s])) + 1;     // cell index inside the segment
+  if (z == cf && grid_point_goes_left(c.c0[s] + ci)) {
+    // on the grid and belonging to the left cell: move its count there
+    atomicSub(&c.cells[c.offset[s] + ci], 1u);
+    ci -= 1;
+    atomicAdd(&c.cells[c.offset[s] + ci], 1u);
+  }
   const long long cc = c.c0[s] + ci;
   // ---- cells -1 / 0 of the main segment: the zero class of x --------------------------
   if (s == 0 && (cc == 0 || cc == -1)) {
@@ -102,25 +119,6 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     int kz = 125 - static_cast<int>((ax - 1u) >> 23);
     kz = max(-1, min(kz, 32));
     atomicAdd(&c.zclass[kz + 1], 1u);
-  }
-  // ---- x on the segment's grid: fix the single coarse level at which it is a tie ----
-  if (z == cf) {
-    if (cc != 0) {
-      const int tz = __ffsll(cc) - 1;          // lowest set bit
-      const int ft = g - 1 - tz;               // the level at which x is a tie
-      if (ft >= 0 && ft < c.n_levels) {
-        const long long a = cc >> (tz + 1);    // floor(x * 2^ft)
-        if ((a & 1ll) == 0) {                  // tie goes down to a; the table counted a + 1
-          const float sc = pow2f(-ft);
-          const int b_up = bin_of(__fmul_rn(__ll2float_rn(a + 1), sc), c.lo, c.scale, c.bmax);
-          const int b_dn = bin_of(__fmul_rn(__ll2float_rn(a), sc), c.lo, c.scale, c.bmax);
-          unsigned* U = c.u_hist + static_cast<size_t>(ft) * B;
-          if (b_up != b_dn) { atomicAdd(&U[b_up], 0xFFFFFFFFu); atomicAdd(&U[b_dn], 1u); }
-          if (a + 1 == 0) atomicAdd(&c.zeros[ft], 0xFFFFFFFFFFFFFFFFull);
-          if (a == 0) atomicAdd(&c.zeros[ft], 1ull);
-        }
-      }
-    }
   }
   // ---- edge cell: float bin, then the fine levels that can still move ----------------
   if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
@@ -157,24 +155,27 @@ struct CellFn {
   float two_g1, magic1;         // auxiliary segment (fast layers only)
 };
 
-// Table position of x.  Fast form: adding the segment's magic constant
-// (1.5 * 2^23 - c0 + offset) to x * 2^G with round-down leaves the position in
-// the low mantissa bits; x is on the grid exactly when round-up gives the same.
+// Table position of x.  Fast form (all cell indices below 2^22 in magnitude): adding the
+// segment's magic constant 1.5 * 2^23 - c0 + offset to x * 2^G with round-down leaves the
+// position in the low mantissa bits; x is on the grid exactly when round-up gives the same.
+// General form (range far from zero): x * 2^G - c0 is formed first - exact, both are close -
+// and the same constant trick is applied to the difference.
 template <bool kFast>
 __device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_grid) {
+  float rd, ru;
   if (kFast) {
     const bool inner = fabsf(x) < f.radius;
     const float s = inner ? f.two_g0 : f.two_g1;
     const float mg = inner ? f.magic0 : f.magic1;
-    const float rd = __fmaf_rd(x, s, mg);
-    const float ru = __fmaf_ru(x, s, mg);
-    *on_grid = (rd == ru);
-    return __float_as_int(rd) - 0x4B400000;
+    rd = __fmaf_rd(x, s, mg);
+    ru = __fmaf_ru(x, s, mg);
+  } else {
+    const float t = __fmaf_rn(x, f.two_g0, -f.c0f0);     // x * 2^G - (c0 + 1), exact
+    rd = __fadd_rd(t, 12582913.0f);
+    ru = __fadd_ru(t, 12582913.0f);
   }
-  const float z = __fmul_rn(x, f.two_g0);
-  const float cf = floorf(z);
-  *on_grid = (z == cf);
-  return __float2int_rz(__fsub_rn(cf, f.c0f0));
+  *on_grid = (rd == ru);
+  return __float_as_int(rd) - 0x4B400000;
 }
 
 // One tile: this thread's four quads are loaded first (guarded loads when the tile is ragged),
@@ -209,25 +210,13 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float x = v[q][k];
-      unsigned o;
-      if (kFast && kFull) {
-        // both segments' products are formed (FMA pipe) and one is kept, instead of selecting
-        // scale and constant first (two selects on the narrower ALU pipe)
-        const bool inner = fabsf(x) < fn.radius;
-        const float rd = inner ? __fmaf_rd(x, fn.two_g0, fn.magic0) : __fmaf_rd(x, fn.two_g1, fn.magic1);
-        const float ru = inner ? __fmaf_ru(x, fn.two_g0, fn.magic0) : __fmaf_ru(x, fn.two_g1, fn.magic1);
-        const bool nz = (x != 0.0f);
-        const int pos = nz ? (__float_as_int(rd) - 0x4B400000) : dummy_pos;
-        o = atomicAdd(&cells[pos], 1u);
-        o = (nz && rd == ru) ? (o | kCellEdge) : o;
-      } else {
-        bool on_grid;
-        int pos = cell_position<kFast>(x, fn, &on_grid);
-        const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
-        pos = nz ? pos : dummy_pos;
-        o = atomicAdd(&cells[pos], 1u);
-        o = (nz && on_grid) ? (o | kCellEdge) : o;   // an on-grid element is queued like an edge one
-      }
+      bool on_grid;
+      int pos = cell_position<kFast>(x, fn, &on_grid);
+      const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
+      pos = nz ? pos : dummy_pos;
+      unsigned o = atomicAdd(&cells[pos], 1u);
+      // an element on the cell grid is queued too: its handler may move it one cell to the left
+      o = (nz && on_grid) ? (o | kCellEdge) : o;
       old[k] = o;
       any |= o;
     }
