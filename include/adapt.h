@@ -84,6 +84,24 @@ typedef struct adapt_search_opts {
                              histogram of candidate c's dequantized tensor      */
   float* range_out;       /* DEVICE, optional: float[n_layers][2] = {min, max}  */
   int32_t algorithm;      /* ADAPT_ALGO_*: which form of the fused kernel runs  */
+  const int32_t* n_bins_per_layer; /* HOST, optional: int32[n_layers], the resolution
+                             r^l of each layer (Sec. 3.3: bins are a per-layer
+                             quantity).  When set, the n_bins argument is ignored
+                             for the bin arithmetic; hist_out and the workspace
+                             are laid out for the largest value, which is also
+                             what adapt_search_workspace_bytes must be asked for;
+                             bins of hist_out beyond a layer's own count are not
+                             written                                             */
+  const int32_t* start_wl_fl; /* HOST, optional: int32[n_layers][2], each layer's
+                             current <WL,FL>.  When set, best_out is PushDown as
+                             Algorithm 3 walks it: from that format step down the
+                             (WL, FL) order of the grid while KLD <= eps and
+                             return the lowest format reached before the first
+                             violation (flag "met eps" cleared and the start
+                             returned if the start itself violates; grid index
+                             -1 if the start is not in the grid).  When NULL,
+                             best_out is the lowest admissible format of the
+                             whole grid                                          */
 } adapt_search_opts;
 
 /* Forms of the fused quantize / zero-count / histogram kernel.  Both give the

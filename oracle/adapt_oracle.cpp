@@ -26,6 +26,7 @@
 //
 // Build: g++ -std=c++17 -O2 -ffp-contract=off -fno-fast-math -shared -fPIC
 
+#include <algorithm>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -213,6 +214,34 @@ void adapt_oracle_select(const double* kld, const int32_t* wl, const int32_t* fl
   out[1] = pick >= 0 ? fl[pick] : 0;
   out[2] = pick;
   out[3] = best_ok >= 0 ? 1 : 0;
+}
+
+// PushDown as a descent from the layer's current format (Algorithm 3: starting at the
+// current <WL,FL>, Decrease and re-test until the divergence tells that a coarser format would
+// lose information).  Candidates are ordered by (WL, FL); Decrease steps to the previous
+// candidate in that order.  The walk starts at the candidate equal to <start_wl, start_fl> and
+// stops before the first candidate whose divergence exceeds eps; it returns the lowest format
+// reached.  If the start itself exceeds eps it is returned with the "met eps" flag cleared;
+// a start that is not in the grid gives grid index -1.
+void adapt_oracle_select_descent(const double* kld, const int32_t* wl, const int32_t* fl,
+                                 int n_cand, double eps, int start_wl, int start_fl,
+                                 int32_t* out) {
+  std::vector<int> order(n_cand);
+  for (int c = 0; c < n_cand; ++c) order[c] = c;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    if (wl[a] != wl[b]) return wl[a] < wl[b];
+    return fl[a] < fl[b];
+  });
+  int pos = -1;
+  for (int i = 0; i < n_cand; ++i)
+    if (wl[order[i]] == start_wl && fl[order[i]] == start_fl) { pos = i; break; }
+  if (pos < 0) { out[0] = start_wl; out[1] = start_fl; out[2] = -1; out[3] = 0; return; }
+  const bool ok = kld[order[pos]] <= eps;
+  if (ok) while (pos > 0 && kld[order[pos - 1]] <= eps) --pos;
+  out[0] = wl[order[pos]];
+  out[1] = fl[order[pos]];
+  out[2] = order[pos];
+  out[3] = ok ? 1 : 0;
 }
 
 // The whole search for one layer, one candidate at a time, in the order the

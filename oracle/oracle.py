@@ -73,6 +73,9 @@ def lib():
                 C.c_void_p, C.c_int64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                 C.c_int, C.c_uint64, C.c_double, C.c_double, C.c_double,
                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+            L.adapt_oracle_select_descent.restype = None
+            L.adapt_oracle_select_descent.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                                                      C.c_double, C.c_int, C.c_int, C.c_void_p]
             L.adapt_oracle_gradient_diversity.restype = None
             L.adapt_oracle_gradient_diversity.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
             _lib = L
@@ -141,6 +144,17 @@ def select(kld_values, wl, fl, eps: float = 0.0):
     out = np.zeros(4, dtype=np.int32)
     lib().adapt_oracle_select(k.ctypes.data, w.ctypes.data, f.ctypes.data, k.size, eps,
                               out.ctypes.data)
+    return out
+
+
+def select_descent(kld_values, wl, fl, start_wl: int, start_fl: int, eps: float = 0.0):
+    """PushDown as a descent from <start_wl, start_fl>; returns int32[4] {wl, fl, index, flags}."""
+    k = np.ascontiguousarray(kld_values, dtype=np.float64)
+    w = np.ascontiguousarray(wl, dtype=np.int32)
+    f = np.ascontiguousarray(fl, dtype=np.int32)
+    out = np.zeros(4, dtype=np.int32)
+    lib().adapt_oracle_select_descent(k.ctypes.data, w.ctypes.data, f.ctypes.data, k.size, eps,
+                                      start_wl, start_fl, out.ctypes.data)
     return out
 
 

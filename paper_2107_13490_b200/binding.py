@@ -45,7 +45,8 @@ class AdaptSearchOpts(C.Structure):
     _fields_ = [("round_mode", C.c_int32), ("layer_base", C.c_int32), ("seed", C.c_uint64),
                 ("eps", C.c_double), ("pseudo_count", C.c_double), ("log_base", C.c_double),
                 ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-                ("hist_out", C.c_void_p), ("range_out", C.c_void_p), ("algorithm", C.c_int32)]
+                ("hist_out", C.c_void_p), ("range_out", C.c_void_p), ("algorithm", C.c_int32),
+                ("n_bins_per_layer", C.c_void_p), ("start_wl_fl", C.c_void_p)]
 
 
 class AdaptError(RuntimeError):
@@ -312,17 +313,26 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
                               stream=None, workspace: Optional[torch.Tensor] = None,
                               want_hist: bool = False, want_range: bool = False,
                               out: Optional[SearchResult] = None,
-                              algorithm: int = ALGO_AUTO) -> SearchResult:
+                              algorithm: int = ALGO_AUTO,
+                              n_bins_per_layer: Optional[Sequence[int]] = None,
+                              start_wl_fl: Optional[Sequence[Sequence[int]]] = None) -> SearchResult:
     dev = tensors[0].device
     assert all(t.is_cuda for t in tensors)
     ptrs, lens = _marshal_tensors(tensors)
     L, Cn = len(tensors), len(grid)
+    per_layer = start = None
+    if n_bins_per_layer is not None:
+        per_layer = np.ascontiguousarray(n_bins_per_layer, dtype=np.int32)
+        assert per_layer.size == L
+        n_bins = int(per_layer.max())          # stride of hist_out and of the workspace
+    if start_wl_fl is not None:
+        start = np.ascontiguousarray(start_wl_fl, dtype=np.int32).reshape(L, 2)
     if out is None:
         out = SearchResult(
             torch.empty((L, Cn), dtype=torch.float64, device=dev),
             torch.empty((L, Cn), dtype=torch.int64, device=dev),
             torch.empty((L, 4), dtype=torch.int32, device=dev),
-            torch.empty((L, Cn + 1, n_bins), dtype=torch.int32, device=dev) if want_hist else None,
+            torch.zeros((L, Cn + 1, n_bins), dtype=torch.int32, device=dev) if want_hist else None,
             torch.empty((L, 2), dtype=torch.float32, device=dev) if want_range else None)
     o = AdaptSearchOpts()
     o.round_mode, o.layer_base, o.seed = round_mode, layer_base, seed
@@ -333,6 +343,8 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
     o.hist_out = out.hist.data_ptr() if out.hist is not None else None
     o.range_out = out.range.data_ptr() if out.range is not None else None
     o.algorithm = algorithm
+    o.n_bins_per_layer = per_layer.ctypes.data if per_layer is not None else None
+    o.start_wl_fl = start.ctypes.data if start is not None else None
     _check(lib().adapt_precision_search_ex(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
                                            n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
                                            out.best.data_ptr(), C.byref(o)),

@@ -168,7 +168,7 @@ struct Plan {
   size_t keyed_smem = 0;
   // byte offsets inside the workspace -- descriptor block (uploaded)
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
-         off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_state = 0, blob_bytes = 0;
+         off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_start = 0, off_state = 0, blob_bytes = 0;
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
   // accumulators (cleared every call)
@@ -235,6 +235,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_order = o;   o = align_up(o + sizeof(int) * C, 16);
   p->off_by_fl = o;   o = align_up(o + sizeof(int) * C, 16);
   p->off_fl_begin = o; o = align_up(o + sizeof(int) * (F + 1), 16);
+  p->off_start = o;   o = align_up(o + sizeof(int) * 2 * L, 16);
   p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
   p->blob_bytes = o;
   p->off_plan = o;      o = align_up(o + sizeof(LayerPlan) * L, 256);
@@ -291,11 +292,11 @@ long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchAr
     d.mis = a.lens[l] > 0 ? mis : 0;
     d.layer_id = a.opts.layer_base + l;
     d.index = l;
-    d.pad_ = 0;
+    d.n_bins = a.opts.n_bins_per_layer ? a.opts.n_bins_per_layer[l] : a.n_bins;
     if (a.lens[l] > 0) tiles += (a.lens[l] + mis + tile - 1) / tile;
   }
   LayerDesc& s = out[k];
-  s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.pad_ = 0;
+  s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.n_bins = 1;
   return tiles;
 }
 
@@ -309,8 +310,18 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   const double base = (o.log_base == 0.0) ? 2.0 : o.log_base;
   if (!(base > 0.0) || base == 1.0 || !std::isfinite(base)) return ADAPT_ERR_INVALID_ARG;
 
+  // per-layer resolutions: the arrays are laid out with the largest one as their stride
+  int bins_stride = a.n_bins;
+  if (o.n_bins_per_layer) {
+    if (a.n_layers < 1) return ADAPT_ERR_INVALID_ARG;
+    bins_stride = 0;
+    for (int l = 0; l < a.n_layers; ++l) {
+      if (o.n_bins_per_layer[l] < 1 || o.n_bins_per_layer[l] > kMaxBins) return ADAPT_ERR_INVALID_ARG;
+      bins_stride = std::max(bins_stride, o.n_bins_per_layer[l]);
+    }
+  }
   Plan plan;
-  if (!make_plan(a.lens, a.n_layers, a.grid, a.n_bins, &plan)) return ADAPT_ERR_INVALID_ARG;
+  if (!make_plan(a.lens, a.n_layers, a.grid, bins_stride, &plan)) return ADAPT_ERR_INVALID_ARG;
   for (int l = 0; l < a.n_layers; ++l) {
     if (a.lens[l] > 0 && !a.tensors[l]) return ADAPT_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(a.tensors[l]) & 3u) return ADAPT_ERR_INVALID_ARG;
@@ -357,6 +368,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   std::memcpy(h + plan.off_order, plan.order.data(), sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_by_fl, plan.by_fl.data(), sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_fl_begin, plan.fl_begin.data(), sizeof(int) * (plan.n_levels + 1));
+  if (o.start_wl_fl) std::memcpy(h + plan.off_start, o.start_wl_fl, sizeof(int) * 2 * a.n_layers);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
   for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
@@ -388,7 +400,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   {
     LaunchScope ls(ADAPT_KERNEL_RANGE_FINALIZE, stream);
     range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
-        d_layers, a.n_layers, a.n_bins, d_state, o.range_out);
+        d_layers, a.n_layers, d_state, o.range_out);
     ADAPT_CUDA(cudaGetLastError());
   }
 
@@ -397,7 +409,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     const int nk = static_cast<int>(keyed.size());
     PlanParams pp;
     pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
-    pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = a.n_bins; pp.cell_cap = plan.cell_cap;
+    pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = bins_stride; pp.cell_cap = plan.cell_cap;
     pp.fine_ratio = ADAPT_FINE_RATIO;
     const int keyed_grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
     pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
@@ -412,7 +424,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
     kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
     kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
-    kp.n_bins = a.n_bins; kp.n_levels = plan.n_levels;
+    kp.n_bins = bins_stride; kp.n_levels = plan.n_levels;
     kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(plan.keyed_smem)));
@@ -427,12 +439,12 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
     ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
     ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
-    ep.n_bins = a.n_bins; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
+    ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
     {
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
       const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / ((plan.n_levels + 1) * nk)));
       expand_kernel<<<dim3(plan.n_levels + 1, nk, slices), kExpandThreads,
-                      sizeof(unsigned) * a.n_bins, stream>>>(ep);
+                      sizeof(unsigned) * bins_stride, stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
   }
@@ -441,10 +453,10 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   if (!direct.empty() && direct_tiles > 0) {
     SearchParams sp;
     sp.layers = d_direct; sp.state = d_state;
-    sp.n_layers = static_cast<int>(direct.size()); sp.n_fl = plan.n_levels; sp.n_bins = a.n_bins;
+    sp.n_layers = static_cast<int>(direct.size()); sp.n_fl = plan.n_levels; sp.n_bins = bins_stride;
     sp.n_tiles = direct_tiles;
     sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed;
-    const size_t per_hist = sizeof(unsigned) * a.n_bins;
+    const size_t per_hist = sizeof(unsigned) * bins_stride;
     const size_t budget = 100 * 1024;
     int fg = static_cast<int>(budget / per_hist) - 1;
     fg = std::max(1, std::min(fg, plan.n_levels));
@@ -477,11 +489,12 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.cand_order = reinterpret_cast<const int*>(ws + plan.off_order);
   kp.cand_by_fl = reinterpret_cast<const int*>(ws + plan.off_by_fl);
   kp.fl_begin = reinterpret_cast<const int*>(ws + plan.off_fl_begin);
-  kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_levels; kp.n_bins = a.n_bins;
+  kp.n_layers = a.n_layers; kp.n_cand = plan.n_cand; kp.n_fl = plan.n_levels; kp.n_bins = bins_stride;
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = o.pseudo_count; kp.inv_ln_base = 1.0 / std::log(base); kp.eps = o.eps;
   kp.kld_out = a.kld_out; kp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
   kp.best_out = a.best_out; kp.hist_out = o.hist_out;
+  kp.start = o.start_wl_fl ? reinterpret_cast<const int*>(ws + plan.off_start) : nullptr;
   {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
     // enough CTAs to fill the GPU when there are few (FL, layer) pairs
@@ -978,7 +991,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   for (int l = 0; l < n_layers; ++l) {
     const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(tensors[l]) >> 2) & 3u);
     hl[l].ptr = tensors[l]; hl[l].n = lens[l]; hl[l].tile_begin = tiles;
-    hl[l].mis = lens[l] > 0 ? mis : 0; hl[l].layer_id = l; hl[l].index = l;
+    hl[l].mis = lens[l] > 0 ? mis : 0; hl[l].layer_id = l; hl[l].index = l; hl[l].n_bins = n_bins;
     if (lens[l] > 0) tiles += (lens[l] + mis + kTile - 1) / kTile;
   }
   hl[n_layers].tile_begin = tiles;
@@ -1017,7 +1030,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
     ADAPT_LAUNCH_OK("range scan launch");
     ++g_launches;
   }
-  range_finalize_kernel<<<1, 128, 0, stream>>>(d_layers, n_layers, n_bins, d_state, nullptr);
+  range_finalize_kernel<<<1, 128, 0, stream>>>(d_layers, n_layers, d_state, nullptr);
   ADAPT_LAUNCH_OK("range finalize launch");
   ++g_launches;
   if (tiles > 0) {
@@ -1053,7 +1066,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = 0.0; kp.inv_ln_base = 1.0 / std::log(2.0); kp.eps = 0.0;
   kp.kld_out = kld_out; kp.zeros_out = reinterpret_cast<long long*>(zeros_out);
-  kp.best_out = best_out; kp.hist_out = nullptr;
+  kp.best_out = best_out; kp.hist_out = nullptr; kp.start = nullptr;
   kld_kernel<<<dim3(n_levels, n_layers), kKldThreads, 0, stream>>>(kp);
   ADAPT_LAUNCH_OK("kld launch");
   ++g_launches;

@@ -21,7 +21,7 @@ struct LayerDesc {
   int mis;               // elements between the 16-byte boundary below ptr and ptr (0..3)
   int layer_id;          // hash layer id
   int index;             // position in the caller's tensor list (addresses state and outputs)
-  int pad_;
+  int n_bins;            // bins of this layer's histograms (<= the stride the arrays use)
 };
 
 // Per-layer state produced on the device by the range scan.

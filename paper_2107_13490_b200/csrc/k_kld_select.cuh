@@ -42,6 +42,7 @@ struct KldParams {
   long long* zeros_out;        // [n_layers][n_cand]
   int* best_out;               // [n_layers][4]
   unsigned* hist_out;          // optional [n_layers][n_cand + 1][n_bins]
+  const int* start;            // optional [n_layers][2]: descent from this <WL,FL> per layer
 };
 
 __device__ __forceinline__ double block_sum(double v, double* s_buf) {
@@ -75,8 +76,9 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   const int f = blockIdx.x, l = blockIdx.y;
   const int c_begin = p.fl_begin[f], c_end = p.fl_begin[f + 1];
   if (c_begin == c_end) return;
-  const int B = p.n_bins;
+  const int stride = p.n_bins;
   const LayerState S = p.state[l];
+  const int B = p.layers[l].n_bins;        // this layer's bins; arrays are laid out with `stride`
   const long long n = p.layers[l].n;
 
   if (S.flags & (kFlagNonfinite | kFlagRange)) {
@@ -88,8 +90,8 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
     }
     return;
   }
-  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + f) * B;
-  const unsigned* Q = p.q_hist + static_cast<size_t>(l) * B;
+  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + f) * stride;
+  const unsigned* Q = p.q_hist + static_cast<size_t>(l) * stride;
   const double n_eff = static_cast<double>(n) + p.alpha * B;
   const double inf_value = __longlong_as_double(0x7ff0000000000000ll);
   const long long zero_count = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + f]);
@@ -117,10 +119,10 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
     const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
     const int bh = bin_of(dequantize(hi_code, f), S.lo, S.scale, S.bmax);
     const int bl = bin_of(dequantize(lo_code, f), S.lo, S.scale, S.bmax);
-    unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * B
+    unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * stride
                              : nullptr;
     unsigned* H0 = (p.hist_out && c == 0)
-                       ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * B : nullptr;
+                       ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * stride : nullptr;
     double k;
     if (bl == 0 && bh == B - 1 && B > 1 && !H) {
       k = unsat;                     // nothing folds: the candidate's histogram is U[FL] itself
@@ -189,6 +191,38 @@ __global__ void select_kernel(const KldParams p) {
     double k2 = __shfl_xor_sync(0xffffffffu, min_k, o);
     int pos2 = __shfl_xor_sync(0xffffffffu, min_pos, o);
     arg_min_merge(min_k, min_pos, k2, pos2);
+  }
+  if (p.start) {
+    // PushDown as a descent (Algorithm 3): from the layer's current format walk down the
+    // (WL, FL) order while the divergence stays <= eps; stop before the first violation
+    const int swl = p.start[2 * l], sfl = p.start[2 * l + 1];
+    int spos = -1;
+    for (int pos = lane; pos < p.n_cand; pos += 32) {
+      const int c = p.cand_order[pos];
+      if (p.cand_wl[c] == swl && p.cand_fl[c] == sfl) spos = (spos < 0) ? pos : min(spos, pos);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const int other = __shfl_xor_sync(0xffffffffu, spos, o);
+      spos = (spos < 0) ? other : (other < 0 ? spos : min(spos, other));
+    }
+    int last_bad = -1;   // highest position below the start whose divergence exceeds eps
+    if (spos >= 0)
+      for (int pos = lane; pos < spos; pos += 32)
+        if (!(kld[p.cand_order[pos]] <= p.eps)) last_bad = max(last_bad, pos);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) last_bad = max(last_bad, __shfl_xor_sync(0xffffffffu, last_bad, o));
+    if (lane == 0) {
+      unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
+      int* o = p.best_out + 4 * l;
+      if (spos < 0) { o[0] = swl; o[1] = sfl; o[2] = -1; o[3] = static_cast<int>(flags); return; }
+      const bool ok = kld[p.cand_order[spos]] <= p.eps;
+      const int pos = ok ? last_bad + 1 : spos;
+      const int c = p.cand_order[pos];
+      if (ok) flags |= 1u;
+      o[0] = p.cand_wl[c]; o[1] = p.cand_fl[c]; o[2] = c; o[3] = static_cast<int>(flags);
+    }
+    return;
   }
   if (lane == 0) {
     unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);

@@ -73,9 +73,9 @@ struct PlanParams {
   int n_layers;              // entries in that list
   const LayerState* state;   // indexed by LayerDesc::index
   LayerPlan* plan;           // indexed by LayerDesc::index
-  float* edges;              // [all layers][n_bins + 1]
+  float* edges;              // [all layers][n_bins + 1] (n_bins = the stride below)
   unsigned* cell_init;       // [all layers][cell_cap]
-  int n_bins;
+  int n_bins;                // stride of the per-bin arrays (the largest layer's bins)
   int cell_cap;              // table entries per layer (memory stride and upper limit)
   int fine_ratio;            // stop refining once a bin holds this many cells
   long long elems_per_cta;   // elements one CTA of the keyed kernel processes
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   const int l = L.index;
   const LayerState S = p.state[l];
   __shared__ LayerPlan s_plan;
-  const int B = p.n_bins;
+  const int B = L.n_bins;      // this layer's own number of bins
 
   if (threadIdx.x == 0) {
     LayerPlan P;
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   if (!P.keyed) return;
 
   // exact lower edge of every bin: smallest float v with bin_of(v) >= b
-  float* E = p.edges + static_cast<size_t>(l) * (B + 1);
+  float* E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
   const unsigned klo = float_key(S.lo), khi = float_key(S.hi);
   // the layer's CTAs (gridDim.y of them) share the edges and the cells
   const int first = blockIdx.y * kPlanThreads + threadIdx.x, stride = kPlanThreads * gridDim.y;

@@ -106,11 +106,12 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
 
 // One thread per layer: decode min/max, derive the bin scale and flags.
 __global__ void range_finalize_kernel(const LayerDesc* __restrict__ layers, int n_layers,
-                                      int n_bins, LayerState* __restrict__ state,
+                                      LayerState* __restrict__ state,
                                       float* __restrict__ range_out) {
   int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l >= n_layers) return;
   LayerState s = state[l];
+  const int n_bins = layers[l].n_bins;
   float lo = 0.0f, hi = 0.0f;
   if (layers[l].n > 0 && !(s.flags & kFlagNonfinite)) {
     lo = key_float(s.min_key);

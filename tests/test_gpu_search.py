@@ -159,6 +159,59 @@ def test_adversarial_value_patterns(B):
                               algorithms=(1, 2))
 
 
+def test_per_layer_resolutions(B):
+    """Each layer with its own number of bins (the paper's per-layer resolution r^l) in one call."""
+    import torch
+    rng = np.random.default_rng(17)
+    xs = [(rng.standard_normal(60000) * 0.1).astype(np.float32),
+          (rng.laplace(0, 1e-3, 40000)).astype(np.float32),
+          np.maximum(rng.standard_normal(70001), 0).astype(np.float32),
+          (rng.standard_normal(333) * 5).astype(np.float32),
+          (rng.standard_normal(50000) * 0.02).astype(np.float32),
+          np.zeros(0, np.float32)]
+    bins = [50, 150, 97, 2048, 1, 64]
+    wl, fl = W.candidate_grid(range(2, 33))
+    grid = B.Grid(wl, fl)
+    dev = G.to_device(xs)
+    ora = [O.precision_search_layer(x, wl, fl, b, want_hist=True) for x, b in zip(xs, bins)]
+    for algo in G.ALGORITHMS:
+        res = B.adapt_precision_search_ex(dev, grid, 7, n_bins_per_layer=bins, want_hist=True,
+                                          want_range=True, algorithm=algo)
+        torch.cuda.synchronize()
+        hist = res.hist.cpu().numpy().view(np.uint32)
+        assert hist.shape[2] == max(bins)
+        for l, b in enumerate(bins):
+            assert np.array_equal(hist[l][:, :b].astype(np.uint64), ora[l]["hist"]), (algo, l)
+            assert not hist[l][:, b:].any()
+            assert np.array_equal(res.zeros.cpu().numpy()[l], ora[l]["zeros"])
+            G.assert_kld_close(res.kld.cpu().numpy()[l], ora[l]["kld"], f"layer {l} algo {algo}")
+            assert list(res.best.cpu().numpy()[l]) == list(ora[l]["best"])
+    with pytest.raises(B.AdaptError):
+        B.adapt_precision_search_ex(dev, grid, 7, n_bins_per_layer=[50, 0, 97, 2048, 1, 64])
+
+
+def test_pushdown_as_a_descent_from_the_current_format(B):
+    import torch
+    w = W.WORKLOADS["resnet20_weights_grads"]
+    xs = W.generate(w)[:8]
+    wl, fl = W.candidate_grid(range(2, 17))
+    grid = B.Grid(wl, fl)
+    dev = G.to_device(xs)
+    ora = O.precision_search(xs, wl, fl, 100, threads=G.host_threads())
+    starts = [(8, 4), (16, 15), (16, 8), (2, 0), (12, 11), (16, 12), (9, 3), (17, 1)]
+    for eps in (0.0, 1e-3):
+        res = B.adapt_precision_search_ex(dev, grid, 100, eps=eps, start_wl_fl=starts)
+        torch.cuda.synchronize()
+        best = res.best.cpu().numpy()
+        for l, (a, b) in enumerate(starts):
+            want = O.select_descent(ora[l]["kld"], wl, fl, a, b, eps)
+            assert list(best[l][:3]) == list(want[:3]), (l, eps)
+            assert (best[l][3] & 1) == want[3]
+    # without start formats the answer is the lowest admissible format of the whole grid
+    res = B.adapt_precision_search_ex(dev, grid, 100)
+    assert [list(r) for r in res.best.cpu().numpy()] == [list(o["best"]) for o in ora]
+
+
 def test_on_grid_tensor_is_lossless(B):
     rng = np.random.default_rng(40)
     x = (rng.integers(-128, 128, 50000) * 2.0 ** -4).astype(np.float32)

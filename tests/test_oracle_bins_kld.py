@@ -226,6 +226,29 @@ def test_select_fallbacks():
     assert list(O.select(k, wl, fl, 0.0)) == [3, 2, 4, 0]     # all inf: last in order
 
 
+def test_select_descent_from_current_format():
+    # order: (2,0) (2,1) (3,0) (3,1) (3,2) (4,0) (4,1) (4,2) (4,3)
+    wl, fl = W.candidate_grid([2, 3, 4])
+    k = np.array([0.5, 0.0, 0.3, 0.0, 0.0, 0.0, 0.0, 0.2, 0.0])
+    # from <4,1>: (4,1) ok, (4,0) ok, (3,2) ok, (3,1) ok, (3,0) loses information -> stop at (3,1)
+    assert list(O.select_descent(k, wl, fl, 4, 1)) == [3, 1, 3, 1]
+    # from <4,3>: (4,2) already loses information -> stays
+    assert list(O.select_descent(k, wl, fl, 4, 3)) == [4, 3, 8, 1]
+    # the start itself loses information: returned with the flag cleared
+    assert list(O.select_descent(k, wl, fl, 4, 2)) == [4, 2, 7, 0]
+    # a descent can end above the global lowest admissible format (2,1)
+    assert list(O.select(k, wl, fl, 0.0))[:2] == [2, 1]
+    # eps widens what counts as lossless: 0.3 admitted, the walk reaches (2,1)
+    assert list(O.select_descent(k, wl, fl, 4, 1, eps=0.3))[:2] == [2, 1]
+    # walking to the very first candidate, and a start outside the grid
+    assert list(O.select_descent(np.zeros(9), wl, fl, 4, 3)) == [2, 0, 0, 1]
+    assert list(O.select_descent(k, wl, fl, 5, 1)) == [5, 1, -1, 0]
+    # array order does not matter
+    perm = np.random.default_rng(1).permutation(9)
+    out = O.select_descent(k[perm], wl[perm], fl[perm], 4, 1)
+    assert list(out[:2]) == [3, 1] and perm[out[2]] == 3
+
+
 # ---- the whole search -------------------------------------------------------
 
 def _by_definition(x, wl, fl, n_bins, mode, seed, layer):
