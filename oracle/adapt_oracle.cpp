@@ -15,6 +15,8 @@
 //   select      - "smallest quantization s.t. KL = 0" (Sec. 3.3; Algorithm 3)
 //   sparsity    - share of non-zero elements (Sec. 3.4 "Inducing Sparsity")
 //   diversity   - gradient diversity of a layer's recent gradients (Sec. 3.3, PushUp)
+//   formats     - block floating point (Sec. 2.1, 2.2) and floating point (Sec. 7) candidates
+//                 through the same EDF / KL steps
 //
 // The paper gives no bit-level rules; the readings taken (saturation,
 // ties-to-even, the stochastic-rounding hash, bin arithmetic, the KLD
@@ -320,6 +322,132 @@ void adapt_oracle_gradient_diversity(const float* const* grads, int n_grads, int
   out[1] = norm_sum;
   out[2] = ds;
   out[3] = (ds > 0.0 && std::isfinite(ds)) ? std::log(ds) : 1.0;
+}
+
+// ---- other number formats through the same EDF / KL machinery ---------------------------
+//
+// The paper names two formats besides fixed point: block floating point (Sec. 2.1
+// "Block-Floating-Point Quantization"; Sec. 2.2, MuPPET's per-layer scale) and, as future work
+// (Sec. 7), floating-point quantization.  A candidate format is a triple (kind, a, b):
+//   kind 0  fixed point      a = WL, b = FL                   (as above)
+//   kind 1  block floating   a = WL, b unused on input: the block is the layer and its scale s
+//                            follows from the layer's extremes; value = code * 2^-s
+//   kind 2  floating point   a = E exponent bits (2..8), b = M mantissa bits (1..23), IEEE-like:
+//                            bias 2^(E-1)-1, the all-ones exponent reserved, gradual underflow
+// The floating-point rules are this build's reading (the paper gives none): parity unpinned by
+// the paper, pinned by the tests against IEEE half precision (numpy) and bfloat16 (torch).
+
+namespace {
+constexpr int kFmtFixed = 0, kFmtBfp = 1, kFmtFloat = 2;
+constexpr int kBfpScaleLimit = 100;  // |s| <= 100 keeps 2^s and 2^-s normal floats
+}  // namespace
+
+// Scale of a block whose extremes are lo <= hi (Sec. 2.2):
+//   s = floor(log2(min((UB + 0.5) / X_max, (LB - 0.5) / X_min))), UB = 2^(WL-1)-1, LB = -2^(WL-1),
+// i.e. the largest integer s with X_max * 2^s <= UB + 0.5 and |X_min| * 2^s <= |LB| + 0.5.
+// A ratio whose extreme has the wrong sign or is zero sets no limit (X_max <= 0, X_min >= 0);
+// with no limit at all (every element zero) s = 0.  s is kept within [-100, 100].
+// The products are exact in double (a float times a power of two), so no logarithm is rounded.
+int adapt_oracle_bfp_scale(float lo, float hi, int wl) {
+  const double ub = std::ldexp(1.0, wl - 1) - 1.0 + 0.5;
+  const double lb = std::ldexp(1.0, wl - 1) + 0.5;
+  const bool lim_hi = hi > 0.0f, lim_lo = lo < 0.0f;
+  if (!lim_hi && !lim_lo) return 0;
+  for (int s = kBfpScaleLimit; s > -kBfpScaleLimit; --s) {
+    const bool ok_hi = !lim_hi || std::ldexp(static_cast<double>(hi), s) <= ub;
+    const bool ok_lo = !lim_lo || std::ldexp(-static_cast<double>(lo), s) <= lb;
+    if (ok_hi && ok_lo) return s;
+  }
+  return -kBfpScaleLimit;
+}
+
+// Value of x in the floating-point format <E,M>: round x to M fraction bits of its own binade
+// (of the lowest normal binade 2^emin when |x| is below it: gradual underflow), then clamp to
+// the largest finite value (2 - 2^-M) * 2^emax (saturation, as for fixed point; no infinities).
+// Rounding is RNE or the SR(x) rule of Sec. 3.2 on the local grid: y = x / quantum is exact,
+// the rest is the fixed-point rule applied to y.
+static float float_format_value(float x, int e_bits, int m_bits, int round_mode, uint32_t k24) {
+  if (x == 0.0f) return 0.0f;
+  const int bias = (1 << (e_bits - 1)) - 1;
+  const int emin = 1 - bias, emax = bias;
+  const int e = std::ilogb(x);                 // floor(log2 |x|), subnormal x included
+  const int ee = std::max(e, emin);
+  const float y = std::ldexp(x, m_bits - ee);  // |y| < 2^(M+1): exact
+  float r;
+  if (round_mode == kRoundNearestEven) {
+    r = std::nearbyintf(y);
+  } else {
+    const float f = std::floor(y);
+    const float frac = y - f;
+    const float p = static_cast<float>(k24) * std::ldexp(1.0f, -24);
+    r = (p < frac) ? f + 1.0f : f;
+  }
+  float v = std::ldexp(r, ee - m_bits);        // integer times a power of two >= 2^-149: exact
+  const float top = std::ldexp(2.0f - std::ldexp(1.0f, -m_bits), emax);
+  if (v > top) v = top;
+  if (v < -top) v = -top;
+  return v;
+}
+
+// One element in one format; for kinds 0 and 1, b is the fraction length / block scale.
+float adapt_oracle_format_value_one(float x, int kind, int a, int b, int round_mode,
+                                    uint32_t k24) {
+  if (kind == kFmtFloat) return float_format_value(x, a, b, round_mode, k24);
+  return dequantize(saturate(round_scaled(x, b, round_mode, k24), a), b);
+}
+
+// A tensor in one format: values_out[i] = the representable value x_i maps to.
+void adapt_oracle_format_quantize(const float* x, int64_t n, int kind, int a, int b,
+                                  int round_mode, uint64_t seed, uint64_t layer,
+                                  float* values_out) {
+  for (int64_t i = 0; i < n; ++i) {
+    const uint32_t k =
+        (round_mode == kRoundStochastic) ? hash24(seed, layer, uint64_t(i)) : 0u;
+    values_out[i] = adapt_oracle_format_value_one(x[i], kind, a, b, round_mode, k);
+  }
+}
+
+// The PushDown body over a list of formats of any kind, one candidate at a time: Quantize ->
+// zero count -> EDF over the shared bins -> KL -> choice.  The candidates are taken in the
+// caller's order (the caller lists them from cheapest to most expensive): the first one whose
+// divergence is <= eps is chosen, else the one of least divergence (first among ties; the last
+// candidate if every divergence is +inf).
+//   kld_out double[n_cand], zeros_out int64[n_cand] (values equal to zero)
+//   b_out   int32[n_cand]: b as used (the derived scale for kind 1, the given b otherwise)
+//   best_out int32[4] = {a, b as used, index, flags}; flags as in adapt_oracle_precision_search
+int adapt_oracle_format_search(const float* x, int64_t n, uint64_t layer, const int32_t* kind,
+                               const int32_t* a, const int32_t* b, int n_cand, int n_bins,
+                               int round_mode, uint64_t seed, double eps, double alpha,
+                               double log_base, double* kld_out, int64_t* zeros_out,
+                               int32_t* b_out, int32_t* best_out, float* range_out) {
+  float lo, hi;
+  const int nonfinite = adapt_oracle_range(x, n, &lo, &hi);
+  if (range_out) { range_out[0] = lo; range_out[1] = hi; }
+  if (nonfinite) return 1;
+  std::vector<uint64_t> q_hist(n_bins), p_hist(n_bins);
+  std::vector<float> values(static_cast<size_t>(n));
+  adapt_oracle_histogram(x, n, lo, hi, n_bins, q_hist.data());
+  for (int c = 0; c < n_cand; ++c) {
+    const int bc = (kind[c] == kFmtBfp) ? adapt_oracle_bfp_scale(lo, hi, a[c]) : b[c];
+    b_out[c] = bc;
+    adapt_oracle_format_quantize(x, n, kind[c], a[c], bc, round_mode, seed, layer, values.data());
+    int64_t zeros = 0;
+    for (int64_t i = 0; i < n; ++i) zeros += (values[i] == 0.0f);
+    zeros_out[c] = zeros;
+    adapt_oracle_histogram(values.data(), n, lo, hi, n_bins, p_hist.data());
+    kld_out[c] = adapt_oracle_kld(p_hist.data(), q_hist.data(), n_bins, alpha, log_base);
+  }
+  int first_ok = -1, least = -1;
+  for (int c = 0; c < n_cand; ++c) {
+    if (first_ok < 0 && kld_out[c] <= eps) first_ok = c;
+    if (std::isfinite(kld_out[c]) && (least < 0 || kld_out[c] < kld_out[least])) least = c;
+  }
+  const int pick = first_ok >= 0 ? first_ok : (least >= 0 ? least : n_cand - 1);
+  best_out[0] = pick >= 0 ? a[pick] : 0;
+  best_out[1] = pick >= 0 ? b_out[pick] : 0;
+  best_out[2] = pick;
+  best_out[3] = (first_ok >= 0 ? 1 : 0) | ((n == 0 || hi == lo) ? 2 : 0);
+  return 0;
 }
 
 }  // extern "C"

@@ -21,6 +21,9 @@ _SO = os.path.join(_HERE, "libadapt_oracle.so")
 
 ROUND_RNE = 0
 ROUND_STOCHASTIC = 1
+FMT_FIXED = 0   # <WL, FL>
+FMT_BFP = 1     # block floating point: word length, scale derived from the layer
+FMT_FLOAT = 2   # <exponent bits, mantissa bits>
 
 _lock = threading.Lock()
 _lib = None
@@ -78,6 +81,20 @@ def lib():
                                                       C.c_double, C.c_int, C.c_int, C.c_void_p]
             L.adapt_oracle_gradient_diversity.restype = None
             L.adapt_oracle_gradient_diversity.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
+            L.adapt_oracle_bfp_scale.restype = C.c_int
+            L.adapt_oracle_bfp_scale.argtypes = [C.c_float, C.c_float, C.c_int]
+            L.adapt_oracle_format_value_one.restype = C.c_float
+            L.adapt_oracle_format_value_one.argtypes = [C.c_float, C.c_int, C.c_int, C.c_int,
+                                                        C.c_int, C.c_uint32]
+            L.adapt_oracle_format_quantize.restype = None
+            L.adapt_oracle_format_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int,
+                                                       C.c_int, C.c_int, C.c_uint64, C.c_uint64,
+                                                       C.c_void_p]
+            L.adapt_oracle_format_search.restype = C.c_int
+            L.adapt_oracle_format_search.argtypes = [
+                C.c_void_p, C.c_int64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int,
+                C.c_int, C.c_int, C.c_uint64, C.c_double, C.c_double, C.c_double,
+                C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
             _lib = L
     return _lib
 
@@ -246,3 +263,45 @@ def gradient_diversity(grads):
     out = np.zeros(4, dtype=np.float64)
     lib().adapt_oracle_gradient_diversity(ptrs, len(arrs), n, out.ctypes.data)
     return out
+
+
+def bfp_scale(lo: float, hi: float, wl: int) -> int:
+    """Block scale s of a layer with extremes lo <= hi at word length wl."""
+    return int(lib().adapt_oracle_bfp_scale(np.float32(lo), np.float32(hi), wl))
+
+
+def format_value_one(x: float, kind: int, a: int, b: int, round_mode: int = ROUND_RNE,
+                     k24: int = 0) -> float:
+    return float(lib().adapt_oracle_format_value_one(np.float32(x), kind, a, b, round_mode, k24))
+
+
+def format_quantize(x, kind: int, a: int, b: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                    layer: int = 0):
+    """The tensor mapped to the representable values of one format; float32[n]."""
+    arr = _as_f32(x)
+    out = np.empty(arr.size, dtype=np.float32)
+    lib().adapt_oracle_format_quantize(arr.ctypes.data, arr.size, kind, a, b, round_mode, seed,
+                                       layer, out.ctypes.data)
+    return out
+
+
+def format_search_layer(x, kind, a, b, n_bins: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                        layer: int = 0, eps: float = 0.0, alpha: float = 0.0,
+                        log_base: float = 2.0):
+    """One layer, every format of the list in the caller's order. Returns a dict."""
+    arr = _as_f32(x)
+    kk = np.ascontiguousarray(kind, dtype=np.int32)
+    aa = np.ascontiguousarray(a, dtype=np.int32)
+    bb = np.ascontiguousarray(b, dtype=np.int32)
+    nc = kk.size
+    kl = np.zeros(nc, dtype=np.float64)
+    zeros = np.zeros(nc, dtype=np.int64)
+    b_used = np.zeros(nc, dtype=np.int32)
+    best = np.zeros(4, dtype=np.int32)
+    rng = np.zeros(2, dtype=np.float32)
+    bad = lib().adapt_oracle_format_search(
+        arr.ctypes.data, arr.size, layer, kk.ctypes.data, aa.ctypes.data, bb.ctypes.data, nc,
+        n_bins, round_mode, seed, eps, alpha, log_base, kl.ctypes.data, zeros.ctypes.data,
+        b_used.ctypes.data, best.ctypes.data, rng.ctypes.data)
+    return {"kld": kl, "zeros": zeros, "b": b_used, "best": best, "range": rng,
+            "nonfinite": int(bad)}
