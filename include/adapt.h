@@ -259,7 +259,11 @@ enum {
   ADAPT_KERNEL_SEARCH_DIRECT = 8,  /* fused kernel, direct form (every FL
                                       evaluated per element)                   */
   ADAPT_KERNEL_DIVERSITY = 9,      /* gradient-diversity reduction              */
-  ADAPT_KERNEL_KINDS = 10
+  ADAPT_KERNEL_FORMAT_RESOLVE = 10,/* format search: per-layer scales and clamps */
+  ADAPT_KERNEL_FORMAT_SEARCH = 11, /* format search: fused round / count / histograms */
+  ADAPT_KERNEL_FORMAT_KLD = 12,    /* format search: divergence per (layer, format) */
+  ADAPT_KERNEL_FORMAT_QUANTIZE = 13, /* stand-alone quantize to a format         */
+  ADAPT_KERNEL_KINDS = 14
 };
 
 /* Switches per-kernel device timing on (non-zero) or off.  While on, every
@@ -315,6 +319,71 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
                                   int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
                                   double* kld_out, int64_t* zeros_out, int32_t* best_out,
                                   void* stream);
+
+/* ---- other number formats ---------------------------------------------------
+ *
+ * The same search (Quantize -> zero count -> histogram over the layer's shared
+ * bins -> KL(P||Q) -> choice; Sec. 3.3, Algorithm 3) over candidate formats of
+ * three kinds, which may be mixed in one list:
+ *   ADAPT_FMT_FIXED  a = WL, b = FL: fixed point as everywhere else in this file.
+ *   ADAPT_FMT_BFP    a = WL (2..32), b ignored: block floating point (Sec. 2.1
+ *       "Block-Floating-Point Quantization") with the layer as the block.  A WL-bit
+ *       signed integer code and a scale s shared by the layer, value = code * 2^-s,
+ *       s from the layer's extremes by the rule of Sec. 2.2:
+ *       s = floor(log2(min((UB+0.5)/X_max, (LB-0.5)/X_min))), UB = 2^(WL-1)-1,
+ *       LB = -2^(WL-1); evaluated exactly as the largest s with X_max*2^s <= UB+0.5
+ *       and |X_min|*2^s <= |LB|+0.5.  An extreme that is zero or of the other sign
+ *       sets no limit; an all-zero layer gets s = 0; s is kept within [-100, 100].
+ *   ADAPT_FMT_FLOAT  a = E exponent bits (2..8), b = M fraction bits (1..23):
+ *       floating point (Sec. 7 names it as the extension of the method), IEEE-like:
+ *       bias 2^(E-1)-1, all-ones exponent reserved, gradual underflow; a value
+ *       beyond the largest finite one, (2-2^-M)*2^bias, saturates to it.  <5,10> is
+ *       half precision, <8,7> bfloat16, <8,23> the identity.
+ * Rounding is opts->round_mode: to nearest even, or the SR(x) rule applied on the
+ * element's local grid, with the same per-element P as everywhere else. */
+enum { ADAPT_FMT_FIXED = 0, ADAPT_FMT_BFP = 1, ADAPT_FMT_FLOAT = 2 };
+typedef struct { int32_t kind, a, b; } adapt_format;
+
+#define ADAPT_MAX_FORMATS 1024
+
+/* Bytes of workspace adapt_format_search needs for these sizes (0 if invalid). */
+size_t adapt_format_search_workspace_bytes(const int64_t* lens, int n_layers,
+                                           const adapt_format* formats, int n_formats,
+                                           int n_bins);
+
+/* Evaluates every format of the list on every layer and chooses one per layer.
+ *   tensors, lens, n_layers   as adapt_precision_search (HOST array of DEVICE pointers)
+ *   formats      HOST array of n_formats (1..ADAPT_MAX_FORMATS) candidates, listed
+ *                from cheapest to most expensive: the choice is the FIRST format
+ *                with KLD <= eps, else the format of least divergence (first among
+ *                ties; the last one if every divergence is +inf)
+ *   n_bins       1..16384, the same for every layer
+ *   kld_out      DEVICE double[n_layers * n_formats]
+ *   zeros_out    DEVICE int64[n_layers * n_formats]: elements whose value in the
+ *                format is zero
+ *   b_out        DEVICE int32[n_layers * n_formats] or NULL: b as used - the layer's
+ *                scale s for ADAPT_FMT_BFP, the given b otherwise
+ *   best_out     DEVICE int32[n_layers * 4] = {a, b as used, index in formats, flags}
+ *   opts         HOST, may be NULL (round to nearest even, eps 0, bits).  Used:
+ *                round_mode, layer_base, seed, eps, pseudo_count, log_base, stream,
+ *                workspace, workspace_bytes, range_out.  hist_out, n_bins_per_layer
+ *                and start_wl_fl must be NULL and algorithm 0: ADAPT_ERR_INVALID_ARG
+ *                otherwise.
+ * Errors as for adapt_precision_search. */
+int adapt_format_search(const float* const* tensors, const int64_t* lens, int n_layers,
+                        const adapt_format* formats, int n_formats, int n_bins,
+                        double* kld_out, int64_t* zeros_out, int32_t* b_out,
+                        int32_t* best_out, const adapt_search_opts* opts);
+
+/* Quantize(L, format): maps x[0..n) to the representable values of one format.
+ *   x           DEVICE float[n]
+ *   kind, a, b  the format; for ADAPT_FMT_BFP b is the scale s (as b_out / best_out
+ *               of adapt_format_search report it), -100 <= s <= 100
+ *   layer       hash layer id for stochastic rounding
+ *   values_out  DEVICE float[n]: the values (code * 2^-b, or the <E,M> value)
+ *   stream      cudaStream_t or NULL */
+int adapt_format_quantize(const float* x, int64_t n, int kind, int a, int b, int round_mode,
+                          uint64_t seed, int layer, float* values_out, void* stream);
 
 /* Frees every library-owned device and pinned buffer of the current device's
  * caches.  Safe to call at any time no library work is in flight. */

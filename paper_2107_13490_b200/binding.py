@@ -30,10 +30,14 @@ EXPORTS = (
     "adapt_precision_switch_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
+    "adapt_format_search_workspace_bytes", "adapt_format_search", "adapt_format_quantize",
 )
+FMT_FIXED, FMT_BFP, FMT_FLOAT = 0, 1, 2
+MAX_FORMATS = 1024
 STATIC_MAX_LAYERS, STATIC_MAX_BINS, STATIC_MAX_CAND = 8, 512, 1024
 KERNEL_KINDS = ("range", "range_finalize", "search", "kld", "select", "quantize", "plan",
-                "expand", "search_direct", "diversity")
+                "expand", "search_direct", "diversity", "format_resolve", "format_search",
+                "format_kld", "format_quantize")
 ALGO_AUTO, ALGO_KEYED, ALGO_DIRECT = 0, 1, 2
 
 
@@ -47,6 +51,10 @@ class AdaptSearchOpts(C.Structure):
                 ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("hist_out", C.c_void_p), ("range_out", C.c_void_p), ("algorithm", C.c_int32),
                 ("n_bins_per_layer", C.c_void_p), ("start_wl_fl", C.c_void_p)]
+
+
+class AdaptFormat(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("a", C.c_int32), ("b", C.c_int32)]
 
 
 class AdaptError(RuntimeError):
@@ -113,6 +121,16 @@ def lib():
         L.adapt_kernel_timing.argtypes = [C.c_int]
         L.adapt_kernel_times.restype = C.c_int
         L.adapt_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_int]
+        L.adapt_format_search_workspace_bytes.restype = C.c_size_t
+        L.adapt_format_search_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int,
+                                                          C.c_int]
+        L.adapt_format_search.restype = C.c_int
+        L.adapt_format_search.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
+                                          C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.POINTER(AdaptSearchOpts)]
+        L.adapt_format_quantize.restype = C.c_int
+        L.adapt_format_quantize.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                            C.c_int, C.c_uint64, C.c_int, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -413,3 +431,71 @@ def adapt_quantize_host(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROU
     _check(lib().adapt_quantize_host(x.data_ptr(), x.numel(), wl, fl, round_mode, seed, layer,
                                      code_bits, codes_out.data_ptr()), "adapt_quantize_host")
     return codes_out
+
+
+def _marshal_formats(formats):
+    """formats: sequence of (kind, a, b) triples -> ctypes array of adapt_format."""
+    arr = (AdaptFormat * len(formats))()
+    for i, (k, a, b) in enumerate(formats):
+        arr[i].kind, arr[i].a, arr[i].b = int(k), int(a), int(b)
+    return arr
+
+
+def adapt_format_search_workspace_bytes(lens: Sequence[int], formats, n_bins: int) -> int:
+    ln = np.ascontiguousarray(lens, dtype=np.int64)
+    arr = _marshal_formats(formats)
+    return int(lib().adapt_format_search_workspace_bytes(
+        ln.ctypes.data, int(ln.size), C.cast(arr, C.c_void_p), len(formats), n_bins))
+
+
+class FormatResult:
+    """Device outputs of adapt_format_search."""
+
+    def __init__(self, kld, zeros, b, best, value_range=None):
+        self.kld, self.zeros, self.b, self.best, self.range = kld, zeros, b, best, value_range
+
+
+def adapt_format_search(tensors: Sequence[torch.Tensor], formats, n_bins: int,
+                        round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                        eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
+                        stream=None, workspace: Optional[torch.Tensor] = None,
+                        want_range: bool = False,
+                        out: Optional[FormatResult] = None) -> FormatResult:
+    """adapt_format_search of adapt.h; formats = sequence of (kind, a, b)."""
+    dev = tensors[0].device
+    assert all(t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(formats)
+    arr = _marshal_formats(formats)
+    if out is None:
+        out = FormatResult(torch.empty((L, Cn), dtype=torch.float64, device=dev),
+                           torch.empty((L, Cn), dtype=torch.int64, device=dev),
+                           torch.empty((L, Cn), dtype=torch.int32, device=dev),
+                           torch.empty((L, 4), dtype=torch.int32, device=dev))
+    if want_range and out.range is None:
+        out.range = torch.empty((L, 2), dtype=torch.float32, device=dev)
+    opts = AdaptSearchOpts()
+    opts.round_mode, opts.layer_base, opts.seed = round_mode, layer_base, seed
+    opts.eps, opts.pseudo_count, opts.log_base = eps, pseudo_count, log_base
+    opts.stream = _stream_handle(stream)
+    if workspace is not None:
+        opts.workspace, opts.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    opts.range_out = out.range.data_ptr() if want_range else None
+    _check(lib().adapt_format_search(ptrs.ctypes.data, lens.ctypes.data, L, C.cast(arr, C.c_void_p),
+                                     Cn, n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
+                                     out.b.data_ptr(), out.best.data_ptr(), C.byref(opts)),
+           "adapt_format_search")
+    return out
+
+
+def adapt_format_quantize(x: torch.Tensor, kind: int, a: int, b: int, round_mode: int = ROUND_RNE,
+                          seed: int = 0, layer: int = 0, out: Optional[torch.Tensor] = None,
+                          stream=None) -> torch.Tensor:
+    """adapt_format_quantize of adapt.h: x mapped to the format's values (float32)."""
+    assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib().adapt_format_quantize(x.data_ptr(), x.numel(), kind, a, b, round_mode, seed, layer,
+                                       out.data_ptr(), _stream_handle(stream)),
+           "adapt_format_quantize")
+    return out

@@ -15,6 +15,7 @@
 #include "common.cuh"
 #include "k_diversity.cuh"
 #include "k_expand.cuh"
+#include "k_formats.cuh"
 #include "k_kld_select.cuh"
 #include "k_plan.cuh"
 #include "k_quantize.cuh"
@@ -894,12 +895,265 @@ int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mod
   return ADAPT_OK;
 }
 
+}  // extern "C"
+
+// ---- other number formats -----------------------------------------------------------------
+
+namespace {
+
+struct FormatPlan {
+  int n_layers = 0, n_cand = 0, n_rules = 0, n_bins = 0;
+  std::vector<FormatCand> cands;
+  std::vector<FormatRule> rules;
+  size_t off_layers = 0, off_cands = 0, off_rules = 0, off_state = 0, blob_bytes = 0;
+  size_t off_level = 0, off_clamp = 0, off_b = 0;
+  size_t accum_begin = 0, off_zeros = 0, off_hist = 0, accum_bytes = 0, total = 0;
+};
+
+bool valid_any_format(const adapt_format& f) {
+  if (f.kind == ADAPT_FMT_FIXED) return valid_format(f.a, f.b);
+  if (f.kind == ADAPT_FMT_BFP) return f.a >= 2 && f.a <= 32;
+  if (f.kind == ADAPT_FMT_FLOAT) return f.a >= 2 && f.a <= 8 && f.b >= 1 && f.b <= 23;
+  return false;
+}
+
+// Validates the sizes, finds the distinct rounding rules and lays out the workspace.
+bool make_format_plan(const int64_t* lens, int n_layers, const adapt_format* formats,
+                      int n_formats, int n_bins, FormatPlan* p) {
+  if (!lens || !formats) return false;
+  if (n_layers < 1 || n_layers > 65535) return false;
+  if (n_formats < 1 || n_formats > ADAPT_MAX_FORMATS) return false;
+  if (n_bins < 1 || n_bins > kMaxBins) return false;
+  for (int l = 0; l < n_layers; ++l)
+    if (lens[l] < 0 || lens[l] >= (1ll << 32)) return false;
+  p->n_layers = n_layers; p->n_cand = n_formats; p->n_bins = n_bins;
+  p->rules.clear();
+  p->rules.push_back(FormatRule{kRuleIdentity, 0, 0, 0});
+  p->cands.resize(n_formats);
+  for (int c = 0; c < n_formats; ++c) {
+    const adapt_format& f = formats[c];
+    if (!valid_any_format(f)) return false;
+    // fixed: one rule per FL; block floating point: per WL; floating point: per (E, M)
+    FormatRule want{f.kind, f.kind == ADAPT_FMT_FIXED ? f.b : f.a,
+                    f.kind == ADAPT_FMT_FLOAT ? f.b : 0, 0};
+    int r = -1;
+    for (size_t i = 1; i < p->rules.size(); ++i)
+      if (p->rules[i].kind == want.kind && p->rules[i].p0 == want.p0 && p->rules[i].p1 == want.p1) {
+        r = static_cast<int>(i);
+        break;
+      }
+    if (r < 0) { r = static_cast<int>(p->rules.size()); p->rules.push_back(want); }
+    p->cands[c] = FormatCand{f.kind, f.a, f.b, r};
+  }
+  p->n_rules = static_cast<int>(p->rules.size());
+  const size_t C = n_formats, L = n_layers, B = n_bins, R = p->n_rules;
+  size_t o = 0;
+  p->off_layers = o;  o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
+  p->off_cands = o;   o = align_up(o + sizeof(FormatCand) * C, 16);
+  p->off_rules = o;   o = align_up(o + sizeof(FormatRule) * R, 16);
+  p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
+  p->blob_bytes = o;
+  p->off_level = o;   o = align_up(o + sizeof(int) * L * R, 256);
+  p->off_clamp = o;   o = align_up(o + sizeof(float2) * L * C, 256);
+  p->off_b = o;       o = align_up(o + sizeof(int) * L * C, 256);
+  p->accum_begin = o;
+  p->off_zeros = o;   o = align_up(o + sizeof(unsigned long long) * L * R, 256);
+  p->off_hist = o;    o = align_up(o + sizeof(unsigned) * L * R * B, 256);
+  p->accum_bytes = o - p->accum_begin;
+  p->total = o;
+  return true;
+}
+
+struct FormatArgs {
+  const float* const* tensors;
+  const int64_t* lens;
+  int n_layers;
+  const adapt_format* formats;
+  int n_formats, n_bins;
+  double* kld_out;
+  int64_t* zeros_out;
+  int32_t* b_out;
+  int32_t* best_out;
+  adapt_search_opts opts;
+};
+
+// Enqueues the whole format search on opts.stream.  Caller holds g_mutex.
+int run_format_search(DeviceCache& dc, const FormatArgs& a) {
+  const adapt_search_opts& o = a.opts;
+  if (!a.tensors || !a.kld_out || !a.zeros_out || !a.best_out) return ADAPT_ERR_INVALID_ARG;
+  if (o.round_mode != ADAPT_ROUND_RNE && o.round_mode != ADAPT_ROUND_STOCHASTIC)
+    return ADAPT_ERR_INVALID_ARG;
+  if (!(o.eps >= 0.0) || !(o.pseudo_count >= 0.0)) return ADAPT_ERR_INVALID_ARG;
+  if (o.hist_out || o.n_bins_per_layer || o.start_wl_fl || o.algorithm != 0) return ADAPT_ERR_INVALID_ARG;
+  const double base = (o.log_base == 0.0) ? 2.0 : o.log_base;
+  if (!(base > 0.0) || base == 1.0 || !std::isfinite(base)) return ADAPT_ERR_INVALID_ARG;
+  FormatPlan plan;
+  if (!make_format_plan(a.lens, a.n_layers, a.formats, a.n_formats, a.n_bins, &plan))
+    return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < a.n_layers; ++l) {
+    if (a.lens[l] > 0 && !a.tensors[l]) return ADAPT_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(a.tensors[l]) & 3u) return ADAPT_ERR_INVALID_ARG;
+  }
+  // shared-memory shape: as many rule histograms per group as fit, at most kMaxRulesPerGroup
+  const size_t per_hist = sizeof(unsigned) * plan.n_bins;
+  const size_t budget = std::min<size_t>(200 * 1024, static_cast<size_t>(dc.max_smem_optin) - 4096);
+  if (per_hist > budget) return ADAPT_ERR_INVALID_ARG;
+
+  char* ws = nullptr;
+  if (o.workspace) {
+    if (reinterpret_cast<uintptr_t>(o.workspace) & 255u) return ADAPT_ERR_INVALID_ARG;
+    if (o.workspace_bytes < plan.total) return ADAPT_ERR_WORKSPACE;
+    ws = static_cast<char*>(o.workspace);
+  } else {
+    int rc = grow_device(&dc.workspace, &dc.workspace_bytes, plan.total);
+    if (rc != ADAPT_OK) return rc;
+    ws = static_cast<char*>(dc.workspace);
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
+
+  PinnedSlot* slot = nullptr;
+  int rc = acquire_slot(dc, plan.blob_bytes, &slot);
+  if (rc != ADAPT_OK) return rc;
+  char* h = static_cast<char*>(slot->host);
+  std::memset(h, 0, plan.blob_bytes);
+  std::vector<int> all(a.n_layers);
+  std::iota(all.begin(), all.end(), 0);
+  SearchArgs la{a.tensors, a.lens, a.n_layers, nullptr, a.n_bins, nullptr, nullptr, nullptr, o};
+  const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, la, kTile);
+  std::memcpy(h + plan.off_cands, plan.cands.data(), sizeof(FormatCand) * plan.n_cand);
+  std::memcpy(h + plan.off_rules, plan.rules.data(), sizeof(FormatRule) * plan.n_rules);
+  LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+  ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
+  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
+
+  FormatParams fp;
+  fp.layers = reinterpret_cast<const LayerDesc*>(ws + plan.off_layers);
+  LayerState* d_state = reinterpret_cast<LayerState*>(ws + plan.off_state);
+  fp.state = d_state;
+  fp.cands = reinterpret_cast<const FormatCand*>(ws + plan.off_cands);
+  fp.rules = reinterpret_cast<const FormatRule*>(ws + plan.off_rules);
+  fp.n_layers = a.n_layers; fp.n_cand = plan.n_cand; fp.n_rules = plan.n_rules; fp.n_bins = plan.n_bins;
+  fp.n_tiles = tiles;
+  fp.level = reinterpret_cast<int*>(ws + plan.off_level);
+  fp.clamp = reinterpret_cast<float2*>(ws + plan.off_clamp);
+  fp.b_used = reinterpret_cast<int*>(ws + plan.off_b);
+  fp.hist = reinterpret_cast<unsigned*>(ws + plan.off_hist);
+  fp.zeros = reinterpret_cast<unsigned long long*>(ws + plan.off_zeros);
+  fp.seed = o.seed;
+  fp.alpha = o.pseudo_count; fp.inv_ln_base = 1.0 / std::log(base); fp.eps = o.eps;
+  fp.kld_out = a.kld_out; fp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
+  fp.b_out = a.b_out; fp.best_out = a.best_out;
+
+  // rule groups: few tiles spread the rules over more CTAs, many tiles fill shared memory
+  int rpg = static_cast<int>(std::min<size_t>(kMaxRulesPerGroup, budget / per_hist));
+  rpg = std::max(1, std::min(rpg, plan.n_rules));
+  const long long want_groups = std::min<long long>(
+      plan.n_rules, std::max<long long>(1, (2ll * dc.sm_count + std::max(1ll, tiles) - 1) / std::max(1ll, tiles)));
+  rpg = std::min<int>(rpg, static_cast<int>((plan.n_rules + want_groups - 1) / want_groups));
+  fp.rules_per_group = rpg;
+  const int groups = (plan.n_rules + rpg - 1) / rpg;
+  const size_t smem = per_hist * rpg;
+
+  if (tiles > 0) {
+    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc.sm_count));
+    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
+    range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(fp.layers, a.n_layers, tiles, d_state);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_RANGE_FINALIZE, stream);
+    range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
+        fp.layers, a.n_layers, d_state, o.range_out);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_FORMAT_RESOLVE, stream);
+    format_resolve_kernel<<<a.n_layers, 128, 0, stream>>>(fp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  if (tiles > 0) {
+    auto kern = (o.round_mode == ADAPT_ROUND_STOCHASTIC) ? format_search_kernel<true>
+                                                         : format_search_kernel<false>;
+    ADAPT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    static_cast<int>(smem)));
+    const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 2048)));
+    dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)), groups);
+    LaunchScope ls(ADAPT_KERNEL_FORMAT_SEARCH, stream);
+    kern<<<grid, kFormatThreads, smem, stream>>>(fp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_FORMAT_KLD, stream);
+    format_kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(fp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  {
+    LaunchScope ls(ADAPT_KERNEL_SELECT, stream);
+    format_select_kernel<<<a.n_layers, 32, 0, stream>>>(fp);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  return ADAPT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t adapt_format_search_workspace_bytes(const int64_t* lens, int n_layers,
+                                           const adapt_format* formats, int n_formats,
+                                           int n_bins) {
+  FormatPlan plan;
+  if (!make_format_plan(lens, n_layers, formats, n_formats, n_bins, &plan)) return 0;
+  return plan.total;
+}
+
+int adapt_format_search(const float* const* tensors, const int64_t* lens, int n_layers,
+                        const adapt_format* formats, int n_formats, int n_bins,
+                        double* kld_out, int64_t* zeros_out, int32_t* b_out,
+                        int32_t* best_out, const adapt_search_opts* opts) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  FormatArgs a{tensors, lens, n_layers, formats, n_formats, n_bins, kld_out, zeros_out, b_out,
+               best_out, opts ? *opts : default_opts()};
+  return run_format_search(*dc, a);
+}
+
+int adapt_format_quantize(const float* x, int64_t n, int kind, int a, int b, int round_mode,
+                          uint64_t seed, int layer, float* values_out, void* stream) {
+  if (n < 0 || (n > 0 && (!x || !values_out))) return ADAPT_ERR_INVALID_ARG;
+  if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
+    return ADAPT_ERR_INVALID_ARG;
+  adapt_format f{kind, a, b};
+  if (kind == ADAPT_FMT_BFP) {
+    if (a < 2 || a > 32 || b < -kBfpScaleLimit || b > kBfpScaleLimit) return ADAPT_ERR_INVALID_ARG;
+  } else if (!valid_any_format(f)) {
+    return ADAPT_ERR_INVALID_ARG;
+  }
+  if (n == 0) return ADAPT_OK;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  FormatQuantParams qp{x, values_out, n, kind, a, b, layer, seed};
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int grid = static_cast<int>(std::min<long long>((n + 255) / 256, 16ll * dc->sm_count));
+  LaunchScope ls(ADAPT_KERNEL_FORMAT_QUANTIZE, s);
+  if (round_mode == ADAPT_ROUND_STOCHASTIC) format_quantize_kernel<true><<<grid, 256, 0, s>>>(qp);
+  else format_quantize_kernel<false><<<grid, 256, 0, s>>>(qp);
+  ADAPT_CUDA(cudaGetLastError());
+  return ADAPT_OK;
+}
+
+}  // extern "C"
+
 // ---- search without any allocation ------------------------------------------------
 //
 // Scratch of adapt_precision_search_static: one fixed device array, part of the library
 // image, so every GPU that loads the library holds it until the process exits.
-
-}  // extern "C"
 
 namespace {
 

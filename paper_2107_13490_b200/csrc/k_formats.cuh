@@ -1,0 +1,369 @@
+// The precision-switch search over other number formats: block floating point (Sec. 2.1
+// "Block-Floating-Point Quantization"; the layer scale of Sec. 2.2) and floating point <E,M>
+// (Sec. 7 names it as the planned extension), next to fixed point, through the same steps:
+// Quantize -> zero count -> histogram over the layer's shared bins -> KL(P||Q) -> choice.
+//
+// Every format rounds an element on a power-of-two grid and then clamps it to the format's
+// range.  The grid is the same for all elements (fixed point: 2^-FL; block floating point:
+// 2^-s with the scale s of the layer) or follows the element's own binade (floating point:
+// 2^(e-M), e >= emin).  Clamping commutes with the monotone bin function, so the kernels build
+// one UNCLAMPED histogram per distinct rounding rule and the divergence kernel folds the two
+// tails into the bins of the clamp values; formats that share a rule share a histogram.
+#pragma once
+
+#include "common.cuh"
+#include "k_kld_select.cuh"
+#include "k_range.cuh"
+
+namespace adapt {
+
+constexpr int kFmtFixed = 0, kFmtBfp = 1, kFmtFloat = 2;
+constexpr int kRuleIdentity = 3;     // the float tensor itself (histogram Q)
+constexpr int kBfpScaleLimit = 100;  // |s| <= 100: 2^s and 2^-s stay normal floats
+constexpr int kFormatThreads = 256;
+constexpr int kMaxRulesPerGroup = 64;
+
+struct FormatCand { int kind, a, b, rule; };   // rule: index of the candidate's rounding rule
+struct FormatRule { int kind, p0, p1, pad; };  // fixed: p0 = FL; bfp: p0 = WL; float: p0 = E, p1 = M
+
+struct FormatParams {
+  const LayerDesc* layers;
+  const LayerState* state;
+  const FormatCand* cands;      // [n_cand]
+  const FormatRule* rules;      // [n_rules]; rule 0 is the identity
+  int n_layers, n_cand, n_rules, n_bins;
+  int rules_per_group;          // rules handled by one blockIdx.y
+  long long n_tiles;
+  int* level;                   // [n_layers][n_rules] grid level of fixed / bfp rules, per layer
+  float2* clamp;                // [n_layers][n_cand] lowest and highest representable value
+  int* b_used;                  // [n_layers][n_cand] b as used (bfp: the layer's scale)
+  unsigned* hist;               // [n_layers][n_rules][n_bins]
+  unsigned long long* zeros;    // [n_layers][n_rules]
+  unsigned long long seed;
+  double alpha, inv_ln_base, eps;
+  double* kld_out;              // [n_layers][n_cand]
+  long long* zeros_out;         // [n_layers][n_cand]
+  int* b_out;                   // optional [n_layers][n_cand]
+  int* best_out;                // [n_layers][4]
+};
+
+// x * 2^k for -149 <= k <= 149 in two exact steps (a single 2^k may not be a normal float).
+__device__ __forceinline__ float scale_pow2(float x, int k) {
+  const int k1 = max(-100, min(100, k));
+  return __fmul_rn(__fmul_rn(x, pow2f(k1)), pow2f(k - k1));
+}
+
+// Largest finite value of <E,M>: (2 - 2^-M) * 2^emax, emax = 2^(E-1) - 1.
+__device__ __forceinline__ float float_format_top(int e_bits, int m_bits) {
+  const int emax = (1 << (e_bits - 1)) - 1;
+  return __fmul_rn(__fsub_rn(2.0f, pow2f(-m_bits)), pow2f(emax));
+}
+
+// Scale of a block with extremes lo <= hi (Sec. 2.2): the largest s with
+// hi * 2^s <= UB + 0.5 and -lo * 2^s <= -LB + 0.5; products of a float and a power of two are
+// exact in double.  An extreme of the wrong sign sets no limit; no limit at all gives 0.
+__device__ inline int bfp_scale(float lo, float hi, int wl) {
+  const double ub = ldexp(1.0, wl - 1) - 0.5;
+  const double lb = ldexp(1.0, wl - 1) + 0.5;
+  const bool lim_hi = hi > 0.0f, lim_lo = lo < 0.0f;
+  if (!lim_hi && !lim_lo) return 0;
+  for (int s = kBfpScaleLimit; s > -kBfpScaleLimit; --s) {
+    const bool ok_hi = !lim_hi || ldexp(static_cast<double>(hi), s) <= ub;
+    const bool ok_lo = !lim_lo || ldexp(-static_cast<double>(lo), s) <= lb;
+    if (ok_hi && ok_lo) return s;
+  }
+  return -kBfpScaleLimit;
+}
+
+// Rounds y to an integer: RNE, or SR(x) of Sec. 3.2 with P = pr.
+template <bool kStochastic>
+__device__ __forceinline__ float round_to_grid(float y, float pr) {
+  if (!kStochastic) return rintf(y);
+  const float f = floorf(y);
+  const float frac = __fsub_rn(y, f);
+  return (pr < frac) ? __fadd_rn(f, 1.0f) : f;
+}
+
+// Unclamped value of x on the grid 2^-level.
+template <bool kStochastic>
+__device__ __forceinline__ float level_value(float x, float two_l, float inv_l, float pr) {
+  return __fmul_rn(round_to_grid<kStochastic>(__fmul_rn(x, two_l), pr), inv_l);
+}
+
+// Unclamped value of x in <E,M>: M fraction bits of its own binade, of binade emin below it.
+template <bool kStochastic>
+__device__ __forceinline__ float float_value(float x, int emin, int m_bits, float pr) {
+  const int e = static_cast<int>((__float_as_uint(x) >> 23) & 0xffu) - 127;  // subnormal: -127
+  const int k = m_bits - max(e, emin);
+  const float y = scale_pow2(x, k);                   // |y| < 2^(M+1): exact
+  return scale_pow2(round_to_grid<kStochastic>(y, pr), -k);
+}
+
+// One CTA per layer: grid level of every rule, clamp values and b-as-used of every candidate.
+__global__ void format_resolve_kernel(const FormatParams p) {
+  const int l = blockIdx.x;
+  const LayerState S = p.state[l];
+  for (int r = threadIdx.x; r < p.n_rules; r += blockDim.x) {
+    const FormatRule R = p.rules[r];
+    int lev = 0;
+    if (R.kind == kFmtFixed) lev = R.p0;
+    else if (R.kind == kFmtBfp) lev = bfp_scale(S.lo, S.hi, R.p0);
+    p.level[static_cast<size_t>(l) * p.n_rules + r] = lev;
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < p.n_cand; c += blockDim.x) {
+    const FormatCand K = p.cands[c];
+    const size_t at = static_cast<size_t>(l) * p.n_cand + c;
+    float2 cl;
+    int b = K.b;
+    if (K.kind == kFmtFloat) {
+      const float top = float_format_top(K.a, K.b);
+      cl = make_float2(-top, top);
+    } else {
+      const int lev = p.level[static_cast<size_t>(l) * p.n_rules + K.rule];
+      b = lev;
+      const float inv = pow2f(-lev);
+      const int hi_code = static_cast<int>((1ll << (K.a - 1)) - 1);
+      const int lo_code = static_cast<int>(-(1ll << (K.a - 1)));
+      cl = make_float2(__fmul_rn(__int2float_rn(lo_code), inv), __fmul_rn(__int2float_rn(hi_code), inv));
+    }
+    p.clamp[at] = cl;
+    p.b_used[at] = b;
+    if (p.b_out) p.b_out[at] = b;
+  }
+}
+
+// Builds the unclamped histogram and the zero count of every rule, every layer.  The rules are
+// cut into groups of rules_per_group (blockIdx.y) so that a group's histograms fit in shared
+// memory; each group reads the tensors once.
+template <bool kStochastic>
+__global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const FormatParams p) {
+  extern __shared__ unsigned s_fhist[];   // [rules in the group][n_bins]
+  __shared__ int s_kind[kMaxRulesPerGroup], s_i0[kMaxRulesPerGroup], s_i1[kMaxRulesPerGroup];
+  __shared__ float s_f0[kMaxRulesPerGroup], s_f1[kMaxRulesPerGroup];
+  __shared__ unsigned s_zero[kMaxRulesPerGroup];
+
+  const int B = p.n_bins;
+  const int r0 = blockIdx.y * p.rules_per_group;
+  const int nr = min(p.rules_per_group, p.n_rules - r0);
+  const int lane = threadIdx.x & 31;
+
+  const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
+  long long t = per * blockIdx.x;
+  const long long t_end = min(p.n_tiles, t + per);
+  if (t >= t_end) return;
+
+  for (int i = threadIdx.x; i < nr * B; i += blockDim.x) s_fhist[i] = 0;
+  if (threadIdx.x < kMaxRulesPerGroup) s_zero[threadIdx.x] = 0;
+
+  int l = layer_of_tile(p.layers, p.n_layers, t);
+  while (t < t_end) {
+    const LayerDesc L = p.layers[l];
+    const int gl = L.index;
+    const LayerState S = p.state[gl];
+    const long long layer_tiles_end = min(t_end, p.layers[l + 1].tile_begin);
+    const float* base = L.ptr - L.mis;
+    const long long jbeg = L.mis, jend = L.mis + L.n;
+    const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
+
+    // this layer's form of the group's rules
+    if (threadIdx.x < nr) {
+      const FormatRule R = p.rules[r0 + threadIdx.x];
+      s_kind[threadIdx.x] = R.kind;
+      if (R.kind == kFmtFloat) {
+        s_i0[threadIdx.x] = 2 - (1 << (R.p0 - 1));   // emin = 1 - bias
+        s_i1[threadIdx.x] = R.p1;
+      } else if (R.kind != kRuleIdentity) {
+        const int lev = p.level[static_cast<size_t>(gl) * p.n_rules + r0 + threadIdx.x];
+        s_f0[threadIdx.x] = pow2f(lev);
+        s_f1[threadIdx.x] = pow2f(-lev);
+      }
+    }
+    __syncthreads();
+
+    for (; t < layer_tiles_end; ++t) {
+      if (!layer_ok) continue;
+      const long long j_tile = (t - L.tile_begin) * kTile;
+      for (int q = 0; q < kTile / 4 / kFormatThreads; ++q) {
+        const long long j0 = j_tile + 4ll * (q * kFormatThreads + threadIdx.x);
+        float v[4];
+        unsigned m = 0;
+        if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
+        else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const bool valid = (m >> k) & 1u;
+          const float x = v[k];
+          float pr = 0.0f;
+          if (kStochastic) {
+            const unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
+                                      static_cast<unsigned long long>(j0 + k - jbeg));
+            pr = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+          }
+          for (int r = 0; r < nr; ++r) {
+            const int kind = s_kind[r];
+            float xq;
+            if (kind == kRuleIdentity) xq = x;
+            else if (kind == kFmtFloat) xq = float_value<kStochastic>(x, s_i0[r], s_i1[r], pr);
+            else xq = level_value<kStochastic>(x, s_f0[r], s_f1[r], pr);
+            const int b = bin_of(xq, S.lo, S.scale, S.bmax);
+            if (valid) atomicAdd(&s_fhist[r * B + b], 1u);
+            const unsigned zm = __ballot_sync(0xffffffffu, valid && xq == 0.0f);
+            if (lane == 0 && zm) atomicAdd(&s_zero[r], __popc(zm));
+          }
+        }
+      }
+    }
+    __syncthreads();
+    if (layer_ok) {
+      for (int i = threadIdx.x; i < nr * B; i += blockDim.x) {
+        const unsigned c = s_fhist[i];
+        if (c) {
+          const int r = i / B, b = i - r * B;
+          atomicAdd(&p.hist[(static_cast<size_t>(gl) * p.n_rules + r0 + r) * B + b], c);
+          s_fhist[i] = 0;
+        }
+      }
+      if (threadIdx.x < nr) {
+        const unsigned c = s_zero[threadIdx.x];
+        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_rules + r0 + threadIdx.x],
+                         static_cast<unsigned long long>(c));
+        s_zero[threadIdx.x] = 0;
+      }
+    }
+    __syncthreads();
+    ++l;
+    while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
+  }
+}
+
+// One CTA per (candidate, layer): the rule's histogram with both tails folded into the bins
+// of the candidate's clamp values, then KL(P||Q) against the identity rule's histogram.
+__global__ void __launch_bounds__(kKldThreads) format_kld_kernel(const FormatParams p) {
+  __shared__ double s_buf[kKldThreads / 32];
+  __shared__ int s_inf;
+  const int c = blockIdx.x, l = blockIdx.y;
+  const int B = p.n_bins;
+  const LayerState S = p.state[l];
+  const long long n = p.layers[l].n;
+  const size_t out = static_cast<size_t>(l) * p.n_cand + c;
+  if (S.flags & (kFlagNonfinite | kFlagRange)) {
+    if (threadIdx.x == 0) {
+      p.kld_out[out] = __longlong_as_double(0x7ff8000000000000ll);  // NaN: unspecified output
+      p.zeros_out[out] = 0;
+    }
+    return;
+  }
+  const int rule = p.cands[c].rule;
+  const unsigned* U = p.hist + (static_cast<size_t>(l) * p.n_rules + rule) * B;
+  const unsigned* Q = p.hist + static_cast<size_t>(l) * p.n_rules * B;
+  const float2 cl = p.clamp[out];
+  const int bl = bin_of(cl.x, S.lo, S.scale, S.bmax);
+  const int bh = bin_of(cl.y, S.lo, S.scale, S.bmax);
+  const double n_eff = static_cast<double>(n) + p.alpha * B;
+
+  double lo_mass = 0.0, hi_mass = 0.0;
+  for (int b = threadIdx.x; b < B; b += kKldThreads) {
+    const unsigned u = U[b];
+    if (b <= bl) lo_mass += u;
+    if (b >= bh) hi_mass += u;
+  }
+  lo_mass = block_sum(lo_mass, s_buf);
+  hi_mass = block_sum(hi_mass, s_buf);
+  if (threadIdx.x == 0) s_inf = 0;
+  __syncthreads();
+  double sum = 0.0;
+  bool inf = false;
+  for (int b = threadIdx.x; b < B; b += kKldThreads) {
+    long long pc;
+    if (bl == bh) pc = (b == bl) ? n : 0;
+    else if (b < bl || b > bh) pc = 0;
+    else if (b == bl) pc = static_cast<long long>(lo_mass);
+    else if (b == bh) pc = static_cast<long long>(hi_mass);
+    else pc = U[b];
+    sum += kld_term(pc, Q[b], p.alpha, &inf);
+  }
+  if (inf) s_inf = 1;
+  sum = block_sum(sum, s_buf);
+  if (threadIdx.x == 0) {
+    double k;
+    if (n_eff <= 0.0) k = 0.0;
+    else if (s_inf) k = __longlong_as_double(0x7ff0000000000000ll);
+    else { k = sum * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
+    p.kld_out[out] = k;
+    p.zeros_out[out] = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_rules + rule]);
+  }
+}
+
+// One warp per layer: the first format of the caller's list with KLD <= eps, else the one of
+// least divergence (first among ties; the last one if every divergence is +inf).
+__global__ void format_select_kernel(const FormatParams p) {
+  const int l = blockIdx.x, lane = threadIdx.x;
+  const double* kld = p.kld_out + static_cast<size_t>(l) * p.n_cand;
+  int first_ok = 0x7fffffff, min_pos = -1;
+  double min_k = 0.0;
+  for (int c = lane; c < p.n_cand; c += 32) {
+    const double k = kld[c];
+    if (k <= p.eps) first_ok = min(first_ok, c);
+    if (k < __longlong_as_double(0x7ff0000000000000ll)) arg_min_merge(min_k, min_pos, k, c);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    first_ok = min(first_ok, __shfl_xor_sync(0xffffffffu, first_ok, o));
+    const double k2 = __shfl_xor_sync(0xffffffffu, min_k, o);
+    const int pos2 = __shfl_xor_sync(0xffffffffu, min_pos, o);
+    arg_min_merge(min_k, min_pos, k2, pos2);
+  }
+  if (lane == 0) {
+    unsigned flags = p.state[l].flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
+    int c;
+    if (first_ok != 0x7fffffff) { c = first_ok; flags |= 1u; }
+    else if (min_pos >= 0) c = min_pos;
+    else c = p.n_cand - 1;
+    int* o = p.best_out + 4 * l;
+    o[0] = p.cands[c].a;
+    o[1] = p.b_used[static_cast<size_t>(l) * p.n_cand + c];
+    o[2] = c;
+    o[3] = static_cast<int>(flags);
+  }
+}
+
+// Quantize(L, format): the tensor mapped to the format's representable values (fp32 out).
+struct FormatQuantParams {
+  const float* x;
+  float* out;
+  long long n;
+  int kind, a, b, layer_id;
+  unsigned long long seed;
+};
+
+template <bool kStochastic>
+__global__ void __launch_bounds__(256) format_quantize_kernel(const FormatQuantParams p) {
+  float lo_v, hi_v, two_l = 1.0f, inv_l = 1.0f;
+  int emin = 0;
+  if (p.kind == kFmtFloat) {
+    hi_v = float_format_top(p.a, p.b);
+    lo_v = -hi_v;
+    emin = 2 - (1 << (p.a - 1));
+  } else {
+    two_l = pow2f(p.b);
+    inv_l = pow2f(-p.b);
+    hi_v = __fmul_rn(__int2float_rn(static_cast<int>((1ll << (p.a - 1)) - 1)), inv_l);
+    lo_v = __fmul_rn(__int2float_rn(static_cast<int>(-(1ll << (p.a - 1)))), inv_l);
+  }
+  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+  for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < p.n; i += stride) {
+    const float x = __ldg(p.x + i);
+    float pr = 0.0f;
+    if (kStochastic)
+      pr = __fmul_rn(__uint2float_rn(hash24(p.seed, static_cast<unsigned long long>(p.layer_id),
+                                            static_cast<unsigned long long>(i))),
+                     5.9604644775390625e-8f);
+    float v = (p.kind == kFmtFloat) ? float_value<kStochastic>(x, emin, p.b, pr)
+                                    : level_value<kStochastic>(x, two_l, inv_l, pr);
+    v = fminf(fmaxf(v, lo_v), hi_v);
+    p.out[i] = __fadd_rn(v, 0.0f);   // -0 becomes +0, as a code of zero would
+  }
+}
+
+}  // namespace adapt
