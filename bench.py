@@ -46,7 +46,7 @@ def parse_args():
                     help="elements of the workload the CPU baseline is timed on")
     ap.add_argument("--elements", type=int, default=0,
                     help="profiling aid: shrink a single-layer workload to this many elements")
-    ap.add_argument("--path", default="search", choices=["search", "diversity"],
+    ap.add_argument("--path", default="search", choices=["search", "diversity", "formats"],
                     help="search: the precision-switch search step (default); diversity: the "
                          "gradient-diversity reduction that feeds PushUp")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -257,12 +257,99 @@ def run_diversity(args):
     return 0
 
 
+def bench_formats():
+    """Block floating point at word lengths 2..16 and twelve float formats <E,M>."""
+    f = [(1, wl, 0) for wl in range(2, 17)]
+    f += [(2, e, m) for e in (4, 5, 8) for m in (2, 3, 7, 10)]
+    return f
+
+
+def run_formats(args):
+    """The search over block-floating-point and floating-point candidates (27 formats) on the
+    AlexNet weight tensors (or --workload / --elements)."""
+    import torch
+    from paper_2107_13490_b200 import binding as B
+    from paper_2107_13490_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    name = args.workload if args.workload != "stress_1g" or args.elements else "alexnet_weights"
+    w = W.WORKLOADS[name]
+    if args.elements:
+        w = W.scaled(w, args.elements)
+    formats = bench_formats()
+    host = W.generate(w)
+    xs = [torch.from_numpy(x).cuda() for x in host]
+    lens = [x.numel() for x in xs]
+    total = sum(lens)
+    ws = torch.empty(B.adapt_format_search_workspace_bytes(lens, formats, w.n_bins),
+                     dtype=torch.uint8, device="cuda")
+    out = None
+    sampler = ClockSampler(0)
+    sampler.start()            # started early: the first sample takes a while to arrive
+    for _ in range(max(args.warmup, 3)):
+        out = B.adapt_format_search(xs, formats, w.n_bins, workspace=ws, out=out)
+    torch.cuda.synchronize()
+    B.adapt_kernel_times(reset=True)
+    B.adapt_kernel_timing(True)
+    n0 = B.adapt_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    e0.record()
+    for _ in range(args.steps):
+        B.adapt_format_search(xs, formats, w.n_bins, workspace=ws, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    B.adapt_kernel_timing(False)
+    launches = B.adapt_kernel_launch_count() - n0
+    ms = e0.elapsed_time(e1) / args.steps
+    kt = B.adapt_kernel_times(reset=True)
+    k_ms = kt["format_search"][0] / args.steps
+    # Issue-bound kernel: one (element, rounding rule) evaluation needs at least 10 lane
+    # instructions (scale, round, rescale; subtract, multiply, floor, two clamps, convert;
+    # one shared atomic), and an SM issues 128 lane instructions per clock.
+    sm_count = torch.cuda.get_device_properties(0).multi_processor_count
+    sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+    n_rules = 1 + len({(k, b if k == 0 else a, b if k == 2 else 0) for k, a, b in formats})
+    peak = sm_count * 128 * sm_mhz * 1e6 / 10.0 / 1e9
+    achieved = total * n_rules / (k_ms * 1e-3) / 1e9
+    line = {"metric": "format-search element-formats/s", "value": total * len(formats) / (ms * 1e-3),
+            "unit": "element-formats/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": ms, "higher_is_better": True,
+            "dtype": "f32", "data": "synthetic", "gpu_launches": int(launches), "clocks": clocks,
+            "config": {"workload": f"{w.name}: {len(xs)} layers, {total} elements, {len(formats)} formats "
+                                   f"(15 block floating point, 12 floating point), {n_rules} rounding rules, "
+                                   f"{w.n_bins} bins",
+                       "l2": "inputs exceed L2" if 4 * total > 126e6 else "inputs fit in L2"},
+            "kernel_ms": {k: v[0] / args.steps for k, v in kt.items() if v[1]},
+            "roofline": {"bound": "alu", "kernel": "format_search", "achieved": achieved, "peak": peak,
+                         "peak_kind": "SMs x 128 lanes x sampled SM clock / 10 instructions per evaluation",
+                         "unit": "G element-rule evaluations/s", "frac": achieved / peak,
+                         "hbm_gbs": 4.0 * total / (k_ms * 1e-3) / 1e9, "traffic": None}}
+    if not args.no_cpu_baseline:
+        from oracle import oracle as O
+        l = max(range(len(host)), key=lambda i: host[i].size)
+        m = min(host[l].size, 1 << 19)
+        t0 = time.perf_counter()
+        O.format_search_layer(host[l][:m], [f[0] for f in formats], [f[1] for f in formats],
+                              [f[2] for f in formats], w.n_bins)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": m * len(formats) / dt, "unit": "element-formats/s", "cores": 1,
+                                "kind": "oracle", "sample": f"first {m} elements of the largest layer"}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
     if args.path == "diversity":
         return run_diversity(args)
+    if args.path == "formats":
+        return run_formats(args)
 
     import torch
     from paper_2107_13490_b200 import binding as B

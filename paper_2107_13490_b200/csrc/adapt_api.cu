@@ -1078,7 +1078,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
                                                          : format_search_kernel<false>;
     ADAPT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(smem)));
-    const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 2048)));
+    const int ctas_per_sm = std::max<int>(1, std::min<size_t>(2, (200 * 1024) / (smem + 2048)));
     dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)), groups);
     LaunchScope ls(ADAPT_KERNEL_FORMAT_SEARCH, stream);
     kern<<<grid, kFormatThreads, smem, stream>>>(fp);

@@ -20,7 +20,7 @@ namespace adapt {
 constexpr int kFmtFixed = 0, kFmtBfp = 1, kFmtFloat = 2;
 constexpr int kRuleIdentity = 3;     // the float tensor itself (histogram Q)
 constexpr int kBfpScaleLimit = 100;  // |s| <= 100: 2^s and 2^-s stay normal floats
-constexpr int kFormatThreads = 256;
+constexpr int kFormatThreads = 1024;   // one or two CTAs per SM own its shared memory
 constexpr int kMaxRulesPerGroup = 64;
 
 struct FormatCand { int kind, a, b, rule; };   // rule: index of the candidate's rounding rule
