@@ -26,7 +26,8 @@
 // This kernel chooses the segments, computes the exact bin edges (smallest
 // float of each bin, by bisection over the float order with the bin function
 // itself), and marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0 of
-// the main segment.
+// the main segment.  (Bit 29 is left to the counting kernel, which adds it to the word an
+// atomic returns when the element sits exactly on the cell grid.)
 #pragma once
 
 #include "common.cuh"
@@ -36,7 +37,8 @@ namespace adapt {
 
 constexpr unsigned kCellEdge = 0x80000000u;
 constexpr unsigned kCellNearZero = 0x40000000u;
-constexpr unsigned kCellCountMask = 0x3FFFFFFFu;
+constexpr unsigned kCellOnGrid = 0x20000000u;     // added to a returned word, never stored
+constexpr unsigned kCellCountMask = 0x1FFFFFFFu;
 constexpr int kPlanThreads = 256;
 
 // Tunables of the table shape (performance only).

@@ -3,9 +3,10 @@
 // common path.  See k_plan.cuh for the cell decomposition this relies on.
 //
 // Per element x != 0:   pos = table position of x's cell;  old = atomicAdd(cell[pos], 1)
-// The returned word carries the cell's marks in its two top bits:
-//   bit 30 (cell -1 / 0 of the main segment) or bit 31 (edge cell): the element goes to
-//          a per-warp queue that the warp drains 32 entries at a time:
+// The returned word carries the cell's marks in its top bits, and bit 29 is added to it when
+// the element sits exactly on the cell grid:
+//   bit 30 (cell -1 / 0 of the main segment), bit 31 (edge cell) or bit 29: the element goes
+//          to a per-warp queue that the warp drains 32 entries at a time:
 //            cell -1 / 0: the element is added to the class counter "highest level at
 //              which it still rounds to zero";
 //            edge entry: b0 = bin(x) into the segment's edge-element histogram,
@@ -16,7 +17,8 @@
 // the parity rule of grid_point_goes_left (its handler moves the count when it belongs left),
 // which makes every coarse rounding tie come out even.
 // Exact zeros are sent to per-lane dummy slots (their number is the layer size
-// minus the sum of the cell counts).  Everything else about an element - the
+// minus the sum of the cell counts).  A dummy slot starts with all three top bits set; zero is
+// on every grid, so the added bit 29 wraps the returned word around to a plain small count.  Everything else about an element - the
 // float histogram, all coarse levels, all fine levels of interior cells - is
 // derived from the cell counts by the expand kernel.
 //
@@ -155,17 +157,18 @@ struct CellFn {
   float two_g1, magic1;         // auxiliary segment (fast layers only)
 };
 
-// Table position of x.  Fast form (all cell indices below 2^22 in magnitude): adding the
-// segment's magic constant 1.5 * 2^23 - c0 + offset to x * 2^G with round-down leaves the
-// position in the low mantissa bits; x is on the grid exactly when round-up gives the same.
-// General form (range far from zero): x * 2^G - c0 is formed first - exact, both are close -
-// and the same constant trick is applied to the difference.
+// Table position of x, and in *grid_bit kCellOnGrid if x lies exactly on the cell grid, else 0.
+// Fast form (all cell indices below 2^22 in magnitude): adding the segment's magic constant
+// 1.5 * 2^23 - c0 + offset to x * 2^G with round-down leaves the position in the low mantissa
+// bits; x is on the grid exactly when round-up gives the same.  General form (range far from
+// zero, one segment): x * 2^G - c0 is formed first - exact, both are close - and the same
+// constant trick is applied to the difference.
 template <bool kFast>
-__device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_grid) {
+__device__ __forceinline__ int cell_position(float x, const CellFn& f, unsigned* grid_bit) {
   float rd, ru;
   if (kFast) {
     // both segments' products are written out and one is kept: measured faster than selecting
-    // the scale and the constant first
+    // the scale and the constant first, by compare-and-select or arithmetically
     const bool inner = fabsf(x) < f.radius;
     rd = inner ? __fmaf_rd(x, f.two_g0, f.magic0) : __fmaf_rd(x, f.two_g1, f.magic1);
     ru = inner ? __fmaf_ru(x, f.two_g0, f.magic0) : __fmaf_ru(x, f.two_g1, f.magic1);
@@ -174,7 +177,9 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, bool* on_
     rd = __fadd_rd(t, 12582913.0f);
     ru = __fadd_ru(t, 12582913.0f);
   }
-  *on_grid = (rd == ru);
+  // A zero is on every grid: in the fast form rd == ru holds for it by itself; in the general
+  // form (where only padding can be zero) it lies far outside the table and is named here.
+  *grid_bit = (rd == ru || (!kFast && x == 0.0f)) ? kCellOnGrid : 0u;
   return __float_as_int(rd) - 0x4B400000;
 }
 
@@ -188,45 +193,41 @@ __device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, i
                                            long long jbeg, long long jend,
                                            const float4* src) {
   float v[kKeyedQuads][4];
-  unsigned vm[kKeyedQuads];
 #pragma unroll
   for (int q = 0; q < kKeyedQuads; ++q) {
     if (kFull) {      // src = this thread's first quad of the tile
       const float4 t = __ldcs(src + q * kKeyedThreads);
       v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
-      vm[q] = 0xFu;
     } else {
       const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
-      vm[q] = 0;
       v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
-      if (j0 < jend) vm[q] = load_quad(base, j0, jbeg, jend, v[q]);
+      if (j0 < jend) load_quad(base, j0, jbeg, jend, v[q]);
     }
   }
 #pragma unroll
   for (int q = 0; q < kKeyedQuads; ++q) {
-    // phase A (no branches): four atomics in flight; exact zeros go to a dummy slot
+    // phase A (no branches): four atomics in flight; exact zeros go to a dummy slot.  An
+    // element on the cell grid gets bit 29 added to its word and is queued too: its handler
+    // may move it one cell to the left.  (Slots that are not loaded hold zeros.)
     unsigned old[4];
     unsigned any = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float x = v[q][k];
-      bool on_grid;
-      int pos = cell_position<kFast>(x, fn, &on_grid);
-      const bool nz = (x != 0.0f) && (kFull || ((vm[q] >> k) & 1u));
-      pos = nz ? pos : dummy_pos;
-      unsigned o = atomicAdd(&cells[pos], 1u);
-      // an element on the cell grid is queued too: its handler may move it one cell to the left
-      o = (nz && on_grid) ? (o | kCellEdge) : o;
+      unsigned grid_bit;
+      int pos = cell_position<kFast>(x, fn, &grid_bit);
+      pos = (x != 0.0f) ? pos : dummy_pos;
+      const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
       old[k] = o;
       any |= o;
     }
     // phase B (rare): elements of marked cells and on-grid elements join the warp's queue;
     // the whole warp enters so that the queue position can stay in a register
-    if (__any_sync(0xffffffffu, any >= kCellNearZero)) {
+    if (__any_sync(0xffffffffu, any >= kCellOnGrid)) {
       const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
-        const bool push = old[k] >= kCellNearZero;
+        const bool push = old[k] >= kCellOnGrid;
         const unsigned pm = __ballot_sync(0xffffffffu, push);
         if (pm) {
           if (push) queue[qn + __popc(pm & lt)] = v[q][k];
@@ -336,7 +337,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
       for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
-      if (threadIdx.x < kDummySlots) cells[p.cell_cap + threadIdx.x] = 0;
+      if (threadIdx.x < kDummySlots)
+        cells[p.cell_cap + threadIdx.x] = kCellEdge | kCellNearZero | kCellOnGrid;
     }
     __syncthreads();
 
