@@ -111,7 +111,7 @@ typedef struct adapt_search_opts {
  * n_bins <= 8192).  DIRECT: the direct form everywhere. */
 enum { ADAPT_ALGO_AUTO = 0, ADAPT_ALGO_KEYED = 1, ADAPT_ALGO_DIRECT = 2 };
 
-/* Library version string, e.g. "adapt-b200 0.4". Never NULL. */
+/* Library version string, e.g. "adapt-b200 0.5". Never NULL. */
 const char* adapt_version(void);
 
 /* Static English text for an adapt_status value. Never NULL. */
