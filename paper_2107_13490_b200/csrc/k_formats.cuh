@@ -133,15 +133,39 @@ __global__ void format_resolve_kernel(const FormatParams p) {
   }
 }
 
+// Exponent classes for the zero counts under round-to-nearest-even: an element rounds to zero
+// exactly when |x| <= 2^t, t = -(level + 1) for a grid rule, emin - M - 1 for a float rule, and
+// that only depends on floor(log2 |x|) and on whether |x| is a power of two.  Class 0 holds the
+// exact zeros, class e + 150 the elements with floor(log2 |x|) = e (-149 <= e <= 127).
+constexpr int kExpClasses = 288;
+
+// Bin index by one convert-with-floor and two integer clamps; equal to bin_of for every input
+// (a NaN converts to 0, out-of-range values saturate and are clamped).
+__device__ __forceinline__ int bin_fast(float v, float lo, float scale, int bmax) {
+  const int b = __float2int_rd(__fmul_rn(__fsub_rn(v, lo), scale));
+  return min(max(b, 0), bmax);
+}
+
+// Float rule with the scaling by 2^k as single multiplications when 2^k and 2^-k are normal.
+template <bool kStochastic>
+__device__ __forceinline__ float float_value_fast(float x, int emin, int m_bits, float pr) {
+  const int e = static_cast<int>((__float_as_uint(x) >> 23) & 0xffu) - 127;
+  const int k = m_bits - max(e, emin);
+  if (k > 126) return float_value<kStochastic>(x, emin, m_bits, pr);   // only |x| < 2^(M-126)
+  return __fmul_rn(round_to_grid<kStochastic>(__fmul_rn(x, pow2f(k)), pr), pow2f(-k));
+}
+
 // Builds the unclamped histogram and the zero count of every rule, every layer.  The rules are
 // cut into groups of rules_per_group (blockIdx.y) so that a group's histograms fit in shared
-// memory; each group reads the tensors once.
+// memory; each group reads the tensors once.  A thread holds four elements and walks the
+// group's rules with them, so a rule's constants are fetched once per four evaluations.
 template <bool kStochastic>
 __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const FormatParams p) {
   extern __shared__ unsigned s_fhist[];   // [rules in the group][n_bins]
   __shared__ int s_kind[kMaxRulesPerGroup], s_i0[kMaxRulesPerGroup], s_i1[kMaxRulesPerGroup];
   __shared__ float s_f0[kMaxRulesPerGroup], s_f1[kMaxRulesPerGroup];
   __shared__ unsigned s_zero[kMaxRulesPerGroup];
+  __shared__ unsigned s_cls[2][kExpClasses];   // [0] all elements, [1] powers of two
 
   const int B = p.n_bins;
   const int r0 = blockIdx.y * p.rules_per_group;
@@ -155,6 +179,7 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
 
   for (int i = threadIdx.x; i < nr * B; i += blockDim.x) s_fhist[i] = 0;
   if (threadIdx.x < kMaxRulesPerGroup) s_zero[threadIdx.x] = 0;
+  if (threadIdx.x < 2 * kExpClasses) (&s_cls[0][0])[threadIdx.x] = 0;
 
   int l = layer_of_tile(p.layers, p.n_layers, t);
   while (t < t_end) {
@@ -165,8 +190,9 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
     const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
+    const int bmax = __float2int_rz(S.bmax);
 
-    // this layer's form of the group's rules
+    // this layer's form of the group's rules; s_i0 of a grid rule = its level
     if (threadIdx.x < nr) {
       const FormatRule R = p.rules[r0 + threadIdx.x];
       s_kind[threadIdx.x] = R.kind;
@@ -175,6 +201,7 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
         s_i1[threadIdx.x] = R.p1;
       } else if (R.kind != kRuleIdentity) {
         const int lev = p.level[static_cast<size_t>(gl) * p.n_rules + r0 + threadIdx.x];
+        s_i0[threadIdx.x] = lev;
         s_f0[threadIdx.x] = pow2f(lev);
         s_f1[threadIdx.x] = pow2f(-lev);
       }
@@ -186,30 +213,61 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
       const long long j_tile = (t - L.tile_begin) * kTile;
       for (int q = 0; q < kTile / 4 / kFormatThreads; ++q) {
         const long long j0 = j_tile + 4ll * (q * kFormatThreads + threadIdx.x);
-        float v[4];
+        float v[4], pr[4];
         unsigned m = 0;
         if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
         else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const bool valid = (m >> k) & 1u;
-          const float x = v[k];
-          float pr = 0.0f;
+          pr[k] = 0.0f;
           if (kStochastic) {
             const unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
                                       static_cast<unsigned long long>(j0 + k - jbeg));
-            pr = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+            pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+          } else if ((m >> k) & 1u) {
+            // exponent class of the element (zero counts of all rules come from these)
+            const unsigned ax = __float_as_uint(v[k]) & 0x7fffffffu;
+            int cls = 0;
+            bool p2 = false;
+            if (ax) {
+              const unsigned eb = ax >> 23, mant = ax & 0x7fffffu;
+              cls = eb ? static_cast<int>(eb) + 23 : 32 - __clz(mant);   // e + 150
+              p2 = eb ? (mant == 0u) : ((mant & (mant - 1u)) == 0u);
+            }
+            atomicAdd(&s_cls[0][cls], 1u);
+            if (p2) atomicAdd(&s_cls[1][cls], 1u);
           }
-          for (int r = 0; r < nr; ++r) {
-            const int kind = s_kind[r];
-            float xq;
-            if (kind == kRuleIdentity) xq = x;
-            else if (kind == kFmtFloat) xq = float_value<kStochastic>(x, s_i0[r], s_i1[r], pr);
-            else xq = level_value<kStochastic>(x, s_f0[r], s_f1[r], pr);
-            const int b = bin_of(xq, S.lo, S.scale, S.bmax);
-            if (valid) atomicAdd(&s_fhist[r * B + b], 1u);
-            const unsigned zm = __ballot_sync(0xffffffffu, valid && xq == 0.0f);
-            if (lane == 0 && zm) atomicAdd(&s_zero[r], __popc(zm));
+        }
+        for (int r = 0; r < nr; ++r) {
+          const int kind = s_kind[r];
+          unsigned* H = s_fhist + r * B;
+          if (kind == kRuleIdentity) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              if ((m >> k) & 1u) atomicAdd(&H[bin_fast(v[k], S.lo, S.scale, bmax)], 1u);
+            continue;
+          }
+          float xq[4];
+          if (kind == kFmtFloat) {
+            const int emin = s_i0[r], mb = s_i1[r];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) xq[k] = float_value_fast<kStochastic>(v[k], emin, mb, pr[k]);
+          } else {
+            const float two_l = s_f0[r], inv_l = s_f1[r];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) xq[k] = level_value<kStochastic>(v[k], two_l, inv_l, pr[k]);
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if ((m >> k) & 1u) atomicAdd(&H[bin_fast(xq[k], S.lo, S.scale, bmax)], 1u);
+          if (kStochastic) {
+            // zero count by vote (the stochastic threshold is per element)
+            unsigned nz = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) nz += (((m >> k) & 1u) && xq[k] == 0.0f) ? 1u : 0u;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nz += __shfl_xor_sync(0xffffffffu, nz, o);
+            if (lane == 0 && nz) atomicAdd(&s_zero[r], nz);
           }
         }
       }
@@ -225,13 +283,23 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
         }
       }
       if (threadIdx.x < nr) {
-        const unsigned c = s_zero[threadIdx.x];
-        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_rules + r0 + threadIdx.x],
-                         static_cast<unsigned long long>(c));
+        unsigned long long c = s_zero[threadIdx.x];
+        if (!kStochastic && s_kind[threadIdx.x] != kRuleIdentity) {
+          // |x| <= 2^t rounds to zero: everything below binade t, the value 2^t itself, zeros
+          const int tz = (s_kind[threadIdx.x] == kFmtFloat)
+                             ? s_i0[threadIdx.x] - s_i1[threadIdx.x] - 1 : -(s_i0[threadIdx.x] + 1);
+          const int ct = tz + 150;           // class of binade t
+          c = s_cls[0][0];
+          for (int i = 1; i < kExpClasses; ++i)
+            if (i < ct) c += s_cls[0][i];
+          if (ct >= 1 && ct < kExpClasses) c += s_cls[1][ct];
+        }
+        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_rules + r0 + threadIdx.x], c);
         s_zero[threadIdx.x] = 0;
       }
     }
     __syncthreads();
+    if (threadIdx.x < 2 * kExpClasses) (&s_cls[0][0])[threadIdx.x] = 0;
     ++l;
     while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
   }
