@@ -36,12 +36,29 @@ struct SearchParams {
   unsigned long long seed;
 };
 
+// Bin index by one convert-with-floor and two integer clamps; equal to bin_of for every input
+// (a NaN converts to 0, out-of-range values saturate and are clamped).
+__device__ __forceinline__ int bin_index_fast(float v, float lo, float scale, int bmax) {
+  const int b = __float2int_rd(__fmul_rn(__fsub_rn(v, lo), scale));
+  return min(max(b, 0), bmax);
+}
+
+// Under round-to-nearest-even an element rounds to zero at fraction length f exactly when
+// |x| <= 2^-(f+1).  kz = the largest such f (capped to -1..32), from the exponent field alone.
+__device__ __forceinline__ int highest_zero_level(float x) {
+  const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
+  if (ax == 0u) return 32;
+  const int kz = 125 - static_cast<int>((ax - 1u) >> 23);
+  return max(-1, min(kz, 32));
+}
+
 template <bool kStochastic>
 __global__ void __launch_bounds__(kSearchThreads)
 search_direct_kernel(const SearchParams p) {
   extern __shared__ unsigned s_hist[];  // [(fl_per_group + 1)][n_bins]
   __shared__ float s_two[kMaxFl], s_inv[kMaxFl];
   __shared__ unsigned s_zero[kMaxFl];
+  __shared__ unsigned s_zlevel[kMaxFl + 2];   // RNE: elements by highest zero level (-1..32)
 
   const int B = p.n_bins;
   const int f0 = blockIdx.y * p.fl_per_group;
@@ -63,6 +80,7 @@ search_direct_kernel(const SearchParams p) {
       s_inv[threadIdx.x] = pow2f(-fl);
     }
   }
+  if (threadIdx.x < kMaxFl + 2) s_zlevel[threadIdx.x] = 0;
   __syncthreads();
 
   int l = layer_of_tile(p.layers, p.n_layers, t);
@@ -74,34 +92,48 @@ search_direct_kernel(const SearchParams p) {
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
     const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
+    const int bmax = __float2int_rz(S.bmax);
 
     for (; t < layer_tiles_end; ++t) {
       if (!layer_ok) continue;
       const long long j_tile = (t - L.tile_begin) * kTile;
       for (int q = 0; q < kTile / 4 / kSearchThreads; ++q) {
         const long long j0 = j_tile + 4ll * (q * kSearchThreads + threadIdx.x);
-        float v[4];
+        float v[4], pr[4];
         unsigned m = 0;
         if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
         else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const bool valid = (m >> k) & 1u;
-          const float x = v[k];
-          if (valid && do_q) atomicAdd(&s_hist[bin_of(x, S.lo, S.scale, S.bmax)], 1u);
-          float pr = 0.0f;
+          pr[k] = 0.0f;
+          if (valid && do_q) atomicAdd(&s_hist[bin_index_fast(v[k], S.lo, S.scale, bmax)], 1u);
           if (kStochastic) {
             unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
                                 static_cast<unsigned long long>(j0 + k - jbeg));
-            pr = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+            pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+          } else if (valid) {
+            atomicAdd(&s_zlevel[highest_zero_level(v[k]) + 1], 1u);
           }
-          for (int f = 0; f < nf; ++f) {
-            float r = round_scaled<kStochastic>(x, s_two[f], pr);
-            float xq = __fmul_rn(r, s_inv[f]);
-            int b = bin_of(xq, S.lo, S.scale, S.bmax);
-            if (valid) atomicAdd(&s_hist[(f + 1) * B + b], 1u);
-            unsigned zm = __ballot_sync(0xffffffffu, valid && r == 0.0f);
-            if (lane == 0 && zm) atomicAdd(&s_zero[f], __popc(zm));
+        }
+        // a thread walks the fraction lengths with its four elements in registers
+        for (int f = 0; f < nf; ++f) {
+          const float two_f = s_two[f], inv_f = s_inv[f];
+          unsigned* H = s_hist + (f + 1) * B;
+          unsigned nz = 0;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float r = round_scaled<kStochastic>(v[k], two_f, pr[k]);
+            const int b = bin_index_fast(__fmul_rn(r, inv_f), S.lo, S.scale, bmax);
+            if ((m >> k) & 1u) {
+              atomicAdd(&H[b], 1u);
+              if (kStochastic) nz += (r == 0.0f) ? 1u : 0u;
+            }
+          }
+          if (kStochastic) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) nz += __shfl_xor_sync(0xffffffffu, nz, o);
+            if (lane == 0 && nz) atomicAdd(&s_zero[f], nz);
           }
         }
       }
@@ -122,13 +154,19 @@ search_direct_kernel(const SearchParams p) {
         }
       }
       if (threadIdx.x < nf) {
-        unsigned c = s_zero[threadIdx.x];
-        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_fl + f0 + threadIdx.x],
-                         static_cast<unsigned long long>(c));
+        unsigned long long c = s_zero[threadIdx.x];
+        if (!kStochastic) {
+          // zero at fraction length f: every element whose highest zero level is >= f
+          const int f = f0 + threadIdx.x;
+          c = 0;
+          for (int kz = f; kz <= 32; ++kz) c += s_zlevel[kz + 1];
+        }
+        if (c) atomicAdd(&p.zeros[static_cast<size_t>(gl) * p.n_fl + f0 + threadIdx.x], c);
         s_zero[threadIdx.x] = 0;
       }
     }
     __syncthreads();
+    if (threadIdx.x < kMaxFl + 2) s_zlevel[threadIdx.x] = 0;
     ++l;
     while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
   }
