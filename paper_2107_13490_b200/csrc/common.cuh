@@ -31,6 +31,8 @@ struct LayerState {
   unsigned flags;    // ADAPT_FLAG_NONFINITE / ADAPT_FLAG_RANGE / ADAPT_FLAG_DEGENERATE
   float lo, hi, scale, bmax;
   float abs_sum;     // sum of |x| (any summation order; only steers table shapes, never results)
+  unsigned zero_count;  // estimate of the exact zeros (the range scan samples one element in
+                        // eight; steers the choice of loop form only, never results)
 };
 
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).

@@ -68,7 +68,26 @@ struct LayerPlan {
   int keyed;        // 1 if the layer goes through the keyed kernel
   int fast;         // 1 if every cell index is below 2^22 in magnitude
   int total_cells;  // seg[0].cells + seg[1].cells
+  unsigned grid_mask;  // low mantissa bits that are zero in every element on its segment's grid
+  int masked;       // 1 if the counting kernel may take "those bits are zero" as its grid-point flag
+  int dense;        // 1 if, besides, exact zeros are so rare that they may go through the handler
+  unsigned grid_mul;   // 2^(32 - bits of grid_mask): x's bit pattern times this is 0 exactly when those bits are
 };
+
+// A float x = M 2^(E-23) (M its 24-bit significand) lies on the grid of level G exactly when
+// M 2^(E-23+G) is an integer, i.e. when M ends in at least 23 - E - G zero bits.  Over a
+// segment whose largest magnitude has exponent E_max, every grid point therefore ends in at
+// least T = 23 - E_max - G zero bits: "the low T bits are zero" flags a superset of the grid
+// points (about one element in 2^T besides them), which the element handler then tests
+// exactly.  Below this many bits the superset is too large to be worth it.
+#ifndef ADAPT_MIN_GRID_MASK_BITS
+#define ADAPT_MIN_GRID_MASK_BITS 8
+#endif
+constexpr int kMinGridMaskBits = ADAPT_MIN_GRID_MASK_BITS;
+#ifndef ADAPT_DENSE_ZERO_RATIO
+#define ADAPT_DENSE_ZERO_RATIO 2048
+#endif
+constexpr long long kDenseZeroRatio = ADAPT_DENSE_ZERO_RATIO;   // <= 0 switches the dense form off
 
 struct PlanParams {
   const LayerDesc* layers;   // keyed layer list
@@ -176,6 +195,21 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     for (int s = 0; s < 2; ++s)
       P.seg[s].magic = 12582912.0f - static_cast<float>(P.seg[s].c0) +
                        static_cast<float>(P.seg[s].offset);
+    int zero_bits = 23;
+    for (int s = 0; s < 2; ++s) {
+      if (s == 1 && P.seg[1].cells == 0) break;
+      // largest magnitude the segment sees: the main segment of two stops below the radius
+      float top = amax;
+      if (s == 0 && P.seg[1].cells > 0) top = __uint_as_float(__float_as_uint(P.radius) - 1u);
+      const int biased = max(1, static_cast<int>((__float_as_uint(top) >> 23) & 0xFFu));
+      zero_bits = min(zero_bits, 23 - (biased - 127) - P.seg[s].g);
+    }
+    P.grid_mask = zero_bits >= 1 ? (1u << zero_bits) - 1u : 0u;
+    P.masked = (P.fast && zero_bits >= kMinGridMaskBits) ? 1 : 0;
+    P.grid_mul = zero_bits >= 1 ? 1u << (32 - zero_bits) : 0u;
+    // zeros handled one by one cost about as much as edge elements: fine below one in 2048
+    P.dense = (kDenseZeroRatio > 0 && P.masked && S.lo <= 0.0f && S.hi >= 0.0f &&
+               static_cast<long long>(S.zero_count) * kDenseZeroRatio <= L.n) ? 1 : 0;
     s_plan = P;
     if (blockIdx.y == 0) p.plan[l] = P;   // every CTA of the layer derives the same plan
   }

@@ -33,6 +33,13 @@
 
 namespace adapt {
 
+#ifndef ADAPT_SEGMENT_INLINE
+#define ADAPT_SEGMENT_INLINE __noinline__
+#endif
+#ifndef ADAPT_KEYED_PF_DIST
+#define ADAPT_KEYED_PF_DIST 1
+#endif
+
 constexpr int kKeyedThreads = 1024;
 constexpr int kKeyedWarps = kKeyedThreads / 32;
 constexpr int kKeyedQuads = 4;                                  // 128-bit loads per thread per tile
@@ -40,6 +47,7 @@ constexpr int kKeyedTile = kKeyedThreads * kKeyedQuads * 4;     // 16384 element
 constexpr int kQueueCap = 160;      // per-warp queue entries: under 32 left over + at most 128 from one quad
 constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..32
 constexpr int kDummySlots = 32;     // where the atomics of exact zeros land (one per lane)
+constexpr int kKeyedPrefetchTiles = ADAPT_KEYED_PF_DIST;   // L2 prefetch distance in tiles (0: none)
 
 struct KeyedParams {
   const LayerDesc* layers;     // keyed layer list (+ sentinel), tiles of kKeyedTile elements
@@ -85,6 +93,10 @@ struct LayerCtx {
   int n_bins, n_levels, d_levels;
   float magic[2];
   int keyed, fast, total_cells;
+  unsigned grid_mask;
+  int masked, dense;
+  unsigned grid_mul;
+  int zero_pos;                // table position of the main segment's cell [0, 2^-G)
 };
 
 // An element that sits exactly on its segment's grid (x * 2^G = p, an integer) is a rounding
@@ -99,10 +111,16 @@ __device__ __forceinline__ int grid_point_goes_left(long long p) {
   return (p & (low << 1)) == 0 ? 1 : 0;
 }
 
-// Handles one queued element (x != 0, finite).  No warp-level primitive inside:
+// Handles one queued element (finite).  No warp-level primitive inside:
 // any subset of lanes may call it.
 __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   const int B = c.n_bins;
+  if (x == 0.0f) {
+    // only the dense form lets an exact zero through: it was counted in the cell [0, 2^-G),
+    // where no zero belongs (zeros are the layer size minus all cell counts)
+    atomicSub(&c.cells[c.zero_pos], 1u);
+    return;
+  }
   const int s = (fabsf(x) < c.radius) ? 0 : 1;
   const float z = __fmul_rn(x, c.two_g[s]);
   const float cf = floorf(z);
@@ -155,7 +173,18 @@ struct CellFn {
   float radius;
   float two_g0, magic0, c0f0;   // main segment
   float two_g1, magic1;         // auxiliary segment (fast layers only)
+  unsigned grid_mask;           // masked form: low significand bits every grid point has zero
+  unsigned grid_mul;            // dense form: 2^(32 - those bits)
+  unsigned cell_base;           // dense form: shared-memory byte address of position 0, minus 4 * 0x4B400000
 };
+
+// How the counting loop finds an element's table position and its grid-point flag.
+constexpr int kCellGeneral = 0;   // range far from zero: difference to the first cell formed first
+constexpr int kCellFast = 1;      // magic-constant index, grid point = round-down equals round-up
+constexpr int kCellMasked = 2;    // magic-constant index, grid-point flag = low significand bits zero
+constexpr int kCellDense = 3;     // as masked, for layers with (almost) no exact zeros: a zero is
+                                  // not steered to a dummy slot but counted in the cell [0, 2^-G),
+                                  // which is marked, and taken out again by the element handler
 
 // Table position of x, and in *grid_bit kCellOnGrid if x lies exactly on the cell grid, else 0.
 // Fast form (all cell indices below 2^22 in magnitude): adding the segment's magic constant
@@ -163,9 +192,20 @@ struct CellFn {
 // bits; x is on the grid exactly when round-up gives the same.  General form (range far from
 // zero, one segment): x * 2^G - c0 is formed first - exact, both are close - and the same
 // constant trick is applied to the difference.
-template <bool kFast>
+//
+// Masked form: the flag is a cheap superset instead - every grid point of the layer has its
+// low significand bits zero (LayerPlan::grid_mask), so those bits being zero sends the element
+// to its handler, which tests exactly; a zero passes the test too, as it must.
+template <int kMode>
 __device__ __forceinline__ int cell_position(float x, const CellFn& f, unsigned* grid_bit) {
+  constexpr bool kFast = kMode != kCellGeneral;
   float rd, ru;
+  if (kMode == kCellMasked) {
+    const bool inner = fabsf(x) < f.radius;
+    rd = inner ? __fmaf_rd(x, f.two_g0, f.magic0) : __fmaf_rd(x, f.two_g1, f.magic1);
+    *grid_bit = (__float_as_uint(x) & f.grid_mask) == 0u ? kCellOnGrid : 0u;
+    return __float_as_int(rd) - 0x4B400000;
+  }
   if (kFast) {
     // both segments' products are written out and one is kept: measured faster than selecting
     // the scale and the constant first, by compare-and-select or arithmetically
@@ -183,92 +223,145 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, unsigned*
   return __float_as_int(rd) - 0x4B400000;
 }
 
-// One tile: this thread's four quads are loaded first (guarded loads when the tile is ragged),
-// then processed quad by quad.  (Fetching the next tile ahead into the same registers was
-// measured and lost: under the 64-register cap it only bought spills.)
-template <bool kFast, bool kFull>
-__device__ __forceinline__ void keyed_tile(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                           float* queue, unsigned& qn,
-                                           const CellFn& fn, const float* base, long long j_tile,
-                                           long long jbeg, long long jend,
-                                           const float4* src) {
-  float v[kKeyedQuads][4];
+// One quad (four consecutive elements held by this thread): phase A counts them, phase B
+// queues the marked ones and drains the warp's queue when 32 entries have gathered.
+template <int kMode>
+__device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                           float* queue, unsigned& qn, const CellFn& fn,
+                                           const float (&v)[4]) {
+  unsigned old[4];
+  bool enter;
+  if (kMode == kCellDense) {
+    // phase A, dense form: no zero test and no flag arithmetic.  The grid-point test is kept
+    // apart from the returned words: x's bit pattern times grid_mul is 0 exactly when the
+    // low significand bits that every grid point has zero are zero (a zero included, which
+    // lands in the marked cell [0, 2^-G) and is queued anyway).
+    unsigned any = 0, tmin = 0xFFFFFFFFu;
 #pragma unroll
-  for (int q = 0; q < kKeyedQuads; ++q) {
-    if (kFull) {      // src = this thread's first quad of the tile
-      const float4 t = __ldcs(src + q * kKeyedThreads);
-      v[q][0] = t.x; v[q][1] = t.y; v[q][2] = t.z; v[q][3] = t.w;
-    } else {
-      const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
-      v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
-      if (j0 < jend) load_quad(base, j0, jbeg, jend, v[q]);
+    for (int k = 0; k < 4; ++k) {
+      const float x = v[k];
+      const bool inner = fabsf(x) < fn.radius;
+      const float rd = inner ? __fmaf_rd(x, fn.two_g0, fn.magic0) : __fmaf_rd(x, fn.two_g1, fn.magic1);
+      const unsigned addr = __float_as_uint(rd) * 4u + fn.cell_base;
+      unsigned o;
+      asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(o) : "r"(addr) : "memory");
+      old[k] = o;
+      any |= o;
+      tmin = min(tmin, __float_as_uint(x) * fn.grid_mul);
     }
-  }
-#pragma unroll
-  for (int q = 0; q < kKeyedQuads; ++q) {
+    enter = any >= kCellOnGrid || tmin == 0u;
+  } else {
     // phase A (no branches): four atomics in flight; exact zeros go to a dummy slot.  An
     // element on the cell grid gets bit 29 added to its word and is queued too: its handler
     // may move it one cell to the left.  (Slots that are not loaded hold zeros.)
-    unsigned old[4];
     unsigned any = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const float x = v[q][k];
+      const float x = v[k];
       unsigned grid_bit;
-      int pos = cell_position<kFast>(x, fn, &grid_bit);
+      int pos = cell_position<kMode>(x, fn, &grid_bit);
       pos = (x != 0.0f) ? pos : dummy_pos;
       const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
       old[k] = o;
       any |= o;
     }
-    // phase B (rare): elements of marked cells and on-grid elements join the warp's queue;
-    // the whole warp enters so that the queue position can stay in a register
-    if (__any_sync(0xffffffffu, any >= kCellOnGrid)) {
-      const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
+    enter = any >= kCellOnGrid;
+  }
+  // phase B (rare): elements of marked cells and on-grid elements join the warp's queue;
+  // the whole warp enters so that the queue position can stay in a register
+  if (__any_sync(0xffffffffu, enter)) {
+    const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const bool push = old[k] >= kCellOnGrid;
-        const unsigned pm = __ballot_sync(0xffffffffu, push);
-        if (pm) {
-          if (push) queue[qn + __popc(pm & lt)] = v[q][k];
-          qn += __popc(pm);
-        }
-      }
-      if (qn >= 32u) {           // drain full groups of 32 (dense lanes)
-        __syncwarp();
-        do {
-          qn -= 32u;
-          handle_special(c, queue[qn + (threadIdx.x & 31)]);
-        } while (qn >= 32u);
-        __syncwarp();
+    for (int k = 0; k < 4; ++k) {
+      bool push = old[k] >= kCellOnGrid;
+      if (kMode == kCellDense) push = push || __float_as_uint(v[k]) * fn.grid_mul == 0u;
+      const unsigned pm = __ballot_sync(0xffffffffu, push);
+      if (pm) {
+        if (push) queue[qn + __popc(pm & lt)] = v[k];
+        qn += __popc(pm);
       }
     }
+    if (qn >= 32u) {           // drain full groups of 32 (dense lanes)
+      __syncwarp();
+      do {
+        qn -= 32u;
+        handle_special(c, queue[qn + (threadIdx.x & 31)]);
+      } while (qn >= 32u);
+      __syncwarp();
+    }
   }
+}
+
+// A ragged tile (the layer's first one when the tensor does not start on a 16-byte boundary, or
+// its last): guarded loads, slots outside the layer hold zeros.
+template <int kMode>
+__device__ __forceinline__ void keyed_tile_ragged(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                                  float* queue, unsigned& qn, const CellFn& fn,
+                                                  const float* base, long long j_tile,
+                                                  long long jbeg, long long jend) {
+  float v[kKeyedQuads][4];
+#pragma unroll
+  for (int q = 0; q < kKeyedQuads; ++q) {
+    const long long j0 = j_tile + 4ll * (q * kKeyedThreads + threadIdx.x);
+    v[q][0] = v[q][1] = v[q][2] = v[q][3] = 0.0f;
+    if (j0 < jend) load_quad(base, j0, jbeg, jend, v[q]);
+  }
+#pragma unroll
+  for (int q = 0; q < kKeyedQuads; ++q) keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, fn, v[q]);
+}
+
+__device__ __forceinline__ void load_full_quad(const float4* src, float (&v)[4]) {
+  const float4 t = __ldcs(src);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
 }
 
 // All tiles [k0, k1) of one layer that this CTA owns (k counts the layer's own tiles).  Only
 // the layer's first tile (when the tensor does not start on a 16-byte boundary) and its last
 // tile can be ragged; every tile between runs through a loop that carries one running pointer.
-template <bool kFast>
-__device__ __forceinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
+template <int kMode>
+__device__ ADAPT_SEGMENT_INLINE void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
                                               float* queue,
-                                              const CellFn& fn, const float* base, long long jbeg,
+                                              const float* base, long long jbeg,
                                               long long jend, int k0, int k1) {
+  // only the constants this form uses are taken into registers
+  CellFn fn;
+  fn.radius = c.radius;
+  fn.two_g0 = c.two_g[0]; fn.magic0 = c.magic[0]; fn.c0f0 = c.c0f[0];
+  fn.two_g1 = c.two_g[1]; fn.magic1 = c.magic[1];
+  fn.grid_mask = c.grid_mask;
+  fn.grid_mul = c.grid_mul;
+  fn.cell_base = static_cast<unsigned>(__cvta_generic_to_shared(cells)) - 4u * 0x4B400000u;
   unsigned qn = 0;             // entries in this warp's queue (same in every lane)
+  // a ragged tile pads with zeros, which the dense form must not see
+  constexpr int kRagged = kMode == kCellDense ? kCellMasked : kMode;
   const int kf0 = max(k0, jbeg > 0 ? 1 : 0);
   const int kf1 = min(k1, static_cast<int>(jend / kKeyedTile));
   if (k0 < kf0)
-    keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
-                             static_cast<long long>(k0) * kKeyedTile, jbeg, jend, nullptr);
+    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, fn, base,
+                               static_cast<long long>(k0) * kKeyedTile, jbeg, jend);
   if (kf0 < kf1) {
     const float4* src = reinterpret_cast<const float4*>(base + static_cast<long long>(kf0) * kKeyedTile) +
                         threadIdx.x;
-    for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4)
-      keyed_tile<kFast, true>(c, cells, dummy_pos, queue, qn, fn, base, 0, 0, 0, src);
+    for (int k = kf0; k < kf1; ++k, src += kKeyedTile / 4) {
+      // ask for the next tile to be brought into L2 while this one is counted: one bulk
+      // request from one thread (requests cut into per-warp pieces, or reaching further
+      // ahead, were measured to gain less or to lose)
+      if (kKeyedPrefetchTiles > 0 && threadIdx.x == 0 && k + kKeyedPrefetchTiles < kf1)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::
+                     "l"(base + static_cast<long long>(k + kKeyedPrefetchTiles) * kKeyedTile),
+                     "r"(kKeyedTile * 4) : "memory");
+      // the thread's four quads are loaded first, then counted quad by quad.  (Fetching ahead
+      // into registers - the next tile, or half tiles in turn - was measured and lost.)
+      float v[kKeyedQuads][4];
+#pragma unroll
+      for (int q = 0; q < kKeyedQuads; ++q) load_full_quad(src + q * kKeyedThreads, v[q]);
+#pragma unroll
+      for (int q = 0; q < kKeyedQuads; ++q) keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, fn, v[q]);
+    }
   }
   for (int k = max(kf1, kf0); k < k1; ++k)
-    keyed_tile<kFast, false>(c, cells, dummy_pos, queue, qn, fn, base,
-                             static_cast<long long>(k) * kKeyedTile, jbeg, jend, nullptr);
+    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, fn, base,
+                               static_cast<long long>(k) * kKeyedTile, jbeg, jend);
   // what is left in the queue
   __syncwarp();
   if ((threadIdx.x & 31) < qn) handle_special(c, queue[threadIdx.x & 31]);
@@ -310,6 +403,9 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.g[1] = P->seg[1].g; c.fs[1] = P->seg[1].fs; c.offset[1] = P->seg[1].offset;
       c.magic[0] = P->seg[0].magic; c.magic[1] = P->seg[1].magic;
       c.keyed = P->keyed; c.fast = P->fast; c.total_cells = P->total_cells;
+      c.grid_mask = P->grid_mask; c.masked = P->masked; c.dense = P->dense;
+      c.grid_mul = P->grid_mul;
+      c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
       c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
       c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
       c.qe_aux = p.qe_hist + (static_cast<size_t>(l) * 2 + 1) * p.n_bins;
@@ -326,10 +422,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     const bool ok = c.keyed != 0;
     const bool fast = c.fast != 0;
     const int total_cells = c.total_cells;
-    CellFn fn;
-    fn.radius = c.radius;
-    fn.two_g0 = c.two_g[0]; fn.magic0 = c.magic[0]; fn.c0f0 = c.c0f[0];
-    fn.two_g1 = c.two_g[1]; fn.magic1 = c.magic[1];
+    const bool masked = c.masked != 0;
+    const bool dense = c.dense != 0;
 
     // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
@@ -344,8 +438,10 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
 
     if (ok) {
       const int k0 = static_cast<int>(t - L.tile_begin), k1 = static_cast<int>(layer_tiles_end - L.tile_begin);
-      if (fast) keyed_segment<true>(c, cells, dummy_pos, queue, fn, base, jbeg, jend, k0, k1);
-      else keyed_segment<false>(c, cells, dummy_pos, queue, fn, base, jbeg, jend, k0, k1);
+      if (dense) keyed_segment<kCellDense>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else if (masked) keyed_segment<kCellMasked>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else if (fast) keyed_segment<kCellFast>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else keyed_segment<kCellGeneral>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
     }
     t = layer_tiles_end;
     __syncthreads();
