@@ -212,13 +212,13 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   for (int c = 0; c < grid->n_cand; ++c) p->fl_begin[grid->fl[c] + 1] += 1;
   for (int f = 0; f < p->n_levels; ++f) p->fl_begin[f + 1] += p->fl_begin[f];
 
-  // shared-memory shape of the keyed kernel: queue + Qe + a few correction levels + cells
+  // shared-memory shape of the keyed kernel: queue + bin edges + Qe + a few correction levels + cells
   const size_t hist = sizeof(unsigned) * n_bins;
   const size_t queue = keyed_smem_bytes(0, 0, 0);
   p->d_levels = static_cast<int>(std::min<size_t>(6, (32 * 1024) / hist));
   p->d_levels = std::min(p->d_levels, p->n_levels);
   if (n_bins <= kKeyedMaxBins) {
-    p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (1 + p->d_levels)) / 4) - 64;
+    p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (2 + p->d_levels)) / 4) - 64;
     p->cell_cap = std::min(p->cell_cap, 1 << 16);
   } else {
     p->cell_cap = 0;
@@ -563,7 +563,7 @@ int run_quantize(const float* x, int64_t n, int wl, int fl, const int32_t* selec
 
 extern "C" {
 
-const char* adapt_version(void) { return "adapt-b200 0.5"; }
+const char* adapt_version(void) { return "adapt-b200 0.6"; }
 
 const char* adapt_status_string(int status) {
   switch (status) {

@@ -45,6 +45,9 @@ constexpr int kPlanThreads = 256;
 #ifndef ADAPT_CELL_BALANCE
 #define ADAPT_CELL_BALANCE 4    // cells ~ sqrt(balance * n_bins * elements one CTA sees of the layer)
 #endif
+#ifndef ADAPT_RADIUS_FACTOR
+#define ADAPT_RADIUS_FACTOR 8.0   // main segment reaches to the power of two above this many mean magnitudes
+#endif
 #ifndef ADAPT_FINE_RATIO
 #define ADAPT_FINE_RATIO 512    // stop refining once a bin holds this many cells
 #endif
@@ -162,7 +165,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     const float mean = S.abs_sum / static_cast<float>(L.n > 0 ? L.n : 1);
     if (P.keyed && S.lo <= 0.0f && S.hi >= 0.0f && P.seg[0].g < g_want && mean > 0.0f &&
         mean < 3.0e38f) {
-      const int rexp = static_cast<int>(ceil(log2(static_cast<double>(mean) * 8.0)));
+      const int rexp = static_cast<int>(ceil(log2(static_cast<double>(mean) * ADAPT_RADIUS_FACTOR)));
       if (rexp > -100 && rexp < 100) {
         const float r = pow2f(rexp);
         if (r < 0.25f * amax) {

@@ -18,13 +18,23 @@
 // which makes every coarse rounding tie come out even.
 // Exact zeros are sent to per-lane dummy slots (their number is the layer size
 // minus the sum of the cell counts).  A dummy slot starts with all three top bits set; zero is
-// on every grid, so the added bit 29 wraps the returned word around to a plain small count.  Everything else about an element - the
-// float histogram, all coarse levels, all fine levels of interior cells - is
-// derived from the cell counts by the expand kernel.
+// on every grid, so the added bit 29 wraps the returned word around to a plain small count.
+// Everything else about an element - the float histogram, all coarse levels, all fine levels
+// of interior cells - is derived from the cell counts by the expand kernel.
+//
+// Four forms of the counting loop, chosen per layer by the plan (same results, different cost):
+//   general  range far from zero (cell indices of 2^22 and more): difference to the first cell first;
+//   fast     magic-constant index, grid point = "round-down equals round-up" (two more FMAs);
+//   masked   magic-constant index, grid-point flag = "the low significand bits that every grid
+//            point of the layer has zero are zero" (a superset, settled exactly by the handler);
+//   dense    as masked, for layers with (almost) no exact zeros: no zero test, no flag arithmetic
+//            on the returned word; a zero lands in the marked cell [0, 2^-G) and its handler
+//            takes it out again.
 //
 // One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
 // for its tables; each thread handles 16 elements (four 128-bit loads, issued
-// together) per tile.
+// together) per tile, and one thread asks for the CTA's next tile to be brought into L2
+// by a bulk prefetch while the current one is counted.
 #pragma once
 
 #include "common.cuh"
@@ -33,11 +43,8 @@
 
 namespace adapt {
 
-#ifndef ADAPT_SEGMENT_INLINE
-#define ADAPT_SEGMENT_INLINE __noinline__
-#endif
 #ifndef ADAPT_KEYED_PF_DIST
-#define ADAPT_KEYED_PF_DIST 1
+#define ADAPT_KEYED_PF_DIST 1    // tiles between the one being counted and the one asked into L2
 #endif
 
 constexpr int kKeyedThreads = 1024;
@@ -72,6 +79,7 @@ struct KeyedParams {
 __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int d_levels) {
   return sizeof(unsigned) * (static_cast<size_t>(cell_cap) + kDummySlots + n_bins +
                              static_cast<size_t>(d_levels) * n_bins) +
+         sizeof(float) * (static_cast<size_t>(n_bins) + 4) +      // the layer's bin edges
          sizeof(float) * kKeyedWarps * kQueueCap;
 }
 
@@ -82,7 +90,7 @@ struct LayerCtx {
   float two_g[2], c0f[2];      // cell function per segment (general form)
   long long c0[2];
   int g[2], fs[2], offset[2];
-  const float* E;              // exact bin edges [n_bins + 1]
+  const float* E;              // shared copy of the layer's exact bin edges [n_bins + 1]
   unsigned* cells;             // shared cell table (marks in the two top bits)
   unsigned* qe;                // shared [n_bins]: main segment's edge-element histogram
   int* d;                      // shared [d_levels][n_bins]
@@ -144,7 +152,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
   if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
-  const float e_lo = __ldg(c.E + b0), e_hi = __ldg(c.E + b0 + 1);
+  const float e_lo = c.E[b0], e_hi = c.E[b0 + 1];
   // distance to the bin's two edges, rounded down: a level is safe once 2^-(f+1) < margin
   const float m = fminf(__fsub_rd(x, e_lo), __fsub_rd(e_hi, x));
   int f_end = 32;
@@ -223,19 +231,16 @@ __device__ __forceinline__ int cell_position(float x, const CellFn& f, unsigned*
   return __float_as_int(rd) - 0x4B400000;
 }
 
-// One quad (four consecutive elements held by this thread): phase A counts them, phase B
-// queues the marked ones and drains the warp's queue when 32 entries have gathered.
+// Phase A of one quad (four consecutive elements held by this thread), no branches: the four
+// atomics are issued together.  Returns whether one of the four must be looked at in phase B.
 template <int kMode>
-__device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                           float* queue, unsigned& qn, const CellFn& fn,
-                                           const float (&v)[4]) {
-  unsigned old[4];
-  bool enter;
+__device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, const CellFn& fn,
+                                            const float (&v)[4], unsigned (&old)[4]) {
   if (kMode == kCellDense) {
-    // phase A, dense form: no zero test and no flag arithmetic.  The grid-point test is kept
-    // apart from the returned words: x's bit pattern times grid_mul is 0 exactly when the
-    // low significand bits that every grid point has zero are zero (a zero included, which
-    // lands in the marked cell [0, 2^-G) and is queued anyway).
+    // dense form: no zero test and no flag arithmetic.  The grid-point test is kept apart
+    // from the returned words: x's bit pattern times grid_mul is 0 exactly when the low
+    // significand bits that every grid point has zero are zero (a zero included, which lands
+    // in the marked cell [0, 2^-G) and is queued anyway).
     unsigned any = 0, tmin = 0xFFFFFFFFu;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -249,26 +254,32 @@ __device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, i
       any |= o;
       tmin = min(tmin, __float_as_uint(x) * fn.grid_mul);
     }
-    enter = any >= kCellOnGrid || tmin == 0u;
-  } else {
-    // phase A (no branches): four atomics in flight; exact zeros go to a dummy slot.  An
-    // element on the cell grid gets bit 29 added to its word and is queued too: its handler
-    // may move it one cell to the left.  (Slots that are not loaded hold zeros.)
-    unsigned any = 0;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const float x = v[k];
-      unsigned grid_bit;
-      int pos = cell_position<kMode>(x, fn, &grid_bit);
-      pos = (x != 0.0f) ? pos : dummy_pos;
-      const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
-      old[k] = o;
-      any |= o;
-    }
-    enter = any >= kCellOnGrid;
+    return any >= kCellOnGrid || tmin == 0u;
   }
-  // phase B (rare): elements of marked cells and on-grid elements join the warp's queue;
-  // the whole warp enters so that the queue position can stay in a register
+  // exact zeros go to a dummy slot.  An element on the cell grid gets bit 29 added to its
+  // word and is queued too: its handler may move it one cell to the left.  (Slots that are
+  // not loaded hold zeros.)
+  unsigned any = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float x = v[k];
+    unsigned grid_bit;
+    int pos = cell_position<kMode>(x, fn, &grid_bit);
+    pos = (x != 0.0f) ? pos : dummy_pos;
+    const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
+    old[k] = o;
+    any |= o;
+  }
+  return any >= kCellOnGrid;
+}
+
+// Phase B of one quad (rare): elements of marked cells and on-grid elements join the warp's
+// queue, which is drained when 32 entries have gathered; the whole warp enters so that the
+// queue position can stay in a register.
+template <int kMode>
+__device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, unsigned& qn,
+                                            const CellFn& fn, const float (&v)[4],
+                                            const unsigned (&old)[4], bool enter) {
   if (__any_sync(0xffffffffu, enter)) {
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
@@ -290,6 +301,15 @@ __device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, i
       __syncwarp();
     }
   }
+}
+
+template <int kMode>
+__device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                           float* queue, unsigned& qn, const CellFn& fn,
+                                           const float (&v)[4]) {
+  unsigned old[4];
+  const bool enter = keyed_count<kMode>(cells, dummy_pos, fn, v, old);
+  keyed_queue<kMode>(c, queue, qn, fn, v, old, enter);
 }
 
 // A ragged tile (the layer's first one when the tensor does not start on a 16-byte boundary, or
@@ -318,11 +338,12 @@ __device__ __forceinline__ void load_full_quad(const float4* src, float (&v)[4])
 // All tiles [k0, k1) of one layer that this CTA owns (k counts the layer's own tiles).  Only
 // the layer's first tile (when the tensor does not start on a 16-byte boundary) and its last
 // tile can be ragged; every tile between runs through a loop that carries one running pointer.
+// Not inlined: each form then gets its own register allocation under the 64-register cap
+// (inlined side by side the four forms spill inside their loops).
 template <int kMode>
-__device__ ADAPT_SEGMENT_INLINE void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                              float* queue,
-                                              const float* base, long long jbeg,
-                                              long long jend, int k0, int k1) {
+__device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
+                                           float* queue, const float* base, long long jbeg,
+                                           long long jend, int k0, int k1) {
   // only the constants this form uses are taken into registers
   CellFn fn;
   fn.radius = c.radius;
@@ -375,7 +396,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
   unsigned* cells = reinterpret_cast<unsigned*>(s_raw);          // [cell_cap + kDummySlots]
   unsigned* qe = cells + p.cell_cap + kDummySlots;
   int* dtab = reinterpret_cast<int*>(qe + p.n_bins);
-  float* queues = reinterpret_cast<float*>(dtab + static_cast<size_t>(p.d_levels) * p.n_bins);
+  float* edges = reinterpret_cast<float*>(dtab + static_cast<size_t>(p.d_levels) * p.n_bins);   // [n_bins + 4]
+  float* queues = edges + p.n_bins + 4;
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* queue = queues + warp * kQueueCap;
@@ -406,7 +428,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.grid_mask = P->grid_mask; c.masked = P->masked; c.dense = P->dense;
       c.grid_mul = P->grid_mul;
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
-      c.E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
+      c.E = edges;
       c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
       c.qe_aux = p.qe_hist + (static_cast<size_t>(l) * 2 + 1) * p.n_bins;
       c.u_hist = layer_u;
@@ -430,6 +452,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
       for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
       for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
+      const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
+      for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
       if (threadIdx.x < kDummySlots)
         cells[p.cell_cap + threadIdx.x] = kCellEdge | kCellNearZero | kCellOnGrid;
