@@ -152,6 +152,19 @@ def test_adversarial_value_patterns(B):
     cases["narrow_offset"] = (0.75 + rng.integers(0, 50, n) * 2.0 ** -24).astype(np.float32)
     cases["two_values"] = np.where(rng.random(n) < 0.3, 0.1, -0.7).astype(np.float32)
     cases["integers"] = rng.integers(-300, 300, n).astype(np.float32)
+    # the counting loop's forms: a handful of exact zeros among values off and on the cell grid
+    # (the form without zero steering, whose element handler takes the zeros out again), a
+    # positive range away from zero with few zero significand bits to go by, and one with many
+    few = base.copy()
+    few[rng.integers(0, n, 6)] = np.float32([0.0, -0.0, 0.0, 0.0, -0.0, 0.0])
+    cases["few_zeros"] = few
+    grid_few = (rng.integers(1, 4000, n) * rng.choice([-1.0, 1.0], n) * 2.0 ** -9).astype(np.float32)
+    grid_few[rng.integers(0, n, 4)] = 0.0
+    cases["few_zeros_on_grid"] = grid_few
+    off100 = (100.0 + rng.random(n)).astype(np.float32)
+    off100[::7] = (100.0 + rng.integers(0, 2048, off100[::7].size) * 2.0 ** -11).astype(np.float32)
+    cases["offset_100"] = off100
+    cases["half_to_one"] = (0.5 + 0.5 * rng.random(n)).astype(np.float32)
     wl, fl = W.candidate_grid(range(2, 33))
     for name, x in cases.items():
         for n_bins in (100, 2048):
