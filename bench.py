@@ -49,6 +49,11 @@ def parse_args():
     ap.add_argument("--path", default="search", choices=["search", "diversity", "formats"],
                     help="search: the precision-switch search step (default); diversity: the "
                          "gradient-diversity reduction that feeds PushUp")
+    ap.add_argument("--algorithm", default="auto", choices=["auto", "keyed", "direct"],
+                    help="profiling aid: which form of the fused search kernel runs (auto: the "
+                         "library's own choice; keyed serves round-to-nearest-even only)")
+    ap.add_argument("--round-mode", default="workload", choices=["workload", "rne", "stochastic"],
+                    help="profiling aid: override the workload's rounding mode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -367,6 +372,8 @@ def main():
     if args.elements:
         base = W.scaled(base, args.elements)
     w = S.rank_workload(base, rank)
+    round_mode = {"workload": w.round_mode, "rne": 0, "stochastic": 1}[args.round_mode]
+    algorithm = {"auto": 0, "keyed": 1, "direct": 2}[args.algorithm]
     wl, fl = w.grid()
     grid = B.Grid(wl, fl)
     n_cand = len(grid)
@@ -384,9 +391,9 @@ def main():
     torch.cuda.synchronize()
 
     def step():
-        B.adapt_precision_search_ex(xs, grid, w.n_bins, round_mode=w.round_mode, seed=w.seed,
-                                    workspace=ws, out=out)
-        B.adapt_quantize_selected_batch(xs, out.best, w.round_mode, w.seed, 0, codes_out=codes)
+        B.adapt_precision_search_ex(xs, grid, w.n_bins, round_mode=round_mode, seed=w.seed,
+                                    workspace=ws, out=out, algorithm=algorithm)
+        B.adapt_quantize_selected_batch(xs, out.best, round_mode, w.seed, 0, codes_out=codes)
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -436,16 +443,34 @@ def main():
     # ---- roofline of the dominant kernel (the fused search kernel) ----------------
     peak, peak_kind = measured_peak_gbs()
     ms_search, n_search = ktimes["search"]
+    ms_direct, n_direct = ktimes.get("search_direct", (0.0, 0))
     algo_bytes = 4.0 * total     # one fp32 read of every element per launch
-    achieved = algo_bytes / (ms_search / n_search * 1e-3) / 1e9 if n_search else None
-    traffic = None
-    if TRAFFIC_CAPTURE["version"] == B.adapt_version() and TRAFFIC_CAPTURE["bytes_per_element"]:
-        traffic = TRAFFIC_CAPTURE["bytes_per_element"] * total
-    roofline = {"bound": "hbm", "kernel": "search (fused quantize/zero-count/histograms)",
-                "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "algorithmic_bytes_per_launch": algo_bytes,
-                "avg_launch_ms": ms_search / n_search if n_search else None}
+    if ms_search >= ms_direct:
+        achieved = algo_bytes / (ms_search / n_search * 1e-3) / 1e9 if n_search else None
+        traffic = None
+        if TRAFFIC_CAPTURE["version"] == B.adapt_version() and TRAFFIC_CAPTURE["bytes_per_element"]:
+            traffic = TRAFFIC_CAPTURE["bytes_per_element"] * total
+        roofline = {"bound": "hbm", "kernel": "search (fused quantize/zero-count/histograms)",
+                    "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                    "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                    "algorithmic_bytes_per_launch": algo_bytes,
+                    "avg_launch_ms": ms_search / n_search if n_search else None}
+    else:
+        # The direct form evaluates every fraction length per element and is issue-bound: one
+        # (element, FL) evaluation needs at least 10 lane instructions (scale, round, rescale;
+        # subtract, multiply, floor, two clamps, convert; one shared atomic), and an SM issues
+        # 128 lane instructions per clock.
+        n_fl = int(max(fl)) + 1
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+        alu_peak = sm_count * 128 * sm_mhz * 1e6 / 10.0 / 1e9
+        achieved = float(total) * n_fl / (ms_direct / args.steps * 1e-3) / 1e9
+        roofline = {"bound": "alu", "kernel": "search_direct (every fraction length per element)",
+                    "achieved": achieved, "peak": alu_peak,
+                    "peak_kind": "SMs x 128 lanes x sampled SM clock / 10 instructions per evaluation",
+                    "unit": "G element-FL evaluations/s", "frac": achieved / alu_peak,
+                    "hbm_gbs": algo_bytes / (ms_direct / args.steps * 1e-3) / 1e9, "traffic": None,
+                    "launches_per_step": n_direct / args.steps}
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps}
                for k, v in ktimes.items() if v[1]}
 
@@ -458,7 +483,7 @@ def main():
         host_codes = [torch.empty(n, dtype=torch.int32).pin_memory() for n in lens]
 
         def e2e_step():
-            B.adapt_precision_switch_host(pinned, grid, w.n_bins, round_mode=w.round_mode,
+            B.adapt_precision_switch_host(pinned, grid, w.n_bins, round_mode=round_mode,
                                           seed=w.seed, out=host_out, codes_out=host_codes)
 
         e2e_step()
@@ -490,7 +515,8 @@ def main():
                 "config": {"workload": base.name, "description": base.description,
                            "elements_per_gpu": total, "layers": len(xs), "candidates": n_cand,
                            "n_bins": w.n_bins,
-                           "round_mode": "rne" if w.round_mode == 0 else "stochastic",
+                           "round_mode": "rne" if round_mode == 0 else "stochastic",
+                           "algorithm": args.algorithm,
                            "step": "adapt_precision_search_ex + adapt_quantize_selected_batch",
                            "l2": "inputs exceed L2" if not fits_l2 else
                                  "L2 flushed (512 MiB write) between timed steps",
