@@ -52,6 +52,65 @@ __device__ __forceinline__ int highest_zero_level(float x) {
   return max(-1, min(kz, 32));
 }
 
+// The bin function without a float-to-int conversion: floor(clamp(u, 0, top)), top the largest
+// float below n_bins, equals clamp(floor(u), 0, n_bins - 1) for every u (a NaN clamps to 0 as
+// fmaxf returns its other operand), and adding 1.5 * 2^23 with round-down leaves that floor in
+// the low mantissa bits.  Returned: the byte offset 4 * bin + 4 * 0x4B400000 (mod 2^32), which
+// the caller adds to a histogram base that has the constant subtracted.
+__device__ __forceinline__ unsigned bin_offset_magic(float v, float lo, float scale, float top) {
+  const float u = __fmul_rn(__fsub_rn(v, lo), scale);
+  const float c = fminf(fmaxf(u, 0.0f), top);
+  return __float_as_uint(__fadd_rd(c, 12582912.0f)) * 4u;
+}
+
+__device__ __forceinline__ void shared_inc(unsigned byte_addr) {
+  asm volatile("red.shared.add.u32 [%0], 1;" :: "r"(byte_addr) : "memory");
+}
+
+// Four elements of one thread through the float histogram, the zero bookkeeping and every
+// fraction length of the group.  kMasked: some of the four lie outside the layer (mask m).
+template <bool kStochastic, bool kMasked>
+__device__ __forceinline__ void direct_quad(const float (&v)[4], unsigned m, long long index0,
+                                            const SearchParams& p, int layer_id, float lo,
+                                            float scale, float top, int nf, bool do_q,
+                                            unsigned hist_base, unsigned hist_stride,
+                                            const float* s_two, const float* s_inv,
+                                            unsigned* s_zero, unsigned* s_zlevel) {
+  float pr[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const bool valid = !kMasked || ((m >> k) & 1u);
+    pr[k] = 0.0f;
+    if (valid && do_q) shared_inc(hist_base + bin_offset_magic(v[k], lo, scale, top));
+    if (kStochastic) {
+      const unsigned h = hash24(p.seed, static_cast<unsigned long long>(layer_id),
+                                static_cast<unsigned long long>(index0 + k));
+      pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+    } else if (valid) {
+      atomicAdd(&s_zlevel[highest_zero_level(v[k]) + 1], 1u);
+    }
+  }
+  // the thread walks the fraction lengths with its four elements in registers
+  unsigned hb = hist_base + hist_stride;
+  for (int f = 0; f < nf; ++f, hb += hist_stride) {
+    const float two_f = s_two[f], inv_f = s_inv[f];
+    unsigned nz = 0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float r = round_scaled<kStochastic>(v[k], two_f, pr[k]);
+      const unsigned off = bin_offset_magic(__fmul_rn(r, inv_f), lo, scale, top);
+      if (!kMasked || ((m >> k) & 1u)) {
+        shared_inc(hb + off);
+        if (kStochastic) nz += (r == 0.0f) ? 1u : 0u;
+      }
+    }
+    if (kStochastic) {
+      nz = __reduce_add_sync(0xffffffffu, nz);
+      if ((threadIdx.x & 31) == 0 && nz) atomicAdd(&s_zero[f], nz);
+    }
+  }
+}
+
 template <bool kStochastic>
 __global__ void __launch_bounds__(kSearchThreads)
 search_direct_kernel(const SearchParams p) {
@@ -64,7 +123,6 @@ search_direct_kernel(const SearchParams p) {
   const int f0 = blockIdx.y * p.fl_per_group;
   const int nf = min(p.fl_per_group, p.n_fl - f0);
   const bool do_q = (blockIdx.y == 0);
-  const int lane = threadIdx.x & 31;
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
@@ -82,6 +140,9 @@ search_direct_kernel(const SearchParams p) {
   }
   if (threadIdx.x < kMaxFl + 2) s_zlevel[threadIdx.x] = 0;
   __syncthreads();
+  // byte address of the float histogram's bin 0, less the constant bin_offset_magic carries
+  const unsigned hist_base = static_cast<unsigned>(__cvta_generic_to_shared(s_hist)) - 4u * 0x4B400000u;
+  const unsigned hist_stride = 4u * static_cast<unsigned>(B);
 
   int l = layer_of_tile(p.layers, p.n_layers, t);
   while (t < t_end) {
@@ -92,50 +153,25 @@ search_direct_kernel(const SearchParams p) {
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
     const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
-    const int bmax = __float2int_rz(S.bmax);
+    // largest float below the number of bins: floor of anything clamped to it is the last bin
+    const float top = __uint_as_float(__float_as_uint(__fadd_rn(S.bmax, 1.0f)) - 1u);
 
     for (; t < layer_tiles_end; ++t) {
       if (!layer_ok) continue;
       const long long j_tile = (t - L.tile_begin) * kTile;
       for (int q = 0; q < kTile / 4 / kSearchThreads; ++q) {
         const long long j0 = j_tile + 4ll * (q * kSearchThreads + threadIdx.x);
-        float v[4], pr[4];
+        float v[4];
         unsigned m = 0;
         if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
         else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const bool valid = (m >> k) & 1u;
-          pr[k] = 0.0f;
-          if (valid && do_q) atomicAdd(&s_hist[bin_index_fast(v[k], S.lo, S.scale, bmax)], 1u);
-          if (kStochastic) {
-            unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
-                                static_cast<unsigned long long>(j0 + k - jbeg));
-            pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
-          } else if (valid) {
-            atomicAdd(&s_zlevel[highest_zero_level(v[k]) + 1], 1u);
-          }
-        }
-        // a thread walks the fraction lengths with its four elements in registers
-        for (int f = 0; f < nf; ++f) {
-          const float two_f = s_two[f], inv_f = s_inv[f];
-          unsigned* H = s_hist + (f + 1) * B;
-          unsigned nz = 0;
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const float r = round_scaled<kStochastic>(v[k], two_f, pr[k]);
-            const int b = bin_index_fast(__fmul_rn(r, inv_f), S.lo, S.scale, bmax);
-            if ((m >> k) & 1u) {
-              atomicAdd(&H[b], 1u);
-              if (kStochastic) nz += (r == 0.0f) ? 1u : 0u;
-            }
-          }
-          if (kStochastic) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) nz += __shfl_xor_sync(0xffffffffu, nz, o);
-            if (lane == 0 && nz) atomicAdd(&s_zero[f], nz);
-          }
-        }
+        // a warp's quads are all inside the layer except at its two ends
+        if (__all_sync(0xffffffffu, m == 0xFu))
+          direct_quad<kStochastic, false>(v, m, j0 - jbeg, p, L.layer_id, S.lo, S.scale, top, nf,
+                                          do_q, hist_base, hist_stride, s_two, s_inv, s_zero, s_zlevel);
+        else
+          direct_quad<kStochastic, true>(v, m, j0 - jbeg, p, L.layer_id, S.lo, S.scale, top, nf,
+                                         do_q, hist_base, hist_stride, s_two, s_inv, s_zero, s_zlevel);
       }
     }
     __syncthreads();
