@@ -139,11 +139,19 @@ __global__ void format_resolve_kernel(const FormatParams p) {
 // exact zeros, class e + 150 the elements with floor(log2 |x|) = e (-149 <= e <= 127).
 constexpr int kExpClasses = 288;
 
-// Bin index by one convert-with-floor and two integer clamps; equal to bin_of for every input
-// (a NaN converts to 0, out-of-range values saturate and are clamped).
-__device__ __forceinline__ int bin_fast(float v, float lo, float scale, int bmax) {
-  const int b = __float2int_rd(__fmul_rn(__fsub_rn(v, lo), scale));
-  return min(max(b, 0), bmax);
+// The bin function without a float-to-int conversion: floor(clamp(u, 0, top)), top the largest
+// float below n_bins, equals clamp(floor(u), 0, n_bins - 1) for every u (a NaN clamps to 0 as
+// fmaxf returns its other operand), and adding 1.5 * 2^23 with round-down leaves that floor in
+// the low mantissa bits.  Returned: the byte offset 4 * bin + 4 * 0x4B400000 (mod 2^32), which
+// the caller adds to a histogram base that has the constant subtracted.
+__device__ __forceinline__ unsigned format_bin_offset(float v, float lo, float scale, float top) {
+  const float u = __fmul_rn(__fsub_rn(v, lo), scale);
+  const float c = fminf(fmaxf(u, 0.0f), top);
+  return __float_as_uint(__fadd_rd(c, 12582912.0f)) * 4u;
+}
+
+__device__ __forceinline__ void format_shared_inc(unsigned byte_addr) {
+  asm volatile("red.shared.add.u32 [%0], 1;" :: "r"(byte_addr) : "memory");
 }
 
 // Float rule with the scaling by 2^k as single multiplications when 2^k and 2^-k are normal.
@@ -153,6 +161,71 @@ __device__ __forceinline__ float float_value_fast(float x, int emin, int m_bits,
   const int k = m_bits - max(e, emin);
   if (k > 126) return float_value<kStochastic>(x, emin, m_bits, pr);   // only |x| < 2^(M-126)
   return __fmul_rn(round_to_grid<kStochastic>(__fmul_rn(x, pow2f(k)), pr), pow2f(-k));
+}
+
+// Four elements of one thread through every rule of the group.  kMasked: some of the four lie
+// outside the layer (mask m).
+template <bool kStochastic, bool kMasked>
+__device__ __forceinline__ void format_quad(const float (&v)[4], unsigned m, long long index0,
+                                            unsigned long long seed, int layer_id, float lo,
+                                            float scale, float top, int nr, unsigned hist_base,
+                                            unsigned hist_stride, const int* s_kind,
+                                            const int* s_i0, const int* s_i1, const float* s_f0,
+                                            const float* s_f1, unsigned* s_zero,
+                                            unsigned (*s_cls)[kExpClasses]) {
+  float pr[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    pr[k] = 0.0f;
+    if (kStochastic) {
+      const unsigned h = hash24(seed, static_cast<unsigned long long>(layer_id),
+                                static_cast<unsigned long long>(index0 + k));
+      pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
+    } else if (!kMasked || ((m >> k) & 1u)) {
+      // exponent class of the element (zero counts of all rules come from these)
+      const unsigned ax = __float_as_uint(v[k]) & 0x7fffffffu;
+      int cls = 0;
+      bool p2 = false;
+      if (ax) {
+        const unsigned eb = ax >> 23, mant = ax & 0x7fffffu;
+        cls = eb ? static_cast<int>(eb) + 23 : 32 - __clz(mant);   // e + 150
+        p2 = eb ? (mant == 0u) : ((mant & (mant - 1u)) == 0u);
+      }
+      atomicAdd(&s_cls[0][cls], 1u);
+      if (p2) atomicAdd(&s_cls[1][cls], 1u);
+    }
+  }
+  unsigned hb = hist_base;
+  for (int r = 0; r < nr; ++r, hb += hist_stride) {
+    const int kind = s_kind[r];
+    if (kind == kRuleIdentity) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (!kMasked || ((m >> k) & 1u)) format_shared_inc(hb + format_bin_offset(v[k], lo, scale, top));
+      continue;
+    }
+    float xq[4];
+    if (kind == kFmtFloat) {
+      const int emin = s_i0[r], mb = s_i1[r];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) xq[k] = float_value_fast<kStochastic>(v[k], emin, mb, pr[k]);
+    } else {
+      const float two_l = s_f0[r], inv_l = s_f1[r];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) xq[k] = level_value<kStochastic>(v[k], two_l, inv_l, pr[k]);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      if (!kMasked || ((m >> k) & 1u)) format_shared_inc(hb + format_bin_offset(xq[k], lo, scale, top));
+    if (kStochastic) {
+      // zero count by a warp reduction (the stochastic threshold is per element)
+      unsigned nz = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) nz += ((!kMasked || ((m >> k) & 1u)) && xq[k] == 0.0f) ? 1u : 0u;
+      nz = __reduce_add_sync(0xffffffffu, nz);
+      if ((threadIdx.x & 31) == 0 && nz) atomicAdd(&s_zero[r], nz);
+    }
+  }
 }
 
 // Builds the unclamped histogram and the zero count of every rule, every layer.  The rules are
@@ -170,7 +243,6 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
   const int B = p.n_bins;
   const int r0 = blockIdx.y * p.rules_per_group;
   const int nr = min(p.rules_per_group, p.n_rules - r0);
-  const int lane = threadIdx.x & 31;
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
@@ -180,6 +252,9 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
   for (int i = threadIdx.x; i < nr * B; i += blockDim.x) s_fhist[i] = 0;
   if (threadIdx.x < kMaxRulesPerGroup) s_zero[threadIdx.x] = 0;
   if (threadIdx.x < 2 * kExpClasses) (&s_cls[0][0])[threadIdx.x] = 0;
+  // byte address of the first rule's bin 0, less the constant format_bin_offset carries
+  const unsigned hist_base = static_cast<unsigned>(__cvta_generic_to_shared(s_fhist)) - 4u * 0x4B400000u;
+  const unsigned hist_stride = 4u * static_cast<unsigned>(B);
 
   int l = layer_of_tile(p.layers, p.n_layers, t);
   while (t < t_end) {
@@ -190,7 +265,8 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
     const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
-    const int bmax = __float2int_rz(S.bmax);
+    // largest float below the number of bins: floor of anything clamped to it is the last bin
+    const float top = __uint_as_float(__float_as_uint(__fadd_rn(S.bmax, 1.0f)) - 1u);
 
     // this layer's form of the group's rules; s_i0 of a grid rule = its level
     if (threadIdx.x < nr) {
@@ -213,63 +289,19 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
       const long long j_tile = (t - L.tile_begin) * kTile;
       for (int q = 0; q < kTile / 4 / kFormatThreads; ++q) {
         const long long j0 = j_tile + 4ll * (q * kFormatThreads + threadIdx.x);
-        float v[4], pr[4];
+        float v[4];
         unsigned m = 0;
         if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
         else { v[0] = v[1] = v[2] = v[3] = 0.0f; }
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          pr[k] = 0.0f;
-          if (kStochastic) {
-            const unsigned h = hash24(p.seed, static_cast<unsigned long long>(L.layer_id),
-                                      static_cast<unsigned long long>(j0 + k - jbeg));
-            pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
-          } else if ((m >> k) & 1u) {
-            // exponent class of the element (zero counts of all rules come from these)
-            const unsigned ax = __float_as_uint(v[k]) & 0x7fffffffu;
-            int cls = 0;
-            bool p2 = false;
-            if (ax) {
-              const unsigned eb = ax >> 23, mant = ax & 0x7fffffu;
-              cls = eb ? static_cast<int>(eb) + 23 : 32 - __clz(mant);   // e + 150
-              p2 = eb ? (mant == 0u) : ((mant & (mant - 1u)) == 0u);
-            }
-            atomicAdd(&s_cls[0][cls], 1u);
-            if (p2) atomicAdd(&s_cls[1][cls], 1u);
-          }
-        }
-        for (int r = 0; r < nr; ++r) {
-          const int kind = s_kind[r];
-          unsigned* H = s_fhist + r * B;
-          if (kind == kRuleIdentity) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              if ((m >> k) & 1u) atomicAdd(&H[bin_fast(v[k], S.lo, S.scale, bmax)], 1u);
-            continue;
-          }
-          float xq[4];
-          if (kind == kFmtFloat) {
-            const int emin = s_i0[r], mb = s_i1[r];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) xq[k] = float_value_fast<kStochastic>(v[k], emin, mb, pr[k]);
-          } else {
-            const float two_l = s_f0[r], inv_l = s_f1[r];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) xq[k] = level_value<kStochastic>(v[k], two_l, inv_l, pr[k]);
-          }
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            if ((m >> k) & 1u) atomicAdd(&H[bin_fast(xq[k], S.lo, S.scale, bmax)], 1u);
-          if (kStochastic) {
-            // zero count by vote (the stochastic threshold is per element)
-            unsigned nz = 0;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) nz += (((m >> k) & 1u) && xq[k] == 0.0f) ? 1u : 0u;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) nz += __shfl_xor_sync(0xffffffffu, nz, o);
-            if (lane == 0 && nz) atomicAdd(&s_zero[r], nz);
-          }
-        }
+        // a warp's quads are all inside the layer except at its two ends
+        if (__all_sync(0xffffffffu, m == 0xFu))
+          format_quad<kStochastic, false>(v, m, j0 - jbeg, p.seed, L.layer_id, S.lo, S.scale, top, nr,
+                                          hist_base, hist_stride, s_kind, s_i0, s_i1, s_f0, s_f1,
+                                          s_zero, s_cls);
+        else
+          format_quad<kStochastic, true>(v, m, j0 - jbeg, p.seed, L.layer_id, S.lo, S.scale, top, nr,
+                                         hist_base, hist_stride, s_kind, s_i0, s_i1, s_f0, s_f1,
+                                         s_zero, s_cls);
       }
     }
     __syncthreads();
