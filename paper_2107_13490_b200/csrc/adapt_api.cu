@@ -458,7 +458,13 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     sp.n_tiles = direct_tiles;
     sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed;
     const size_t per_hist = sizeof(unsigned) * bins_stride;
-    const size_t budget = 100 * 1024;
+    // When the histograms of all fraction lengths overflow half an SM's shared memory and there
+    // is work for every SM, one CTA of 1024 threads takes the whole of it: fewer FL groups (each
+    // group re-reads the tensors) and twice the resident warps of two 256-thread CTAs.
+    const bool wide = per_hist * (plan.n_levels + 1) > 100 * 1024 && direct_tiles >= 2ll * dc.sm_count &&
+                      dc.max_smem_optin >= 200 * 1024 + 1024;
+    const int threads = wide ? kSearchThreadsWide : kSearchThreads;
+    const size_t budget = (wide ? 200 : 100) * 1024;
     int fg = static_cast<int>(budget / per_hist) - 1;
     fg = std::max(1, std::min(fg, plan.n_levels));
     // few tiles: spread the fraction lengths over more CTAs instead of looping over them in one
@@ -473,11 +479,11 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
                                                          : search_direct_kernel<false>;
     ADAPT_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(smem)));
-    const int ctas_per_sm = std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
+    const int ctas_per_sm = wide ? 1 : std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
     dim3 grid(static_cast<unsigned>(std::min<long long>(direct_tiles, 1ll * ctas_per_sm * dc.sm_count)),
               groups);
     LaunchScope ls(ADAPT_KERNEL_SEARCH_DIRECT, stream);
-    kern<<<grid, kSearchThreads, smem, stream>>>(sp);
+    kern<<<grid, threads, smem, stream>>>(sp);
     ADAPT_CUDA(cudaGetLastError());
   }
 

@@ -20,7 +20,8 @@
 
 namespace adapt {
 
-constexpr int kSearchThreads = 256;
+constexpr int kSearchThreads = 256;       // threads per CTA when several CTAs share an SM
+constexpr int kSearchThreadsWide = 1024;  // one CTA per SM owning all of its shared memory
 
 struct SearchParams {
   const LayerDesc* layers;
@@ -112,7 +113,7 @@ __device__ __forceinline__ void direct_quad(const float (&v)[4], unsigned m, lon
 }
 
 template <bool kStochastic>
-__global__ void __launch_bounds__(kSearchThreads)
+__global__ void __launch_bounds__(kSearchThreadsWide)
 search_direct_kernel(const SearchParams p) {
   extern __shared__ unsigned s_hist[];  // [(fl_per_group + 1)][n_bins]
   __shared__ float s_two[kMaxFl], s_inv[kMaxFl];
@@ -159,8 +160,8 @@ search_direct_kernel(const SearchParams p) {
     for (; t < layer_tiles_end; ++t) {
       if (!layer_ok) continue;
       const long long j_tile = (t - L.tile_begin) * kTile;
-      for (int q = 0; q < kTile / 4 / kSearchThreads; ++q) {
-        const long long j0 = j_tile + 4ll * (q * kSearchThreads + threadIdx.x);
+      for (int q = 0; q < kTile / 4 / static_cast<int>(blockDim.x); ++q) {
+        const long long j0 = j_tile + 4ll * (q * static_cast<int>(blockDim.x) + threadIdx.x);
         float v[4];
         unsigned m = 0;
         if (j0 < jend) m = load_quad(base, j0, jbeg, jend, v);
