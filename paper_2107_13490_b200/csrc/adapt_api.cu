@@ -219,7 +219,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->d_levels = std::min(p->d_levels, p->n_levels);
   if (n_bins <= kKeyedMaxBins) {
     p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (2 + p->d_levels)) / 4) - 64;
-    p->cell_cap = std::min(p->cell_cap, 1 << 16);
+    p->cell_cap = std::min(p->cell_cap, 1 << 16) & ~3;   // rows of the cell arrays stay 16-byte aligned
   } else {
     p->cell_cap = 0;
   }

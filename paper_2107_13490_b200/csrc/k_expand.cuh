@@ -61,27 +61,40 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
   unsigned long long zero = 0;
   // the cells are shared by the gridDim.z CTAs of this (level, layer), a contiguous slice each
-  const int per_slice = (P.total_cells + gridDim.z - 1) / gridDim.z;
+  const int per_slice = ((P.total_cells + gridDim.z - 1) / gridDim.z + 3) & ~3;
   const int i_end = min(P.total_cells, static_cast<int>(blockIdx.z + 1) * per_slice);
-  for (int i = blockIdx.z * per_slice + threadIdx.x; i < i_end; i += kExpandThreads) {
-    const unsigned m = count[i];
-    if (m == 0) continue;
-    const int s = (P.seg[1].cells > 0 && i >= P.seg[1].offset) ? 1 : 0;
-    const SegPlan& sp = P.seg[s];
-    const long long cc = sp.c0 + (i - sp.offset);
-    if (is_q || f >= sp.g) {
-      if (!(init[i] & kCellEdge)) {
-        const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
-        atomicAdd(&s_hist[bin_of(lf, S.lo, S.scale, S.bmax)], m);
+  // four cells per thread and trip, counts and marks fetched as 128-bit words (slices start on
+  // multiples of four cells; the rows are 16-byte aligned and a multiple of four cells long)
+  const uint4* count4 = reinterpret_cast<const uint4*>(count);
+  const uint4* init4 = reinterpret_cast<const uint4*>(init);
+#pragma unroll 2
+  for (int i0 = blockIdx.z * per_slice + 4 * threadIdx.x; i0 < i_end; i0 += 4 * kExpandThreads) {
+    const uint4 m4 = __ldg(count4 + (i0 >> 2));
+    const uint4 k4 = __ldg(init4 + (i0 >> 2));
+    const unsigned ms[4] = {m4.x, m4.y, m4.z, m4.w};
+    const unsigned ks[4] = {k4.x, k4.y, k4.z, k4.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int i = i0 + e;
+      const unsigned m = ms[e];
+      if (m == 0 || i >= i_end) continue;
+      const int s = (P.seg[1].cells > 0 && i >= P.seg[1].offset) ? 1 : 0;
+      const SegPlan& sp = P.seg[s];
+      const long long cc = sp.c0 + (i - sp.offset);
+      if (is_q || f >= sp.g) {
+        if (!(ks[e] & kCellEdge)) {
+          const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
+          atomicAdd(&s_hist[bin_of(lf, S.lo, S.scale, S.bmax)], m);
+        }
+      } else {
+        const int d = sp.g - f;                      // 1..32
+        const long long a = cc >> d;                 // floor(c / 2^d)
+        const long long rem = cc - (a << d);
+        const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
+        const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
+        atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+        if (r == 0) zero += m;
       }
-    } else {
-      const int d = sp.g - f;                      // 1..32
-      const long long a = cc >> d;                 // floor(c / 2^d)
-      const long long rem = cc - (a << d);
-      const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
-      const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
-      atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
-      if (r == 0) zero += m;
     }
   }
 #pragma unroll

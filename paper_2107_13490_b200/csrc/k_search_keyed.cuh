@@ -446,7 +446,13 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
       const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
-      for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) cells[i] = __ldg(init + i);
+      // 128-bit copies, several in flight per thread (the table and its rows are 16-byte aligned,
+      // the row has room for the last quad: the table size is a multiple of four)
+      const uint4* init4 = reinterpret_cast<const uint4*>(init);
+      uint4* cells4 = reinterpret_cast<uint4*>(cells);
+      const int n4 = (total_cells + 3) >> 2;
+#pragma unroll 4
+      for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = __ldg(init4 + i);
       for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
       const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
       for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
