@@ -37,7 +37,7 @@ TRAFFIC_CAPTURE = {"version": "adapt-b200 0.6", "bytes_per_element": 4.161}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="stress_1g")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

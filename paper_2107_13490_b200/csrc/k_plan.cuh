@@ -74,6 +74,7 @@ struct LayerPlan {
   unsigned grid_mask;  // low mantissa bits that are zero in every element on its segment's grid
   int masked;       // 1 if the counting kernel may take "those bits are zero" as its grid-point flag
   int dense;        // 1 if, besides, exact zeros are so rare that they may go through the handler
+  unsigned grid_mul;   // 2^(32 - bits of grid_mask): x's bit pattern times this is 0 exactly when those bits are
 };
 
 // A float x = M 2^(E-23) (M its 24-bit significand) lies on the grid of level G exactly when
@@ -208,6 +209,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     }
     P.grid_mask = zero_bits >= 1 ? (1u << zero_bits) - 1u : 0u;
     P.masked = (P.fast && zero_bits >= kMinGridMaskBits) ? 1 : 0;
+    P.grid_mul = zero_bits >= 1 ? 1u << (32 - zero_bits) : 0u;
     // zeros handled one by one cost about as much as edge elements: fine below one in 2048
     P.dense = (kDenseZeroRatio > 0 && P.masked && S.lo <= 0.0f && S.hi >= 0.0f &&
                static_cast<long long>(S.zero_count) * kDenseZeroRatio <= L.n) ? 1 : 0;

@@ -103,6 +103,7 @@ struct LayerCtx {
   int keyed, fast, total_cells;
   unsigned grid_mask;
   int masked, dense;
+  unsigned grid_mul;
   int zero_pos;                // table position of the main segment's cell [0, 2^-G)
 };
 
@@ -181,6 +182,7 @@ struct CellFn {
   float two_g0, magic0, c0f0;   // main segment
   float two_g1, magic1;         // auxiliary segment (fast layers only)
   unsigned grid_mask;           // masked form: low significand bits every grid point has zero
+  unsigned grid_mul;            // dense form: 2^(32 - those bits)
   unsigned cell_base;           // dense form: shared-memory byte address of position 0, minus 4 * 0x4B400000
 };
 
@@ -235,12 +237,11 @@ template <int kMode>
 __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, const CellFn& fn,
                                             const float (&v)[4], unsigned (&old)[4]) {
   if (kMode == kCellDense) {
-    // dense form: no zero test.  The grid-point flag rides on the returned words: the low
-    // significand bits that every grid point of the layer has zero, minus one, are all ones
-    // exactly when those bits are zero (a zero included, which lands in the marked cell
-    // [0, 2^-G) and is queued anyway) and a small number otherwise, so OR-ing them in leaves
-    // the test "some word >= 2^29" to answer for marks and grid points at once.
-    unsigned any = 0;
+    // dense form: no zero test and no flag arithmetic.  The grid-point test is kept apart
+    // from the returned words: x's bit pattern times grid_mul is 0 exactly when the low
+    // significand bits that every grid point has zero are zero (a zero included, which lands
+    // in the marked cell [0, 2^-G) and is queued anyway).
+    unsigned any = 0, tmin = 0xFFFFFFFFu;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const float x = v[k];
@@ -249,11 +250,11 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
       const unsigned addr = __float_as_uint(rd) * 4u + fn.cell_base;
       unsigned o;
       asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(o) : "r"(addr) : "memory");
-      o |= (__float_as_uint(x) & fn.grid_mask) - 1u;
       old[k] = o;
       any |= o;
+      tmin = min(tmin, __float_as_uint(x) * fn.grid_mul);
     }
-    return any >= kCellOnGrid;
+    return any >= kCellOnGrid || tmin == 0u;
   }
   // exact zeros go to a dummy slot.  An element on the cell grid gets bit 29 added to its
   // word and is queued too: its handler may move it one cell to the left.  (Slots that are
@@ -283,7 +284,8 @@ __device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, uns
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const bool push = old[k] >= kCellOnGrid;
+      bool push = old[k] >= kCellOnGrid;
+      if (kMode == kCellDense) push = push || __float_as_uint(v[k]) * fn.grid_mul == 0u;
       const unsigned pm = __ballot_sync(0xffffffffu, push);
       if (pm) {
         if (push) queue[qn + __popc(pm & lt)] = v[k];
@@ -348,6 +350,7 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
   fn.two_g0 = c.two_g[0]; fn.magic0 = c.magic[0]; fn.c0f0 = c.c0f[0];
   fn.two_g1 = c.two_g[1]; fn.magic1 = c.magic[1];
   fn.grid_mask = c.grid_mask;
+  fn.grid_mul = c.grid_mul;
   fn.cell_base = static_cast<unsigned>(__cvta_generic_to_shared(cells)) - 4u * 0x4B400000u;
   unsigned qn = 0;             // entries in this warp's queue (same in every lane)
   // a ragged tile pads with zeros, which the dense form must not see
@@ -423,6 +426,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.magic[0] = P->seg[0].magic; c.magic[1] = P->seg[1].magic;
       c.keyed = P->keyed; c.fast = P->fast; c.total_cells = P->total_cells;
       c.grid_mask = P->grid_mask; c.masked = P->masked; c.dense = P->dense;
+      c.grid_mul = P->grid_mul;
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
       c.E = edges;
       c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
