@@ -162,6 +162,21 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                                   uint64_t seed, int32_t layer_base,
                                   int32_t* const* codes_out, void* stream);
 
+/* The same loop with the dequantized values as output: values_out[l][i] =
+ * code * 2^-FL as fp32, code as adapt_quantize_selected_batch would write it.
+ * This is the layer as a float32 simulation of fixed-point training continues
+ * with it (Sec. 4.1: the quantized network is simulated in float32; Algorithm 1,
+ * Quantize of every layer after the precision switch).
+ *   values_out HOST array of n_layers DEVICE pointers, fp32[lens[l]] each;
+ *              values_out[l] may be tensors[l] itself (in place), but must not
+ *              overlap it otherwise
+ * Other arguments, the untouched layers and the library-owned layer table as
+ * for adapt_quantize_selected_batch. */
+int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* lens,
+                                    int n_layers, const int32_t* best, int round_mode,
+                                    uint64_t seed, int32_t layer_base,
+                                    float* const* values_out, void* stream);
+
 /* Gradient diversity of each layer over its last n_grads gradient tensors -
  * the quantity PushUp reads (Sec. 3.3, the gradient-diversity equation and its
  * log form):  delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2, and

@@ -25,6 +25,7 @@ OK, ERR_INVALID_ARG, ERR_NONFINITE, ERR_RANGE, ERR_CUDA, ERR_WORKSPACE = range(6
 EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
+    "adapt_requantize_selected_batch",
     "adapt_search_workspace_bytes", "adapt_gradient_diversity",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_precision_switch_host",
@@ -95,6 +96,8 @@ def lib():
         L.adapt_quantize_selected_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                                     C.c_int, C.c_uint64, C.c_int32, C.c_void_p,
                                                     C.c_void_p]
+        L.adapt_requantize_selected_batch.restype = C.c_int
+        L.adapt_requantize_selected_batch.argtypes = L.adapt_quantize_selected_batch.argtypes
         L.adapt_gradient_diversity.restype = C.c_int
         L.adapt_gradient_diversity.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                C.c_void_p]
@@ -242,6 +245,25 @@ def adapt_quantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.T
                                                outs.ctypes.data, _stream_handle(stream)),
            "adapt_quantize_selected_batch")
     return codes_out
+
+
+def adapt_requantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.Tensor,
+                                    round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
+                                    values_out: Optional[Sequence[torch.Tensor]] = None, stream=None):
+    """All layers replaced by their dequantized values code * 2^-FL (fp32) at the <WL,FL> a search
+    left in ``best``; ``values_out`` defaults to new tensors and may be ``tensors`` (in place)."""
+    assert best.is_cuda and best.dtype == torch.int32 and best.numel() >= 4 * len(tensors)
+    if values_out is None:
+        values_out = [torch.empty(t.numel(), dtype=torch.float32, device=t.device) for t in tensors]
+    ptrs, lens = _marshal_tensors(tensors)
+    outs = np.array([c.data_ptr() for c in values_out], dtype=np.uint64)
+    assert all(c.dtype == torch.float32 and c.is_cuda and c.is_contiguous() and c.numel() == t.numel()
+               for c, t in zip(values_out, tensors))
+    _check(lib().adapt_requantize_selected_batch(ptrs.ctypes.data, lens.ctypes.data, len(tensors),
+                                                 best.data_ptr(), round_mode, seed, layer_base,
+                                                 outs.ctypes.data, _stream_handle(stream)),
+           "adapt_requantize_selected_batch")
+    return values_out
 
 
 def adapt_gradient_diversity(grads: Sequence[Sequence[torch.Tensor]],

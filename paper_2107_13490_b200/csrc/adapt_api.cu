@@ -634,7 +634,7 @@ namespace {
 // Body of adapt_quantize_selected_batch.  Caller holds g_mutex.
 int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_layers,
                        const int32_t* best, int round_mode, uint64_t seed, int32_t layer_base,
-                       int32_t* const* codes_out, void* stream_handle) {
+                       void* const* codes_out, bool dequant, void* stream_handle) {
   if (!tensors || !lens || !best || !codes_out) return ADAPT_ERR_INVALID_ARG;
   if (n_layers < 1 || n_layers > 65535) return ADAPT_ERR_INVALID_ARG;
   if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
@@ -670,10 +670,10 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
   const int grid = static_cast<int>(std::min<long long>(tiles, 32ll * dc->sm_count));
   const QuantLayer* d = static_cast<const QuantLayer*>(dc->batch_tab);
   LaunchScope ls(ADAPT_KERNEL_QUANTIZE, stream);
-  if (round_mode == ADAPT_ROUND_STOCHASTIC)
-    quantize_batch_kernel<true><<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
-  else
-    quantize_batch_kernel<false><<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
+  const bool sr = round_mode == ADAPT_ROUND_STOCHASTIC;
+  auto kern = dequant ? (sr ? quantize_batch_kernel<true, true> : quantize_batch_kernel<false, true>)
+                      : (sr ? quantize_batch_kernel<true, false> : quantize_batch_kernel<false, false>);
+  kern<<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
   ADAPT_CUDA(cudaGetLastError());
   return ADAPT_OK;
 }
@@ -685,8 +685,16 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                                   const int32_t* best, int round_mode, uint64_t seed,
                                   int32_t layer_base, int32_t* const* codes_out, void* stream_handle) {
   std::lock_guard<std::mutex> lock(g_mutex);
-  return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base, codes_out,
-                            stream_handle);
+  return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base,
+                            reinterpret_cast<void* const*>(codes_out), false, stream_handle);
+}
+
+int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* lens, int n_layers,
+                                    const int32_t* best, int round_mode, uint64_t seed,
+                                    int32_t layer_base, float* const* values_out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base,
+                            reinterpret_cast<void* const*>(values_out), true, stream_handle);
 }
 
 int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
@@ -837,7 +845,8 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
       dcodes[l] = reinterpret_cast<int32_t*>(static_cast<char*>(dc->stage_codes) + off[l]);
     }
     rc = run_quantize_batch(dptr.data(), lens, n_layers, a.best_out, o.round_mode, o.seed,
-                            o.layer_base, dcodes.data(), o.stream);
+                            o.layer_base, reinterpret_cast<void* const*>(dcodes.data()), false,
+                            o.stream);
     if (rc != ADAPT_OK) return rc;
     for (int l = 0; l < n_layers; ++l)
       if (lens[l] > 0)

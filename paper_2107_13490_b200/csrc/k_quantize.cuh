@@ -75,7 +75,7 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const QuantPara
 // device for it, in one launch (Algorithm 1: for l in L: L^[l] = Quantize(L[l], Q[l].quant)).
 struct QuantLayer {
   const float* x;
-  int* out;
+  void* out;              // int32 codes, or fp32 dequantized values (kDequant)
   long long n;
   long long tile_begin;   // first tile of the layer in the launch's tile list (4096 elements each)
   int layer_id;           // hash layer id
@@ -84,7 +84,10 @@ struct QuantLayer {
 
 constexpr int kQuantTile = 4096;
 
-template <bool kStochastic>
+// kDequant: instead of the codes the kernel writes the dequantized values code * 2^-FL as
+// fp32 - the tensor a float32 simulation of fixed-point training goes on with (Sec. 4.1); out
+// may be x itself (every element is read and written by the same thread).
+template <bool kStochastic, bool kDequant>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long long n_tiles,
                       const int* __restrict__ best, unsigned long long seed) {
@@ -102,7 +105,6 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
     const long long i1 = min(L.n, i0 + kQuantTile);
     if (L.vec && i1 - i0 == kQuantTile) {
       const float4* x4 = reinterpret_cast<const float4*>(L.x + i0);
-      int4* o4 = reinterpret_cast<int4*>(L.out + i0);
       for (int q = threadIdx.x; q < kQuantTile / 4; q += kQuantThreads) {
         const float4 v = __ldcs(x4 + q);
         const long long i = i0 + 4ll * q;
@@ -111,11 +113,20 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
         c.y = quantize_one<kStochastic>(v.y, two_fl, wl, seed, L.layer_id, i + 1);
         c.z = quantize_one<kStochastic>(v.z, two_fl, wl, seed, L.layer_id, i + 2);
         c.w = quantize_one<kStochastic>(v.w, two_fl, wl, seed, L.layer_id, i + 3);
-        __stcs(o4 + q, c);
+        if (kDequant) {
+          const float4 d = make_float4(dequantize(c.x, fl), dequantize(c.y, fl), dequantize(c.z, fl),
+                                       dequantize(c.w, fl));
+          __stcs(reinterpret_cast<float4*>(static_cast<float*>(L.out) + i0) + q, d);
+        } else {
+          __stcs(reinterpret_cast<int4*>(static_cast<int*>(L.out) + i0) + q, c);
+        }
       }
     } else {
-      for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads)
-        L.out[i] = quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i);
+      for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads) {
+        const int c = quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i);
+        if (kDequant) static_cast<float*>(L.out)[i] = dequantize(c, fl);
+        else static_cast<int*>(L.out)[i] = c;
+      }
     }
   }
 }

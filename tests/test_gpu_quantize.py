@@ -106,6 +106,16 @@ def test_batched_quantize_at_device_resident_selections(B):
             want, _ = O.quantize(xs[i], int(ora[j]["best"][0]), int(ora[j]["best"][1]), mode, 7, 2 + j)
             assert np.array_equal(codes[j].cpu().numpy(), want), (mode, i)
         assert codes[-1].numel() == 0
+        # the same loop with dequantized fp32 values as output, to new tensors and in place
+        vals = B.adapt_requantize_selected_batch(bufs, res.best, mode, seed=7, layer_base=2)
+        torch.cuda.synchronize()
+        for j, i in enumerate(pick):
+            _, xhat = O.quantize(xs[i], int(ora[j]["best"][0]), int(ora[j]["best"][1]), mode, 7, 2 + j)
+            assert np.array_equal(vals[j].cpu().numpy().view(np.uint32), xhat.view(np.uint32)), (mode, i)
+        B.adapt_requantize_selected_batch(bufs, res.best, mode, seed=7, layer_base=2, values_out=bufs)
+        torch.cuda.synchronize()
+        for j in range(len(pick)):
+            assert torch.equal(bufs[j], vals[j]), (mode, j)
 
 
 def test_quantize_argument_errors_and_host_form(B):
