@@ -162,6 +162,21 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                                   uint64_t seed, int32_t layer_base,
                                   int32_t* const* codes_out, void* stream);
 
+/* adapt_quantize_selected_batch with packed codes: codes_out[l] is DEVICE
+ * int8[lens[l]] (code_bits 8), int16[...] (16) or int32[...] (32), aligned to
+ * its element size.  The word length of a layer is only known on the device: a
+ * layer whose selected WL exceeds code_bits is left untouched and, when
+ * unfit_out is given (DEVICE int32[n_layers], cleared by the call), reported
+ * there as unfit_out[l] = WL; all other entries stay 0.  (Algorithm 1, the
+ * Quantize of every layer after the switch; the packed forms pay once the
+ * search has settled on short word lengths: 1 or 2 bytes written per element
+ * instead of 4.) */
+int adapt_quantize_selected_batch_packed(const float* const* tensors, const int64_t* lens,
+                                         int n_layers, const int32_t* best, int round_mode,
+                                         uint64_t seed, int32_t layer_base, int code_bits,
+                                         void* const* codes_out, int32_t* unfit_out,
+                                         void* stream);
+
 /* The same loop with the dequantized values as output: values_out[l][i] =
  * code * 2^-FL as fp32, code as adapt_quantize_selected_batch would write it.
  * This is the layer as a float32 simulation of fixed-point training continues

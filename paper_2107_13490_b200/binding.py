@@ -25,7 +25,7 @@ OK, ERR_INVALID_ARG, ERR_NONFINITE, ERR_RANGE, ERR_CUDA, ERR_WORKSPACE = range(6
 EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
-    "adapt_requantize_selected_batch",
+    "adapt_requantize_selected_batch", "adapt_quantize_selected_batch_packed",
     "adapt_search_workspace_bytes", "adapt_gradient_diversity",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_precision_switch_host",
@@ -96,6 +96,10 @@ def lib():
         L.adapt_quantize_selected_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                                     C.c_int, C.c_uint64, C.c_int32, C.c_void_p,
                                                     C.c_void_p]
+        L.adapt_quantize_selected_batch_packed.restype = C.c_int
+        L.adapt_quantize_selected_batch_packed.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                                           C.c_int, C.c_uint64, C.c_int32, C.c_int,
+                                                           C.c_void_p, C.c_void_p, C.c_void_p]
         L.adapt_requantize_selected_batch.restype = C.c_int
         L.adapt_requantize_selected_batch.argtypes = L.adapt_quantize_selected_batch.argtypes
         L.adapt_gradient_diversity.restype = C.c_int
@@ -245,6 +249,33 @@ def adapt_quantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.T
                                                outs.ctypes.data, _stream_handle(stream)),
            "adapt_quantize_selected_batch")
     return codes_out
+
+
+def adapt_quantize_selected_batch_packed(tensors: Sequence[torch.Tensor], best: torch.Tensor,
+                                         code_bits: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                                         layer_base: int = 0,
+                                         codes_out: Optional[Sequence[torch.Tensor]] = None,
+                                         unfit_out: Optional[torch.Tensor] = None, stream=None):
+    """adapt_quantize_selected_batch with int8 / int16 / int32 codes.  Returns (codes, unfit):
+    unfit is device int32[L], the word length of every layer that did not fit ``code_bits``
+    (such a layer's codes are left untouched), 0 elsewhere."""
+    dt = {8: torch.int8, 16: torch.int16, 32: torch.int32}[code_bits]
+    assert best.is_cuda and best.dtype == torch.int32 and best.numel() >= 4 * len(tensors)
+    if codes_out is None:
+        codes_out = [torch.empty(t.numel(), dtype=dt, device=t.device) for t in tensors]
+    if unfit_out is None:
+        unfit_out = torch.empty(len(tensors), dtype=torch.int32, device=best.device)
+    assert unfit_out.is_cuda and unfit_out.dtype == torch.int32 and unfit_out.numel() >= len(tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    outs = np.array([c.data_ptr() for c in codes_out], dtype=np.uint64)
+    assert all(c.dtype == dt and c.is_cuda and c.is_contiguous() and c.numel() == t.numel()
+               for c, t in zip(codes_out, tensors))
+    _check(lib().adapt_quantize_selected_batch_packed(ptrs.ctypes.data, lens.ctypes.data, len(tensors),
+                                                      best.data_ptr(), round_mode, seed, layer_base,
+                                                      code_bits, outs.ctypes.data, unfit_out.data_ptr(),
+                                                      _stream_handle(stream)),
+           "adapt_quantize_selected_batch_packed")
+    return codes_out, unfit_out
 
 
 def adapt_requantize_selected_batch(tensors: Sequence[torch.Tensor], best: torch.Tensor,

@@ -632,17 +632,21 @@ int adapt_quantize_selected(const float* x, int64_t n, const int32_t* selected, 
 
 namespace {
 // Body of adapt_quantize_selected_batch.  Caller holds g_mutex.
+// out_bits: 8, 16 or 32 for integer codes of that width, 0 for dequantized fp32 values.
 int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_layers,
                        const int32_t* best, int round_mode, uint64_t seed, int32_t layer_base,
-                       void* const* codes_out, bool dequant, void* stream_handle) {
+                       void* const* codes_out, int out_bits, int32_t* unfit, void* stream_handle) {
   if (!tensors || !lens || !best || !codes_out) return ADAPT_ERR_INVALID_ARG;
   if (n_layers < 1 || n_layers > 65535) return ADAPT_ERR_INVALID_ARG;
   if (round_mode != ADAPT_ROUND_RNE && round_mode != ADAPT_ROUND_STOCHASTIC)
     return ADAPT_ERR_INVALID_ARG;
+  if (out_bits != 0 && out_bits != 8 && out_bits != 16 && out_bits != 32) return ADAPT_ERR_INVALID_ARG;
+  const uintptr_t elem = out_bits == 0 ? 4u : static_cast<uintptr_t>(out_bits / 8);
   for (int l = 0; l < n_layers; ++l) {
     if (lens[l] < 0) return ADAPT_ERR_INVALID_ARG;
     if (lens[l] > 0 && (!tensors[l] || !codes_out[l])) return ADAPT_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(tensors[l]) & 3u) || (reinterpret_cast<uintptr_t>(codes_out[l]) & 3u))
+    if ((reinterpret_cast<uintptr_t>(tensors[l]) & 3u) ||
+        (reinterpret_cast<uintptr_t>(codes_out[l]) & (elem - 1u)))
       return ADAPT_ERR_INVALID_ARG;
   }
   DeviceCache* dc = nullptr;
@@ -660,20 +664,26 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
     h[l].x = tensors[l]; h[l].out = codes_out[l]; h[l].n = lens[l]; h[l].tile_begin = tiles;
     h[l].layer_id = layer_base + l;
     h[l].vec = !(reinterpret_cast<uintptr_t>(tensors[l]) & 15u) &&
-               !(reinterpret_cast<uintptr_t>(codes_out[l]) & 15u);
+               !(reinterpret_cast<uintptr_t>(codes_out[l]) & (4u * elem - 1u));
     tiles += (lens[l] + kQuantTile - 1) / kQuantTile;
   }
-  if (tiles == 0) return ADAPT_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+  if (unfit) ADAPT_CUDA(cudaMemsetAsync(unfit, 0, sizeof(int32_t) * static_cast<size_t>(n_layers), stream));
+  if (tiles == 0) return ADAPT_OK;
   ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, h, bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
   const int grid = static_cast<int>(std::min<long long>(tiles, 32ll * dc->sm_count));
   const QuantLayer* d = static_cast<const QuantLayer*>(dc->batch_tab);
   LaunchScope ls(ADAPT_KERNEL_QUANTIZE, stream);
   const bool sr = round_mode == ADAPT_ROUND_STOCHASTIC;
-  auto kern = dequant ? (sr ? quantize_batch_kernel<true, true> : quantize_batch_kernel<false, true>)
-                      : (sr ? quantize_batch_kernel<true, false> : quantize_batch_kernel<false, false>);
-  kern<<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed);
+  void (*kern)(const QuantLayer*, int, long long, const int*, unsigned long long, int*) = nullptr;
+  switch (out_bits) {
+    case 0:  kern = sr ? quantize_batch_kernel<true, float>   : quantize_batch_kernel<false, float>;   break;
+    case 8:  kern = sr ? quantize_batch_kernel<true, int8_t>  : quantize_batch_kernel<false, int8_t>;  break;
+    case 16: kern = sr ? quantize_batch_kernel<true, int16_t> : quantize_batch_kernel<false, int16_t>; break;
+    default: kern = sr ? quantize_batch_kernel<true, int32_t> : quantize_batch_kernel<false, int32_t>; break;
+  }
+  kern<<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed, unfit);
   ADAPT_CUDA(cudaGetLastError());
   return ADAPT_OK;
 }
@@ -686,7 +696,18 @@ int adapt_quantize_selected_batch(const float* const* tensors, const int64_t* le
                                   int32_t layer_base, int32_t* const* codes_out, void* stream_handle) {
   std::lock_guard<std::mutex> lock(g_mutex);
   return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base,
-                            reinterpret_cast<void* const*>(codes_out), false, stream_handle);
+                            reinterpret_cast<void* const*>(codes_out), 32, nullptr, stream_handle);
+}
+
+int adapt_quantize_selected_batch_packed(const float* const* tensors, const int64_t* lens,
+                                         int n_layers, const int32_t* best, int round_mode,
+                                         uint64_t seed, int32_t layer_base, int code_bits,
+                                         void* const* codes_out, int32_t* unfit_out,
+                                         void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (code_bits != 8 && code_bits != 16 && code_bits != 32) return ADAPT_ERR_INVALID_ARG;
+  return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base, codes_out,
+                            code_bits, unfit_out, stream_handle);
 }
 
 int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* lens, int n_layers,
@@ -694,7 +715,7 @@ int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* 
                                     int32_t layer_base, float* const* values_out, void* stream_handle) {
   std::lock_guard<std::mutex> lock(g_mutex);
   return run_quantize_batch(tensors, lens, n_layers, best, round_mode, seed, layer_base,
-                            reinterpret_cast<void* const*>(values_out), true, stream_handle);
+                            reinterpret_cast<void* const*>(values_out), 0, nullptr, stream_handle);
 }
 
 int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
@@ -845,7 +866,7 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
       dcodes[l] = reinterpret_cast<int32_t*>(static_cast<char*>(dc->stage_codes) + off[l]);
     }
     rc = run_quantize_batch(dptr.data(), lens, n_layers, a.best_out, o.round_mode, o.seed,
-                            o.layer_base, reinterpret_cast<void* const*>(dcodes.data()), false,
+                            o.layer_base, reinterpret_cast<void* const*>(dcodes.data()), 32, nullptr,
                             o.stream);
     if (rc != ADAPT_OK) return rc;
     for (int l = 0; l < n_layers; ++l)

@@ -75,22 +75,33 @@ __global__ void __launch_bounds__(kQuantThreads) quantize_kernel(const QuantPara
 // device for it, in one launch (Algorithm 1: for l in L: L^[l] = Quantize(L[l], Q[l].quant)).
 struct QuantLayer {
   const float* x;
-  void* out;              // int32 codes, or fp32 dequantized values (kDequant)
+  void* out;              // int8 / int16 / int32 codes, or fp32 dequantized values
   long long n;
   long long tile_begin;   // first tile of the layer in the launch's tile list (4096 elements each)
   int layer_id;           // hash layer id
-  int vec;                // x is 16-byte aligned and out 16-byte aligned: 128-bit accesses
+  int vec;                // x is 16-byte aligned and out aligned for a 4-element store
 };
 
 constexpr int kQuantTile = 4096;
 
-// kDequant: instead of the codes the kernel writes the dequantized values code * 2^-FL as
-// fp32 - the tensor a float32 simulation of fixed-point training goes on with (Sec. 4.1); out
-// may be x itself (every element is read and written by the same thread).
-template <bool kStochastic, bool kDequant>
+// Output of the batched kernel: int32 / int16 / int8 codes, or (float) the dequantized values
+// code * 2^-FL as fp32 - the tensor a float32 simulation of fixed-point training goes on with
+// (Sec. 4.1); the float output may be x itself (every element is read and written by the same
+// thread).  A layer whose selected word length does not fit the code type is left untouched
+// and, if `unfit` is given, reported there (unfit[layer] = its word length).
+template <typename T> struct Pack4;
+template <> struct Pack4<float> { using type = float4; };
+
+template <typename T>
+__device__ __forceinline__ T quant_out(int code, int fl) { return static_cast<T>(code); }
+template <>
+__device__ __forceinline__ float quant_out<float>(int code, int fl) { return dequantize(code, fl); }
+
+template <bool kStochastic, typename T>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long long n_tiles,
-                      const int* __restrict__ best, unsigned long long seed) {
+                      const int* __restrict__ best, unsigned long long seed, int* __restrict__ unfit) {
+  constexpr int kBits = sizeof(T) == 1 ? 8 : (sizeof(T) == 2 ? 16 : 32);   // float carries any code
   for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
     int lo = 0, hi = n_layers - 1;                 // layer that owns tile t
     while (lo < hi) {
@@ -100,33 +111,31 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
     const QuantLayer L = layers[lo];
     const int wl = best[4 * lo], fl = best[4 * lo + 1];
     if (wl < 2 || wl > 32 || fl < 0 || fl >= wl) continue;   // layer without a valid selection
+    if (wl > kBits) {
+      if (unfit && t == L.tile_begin && threadIdx.x == 0) unfit[lo] = wl;
+      continue;
+    }
     const float two_fl = pow2f(fl);
     const long long i0 = (t - L.tile_begin) * kQuantTile;
     const long long i1 = min(L.n, i0 + kQuantTile);
+    T* out = static_cast<T*>(L.out);
     if (L.vec && i1 - i0 == kQuantTile) {
+      using P4 = typename Pack4<T>::type;
       const float4* x4 = reinterpret_cast<const float4*>(L.x + i0);
+      P4* o4 = reinterpret_cast<P4*>(out + i0);
       for (int q = threadIdx.x; q < kQuantTile / 4; q += kQuantThreads) {
         const float4 v = __ldcs(x4 + q);
         const long long i = i0 + 4ll * q;
-        int4 c;
-        c.x = quantize_one<kStochastic>(v.x, two_fl, wl, seed, L.layer_id, i + 0);
-        c.y = quantize_one<kStochastic>(v.y, two_fl, wl, seed, L.layer_id, i + 1);
-        c.z = quantize_one<kStochastic>(v.z, two_fl, wl, seed, L.layer_id, i + 2);
-        c.w = quantize_one<kStochastic>(v.w, two_fl, wl, seed, L.layer_id, i + 3);
-        if (kDequant) {
-          const float4 d = make_float4(dequantize(c.x, fl), dequantize(c.y, fl), dequantize(c.z, fl),
-                                       dequantize(c.w, fl));
-          __stcs(reinterpret_cast<float4*>(static_cast<float*>(L.out) + i0) + q, d);
-        } else {
-          __stcs(reinterpret_cast<int4*>(static_cast<int*>(L.out) + i0) + q, c);
-        }
+        P4 c;
+        c.x = quant_out<T>(quantize_one<kStochastic>(v.x, two_fl, wl, seed, L.layer_id, i + 0), fl);
+        c.y = quant_out<T>(quantize_one<kStochastic>(v.y, two_fl, wl, seed, L.layer_id, i + 1), fl);
+        c.z = quant_out<T>(quantize_one<kStochastic>(v.z, two_fl, wl, seed, L.layer_id, i + 2), fl);
+        c.w = quant_out<T>(quantize_one<kStochastic>(v.w, two_fl, wl, seed, L.layer_id, i + 3), fl);
+        __stcs(o4 + q, c);
       }
     } else {
-      for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads) {
-        const int c = quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i);
-        if (kDequant) static_cast<float*>(L.out)[i] = dequantize(c, fl);
-        else static_cast<int*>(L.out)[i] = c;
-      }
+      for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads)
+        out[i] = quant_out<T>(quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i), fl);
     }
   }
 }

@@ -106,6 +106,23 @@ def test_batched_quantize_at_device_resident_selections(B):
             want, _ = O.quantize(xs[i], int(ora[j]["best"][0]), int(ora[j]["best"][1]), mode, 7, 2 + j)
             assert np.array_equal(codes[j].cpu().numpy(), want), (mode, i)
         assert codes[-1].numel() == 0
+        # packed codes: a layer whose selected word length exceeds the code width is reported
+        # and left untouched, the others hold the oracle's codes
+        sel = [int(ora[j]["best"][0]) for j in range(len(pick))]
+        for bits, dt in ((8, np.int8), (16, np.int16), (32, np.int32)):
+            outs = [torch.full((b.numel() + 3,), 77, dtype={8: torch.int8, 16: torch.int16, 32: torch.int32}[bits],
+                               device="cuda")[(j % 3):(j % 3) + b.numel()] for j, b in enumerate(bufs)]
+            packed, unfit = B.adapt_quantize_selected_batch_packed(bufs, res.best, bits, mode, seed=7,
+                                                                   layer_base=2, codes_out=outs)
+            torch.cuda.synchronize()
+            unfit = unfit.cpu().numpy()
+            for j, i in enumerate(pick):
+                if sel[j] > bits:
+                    assert unfit[j] == sel[j] and (packed[j] == 77).all(), (mode, bits, i)
+                else:
+                    want, _ = O.quantize(xs[i], sel[j], int(ora[j]["best"][1]), mode, 7, 2 + j)
+                    assert unfit[j] == 0 and np.array_equal(packed[j].cpu().numpy(), want.astype(dt)), (mode, bits, i)
+            assert unfit[-1] == 0
         # the same loop with dequantized fp32 values as output, to new tensors and in place
         vals = B.adapt_requantize_selected_batch(bufs, res.best, mode, seed=7, layer_base=2)
         torch.cuda.synchronize()
