@@ -10,6 +10,8 @@
 //                 Quantization"; Sec. 3.2 "Precision Levels", the SR(x) rule)
 //   range/bins  - discretisation "via binning" at resolution r (Sec. 3.3,
 //                 the EDF equation), read as r equal-width bins on [min,max]
+//   normalize   - gradient normalisation g / ||g||_2 (Sec. 3.3, the paragraph on the
+//                 limited range of fixed point)
 //   kld         - discrete Kullback-Leibler divergence KL(P||Q), P the
 //                 quantized tensor, Q the float tensor (Sec. 3.3, Eq. dkld)
 //   select      - "smallest quantization s.t. KL = 0" (Sec. 3.3; Algorithm 3)
@@ -302,6 +304,18 @@ int adapt_oracle_precision_search(const float* x, int64_t n, uint64_t layer,
 // grads[k] points to n fp32 values; everything is accumulated in double, in index order.
 // out = {sum of norms, norm of the sum, delta_s, log form}.  0/0 gives NaN for delta_s
 // (log form 1); x/0 gives +inf (log form 1).
+// Gradient normalisation of Sec. 3.3 ("Dealing with Fixed-Points Limited Range"):
+// g <- g / ||g||_2.  The norm is the square root of the sum of squares taken in double,
+// elements in order; each quotient is formed in double and rounded to float.  A gradient
+// whose norm is 0 (all zeros) is returned unchanged (the paper does not say; 0/0 has no value).
+void adapt_oracle_normalize_gradient(const float* g, int64_t n, float* out) {
+  double sq = 0.0;
+  for (int64_t i = 0; i < n; ++i) sq += static_cast<double>(g[i]) * g[i];
+  const double norm = std::sqrt(sq);
+  for (int64_t i = 0; i < n; ++i)
+    out[i] = norm > 0.0 ? static_cast<float>(static_cast<double>(g[i]) / norm) : g[i];
+}
+
 void adapt_oracle_gradient_diversity(const float* const* grads, int n_grads, int64_t n,
                                      double* out) {
   double sum_norms = 0.0;

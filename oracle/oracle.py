@@ -81,6 +81,8 @@ def lib():
                                                       C.c_double, C.c_int, C.c_int, C.c_void_p]
             L.adapt_oracle_gradient_diversity.restype = None
             L.adapt_oracle_gradient_diversity.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
+            L.adapt_oracle_normalize_gradient.restype = None
+            L.adapt_oracle_normalize_gradient.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
             L.adapt_oracle_bfp_scale.restype = C.c_int
             L.adapt_oracle_bfp_scale.argtypes = [C.c_float, C.c_float, C.c_int]
             L.adapt_oracle_format_value_one.restype = C.c_float
@@ -262,6 +264,14 @@ def gradient_diversity(grads):
     ptrs = (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
     out = np.zeros(4, dtype=np.float64)
     lib().adapt_oracle_gradient_diversity(ptrs, len(arrs), n, out.ctypes.data)
+    return out
+
+
+def normalize_gradient(g):
+    """g / ||g||_2 as fp32 (norm and quotients in double); an all-zero gradient comes back as is."""
+    a = _as_f32(g)
+    out = np.empty_like(a)
+    lib().adapt_oracle_normalize_gradient(a.ctypes.data, a.size, out.ctypes.data)
     return out
 
 

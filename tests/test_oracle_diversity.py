@@ -66,3 +66,29 @@ def test_matches_numpy_norms():
     assert out[1] == pytest.approx(norm_sum, rel=1e-12)
     assert out[2] == pytest.approx(sum_norms / norm_sum, rel=1e-12)
     assert out[3] == pytest.approx(math.log(sum_norms / norm_sum), rel=1e-11)
+
+
+def test_normalized_gradient_pins():
+    """g / ||g||_2 (Sec. 3.3): hand-worked 3-4-5 triangle, unit norm, exact invariance under a
+    power-of-two scale and a sign flip, exact rational quotients, the all-zero gradient."""
+    from fractions import Fraction
+    out = O.normalize_gradient(np.float32([3.0, 4.0]))
+    assert out[0] == np.float32(0.6) and out[1] == np.float32(0.8)
+    out = O.normalize_gradient(np.float32([0.0, -2.0, 0.0]))
+    assert list(out) == [0.0, -1.0, 0.0]
+    rng = np.random.default_rng(5)
+    g = (rng.standard_normal(10001) * 1e-3).astype(np.float32)
+    out = O.normalize_gradient(g)
+    assert abs(np.linalg.norm(out.astype(np.float64)) - 1.0) < 1e-7
+    assert np.array_equal(O.normalize_gradient(g * np.float32(1024.0)), out)     # exact scaling
+    assert np.array_equal(O.normalize_gradient(-g), -out)
+    want = (g.astype(np.float64) / np.linalg.norm(g.astype(np.float64))).astype(np.float32)
+    assert np.max(np.abs(out.view(np.int32).astype(np.int64) - want.view(np.int32))) <= 1
+    # small case against exact rational arithmetic: squares sum to 49 = 7^2
+    h = np.float32([2.0, 3.0, 6.0])
+    out = O.normalize_gradient(h)
+    for o, x in zip(out, h):
+        assert o == np.float32(float(Fraction(int(x), 7)))
+    z = np.zeros(17, dtype=np.float32)
+    assert np.array_equal(O.normalize_gradient(z), z)
+    assert O.normalize_gradient(np.zeros(0, dtype=np.float32)).size == 0
