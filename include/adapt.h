@@ -208,6 +208,24 @@ int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* 
 int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
                              int n_grads, double* out, void* stream);
 
+/* Gradient normalisation of Sec. 3.3 ("Dealing with Fixed-Points Limited
+ * Range"): every layer's gradient is divided by its own L2 norm,
+ * out[l][i] = grads[l][i] / ||grads[l]||_2, so that an update step cannot move
+ * weights out of the representable range.  The norm is the square root of the
+ * sum of squares accumulated in double, each quotient is formed in double (as a
+ * product with the norm's reciprocal) and rounded to fp32: within one fp32 ulp
+ * of the correctly rounded quotient; a layer whose norm is 0 is copied unchanged.
+ *   grads     HOST array of n_layers DEVICE pointers (fp32, 4-byte aligned)
+ *   lens      HOST array of element counts (0 allowed)
+ *   out       HOST array of n_layers DEVICE pointers, fp32[lens[l]] each;
+ *             out[l] may be grads[l] itself (in place), no other overlap
+ *   norms_out optional DEVICE double[n_layers]: the SUMS OF SQUARES ||g||_2^2
+ * Two launches (reduction, scaling): 4 + 8 bytes per element.  Uses the same
+ * library-owned device buffer as adapt_gradient_diversity (allocated and grown
+ * inside the call); calls that use it must not overlap on the device. */
+int adapt_normalize_gradients(const float* const* grads, const int64_t* lens, int n_layers,
+                              float* const* out, double* norms_out, void* stream);
+
 /* Bytes of DEVICE workspace the search needs for these sizes (0 on invalid
  * arguments).  lens is a HOST array. */
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers,

@@ -26,7 +26,7 @@ EXPORTS = (
     "adapt_version", "adapt_status_string", "adapt_last_error", "adapt_quantize",
     "adapt_quantize_ex", "adapt_quantize_selected", "adapt_quantize_selected_batch",
     "adapt_requantize_selected_batch", "adapt_quantize_selected_batch_packed",
-    "adapt_search_workspace_bytes", "adapt_gradient_diversity",
+    "adapt_search_workspace_bytes", "adapt_gradient_diversity", "adapt_normalize_gradients",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
     "adapt_precision_switch_host",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
@@ -100,6 +100,9 @@ def lib():
         L.adapt_quantize_selected_batch_packed.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
                                                            C.c_int, C.c_uint64, C.c_int32, C.c_int,
                                                            C.c_void_p, C.c_void_p, C.c_void_p]
+        L.adapt_normalize_gradients.restype = C.c_int
+        L.adapt_normalize_gradients.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p,
+                                                C.c_void_p]
         L.adapt_requantize_selected_batch.restype = C.c_int
         L.adapt_requantize_selected_batch.argtypes = L.adapt_quantize_selected_batch.argtypes
         L.adapt_gradient_diversity.restype = C.c_int
@@ -316,6 +319,25 @@ def adapt_gradient_diversity(grads: Sequence[Sequence[torch.Tensor]],
                                           out.data_ptr(), _stream_handle(stream)),
            "adapt_gradient_diversity")
     return out
+
+
+def adapt_normalize_gradients(grads: Sequence[torch.Tensor],
+                              out: Optional[Sequence[torch.Tensor]] = None,
+                              want_sumsq: bool = False, stream=None):
+    """Every layer's gradient divided by its L2 norm (``out`` defaults to new tensors and may be
+    ``grads``: in place).  Returns out, or (out, device float64[L] sums of squares)."""
+    if out is None:
+        out = [torch.empty_like(g) for g in grads]
+    ptrs, lens = _marshal_tensors(grads)
+    assert all(o.is_cuda and o.dtype == torch.float32 and o.is_contiguous() and o.numel() == g.numel()
+               for o, g in zip(out, grads))
+    outs = np.array([o.data_ptr() for o in out], dtype=np.uint64)
+    sumsq = torch.empty(len(grads), dtype=torch.float64, device=grads[0].device) if want_sumsq else None
+    _check(lib().adapt_normalize_gradients(ptrs.ctypes.data, lens.ctypes.data, len(grads),
+                                           outs.ctypes.data, sumsq.data_ptr() if want_sumsq else None,
+                                           _stream_handle(stream)),
+           "adapt_normalize_gradients")
+    return (out, sumsq) if want_sumsq else out
 
 
 def adapt_search_workspace_bytes(lens: Sequence[int], grid: Grid, n_bins: int) -> int:

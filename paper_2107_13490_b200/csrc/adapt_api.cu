@@ -778,6 +778,71 @@ int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int
   return ADAPT_OK;
 }
 
+int adapt_normalize_gradients(const float* const* grads, const int64_t* lens, int n_layers,
+                              float* const* out, double* norms_out, void* stream_handle) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (!grads || !lens || !out) return ADAPT_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > 65535) return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    if (lens[l] < 0) return ADAPT_ERR_INVALID_ARG;
+    if (lens[l] > 0 && (!grads[l] || !out[l])) return ADAPT_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(grads[l]) & 3u) || (reinterpret_cast<uintptr_t>(out[l]) & 3u))
+      return ADAPT_ERR_INVALID_ARG;
+  }
+  DeviceCache* dc = nullptr;
+  int rc = current_cache(&dc);
+  if (rc != ADAPT_OK) return rc;
+  // layer table, the two pointer lists, then the sums of squares (two doubles per layer)
+  const size_t L = n_layers;
+  const size_t off_g = align_up(sizeof(DivLayer) * (L + 1), 256);
+  const size_t off_o = align_up(off_g + sizeof(float*) * L, 256);
+  const size_t blob = align_up(off_o + sizeof(float*) * L, 256);
+  const size_t sums = sizeof(double) * L * 2;
+  rc = grow_device(&dc->div_buf, &dc->div_buf_bytes, align_up(blob + sums, 4096));
+  if (rc != ADAPT_OK) return rc;
+  PinnedSlot* slot = nullptr;
+  rc = acquire_slot(*dc, blob, &slot);
+  if (rc != ADAPT_OK) return rc;
+  char* h = static_cast<char*>(slot->host);
+  DivLayer* hl = reinterpret_cast<DivLayer*>(h);
+  long long tiles = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    hl[l].n = lens[l]; hl[l].tile_begin = tiles; hl[l].pad_ = 0;
+    hl[l].vec = !(reinterpret_cast<uintptr_t>(grads[l]) & 15u) && !(reinterpret_cast<uintptr_t>(out[l]) & 15u);
+    tiles += (lens[l] + kDivTile - 1) / kDivTile;
+  }
+  hl[n_layers].n = 0; hl[n_layers].tile_begin = tiles; hl[n_layers].vec = 0; hl[n_layers].pad_ = 0;
+  std::memcpy(h + off_g, grads, sizeof(float*) * L);
+  std::memcpy(h + off_o, out, sizeof(float*) * L);
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+  char* d = static_cast<char*>(dc->div_buf);
+  ADAPT_CUDA(cudaMemcpyAsync(d, h, blob, cudaMemcpyHostToDevice, stream));
+  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  ADAPT_CUDA(cudaMemsetAsync(d + blob, 0, sums, stream));
+  DivParams dp;
+  dp.layers = reinterpret_cast<const DivLayer*>(d);
+  dp.grads = reinterpret_cast<const float* const*>(d + off_g);
+  dp.sumsq = reinterpret_cast<double*>(d + blob);
+  dp.n_layers = n_layers; dp.n_grads = 1; dp.n_tiles = tiles;
+  if (tiles > 0) {
+    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc->sm_count));
+    {
+      LaunchScope ls(ADAPT_KERNEL_DIVERSITY, stream);
+      diversity_kernel<<<grid, kDivThreads, 0, stream>>>(dp);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+    LaunchScope ls(ADAPT_KERNEL_DIVERSITY, stream);
+    normalize_kernel<<<grid, kDivThreads, 0, stream>>>(dp.layers, dp.grads,
+                                                       reinterpret_cast<float* const*>(d + off_o),
+                                                       dp.sumsq, n_layers, tiles);
+    ADAPT_CUDA(cudaGetLastError());
+  }
+  if (norms_out)   // the sums of squares sit two doubles apart: strided copy of the first of each
+    ADAPT_CUDA(cudaMemcpy2DAsync(norms_out, sizeof(double), dp.sumsq, 2 * sizeof(double),
+                                 sizeof(double), L, cudaMemcpyDeviceToDevice, stream));
+  return ADAPT_OK;
+}
+
 size_t adapt_search_workspace_bytes(const int64_t* lens, int n_layers, const adapt_grid* grid,
                                     int n_bins) {
   Plan plan;

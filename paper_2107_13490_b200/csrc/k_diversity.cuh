@@ -106,6 +106,54 @@ __global__ void __launch_bounds__(kDivThreads) diversity_kernel(const DivParams 
   }
 }
 
+// Gradient normalisation (Sec. 3.3, "Dealing with Fixed-Points Limited Range"):
+// out = g / ||g||_2 per layer, the norm taken from the sums of squares the reduction above left
+// in sumsq (one gradient per layer: sumsq[2 l]).  The quotient is formed in double, as a product
+// with the reciprocal of the norm (a double division per element would make the kernel
+// FP64-bound), and rounded to float: like the norm's summation order this can move a result by
+// one fp32 ulp where the quotient sits on a rounding boundary, never more.  A layer whose norm
+// is 0 is copied.  out may be g itself.  8 B per element.
+__global__ void __launch_bounds__(kDivThreads)
+normalize_kernel(const DivLayer* __restrict__ layers, const float* const* __restrict__ grads,
+                 float* const* __restrict__ outs, const double* __restrict__ sumsq, int n_layers,
+                 long long n_tiles) {
+  for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+    int lo = 0, hi = n_layers - 1;          // layer that owns tile t
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (layers[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
+    }
+    const DivLayer L = layers[lo];
+    const float* g = grads[lo];
+    float* out = outs[lo];
+    const double norm = sqrt(sumsq[2 * lo]);
+    const bool scale = norm > 0.0;
+    const double inv = scale ? 1.0 / norm : 0.0;
+    const long long i0 = (t - L.tile_begin) * kDivTile;
+    const long long i1 = min(L.n, i0 + kDivTile);
+    if (L.vec && i1 - i0 == kDivTile) {
+      const float4* g4 = reinterpret_cast<const float4*>(g + i0);
+      float4* o4 = reinterpret_cast<float4*>(out + i0);
+#pragma unroll
+      for (int q = 0; q < kDivPerThread / 4; ++q) {
+        float4 v = __ldcs(g4 + q * kDivThreads + threadIdx.x);
+        if (scale) {
+          v.x = __double2float_rn(__dmul_rn(static_cast<double>(v.x), inv));
+          v.y = __double2float_rn(__dmul_rn(static_cast<double>(v.y), inv));
+          v.z = __double2float_rn(__dmul_rn(static_cast<double>(v.z), inv));
+          v.w = __double2float_rn(__dmul_rn(static_cast<double>(v.w), inv));
+        }
+        __stcs(o4 + q * kDivThreads + threadIdx.x, v);
+      }
+    } else {
+      for (long long i = i0 + threadIdx.x; i < i1; i += kDivThreads) {
+        const float x = __ldcs(g + i);
+        out[i] = scale ? __double2float_rn(__dmul_rn(static_cast<double>(x), inv)) : x;
+      }
+    }
+  }
+}
+
 // One thread per layer: norms from the sums of squares, then the two forms of the diversity.
 __global__ void diversity_finalize_kernel(const double* __restrict__ sumsq, int n_layers,
                                           int n_grads, double* __restrict__ out) {

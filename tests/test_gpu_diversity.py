@@ -84,3 +84,40 @@ def test_large_multi_tile(B):
     dev = [torch.from_numpy(g).cuda() for g in host]
     out = B.adapt_gradient_diversity([dev]).cpu().numpy()
     _close(out[0], O.gradient_diversity(host))
+
+
+def test_gradient_normalisation_matches_the_oracle(B):
+    """g / ||g||_2 per layer (Sec. 3.3).  The norm's summation order differs (sequential on the
+    CPU, tree on the GPU): its relative error stays below n * 2^-53, far inside half an fp32 ulp
+    of every quotient except at rounding boundaries - so at most one ulp of fp32 per element,
+    and the sums of squares agree to 1e-12."""
+    import torch
+    rng = np.random.default_rng(11)
+    host = [(rng.laplace(0, 1e-4, n)).astype(np.float32) for n in (1, 5, 2047, 2048, 2049, 70001, 1 << 20)]
+    host.append(np.zeros(300, dtype=np.float32))            # zero norm: copied
+    host.append(np.zeros(0, dtype=np.float32))              # empty layer
+    host.append(np.float32([3.0, 4.0]))
+    dev = []
+    for j, h in enumerate(host):                              # odd phases: scalar path too
+        b = torch.zeros(h.size + 4, dtype=torch.float32, device="cuda")
+        b[j % 4:j % 4 + h.size] = torch.from_numpy(h).cuda()
+        dev.append(b[j % 4:j % 4 + h.size])
+    out, sumsq = B.adapt_normalize_gradients(dev, want_sumsq=True)
+    torch.cuda.synchronize()
+    sumsq = sumsq.cpu().numpy()
+    for j, h in enumerate(host):
+        want = O.normalize_gradient(h)
+        got = out[j].cpu().numpy()
+        assert got.shape == want.shape
+        if h.size:
+            d = np.abs(got.view(np.int32).astype(np.int64) - want.view(np.int32).astype(np.int64))
+            assert d.max() <= 1, (j, int(d.max()))
+            ss = float(np.sum(h.astype(np.float64) ** 2))
+            assert sumsq[j] == pytest.approx(ss, rel=1e-12, abs=0.0)
+    assert list(out[-1].cpu().numpy()) == [np.float32(0.6), np.float32(0.8)]
+    # in place
+    ref = [o.clone() for o in out]
+    B.adapt_normalize_gradients(dev, out=dev)
+    torch.cuda.synchronize()
+    for a, b in zip(dev, ref):
+        assert torch.equal(a, b)
