@@ -46,9 +46,11 @@ def parse_args():
                     help="elements of the workload the CPU baseline is timed on")
     ap.add_argument("--elements", type=int, default=0,
                     help="profiling aid: shrink a single-layer workload to this many elements")
-    ap.add_argument("--path", default="search", choices=["search", "diversity", "formats"],
+    ap.add_argument("--path", default="search", choices=["search", "diversity", "normalize", "formats"],
                     help="search: the precision-switch search step (default); diversity: the "
-                         "gradient-diversity reduction that feeds PushUp")
+                         "gradient-diversity reduction that feeds PushUp; normalize: g / ||g||_2 per "
+                         "layer; formats: the search over block-floating-point and floating-point "
+                         "candidates")
     ap.add_argument("--algorithm", default="auto", choices=["auto", "keyed", "direct"],
                     help="profiling aid: which form of the fused search kernel runs (auto: the "
                          "library's own choice; keyed serves round-to-nearest-even only)")
@@ -210,6 +212,56 @@ def run_reference(args):
     return 0
 
 
+def run_normalize(args):
+    """Gradient normalisation g / ||g||_2: one layer of 2^28 elements (or --elements N); one
+    read for the norm, one read and one write for the scaling = 12 B per element."""
+    import torch
+    from paper_2107_13490_b200 import binding as B
+    from paper_2107_13490_b200 import workloads as W
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    B.lib()
+    n = args.elements or (1 << 28)
+    host = W.generate_layer(W.LayerSpec("g", (n,), "laplace", 1e-4, zero_frac=0.05), 7, 0)
+    g = [torch.from_numpy(host).cuda()]
+    out = [torch.empty_like(g[0])]
+    for _ in range(max(args.warmup, 3)):
+        B.adapt_normalize_gradients(g, out=out)
+    torch.cuda.synchronize()
+    n0 = B.adapt_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        B.adapt_normalize_gradients(g, out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    peak, kind = measured_peak_gbs()
+    achieved = 12.0 * n / (ms * 1e-3) / 1e9
+    line = {"metric": "gradient-normalisation elements/s", "value": n / (ms * 1e-3), "unit": "elements/s",
+            "n_gpus": 1, "steps": args.steps, "ms_per_step": ms, "dtype": "f64", "data": "synthetic",
+            "gpu_launches": int(B.adapt_kernel_launch_count() - n0),
+            "config": {"workload": f"one layer, {n} elements, Laplace(0,1e-4) with 5% zeros",
+                       "l2": "inputs exceed L2" if 4 * n > 126e6 else "inputs may sit in L2"},
+            "roofline": {"bound": "hbm", "kernel": "diversity (norm) + normalize (scaling), whole call",
+                         "achieved": achieved, "peak": peak, "peak_kind": kind, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": None}}
+    if not args.no_cpu_baseline:
+        from oracle import oracle as O
+        m = min(n, 1 << 24)
+        t0 = time.perf_counter()
+        want = O.normalize_gradient(host[:m])
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": m / dt, "unit": "elements/s", "cores": 1, "kind": "oracle",
+                                "sample": f"first {m} elements"}
+        if m == n:
+            got = out[0].cpu().numpy()
+            line["parity_max_ulp"] = int(np.abs(got.view(np.int32).astype(np.int64) -
+                                                want.view(np.int32).astype(np.int64)).max())
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def run_diversity(args):
     """Gradient-diversity reduction: one layer of 2^24 elements with 32 recent gradients
     (2 GiB read per step), or --elements N."""
@@ -353,6 +405,8 @@ def main():
         return run_reference(args)
     if args.path == "diversity":
         return run_diversity(args)
+    if args.path == "normalize":
+        return run_normalize(args)
     if args.path == "formats":
         return run_formats(args)
 
