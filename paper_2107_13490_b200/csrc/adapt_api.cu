@@ -173,7 +173,7 @@ struct Plan {
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
   // accumulators (cleared every call)
-  size_t off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
+  size_t off_sub = 0, off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
          off_zclass = 0, off_nzero = 0, accum_begin = 0, accum_bytes = 0;
   size_t total = 0;
 };
@@ -249,6 +249,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_q = o;       o = align_up(o + sizeof(unsigned) * L * B, 256);
   p->off_qe = o;      o = align_up(o + sizeof(unsigned) * L * B * 2, 256);
   p->off_cells = o;   o = align_up(o + sizeof(unsigned) * L * K, 256);
+  p->off_sub = o;     o = align_up(o + sizeof(unsigned) * (K ? L * 2 * B * kSubCells : 0), 256);
   p->off_u = o;       o = align_up(o + sizeof(unsigned) * L * F * B, 256);
   p->accum_bytes = o - p->accum_begin;
   p->total = o;
@@ -389,6 +390,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   unsigned* d_q = reinterpret_cast<unsigned*>(ws + plan.off_q);
   unsigned* d_qe = reinterpret_cast<unsigned*>(ws + plan.off_qe);
   unsigned* d_cells = reinterpret_cast<unsigned*>(ws + plan.off_cells);
+  unsigned* d_sub = reinterpret_cast<unsigned*>(ws + plan.off_sub);
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + plan.off_u);
 
   // K1: range scan over every layer, then bin origin / scale per layer
@@ -424,6 +426,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
     kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
+    kp.sub_count = d_sub;
     kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
     kp.n_bins = bins_stride; kp.n_levels = plan.n_levels;
     kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
@@ -438,6 +441,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ExpandParams ep;
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
     ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
+    ep.sub_count = d_sub; ep.edges = d_edges;
     ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
     ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
     ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
@@ -569,7 +573,7 @@ int run_quantize(const float* x, int64_t n, int wl, int fl, const int32_t* selec
 
 extern "C" {
 
-const char* adapt_version(void) { return "adapt-b200 0.7"; }
+const char* adapt_version(void) { return "adapt-b200 0.8"; }
 
 const char* adapt_status_string(int status) {
   switch (status) {

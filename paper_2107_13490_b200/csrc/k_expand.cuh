@@ -33,6 +33,8 @@ struct ExpandParams {
   const unsigned* cell_init;   // [layer][cell_cap]
   const unsigned* cell_count;  // [layer][cell_cap]
   const unsigned* qe_hist;     // [layer][2][n_bins]
+  const unsigned* sub_count;   // [layer][2][n_bins][kSubCells]  sub-cell counts of the edge cells
+  const float* edges;          // [layer][n_bins + 1]  exact bin edges
   unsigned* q_hist;            // [layer][n_bins]
   unsigned* u_hist;            // [layer][n_levels][n_bins]
   unsigned long long* zeros;   // [layer][n_levels]
@@ -97,6 +99,53 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
       }
     }
   }
+  // sub-cells of the edge cells (refined layers).  Entry (segment, id, j): sub-cell j of the edge
+  // cell whose left end lies in bin id, i.e. the cell that holds the bin edge E[id + 1] (the
+  // cell to its left when that edge sits exactly on the cell grid).  Levels below the
+  // segment's G are served by the cell itself; for G <= f < G + kSubBits the sub-cell index
+  // fixes the rounded value; for finer levels and the float histogram an interior sub-cell
+  // puts its elements into its bin (those of a sub-cell with a bin edge inside were binned one
+  // by one).  Sub-cells never add to the zero counts: next to zero the zero classes do.
+  if (P.refined) {
+    const float* E = p.edges + static_cast<size_t>(l) * (B + 1);
+    const unsigned* sub = p.sub_count + static_cast<size_t>(l) * 2 * B * kSubCells;
+    for (int s = 0; s < 2; ++s) {
+      const SegPlan& sp = P.seg[s];
+      if (sp.cells == 0) continue;
+      if (!is_q && f < sp.fs) continue;
+      const int gs = sp.g + kSubBits;
+      const int n_sub = L.n_bins * kSubCells;
+      const int per_z = ((n_sub + gridDim.z - 1) / gridDim.z + 3) & ~3;
+      const int k_end = min(n_sub, static_cast<int>(blockIdx.z + 1) * per_z);
+      const uint4* sub4 = reinterpret_cast<const uint4*>(sub + static_cast<size_t>(s) * B * kSubCells);
+      for (int k0 = blockIdx.z * per_z + 4 * threadIdx.x; k0 < k_end; k0 += 4 * kExpandThreads) {
+        const uint4 m4 = __ldg(sub4 + (k0 >> 2));
+        const unsigned ms[4] = {m4.x, m4.y, m4.z, m4.w};
+        if ((m4.x | m4.y | m4.z | m4.w) == 0u) continue;
+        const int id = k0 / kSubCells;                      // the four share their edge cell
+        const long long cc = static_cast<long long>(ceil(ldexp(static_cast<double>(E[id + 1]), sp.g))) - 1;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const unsigned m = ms[e];
+          if (m == 0) continue;
+          const long long jj = cc * kSubCells + ((k0 + e) & (kSubCells - 1));
+          if (is_q || f >= gs) {
+            const float l2 = __double2float_rd(ldexp(static_cast<double>(jj), -gs));
+            const float r2 = __double2float_ru(ldexp(static_cast<double>(jj + 1), -gs));
+            const int bl = bin_of(l2, S.lo, S.scale, S.bmax);
+            if (bl == bin_of(r2, S.lo, S.scale, S.bmax)) atomicAdd(&s_hist[bl], m);
+          } else {
+            const int d = gs - f;                        // 1..kSubBits
+            const long long a = jj >> d;
+            const long long rem = jj - (a << d);
+            const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
+            const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
+            atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+          }
+        }
+      }
+    }
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) zero += __shfl_xor_sync(0xffffffffu, zero, o);
   if ((threadIdx.x & 31) == 0 && zero) atomicAdd(&s_zero, zero);
@@ -109,8 +158,11 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   const int bz = bin_of(0.0f, S.lo, S.scale, S.bmax);
   const unsigned* qe0 = p.qe_hist + static_cast<size_t>(l) * 2 * B;
   const unsigned* qe1 = qe0 + B;
-  const bool fine0 = lead && (is_q || f >= P.seg[0].fs);
-  const bool fine1 = lead && P.seg[1].cells > 0 && (is_q || f >= P.seg[1].fs);
+  // the edge-element histograms hold what the level loop looked at: from the sub-cells' level on
+  const int fe0 = P.refined ? max(P.seg[0].g + kSubBits, 0) : P.seg[0].fs;
+  const int fe1 = P.refined ? max(P.seg[1].g + kSubBits, 0) : P.seg[1].fs;
+  const bool fine0 = lead && (is_q || f >= fe0);
+  const bool fine1 = lead && P.seg[1].cells > 0 && (is_q || f >= fe1);
   unsigned* out = is_q ? p.q_hist + static_cast<size_t>(l) * B
                        : p.u_hist + (static_cast<size_t>(l) * p.n_levels + f) * B;
   for (int b = threadIdx.x; b < B; b += kExpandThreads) {

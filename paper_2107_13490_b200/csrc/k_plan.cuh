@@ -41,6 +41,20 @@ constexpr unsigned kCellOnGrid = 0x20000000u;     // added to a returned word, n
 constexpr unsigned kCellCountMask = 0x1FFFFFFFu;
 constexpr int kPlanThreads = 256;
 
+// Second level under the edge cells.  An element of an edge cell is counted again in one of
+// kSubCells sub-cells (2^-(G + kSubBits) wide) of a table in global memory, indexed by segment,
+// by the bin of the edge cell's left end (no two edge cells of a segment share it) and by the
+// sub-cell.  Towards the levels G .. G + kSubBits - 1 a sub-cell is what a cell is towards the
+// coarse levels, towards the finer levels and the float histogram an interior sub-cell is what
+// an interior cell is; only the elements of sub-cells that themselves hold a bin edge still go
+// through the level loop.  Used for layers in the magic-constant forms (cell indices below 2^22).
+constexpr int kSubBits = 5;
+constexpr int kSubCells = 1 << kSubBits;
+// The main segment's edge cells sit where the mass is: a few cells can take a large share of all
+// sub-cell counts, so they are kept per CTA in shared memory when the segment's cells start in at
+// most this many bins (reductions of all SMs into one line of global memory would serialise).
+constexpr int kSubSharedIds = 128;
+
 // Tunables of the table shape (performance only).
 #ifndef ADAPT_CELL_BALANCE
 #define ADAPT_CELL_BALANCE 4    // cells ~ sqrt(balance * n_bins * elements one CTA sees of the layer)
@@ -74,6 +88,10 @@ struct LayerPlan {
   unsigned grid_mask;  // low mantissa bits that are zero in every element on its segment's grid
   int masked;       // 1 if the counting kernel may take "those bits are zero" as its grid-point flag
   int dense;        // 1 if, besides, exact zeros are so rare that they may go through the handler
+  int refined;      // 1 if the elements of edge cells are counted once more, in sub-cells
+  int sub_base;     // main segment: bin of its first cell's left end, or -1 if the bins its cells
+                    // start in number more than kSubSharedIds (its sub-cell counts then go
+                    // straight to global memory like the auxiliary segment's)
   unsigned grid_mul;   // 2^(32 - bits of grid_mask): x's bit pattern times this is 0 exactly when those bits are
 };
 
@@ -206,6 +224,15 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
       if (s == 0 && P.seg[1].cells > 0) top = __uint_as_float(__float_as_uint(P.radius) - 1u);
       const int biased = max(1, static_cast<int>((__float_as_uint(top) >> 23) & 0xFFu));
       zero_bits = min(zero_bits, 23 - (biased - 127) - P.seg[s].g);
+    }
+    P.refined = (P.keyed && P.fast) ? 1 : 0;
+    P.sub_base = -1;
+    if (P.refined) {
+      const SegPlan& m0 = P.seg[0];
+      const float first = __double2float_rd(ldexp(static_cast<double>(m0.c0), -m0.g));
+      const float last = __double2float_rd(ldexp(static_cast<double>(m0.c0 + m0.cells - 1), -m0.g));
+      const int b_first = bin_of(first, S.lo, S.scale, S.bmax);
+      if (bin_of(last, S.lo, S.scale, S.bmax) - b_first < kSubSharedIds) P.sub_base = b_first;
     }
     P.grid_mask = zero_bits >= 1 ? (1u << zero_bits) - 1u : 0u;
     P.masked = (P.fast && zero_bits >= kMinGridMaskBits) ? 1 : 0;

@@ -67,6 +67,7 @@ struct KeyedParams {
   unsigned* cell_count;        // [layer][cell_cap]      global cell counts
   unsigned* qe_hist;           // [layer][2][n_bins]     float histogram of the edge elements, per segment
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
+  unsigned* sub_count;         // [layer][2][n_bins][kSubCells]  sub-cell counts of the edge cells
   unsigned long long* zeros;   // [layer][n_levels]
   unsigned long long* zero_class;  // [layer][kZeroClasses]
   unsigned long long* cell_total;  // [layer] sum of all cell counts = non-zero elements
@@ -80,6 +81,7 @@ __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int
   return sizeof(unsigned) * (static_cast<size_t>(cell_cap) + kDummySlots + n_bins +
                              static_cast<size_t>(d_levels) * n_bins) +
          sizeof(float) * (static_cast<size_t>(n_bins) + 4) +      // the layer's bin edges
+         sizeof(unsigned) * kSubSharedIds * kSubCells +          // main segment's sub-cell counts
          sizeof(float) * kKeyedWarps * kQueueCap;
 }
 
@@ -105,6 +107,12 @@ struct LayerCtx {
   int masked, dense;
   unsigned grid_mul;
   int zero_pos;                // table position of the main segment's cell [0, 2^-G)
+  int refined;                 // edge cells have sub-cells
+  int fs_edge[2];              // first level the level loop looks at: fs, or the sub-cells' level
+  float sub_two[2];            // 2^(G + kSubBits) per segment
+  unsigned* sub;               // global, this layer's [2][n_bins][kSubCells]
+  unsigned* sub_s;             // shared [kSubSharedIds][kSubCells]: main segment's, when sub_base >= 0
+  int sub_base;
 };
 
 // An element that sits exactly on its segment's grid (x * 2^G = p, an integer) is a rounding
@@ -148,8 +156,40 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     kz = max(-1, min(kz, 32));
     atomicAdd(&c.zclass[kz + 1], 1u);
   }
-  // ---- edge cell: float bin, then the fine levels that can still move ----------------
+  // ---- edge cell: its sub-cell, float bin, then the fine levels that can still move ---------
   if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
+  if (c.refined) {
+    // sub-cell index: x * 2^(G + kSubBits) is exact, the cell's first sub-cell index c * 2^kSubBits
+    // is a float (c < 2^22), and the two lie within 2^kSubBits of each other.  A point of the
+    // sub-grid goes left or right by the same parity rule as a point of the cell grid (for a
+    // point of both grids the two decisions agree: the rule does not depend on the scale).
+    const float zs = __fmul_rn(x, c.sub_two[s]);
+    const float cfs = floorf(zs);
+    int j = __float2int_rz(__fsub_rn(cfs, __ll2float_rn(cc * kSubCells)));
+    if (zs == cfs && grid_point_goes_left(cc * kSubCells + j)) j -= 1;
+    j = max(0, min(j, kSubCells - 1));      // always true by construction; keeps the address in the table
+    const long long jj = cc * kSubCells + j;
+    const int g = c.g[s];
+    // left end of the cell (exact: c < 2^22), then the ends of the sub-cell's closed interval,
+    // rounded outwards (c * 2^kSubBits + j can need 27 bits); in float when the powers of two
+    // involved are normal numbers - the same real numbers rounded the same way as in double
+    float lf, l2, r2;
+    if (g >= -120 && g + kSubBits <= 120) {
+      const float w2 = pow2f(-(g + kSubBits));
+      lf = __fmul_rn(__ll2float_rn(cc), pow2f(-g));
+      l2 = __fadd_rd(lf, __fmul_rn(__int2float_rn(j), w2));
+      r2 = __fadd_ru(lf, __fmul_rn(__int2float_rn(j + 1), w2));
+    } else {
+      lf = __double2float_rd(ldexp(static_cast<double>(cc), -g));
+      l2 = __double2float_rd(ldexp(static_cast<double>(jj), -(g + kSubBits)));
+      r2 = __double2float_ru(ldexp(static_cast<double>(jj + 1), -(g + kSubBits)));
+    }
+    const int id = bin_of(lf, c.lo, c.scale, c.bmax);
+    if (s == 0 && c.sub_base >= 0) atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
+    else atomicAdd(&c.sub[(static_cast<size_t>(s) * B + id) * kSubCells + j], 1u);
+    // an interior sub-cell (its closed interval in one bin) settles the element
+    if (bin_of(l2, c.lo, c.scale, c.bmax) == bin_of(r2, c.lo, c.scale, c.bmax)) return;
+  }
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
   if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
   const float e_lo = c.E[b0], e_hi = c.E[b0 + 1];
@@ -158,7 +198,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   int f_end = 32;
   if (m > 0.0f) f_end = 126 - static_cast<int>((__float_as_uint(m) - 1u) >> 23);
   f_end = min(f_end, c.n_levels);
-  const int fs = c.fs[s];
+  const int fs = c.fs_edge[s];
   for (int f = fs; f < f_end; ++f) {
     const float r = rintf(__fmul_rn(x, pow2f(f)));
     const float v = __fmul_rn(r, pow2f(-f));
@@ -397,7 +437,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
   unsigned* qe = cells + p.cell_cap + kDummySlots;
   int* dtab = reinterpret_cast<int*>(qe + p.n_bins);
   float* edges = reinterpret_cast<float*>(dtab + static_cast<size_t>(p.d_levels) * p.n_bins);   // [n_bins + 4]
-  float* queues = edges + p.n_bins + 4;
+  unsigned* sub_s = reinterpret_cast<unsigned*>(edges + p.n_bins + 4);   // [kSubSharedIds][kSubCells]
+  float* queues = reinterpret_cast<float*>(sub_s + kSubSharedIds * kSubCells);
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* queue = queues + warp * kQueueCap;
@@ -426,6 +467,14 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.magic[0] = P->seg[0].magic; c.magic[1] = P->seg[1].magic;
       c.keyed = P->keyed; c.fast = P->fast; c.total_cells = P->total_cells;
       c.grid_mask = P->grid_mask; c.masked = P->masked; c.dense = P->dense;
+      c.refined = P->refined;
+      for (int sg = 0; sg < 2; ++sg) {
+        const int gs = P->seg[sg].g + kSubBits;
+        c.fs_edge[sg] = P->refined ? max(gs, 0) : P->seg[sg].fs;
+        c.sub_two[sg] = P->refined ? pow2f(max(-126, min(gs, 127))) : 1.0f;
+      }
+      c.sub = p.sub_count + static_cast<size_t>(l) * 2 * p.n_bins * kSubCells;
+      c.sub_s = sub_s; c.sub_base = P->refined ? P->sub_base : -1;
       c.grid_mul = P->grid_mul;
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
       c.E = edges;
@@ -461,6 +510,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
       for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
+      for (int i = threadIdx.x; i < kSubSharedIds * kSubCells; i += kKeyedThreads) sub_s[i] = 0;
       if (threadIdx.x < kDummySlots)
         cells[p.cell_cap + threadIdx.x] = kCellEdge | kCellNearZero | kCellOnGrid;
     }
@@ -493,11 +543,19 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
         const unsigned n = qe[i];
         if (n) atomicAdd(&gq[i], n);
       }
+      if (c.sub_base >= 0) {
+        unsigned* gs = c.sub + static_cast<size_t>(c.sub_base) * kSubCells;     // segment 0, id sub_base
+        const int room = (p.n_bins - c.sub_base) * kSubCells;
+        for (int i = threadIdx.x; i < min(kSubSharedIds * kSubCells, room); i += kKeyedThreads) {
+          const unsigned n = sub_s[i];
+          if (n) atomicAdd(&gs[i], n);
+        }
+      }
       for (int i = threadIdx.x; i < p.n_bins * p.d_levels; i += kKeyedThreads) {
         const int dv = dtab[i];
         if (dv) {
           const int j = i / p.n_bins, b = i - j * p.n_bins;
-          const int f = c.fs[0] + j;
+          const int f = c.fs_edge[0] + j;
           if (f < p.n_levels)
             atomicAdd(&layer_u[static_cast<size_t>(f) * p.n_bins + b], static_cast<unsigned>(dv));
         }
