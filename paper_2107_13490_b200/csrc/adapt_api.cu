@@ -157,6 +157,9 @@ int acquire_slot(DeviceCache& c, size_t bytes, PinnedSlot** out) {
 // ---- search plan ----------------------------------------------------------------
 
 constexpr int kMaxBins = 16384;
+#ifndef ADAPT_D_LEVELS_MAX
+#define ADAPT_D_LEVELS_MAX 6   // fine levels of the main segment whose corrections stay in shared memory
+#endif
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
 constexpr int kKeyedMaxBins = 8192;
 constexpr size_t kKeyedSmemBudget = 224 * 1024; // one CTA per SM owns its shared memory
@@ -215,7 +218,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   // shared-memory shape of the keyed kernel: queue + bin edges + Qe + a few correction levels + cells
   const size_t hist = sizeof(unsigned) * n_bins;
   const size_t queue = keyed_smem_bytes(0, 0, 0);
-  p->d_levels = static_cast<int>(std::min<size_t>(6, (32 * 1024) / hist));
+  p->d_levels = static_cast<int>(std::min<size_t>(ADAPT_D_LEVELS_MAX, (32 * 1024) / hist));
   p->d_levels = std::min(p->d_levels, p->n_levels);
   if (n_bins <= kKeyedMaxBins) {
     p->cell_cap = static_cast<int>((kKeyedSmemBudget - queue - hist * (2 + p->d_levels)) / 4) - 64;

@@ -114,11 +114,14 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
       if (sp.cells == 0) continue;
       if (!is_q && f < sp.fs) continue;
       const int gs = sp.g + kSubBits;
-      const int n_sub = L.n_bins * kSubCells;
-      const int per_z = ((n_sub + gridDim.z - 1) / gridDim.z + 3) & ~3;
-      const int k_end = min(n_sub, static_cast<int>(blockIdx.z + 1) * per_z);
+      // the main segment's counts, when they were kept in shared memory, lie in a short range of ids
+      const bool narrow = (s == 0 && P.sub_base >= 0);
+      const int k_lo = narrow ? P.sub_base * kSubCells : 0;
+      const int k_hi = narrow ? min(L.n_bins, P.sub_base + kSubSharedIds) * kSubCells : L.n_bins * kSubCells;
+      const int per_z = ((k_hi - k_lo + gridDim.z - 1) / gridDim.z + 3) & ~3;
+      const int k_end = min(k_hi, k_lo + static_cast<int>(blockIdx.z + 1) * per_z);
       const uint4* sub4 = reinterpret_cast<const uint4*>(sub + static_cast<size_t>(s) * B * kSubCells);
-      for (int k0 = blockIdx.z * per_z + 4 * threadIdx.x; k0 < k_end; k0 += 4 * kExpandThreads) {
+      for (int k0 = k_lo + blockIdx.z * per_z + 4 * threadIdx.x; k0 < k_end; k0 += 4 * kExpandThreads) {
         const uint4 m4 = __ldg(sub4 + (k0 >> 2));
         const unsigned ms[4] = {m4.x, m4.y, m4.z, m4.w};
         if ((m4.x | m4.y | m4.z | m4.w) == 0u) continue;
