@@ -165,6 +165,12 @@ def test_adversarial_value_patterns(B):
     off100[::7] = (100.0 + rng.integers(0, 2048, off100[::7].size) * 2.0 ** -11).astype(np.float32)
     cases["offset_100"] = off100
     cases["half_to_one"] = (0.5 + 0.5 * rng.random(n)).astype(np.float32)
+    # points of grids finer than the cells but coarser than (or equal to) the sub-cells of the edge
+    # cells: rounding ties at levels between the two, many of them inside edge cells
+    fine = rng.integers(-(1 << 13), 1 << 13, n).astype(np.float64)
+    cases["fine_grid_15"] = (fine * 2.0 ** -15 + 2.0 ** -16).astype(np.float32)
+    cases["fine_grid_mixed"] = np.where(rng.random(n) < 0.5, fine * 2.0 ** -15,
+                                        rng.integers(-(1 << 15), 1 << 15, n) * 2.0 ** -17).astype(np.float32)
     wl, fl = W.candidate_grid(range(2, 33))
     for name, x in cases.items():
         for n_bins in (100, 2048):
