@@ -48,7 +48,10 @@ constexpr int kPlanThreads = 256;
 // coarse levels, towards the finer levels and the float histogram an interior sub-cell is what
 // an interior cell is; only the elements of sub-cells that themselves hold a bin edge still go
 // through the level loop.  Used for layers in the magic-constant forms (cell indices below 2^22).
-constexpr int kSubBits = 5;
+#ifndef ADAPT_SUB_BITS
+#define ADAPT_SUB_BITS 5
+#endif
+constexpr int kSubBits = ADAPT_SUB_BITS;
 constexpr int kSubCells = 1 << kSubBits;
 // The main segment's edge cells sit where the mass is: a few cells can take a large share of all
 // sub-cell counts, so they are kept per CTA in shared memory when the segment's cells start in at
