@@ -111,14 +111,15 @@ typedef struct adapt_search_opts {
  * n_bins <= 8192).  DIRECT: the direct form everywhere. */
 enum { ADAPT_ALGO_AUTO = 0, ADAPT_ALGO_KEYED = 1, ADAPT_ALGO_DIRECT = 2 };
 
-/* Library version string, e.g. "adapt-b200 0.5". Never NULL. */
+/* Library version string: "adapt-b200 <major>.<minor>". Never NULL. */
 const char* adapt_version(void);
 
 /* Static English text for an adapt_status value. Never NULL. */
 const char* adapt_status_string(int status);
 
-/* Text of the last CUDA error seen by the calling thread's most recent failing
- * call ("" if none). Valid until the next call from any thread. */
+/* Detail text of the calling thread's most recent failing call: the CUDA error
+ * string, or the limit that was exceeded ("" if none).  The buffer belongs to the
+ * calling thread and stays valid until that thread's next failing call. */
 const char* adapt_last_error(void);
 
 /* Quantize(L, <WL,FL>) - Algorithm 1 (re-quantisation of each layer after the
@@ -358,7 +359,11 @@ int adapt_kernel_times(double* ms_out, uint64_t* launches_out, int reset);
  *
  * The first call on a device looks up the scratch array's device address
  * (cudaGetSymbolAddress, with that device current) and keeps it; make that
- * first call before any stream capture begins.
+ * first call before any stream capture begins.  Every call copies a small
+ * descriptor block from ordinary (pageable) host memory of the library, so the
+ * host may wait inside the call for earlier work of that stream, and the call
+ * must not be issued on a stream that is being captured: it then returns
+ * ADAPT_ERR_INVALID_ARG without enqueuing anything.
  * Every call uses the same array and clears the parts that must start at zero,
  * so calls that can overlap on the GPU (different streams, different host
  * threads) race with each other: issue them on one stream or order them with

@@ -29,7 +29,7 @@ using namespace adapt;
 
 std::mutex g_mutex;                     // serialises calls that touch library-owned state
 std::atomic<uint64_t> g_launches{0};
-char g_last_error[512] = "";
+thread_local char g_last_error[512] = "";   // per calling thread
 
 // Optional per-kernel device timing: events around each launch, on its stream.
 struct TimedLaunch { int kind; cudaEvent_t start, stop; };
@@ -1344,6 +1344,15 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   rc = static_scratch_address(&ws);
   if (rc != ADAPT_OK) return rc;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
+  // the descriptor block below is re-read from a host array that the next call overwrites:
+  // a captured copy of it would replay stale or foreign contents
+  cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+  ADAPT_CUDA(cudaStreamIsCapturing(stream, &capturing));
+  if (capturing != cudaStreamCaptureStatusNone) {
+    std::snprintf(g_last_error, sizeof(g_last_error),
+                  "adapt_precision_search_static: the stream is being captured");
+    return ADAPT_ERR_INVALID_ARG;
+  }
 
   // descriptor block: layer list, candidates (slot = FL, order by (WL, FL, index)), fresh state
   unsigned char* h = g_static_blob;

@@ -204,6 +204,7 @@ search_direct_kernel(const SearchParams p) {
     }
     __syncthreads();
     if (threadIdx.x < kMaxFl + 2) s_zlevel[threadIdx.x] = 0;
+    __syncthreads();             // the next layer's first atomics must find the cleared classes
     ++l;
     while (l < p.n_layers && p.layers[l + 1].tile_begin <= t) ++l;
   }

@@ -105,6 +105,22 @@ def test_many_layers_with_empty_and_degenerate_ones(B):
         assert not (best[1][3] & B.FLAG_DEGENERATE)
 
 
+def test_thousands_of_small_layers_share_ctas(B):
+    """More layers than the direct kernel has CTAs: every CTA walks several layers in a row and
+    must hand each one clean private counters (round-to-nearest-even zero classes included)."""
+    rng = np.random.default_rng(4242)
+    sizes = rng.integers(1, 1500, 3000)
+    xs = []
+    for l, n in enumerate(sizes):
+        x = (rng.standard_normal(n) * 2.0 ** rng.integers(-12, 2)).astype(np.float32)
+        x[rng.random(n) < 0.2] = 0.0
+        xs.append(x)
+    wl, fl = W.candidate_grid([4, 9, 14])
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        G.run_and_compare(B, xs, wl, fl, 32, round_mode=mode, seed=21, where=f"3000 layers mode={mode}",
+                          algorithms=(0, 2))
+
+
 def test_options_eps_pseudocount_base_and_grid_order(B):
     rng = np.random.default_rng(3)
     xs = [(rng.laplace(0, 0.02, 20000)).astype(np.float32),
