@@ -58,6 +58,8 @@ def parse_args():
                     help="profiling aid: override the workload's rounding mode")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the blocks on the other configs and the other value classes")
     return ap.parse_args()
 
 
@@ -92,15 +94,27 @@ class ClockSampler:
     def stop(self, t0: float, t1: float):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        out = self.window(t0, t1)
+        self.close()
+        return out
+
+    def close(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+            self.proc = None
+
+    def window(self, t0: float, t1: float):
+        """Summary of the samples that fall inside [t0, t1] (the sampler keeps running)."""
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         time.sleep(0.12)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
         sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for stamp, ln in self.lines:
+        for stamp, ln in list(self.lines):
             if not (t0 <= stamp <= t1 + 0.06):     # a sample is read up to one period late
                 continue
             f = [t.strip() for t in ln.split(",")]
@@ -399,6 +413,113 @@ def run_formats(args):
     return 0
 
 
+def _timed_steps(torch, step, steps, flush):
+    """Per-step CUDA-event times (ms) of `steps` calls of step(), L2 flushed before each when a
+    flush buffer is given (the flush lies outside the events)."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(steps)]
+    for a, b in evs:
+        if flush is not None:
+            flush.zero_()
+        a.record()
+        step()
+        b.record()
+    torch.cuda.synchronize()
+    return [a.elapsed_time(b) for a, b in evs]
+
+
+def workloads_block(torch, B, W, dev, sampler, peak, names, steps=30):
+    """The paper's own workload shapes, device-resident, the library's per-kernel events OFF:
+    median step time over L2-flushed steps, launches per step, and the time the step's
+    algorithmic HBM traffic needs at the copy rate (one 4 B/element read for the search - the
+    second read can come from L2 for sets that fit it - plus 8 B/element for the quantize)."""
+    out = {}
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    for name in names:
+        w = W.WORKLOADS[name]
+        wl, fl = w.grid()
+        grid = B.Grid(wl, fl)
+        xs = [torch.from_numpy(x).to(dev) for x in W.generate(w)]
+        lens = [x.numel() for x in xs]
+        total = sum(lens)
+        codes = [torch.empty(n, dtype=torch.int32, device=dev) for n in lens]
+        ws = torch.empty(B.adapt_search_workspace_bytes(lens, grid, w.n_bins), dtype=torch.uint8, device=dev)
+        res = B.SearchResult(torch.empty((len(xs), len(grid)), dtype=torch.float64, device=dev),
+                             torch.empty((len(xs), len(grid)), dtype=torch.int64, device=dev),
+                             torch.empty((len(xs), 4), dtype=torch.int32, device=dev))
+
+        def step():
+            B.adapt_precision_search_ex(xs, grid, w.n_bins, round_mode=w.round_mode, seed=w.seed,
+                                        workspace=ws, out=res)
+            B.adapt_quantize_selected_batch(xs, res.best, w.round_mode, w.seed, 0, codes_out=codes)
+
+        for _ in range(5):
+            step()
+        torch.cuda.synchronize()
+        n0 = B.adapt_kernel_launch_count()
+        t0 = time.time()
+        ms = _timed_steps(torch, step, steps, flush)
+        # keep the region long enough for the clock sampler to see it
+        while time.time() - t0 < 0.35:
+            ms += _timed_steps(torch, step, steps, flush)
+        t1 = time.time()
+        launches = (B.adapt_kernel_launch_count() - n0) / len(ms)
+        med = statistics.median(ms)
+        bound_ms = 12.0 * total / (peak * 1e9) * 1e3
+        out[name] = {"ms_per_step": med, "ms_min": min(ms), "steps": len(ms),
+                     "launches_per_step": launches, "elements": total, "layers": len(xs),
+                     "candidates": len(grid), "n_bins": w.n_bins,
+                     "round_mode": "rne" if w.round_mode == 0 else "stochastic",
+                     "element_candidates_per_s": total * len(grid) / (med * 1e-3),
+                     "hbm_bound_ms": bound_ms, "ratio_to_hbm_bound": med / bound_ms,
+                     "clocks": sampler.window(t0, t1)}
+        del xs, codes, ws, res
+    del flush
+    return out
+
+
+def distributions_block(torch, B, W, dev, sampler, peak, log2_n=28, steps=8):
+    """The fused search kernel alone (library events around its launch) on single tensors of
+    2^log2_n elements of other value classes, full 527-candidate grid, round-to-nearest-even,
+    at 2048 and 512 bins: GB/s over the 4 B/element it must read, and the fraction of the peak."""
+    out = {}
+    n = 1 << log2_n
+    wl, fl = W.candidate_grid(range(2, 33))
+    grid = B.Grid(wl, fl)
+    res = B.SearchResult(torch.empty((1, len(grid)), dtype=torch.float64, device=dev),
+                         torch.empty((1, len(grid)), dtype=torch.int64, device=dev),
+                         torch.empty((1, 4), dtype=torch.int32, device=dev))
+    ws = torch.empty(B.adapt_search_workspace_bytes([n], grid, 2048), dtype=torch.uint8, device=dev)
+    for name, spec in W.distribution_sweep(n):
+        x = torch.from_numpy(W.generate_layer(spec, 11, 0)).to(dev)
+        for n_bins in (2048, 512):
+            def step():
+                B.adapt_precision_search_ex([x], grid, n_bins, workspace=ws, out=res)
+            for _ in range(3):
+                step()
+            torch.cuda.synchronize()
+            B.adapt_kernel_times(reset=True)
+            B.adapt_kernel_timing(True)
+            t0 = time.time()
+            k = 0
+            while k < steps or time.time() - t0 < 0.35:
+                step()
+                k += 1
+            torch.cuda.synchronize()
+            t1 = time.time()
+            B.adapt_kernel_timing(False)
+            kt = B.adapt_kernel_times(reset=True)
+            ms_k, n_k = kt["search"]
+            if not n_k:
+                ms_k, n_k = kt["search_direct"]
+            ms = ms_k / n_k
+            gbs = 4.0 * n / (ms * 1e-3) / 1e9
+            out[f"{name}/{n_bins}"] = {"search_kernel_ms": ms, "gbs": gbs, "frac": gbs / peak,
+                                       "launches": n_k, "clocks": sampler.window(t0, t1)}
+        del x
+    return out
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -487,7 +608,7 @@ def main():
         del flush
     t_region1 = time.time()
     S.barrier()
-    clocks = sampler.stop(t_region0, t_region1)
+    clocks = sampler.window(t_region0, t_region1)
     launches = B.adapt_kernel_launch_count() - launches0
     B.adapt_kernel_timing(False)
     ktimes = B.adapt_kernel_times(reset=True)
@@ -557,6 +678,16 @@ def main():
                "api": "adapt_precision_switch_host (pinned host buffers in, results and codes out)"}
         del host_codes
 
+    # ---- the other configs and other value classes (single GPU, default workload only) -----
+    workloads = distributions = None
+    if world == 1 and args.workload == "stress_1g" and not args.elements and not args.no_extra:
+        del codes, ws
+        workloads = workloads_block(torch, B, W, dev, sampler, peak,
+                                    ("single4k", "alexnet_weights", "resnet20_weights_grads",
+                                     "resnet18_weights_acts"))
+        distributions = distributions_block(torch, B, W, dev, sampler, peak)
+    sampler.close()
+
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline = time_oracle(xs_np, wl, fl, w, args.cpu_sample)
@@ -578,6 +709,7 @@ def main():
                 "hbm_gbs_whole_step": (8.0 * total + 8.0 * total) * args.steps / secs_max / 1e9 * world,
                 "roofline": roofline, "kernels": kernels, "e2e": e2e,
                 "cpu_baseline": cpu_baseline, "gpu_launches": int(launches), "clocks": clocks,
+                "workloads": workloads, "distributions": distributions,
                 "library": B.adapt_version()}
         print(json.dumps(line), flush=True)
     if world > 1:

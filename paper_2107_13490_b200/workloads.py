@@ -33,11 +33,16 @@ ROUND_STOCHASTIC = 1
 class LayerSpec:
     name: str
     shape: Tuple[int, ...]
-    dist: str            # "normal" | "laplace" | "relu_normal" | "laplace_outliers"
-    scale: float         # std (normal), b (laplace), std before ReLU (relu_normal)
+    dist: str            # "normal" | "laplace" | "relu_normal" | "laplace_outliers" | "uniform" |
+                         # "fixed_point"
+    scale: float         # std (normal, fixed_point), b (laplace), std before ReLU (relu_normal),
+                         # half width (uniform)
     zero_frac: float = 0.0      # share of positions forced to exactly 0
     outlier_frac: float = 0.0   # share of positions multiplied by outlier_gain
     outlier_gain: float = 1.0
+    word: Tuple[int, int] = (0, 0)   # "fixed_point": the <WL,FL> whose representable values the
+                                     # tensor is drawn from (a layer as a float32 simulation of
+                                     # fixed-point training holds it, Sec. 4.1)
 
     @property
     def numel(self) -> int:
@@ -147,6 +152,19 @@ WORKLOAD_ORDER = ("single4k", "alexnet_weights", "resnet20_weights_grads",
                   "resnet18_weights_acts", "stress_1g")
 
 
+def distribution_sweep(numel: int) -> List[Tuple[str, LayerSpec]]:
+    """Single-layer tensors of other value classes than the stress workload's, for the bench's
+    sweep of the fused kernel: smooth wide distributions, post-ReLU activations, a mostly-zero
+    tensor, and tensors that already lie on a fixed-point grid."""
+    n = (int(numel),)
+    return [("normal", LayerSpec("t", n, "normal", 1.0)),
+            ("uniform", LayerSpec("t", n, "uniform", 1.0)),
+            ("half_zero_relu", LayerSpec("t", n, "relu_normal", 1.0)),
+            ("zeros_90pct", LayerSpec("t", n, "normal", 1.0, zero_frac=0.9)),
+            ("on_grid_8_4", LayerSpec("t", n, "fixed_point", 1.0, word=(8, 4))),
+            ("on_grid_16_12", LayerSpec("t", n, "fixed_point", 1.0, word=(16, 12)))]
+
+
 def scaled(workload: Workload, numel: int, name: Optional[str] = None) -> Workload:
     """A copy of a single-layer workload with a different element count (same
     distribution, grid, bins); for multi-tile parity cases and size sweeps."""
@@ -180,6 +198,15 @@ def _fill_chunk(spec: LayerSpec, seed: int, layer: int, chunk: int, out: np.ndar
                        np.float32(0.0))
     elif spec.dist in ("laplace", "laplace_outliers"):
         v = _laplace(g, n, spec.scale)
+    elif spec.dist == "uniform":
+        v = ((g.random(n, dtype=np.float32) * np.float32(2.0) - np.float32(1.0)) *
+             np.float32(spec.scale))
+    elif spec.dist == "fixed_point":
+        # integer words with a normal spread, kept inside the word, times the word's unit
+        wl, fl = spec.word
+        k = np.rint(g.standard_normal(n, dtype=np.float32) * np.float32(spec.scale * 2.0 ** fl))
+        k = np.clip(k, -(2.0 ** (wl - 1)), 2.0 ** (wl - 1) - 1.0)
+        v = (k * np.float32(2.0 ** -fl)).astype(np.float32)
     else:
         raise ValueError(spec.dist)
     if spec.outlier_frac > 0.0:
