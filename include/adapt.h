@@ -419,7 +419,9 @@ size_t adapt_format_search_workspace_bytes(const int64_t* lens, int n_layers,
  *   best_out     DEVICE int32[n_layers * 4] = {a, b as used, index in formats, flags}
  *   opts         HOST, may be NULL (round to nearest even, eps 0, bits).  Used:
  *                round_mode, layer_base, seed, eps, pseudo_count, log_base, stream,
- *                workspace, workspace_bytes, range_out.  hist_out, n_bins_per_layer
+ *                workspace, workspace_bytes, range_out, hist_out (DEVICE, optional:
+ *                uint32[n_layers][n_formats+1][n_bins], slot 0 = histogram of the float
+ *                tensor, slot c+1 = histogram of format c's values).  n_bins_per_layer
  *                and start_wl_fl must be NULL and algorithm 0: ADAPT_ERR_INVALID_ARG
  *                otherwise.
  * Errors as for adapt_precision_search. */

@@ -526,15 +526,16 @@ def adapt_format_search_workspace_bytes(lens: Sequence[int], formats, n_bins: in
 class FormatResult:
     """Device outputs of adapt_format_search."""
 
-    def __init__(self, kld, zeros, b, best, value_range=None):
+    def __init__(self, kld, zeros, b, best, value_range=None, hist=None):
         self.kld, self.zeros, self.b, self.best, self.range = kld, zeros, b, best, value_range
+        self.hist = hist
 
 
 def adapt_format_search(tensors: Sequence[torch.Tensor], formats, n_bins: int,
                         round_mode: int = ROUND_RNE, seed: int = 0, layer_base: int = 0,
                         eps: float = 0.0, pseudo_count: float = 0.0, log_base: float = 0.0,
                         stream=None, workspace: Optional[torch.Tensor] = None,
-                        want_range: bool = False,
+                        want_range: bool = False, want_hist: bool = False,
                         out: Optional[FormatResult] = None) -> FormatResult:
     """adapt_format_search of adapt.h; formats = sequence of (kind, a, b)."""
     dev = tensors[0].device
@@ -556,6 +557,9 @@ def adapt_format_search(tensors: Sequence[torch.Tensor], formats, n_bins: int,
     if workspace is not None:
         opts.workspace, opts.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     opts.range_out = out.range.data_ptr() if want_range else None
+    if want_hist and out.hist is None:
+        out.hist = torch.zeros((L, Cn + 1, n_bins), dtype=torch.int32, device=dev)
+    opts.hist_out = out.hist.data_ptr() if want_hist else None
     _check(lib().adapt_format_search(ptrs.ctypes.data, lens.ctypes.data, L, C.cast(arr, C.c_void_p),
                                      Cn, n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
                                      out.b.data_ptr(), out.best.data_ptr(), C.byref(opts)),

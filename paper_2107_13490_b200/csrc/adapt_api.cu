@@ -1092,7 +1092,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   if (o.round_mode != ADAPT_ROUND_RNE && o.round_mode != ADAPT_ROUND_STOCHASTIC)
     return ADAPT_ERR_INVALID_ARG;
   if (!(o.eps >= 0.0) || !(o.pseudo_count >= 0.0)) return ADAPT_ERR_INVALID_ARG;
-  if (o.hist_out || o.n_bins_per_layer || o.start_wl_fl || o.algorithm != 0) return ADAPT_ERR_INVALID_ARG;
+  if (o.n_bins_per_layer || o.start_wl_fl || o.algorithm != 0) return ADAPT_ERR_INVALID_ARG;
   const double base = (o.log_base == 0.0) ? 2.0 : o.log_base;
   if (!(base > 0.0) || base == 1.0 || !std::isfinite(base)) return ADAPT_ERR_INVALID_ARG;
   FormatPlan plan;
@@ -1152,7 +1152,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   fp.seed = o.seed;
   fp.alpha = o.pseudo_count; fp.inv_ln_base = 1.0 / std::log(base); fp.eps = o.eps;
   fp.kld_out = a.kld_out; fp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
-  fp.b_out = a.b_out; fp.best_out = a.best_out;
+  fp.b_out = a.b_out; fp.best_out = a.best_out; fp.hist_out = o.hist_out;
 
   // rule groups: few tiles spread the rules over more CTAs, many tiles fill shared memory
   int rpg = static_cast<int>(std::min<size_t>(kMaxRulesPerGroup, budget / per_hist));

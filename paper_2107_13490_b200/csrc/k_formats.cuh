@@ -45,6 +45,7 @@ struct FormatParams {
   long long* zeros_out;         // [n_layers][n_cand]
   int* b_out;                   // optional [n_layers][n_cand]
   int* best_out;                // [n_layers][4]
+  unsigned* hist_out;           // optional [n_layers][n_cand + 1][n_bins]; slot 0 = float tensor
 };
 
 // x * 2^k for -149 <= k <= 149 in two exact steps (a single 2^k may not be a normal float).
@@ -374,6 +375,8 @@ __global__ void __launch_bounds__(kKldThreads) format_kld_kernel(const FormatPar
   __syncthreads();
   double sum = 0.0;
   bool inf = false;
+  unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * B : nullptr;
+  unsigned* H0 = (p.hist_out && c == 0) ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * B : nullptr;
   for (int b = threadIdx.x; b < B; b += kKldThreads) {
     long long pc;
     if (bl == bh) pc = (b == bl) ? n : 0;
@@ -381,6 +384,8 @@ __global__ void __launch_bounds__(kKldThreads) format_kld_kernel(const FormatPar
     else if (b == bl) pc = static_cast<long long>(lo_mass);
     else if (b == bh) pc = static_cast<long long>(hi_mass);
     else pc = U[b];
+    if (H) H[b] = static_cast<unsigned>(pc);
+    if (H0) H0[b] = Q[b];
     sum += kld_term(pc, Q[b], p.alpha, &inf);
   }
   if (inf) s_inf = 1;

@@ -35,8 +35,9 @@ def run_and_compare(B, tensors_np, formats, n_bins, round_mode=0, seed=0, layer_
     dev = to_device(tensors_np)
     res = B.adapt_format_search(dev, formats, n_bins, round_mode=round_mode, seed=seed,
                                 layer_base=layer_base, eps=eps, pseudo_count=pseudo_count,
-                                want_range=True)
+                                want_range=True, want_hist=True)
     torch.cuda.synchronize()
+    hist = res.hist.cpu().numpy().view(np.uint32)
     kld, zeros = res.kld.cpu().numpy(), res.zeros.cpu().numpy()
     b, best, rng = res.b.cpu().numpy(), res.best.cpu().numpy(), res.range.cpu().numpy()
     kind = [f[0] for f in formats]
@@ -51,6 +52,16 @@ def run_and_compare(B, tensors_np, formats, n_bins, round_mode=0, seed=0, layer_
         assert np.array_equal(zeros[l], o["zeros"]), f"{tag}: zero counts differ"
         assert_kld_close(kld[l], o["kld"], tag)
         assert list(best[l]) == list(o["best"]), f"{tag}: best {best[l]} vs {o['best']}"
+        if t.size == 0 or o["nonfinite"]:
+            continue
+        # every format's histogram bin by bin: the oracle's values of the format through the
+        # oracle's own histogram step, on the float tensor's range
+        lo, hi = o["range"]
+        assert np.array_equal(hist[l][0].astype(np.uint64), O.histogram(t, lo, hi, n_bins)), tag
+        for c, (k, fa, _) in enumerate(formats):
+            vals = O.format_quantize(t, k, fa, int(o["b"][c]), round_mode, seed, layer_base + l)
+            assert np.array_equal(hist[l][c + 1].astype(np.uint64), O.histogram(vals, lo, hi, n_bins)), \
+                f"{tag}: histogram of format {formats[c]} differs"
     return res
 
 

@@ -11,7 +11,11 @@ from tests import gpu_util as G
 
 pytestmark = pytest.mark.gpu
 
-SAMPLED = [(2, 1), (6, 3), (8, 4), (12, 9), (16, 15), (20, 6), (32, 27)]
+# low word lengths as training meets them, plus one candidate in every four fraction lengths up to
+# the finest: the keyed kernel treats a level by where it lies against the cells' and the
+# sub-cells' levels, so the sample walks across all of them
+SAMPLED = [(2, 1), (6, 3), (8, 4), (12, 9), (16, 15), (20, 6),
+           (32, 0), (32, 12), (32, 17), (32, 19), (32, 21), (32, 23), (32, 25), (32, 27), (32, 29), (32, 31)]
 
 
 def test_stress_1g_sampled_candidates_and_invariants():
