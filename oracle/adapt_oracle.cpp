@@ -17,6 +17,8 @@
 //   select      - "smallest quantization s.t. KL = 0" (Sec. 3.3; Algorithm 3)
 //   sparsity    - share of non-zero elements (Sec. 3.4 "Inducing Sparsity")
 //   diversity   - gradient diversity of a layer's recent gradients (Sec. 3.3, PushUp)
+//   pushup      - the suggestions s_1, s_2, the strategy and the new <WL,FL> (Sec. 3.3, PushUp;
+//                 the buffer bits of "Dealing with Fixed-Points Limited Range")
 //   formats     - block floating point (Sec. 2.1, 2.2) and floating point (Sec. 7) candidates
 //                 through the same EDF / KL steps
 //
@@ -297,13 +299,6 @@ int adapt_oracle_precision_search(const float* x, int64_t n, uint64_t layer,
 
 // ---- gradient diversity (PushUp's input) ---------------------------------------------
 
-// Gradient diversity of one layer over its last n_grads gradient tensors (Sec. 3.3, the
-// PushUp heuristic, Eq. ourgd / its log form):
-//   delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2 ,
-//   log form = log(delta_s) if 0 < delta_s < inf, else 1.
-// grads[k] points to n fp32 values; everything is accumulated in double, in index order.
-// out = {sum of norms, norm of the sum, delta_s, log form}.  0/0 gives NaN for delta_s
-// (log form 1); x/0 gives +inf (log form 1).
 // Gradient normalisation of Sec. 3.3 ("Dealing with Fixed-Points Limited Range"):
 // g <- g / ||g||_2.  The norm is the square root of the sum of squares taken in double,
 // elements in order; each quotient is formed in double and rounded to float.  A gradient
@@ -316,6 +311,13 @@ void adapt_oracle_normalize_gradient(const float* g, int64_t n, float* out) {
     out[i] = norm > 0.0 ? static_cast<float>(static_cast<double>(g[i]) / norm) : g[i];
 }
 
+// Gradient diversity of one layer over its last n_grads gradient tensors (Sec. 3.3, the
+// PushUp heuristic, Eq. ourgd / its log form):
+//   delta_s = sum_k ||g_k||_2 / || sum_k g_k ||_2 ,
+//   log form = log(delta_s) if 0 < delta_s < inf, else 1.
+// grads[k] points to n fp32 values; everything is accumulated in double, in index order.
+// out = {sum of norms, norm of the sum, delta_s, log form}.  0/0 gives NaN for delta_s
+// (log form 1); x/0 gives +inf (log form 1).
 void adapt_oracle_gradient_diversity(const float* const* grads, int n_grads, int64_t n,
                                      double* out) {
   double sum_norms = 0.0;
@@ -336,6 +338,47 @@ void adapt_oracle_gradient_diversity(const float* const* grads, int n_grads, int
   out[1] = norm_sum;
   out[2] = ds;
   out[3] = (ds > 0.0 && std::isfinite(ds)) ? std::log(ds) : 1.0;
+}
+
+// ---- PushUp: the new <WL,FL> of a layer from its gradient diversity ------------------------
+//
+// Sec. 3.3 "The PushUp Operation" and "Dealing with Fixed-Points Limited Range", in the
+// paper's order and notation.  Inputs: d = the log form of the gradient diversity (above),
+// <WL_min, FL_min> = what PushDown returned, st = the global strategy (0 min, 1 mean, 2 max),
+// buff = the buffer bits.  Steps:
+//   if d > 0:  s_1 = max(ceil(1 / (d - 1)), 1)
+//              s_2 = max(ceil(min(32 d^2 - 1, 32)) - FL_min, 1)
+//              s   = min(s_1, s_2) | ceil(0.5 (s_1 + s_2)) | max(s_1, s_2)      by st
+//   else       s   = 1
+//   FL = min(FL_min + s, 32);   WL = min(max(WL_min, FL) + 1, 32)
+//   FL = min(FL, 32 - buff);    WL = max(min(FL + buff, 32), WL)
+//   FL = min(FL, WL - 1)        (a word keeps at least its sign bit)
+// Readings where the text leaves a choice: the quotient of s_1 is 1 / (d - 1) as printed (its
+// denominator 0 gives the largest suggestion, and every suggestion is capped at 32, beyond
+// which FL cannot move anyway); the real number inside s_2 is rounded up like every other
+// rounding of the paragraph; the second "if" of the text, printed with the same condition as
+// the first, is its complement; d stands for "log delta_s" also where delta_s is 0 or not
+// finite (d = 1 then); the FL inside WL's max is the new one, since with the old one the word
+// could come out shorter than its fraction; the buffer step works on the values just computed.
+// out = {WL, FL, s_1, s_2, s} (s_1 = s_2 = 0 when d <= 0).  All real arithmetic in double.
+void adapt_oracle_pushup(double d, int wl_min, int fl_min, int st, int buff, int32_t* out) {
+  int s1 = 0, s2 = 0, s = 1;
+  if (d > 0.0) {
+    const double q = 1.0 / (d - 1.0);                 // +inf when d == 1
+    s1 = (q >= 32.0) ? 32 : static_cast<int>(std::fmax(std::ceil(q), 1.0));
+    const double w = std::fmin(32.0 * (d * d) - 1.0, 32.0);
+    s2 = std::max(static_cast<int>(std::ceil(w)) - fl_min, 1);
+    s2 = std::min(s2, 32);
+    if (st == 0) s = std::min(s1, s2);
+    else if (st == 1) s = (s1 + s2 + 1) / 2;          // ceil(0.5 (s_1 + s_2)) for integers
+    else s = std::max(s1, s2);
+  }
+  int fl = std::min(fl_min + s, 32);
+  int wl = std::min(std::max(wl_min, fl) + 1, 32);
+  fl = std::min(fl, 32 - buff);
+  wl = std::max(std::min(fl + buff, 32), wl);
+  fl = std::min(fl, wl - 1);
+  out[0] = wl; out[1] = fl; out[2] = s1; out[3] = s2; out[4] = s;
 }
 
 // ---- other number formats through the same EDF / KL machinery ---------------------------

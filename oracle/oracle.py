@@ -81,6 +81,9 @@ def lib():
                                                       C.c_double, C.c_int, C.c_int, C.c_void_p]
             L.adapt_oracle_gradient_diversity.restype = None
             L.adapt_oracle_gradient_diversity.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
+            L.adapt_oracle_pushup.restype = None
+            L.adapt_oracle_pushup.argtypes = [C.c_double, C.c_int, C.c_int, C.c_int, C.c_int,
+                                              C.c_void_p]
             L.adapt_oracle_normalize_gradient.restype = None
             L.adapt_oracle_normalize_gradient.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
             L.adapt_oracle_bfp_scale.restype = C.c_int
@@ -264,6 +267,17 @@ def gradient_diversity(grads):
     ptrs = (C.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
     out = np.zeros(4, dtype=np.float64)
     lib().adapt_oracle_gradient_diversity(ptrs, len(arrs), n, out.ctypes.data)
+    return out
+
+
+STRATEGY_MIN, STRATEGY_MEAN, STRATEGY_MAX = 0, 1, 2
+
+
+def pushup(log_diversity: float, wl_min: int, fl_min: int, strategy: int, buff: int):
+    """PushUp's scalar step for one layer. Returns int32[5] = {WL, FL, s_1, s_2, s}."""
+    out = np.zeros(5, dtype=np.int32)
+    lib().adapt_oracle_pushup(C.c_double(log_diversity), int(wl_min), int(fl_min), int(strategy),
+                              int(buff), out.ctypes.data)
     return out
 
 
