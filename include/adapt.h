@@ -209,6 +209,36 @@ int adapt_requantize_selected_batch(const float* const* tensors, const int64_t* 
 int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int n_layers,
                              int n_grads, double* out, void* stream);
 
+/* Strategies of PushUp (Sec. 3.3, the strategy equation). */
+enum { ADAPT_STRATEGY_MIN = 0, ADAPT_STRATEGY_MEAN = 1, ADAPT_STRATEGY_MAX = 2 };
+
+/* PushUp's scalar step (Sec. 3.3 "The PushUp Operation"; buffer bits of "Dealing with
+ * Fixed-Points Limited Range"): from each layer's gradient diversity and the format that
+ * PushDown found, the format the layer trains on next.  Host arithmetic only - a handful of
+ * scalar operations per layer; nothing is launched and no device is touched.
+ * With d = diversity[l][3] (the log form adapt_gradient_diversity writes) and
+ * <WL_min, FL_min> = best[l][0..1] (as a search writes it):
+ *   d > 0:  s1 = max(ceil(1 / (d - 1)), 1), s2 = max(ceil(min(32 d^2 - 1, 32)) - FL_min, 1),
+ *           s = min(s1, s2) | ceil((s1 + s2) / 2) | max(s1, s2) by strategy;   else s = 1
+ *   FL = min(FL_min + s, 32),   WL = min(max(WL_min, FL) + 1, 32)
+ *   FL = min(FL, 32 - buff),    WL = max(min(FL + buff, 32), WL),   FL = min(FL, WL - 1)
+ * Readings of the printed text: the quotient's denominator is d - 1 as printed (0 gives the
+ * largest suggestion; suggestions are capped at 32, beyond which FL cannot move); the real
+ * number in s2 is rounded up like the paragraph's other roundings; the text's second case,
+ * printed with the first one's condition, is its complement; the FL inside WL's max is the
+ * new one (with the old one the word could come out shorter than its fraction); the buffer
+ * step works on the values just computed; the last step keeps the sign bit when buff is 0.
+ *   diversity      HOST double[n_layers][4], rows as adapt_gradient_diversity writes them
+ *   best           HOST int32[n_layers][4], rows as a search writes them ({wl, fl, ...})
+ *   strategy       ADAPT_STRATEGY_*
+ *   buff           buffer bits, 0..31 (the paper trains with 4 and 8)
+ *   wl_fl_out      HOST int32[n_layers][2] = {WL, FL}: a valid format, WL >= WL_min
+ *   suggestion_out HOST int32[n_layers][3] = {s1, s2, s} or NULL (s1 = s2 = 0 when d <= 0)
+ * ADAPT_ERR_INVALID_ARG (nothing written) for null pointers, n_layers < 1, an unknown strategy,
+ * buff outside 0..31, or a row of best that is not a format (2 <= WL <= 32, 0 <= FL < WL). */
+int adapt_pushup(const double* diversity, const int32_t* best, int n_layers, int strategy,
+                 int buff, int32_t* wl_fl_out, int32_t* suggestion_out);
+
 /* Gradient normalisation of Sec. 3.3 ("Dealing with Fixed-Points Limited
  * Range"): every layer's gradient is divided by its own L2 norm,
  * out[l][i] = grads[l][i] / ||grads[l]||_2, so that an update step cannot move

@@ -32,7 +32,9 @@ EXPORTS = (
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
     "adapt_format_search_workspace_bytes", "adapt_format_search", "adapt_format_quantize",
+    "adapt_pushup",
 )
+STRATEGY_MIN, STRATEGY_MEAN, STRATEGY_MAX = 0, 1, 2
 FMT_FIXED, FMT_BFP, FMT_FLOAT = 0, 1, 2
 MAX_FORMATS = 1024
 STATIC_MAX_LAYERS, STATIC_MAX_BINS, STATIC_MAX_CAND = 8, 512, 1024
@@ -108,6 +110,9 @@ def lib():
         L.adapt_gradient_diversity.restype = C.c_int
         L.adapt_gradient_diversity.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                C.c_void_p]
+        L.adapt_pushup.restype = C.c_int
+        L.adapt_pushup.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                   C.c_void_p]
         L.adapt_search_workspace_bytes.restype = C.c_size_t
         L.adapt_search_workspace_bytes.argtypes = [C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int]
         search_args = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(AdaptGrid), C.c_int, C.c_void_p,
@@ -319,6 +324,25 @@ def adapt_gradient_diversity(grads: Sequence[Sequence[torch.Tensor]],
                                           out.data_ptr(), _stream_handle(stream)),
            "adapt_gradient_diversity")
     return out
+
+
+def adapt_pushup(diversity, best, strategy: int, buff: int, want_suggestions: bool = False):
+    """adapt_pushup of adapt.h.  diversity: [L][4] doubles and best: [L][4] int32, host arrays or
+    tensors (device tensors are copied to the host first: the call is host arithmetic).
+    Returns int32[L][2] = {WL, FL} (and int32[L][3] = {s1, s2, s} when asked for)."""
+    if isinstance(diversity, torch.Tensor):
+        diversity = diversity.detach().cpu().numpy()
+    if isinstance(best, torch.Tensor):
+        best = best.detach().cpu().numpy()
+    div = np.ascontiguousarray(diversity, dtype=np.float64).reshape(-1, 4)
+    bst = np.ascontiguousarray(best, dtype=np.int32).reshape(-1, 4)
+    assert div.shape[0] == bst.shape[0]
+    out = np.zeros((div.shape[0], 2), dtype=np.int32)
+    sug = np.zeros((div.shape[0], 3), dtype=np.int32) if want_suggestions else None
+    _check(lib().adapt_pushup(div.ctypes.data, bst.ctypes.data, div.shape[0], strategy, buff,
+                              out.ctypes.data, sug.ctypes.data if want_suggestions else None),
+           "adapt_pushup")
+    return (out, sug) if want_suggestions else out
 
 
 def adapt_normalize_gradients(grads: Sequence[torch.Tensor],

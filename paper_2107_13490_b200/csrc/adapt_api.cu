@@ -785,6 +785,46 @@ int adapt_gradient_diversity(const float* const* grads, const int64_t* lens, int
   return ADAPT_OK;
 }
 
+int adapt_pushup(const double* diversity, const int32_t* best, int n_layers, int strategy,
+                 int buff, int32_t* wl_fl_out, int32_t* suggestion_out) {
+  if (!diversity || !best || !wl_fl_out || n_layers < 1) return ADAPT_ERR_INVALID_ARG;
+  if (strategy != ADAPT_STRATEGY_MIN && strategy != ADAPT_STRATEGY_MEAN &&
+      strategy != ADAPT_STRATEGY_MAX) return ADAPT_ERR_INVALID_ARG;
+  if (buff < 0 || buff > 31) return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!valid_format(best[4 * l], best[4 * l + 1])) return ADAPT_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l) {
+    const double d = diversity[4 * l + 3];
+    const int wl_min = best[4 * l], fl_min = best[4 * l + 1];
+    int first = 0, second = 0, step = 1;
+    if (d > 0.0) {
+      // first suggestion: the reciprocal of d - 1, rounded up, between 1 and 32
+      const double recip = 1.0 / (d - 1.0);
+      first = 32;
+      if (recip < 32.0) first = recip > 1.0 ? static_cast<int>(std::ceil(recip)) : 1;
+      // second suggestion: 32 d^2 - 1 (at most 32), rounded up, less the present fraction length
+      double target = 32.0 * (d * d) - 1.0;
+      if (target > 32.0) target = 32.0;
+      second = static_cast<int>(std::ceil(target)) - fl_min;
+      second = std::max(1, std::min(second, 32));
+      if (strategy == ADAPT_STRATEGY_MIN) step = std::min(first, second);
+      else if (strategy == ADAPT_STRATEGY_MAX) step = std::max(first, second);
+      else step = (first + second) / 2 + ((first + second) & 1);
+    }
+    int fl = std::min(fl_min + step, 32);
+    int wl = std::min(std::max(wl_min, fl) + 1, 32);
+    if (fl > 32 - buff) fl = 32 - buff;                 // room for the buffer bits
+    wl = std::max(wl, std::min(fl + buff, 32));
+    if (fl > wl - 1) fl = wl - 1;                       // the sign bit stays
+    wl_fl_out[2 * l] = wl;
+    wl_fl_out[2 * l + 1] = fl;
+    if (suggestion_out) {
+      suggestion_out[3 * l] = first; suggestion_out[3 * l + 1] = second; suggestion_out[3 * l + 2] = step;
+    }
+  }
+  return ADAPT_OK;
+}
+
 int adapt_normalize_gradients(const float* const* grads, const int64_t* lens, int n_layers,
                               float* const* out, double* norms_out, void* stream_handle) {
   std::lock_guard<std::mutex> lock(g_mutex);

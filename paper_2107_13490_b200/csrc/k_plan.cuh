@@ -26,8 +26,7 @@
 // This kernel chooses the segments, computes the exact bin edges (smallest
 // float of each bin, by bisection over the float order with the bin function
 // itself), and marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0 of
-// the main segment.  (Bit 29 is left to the counting kernel, which adds it to the word an
-// atomic returns when the element sits exactly on the cell grid.)
+// the main segment.
 #pragma once
 
 #include "common.cuh"
@@ -37,8 +36,7 @@ namespace adapt {
 
 constexpr unsigned kCellEdge = 0x80000000u;
 constexpr unsigned kCellNearZero = 0x40000000u;
-constexpr unsigned kCellOnGrid = 0x20000000u;     // added to a returned word, never stored
-constexpr unsigned kCellCountMask = 0x1FFFFFFFu;
+constexpr unsigned kCellCountMask = 0x3FFFFFFFu;
 constexpr int kPlanThreads = 256;
 
 // Second level under the edge cells.  An element of an edge cell is counted again in one of
@@ -228,7 +226,10 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
       const int biased = max(1, static_cast<int>((__float_as_uint(top) >> 23) & 0xFFu));
       zero_bits = min(zero_bits, 23 - (biased - 127) - P.seg[s].g);
     }
+    // sub-cells need every cell index exact as a float and 2^-(G + kSubBits) a normal float
     P.refined = (P.keyed && P.fast) ? 1 : 0;
+    for (int s = 0; s < 2; ++s)
+      if (P.seg[s].cells > 0 && (P.seg[s].g < -100 || P.seg[s].g > 100)) P.refined = 0;
     P.sub_base = -1;
     if (P.refined) {
       const SegPlan& m0 = P.seg[0];

@@ -121,3 +121,25 @@ def test_gradient_normalisation_matches_the_oracle(B):
     torch.cuda.synchronize()
     for a, b in zip(dev, ref):
         assert torch.equal(a, b)
+
+
+def test_precision_switch_chain_search_diversity_pushup(B):
+    """One precision switch of a few layers as Algorithm 2 strings it together: PushDown (the
+    search on the weights), the gradient diversity over the lookback, PushUp - every stage through
+    the C ABI, the chosen formats against the same chain on the oracle."""
+    import torch
+    shapes = [s for _, s in W._resnet20_shapes()][:6]
+    k = 25
+    wl, fl = W.candidate_grid(range(2, 17))
+    weights = [W.generate_layer(W._kaiming("w", s), 7, l, threads=1) for l, s in enumerate(shapes)]
+    grads = [_grads(int(np.prod(s)), k, 9, l) for l, s in enumerate(shapes)]
+    res = B.adapt_precision_search_ex([torch.from_numpy(w).cuda() for w in weights], B.Grid(wl, fl), 100)
+    div = B.adapt_gradient_diversity([[torch.from_numpy(g).cuda() for g in gl] for gl in grads])
+    torch.cuda.synchronize()
+    ora = O.precision_search(weights, wl, fl, 100)
+    for st in (B.STRATEGY_MIN, B.STRATEGY_MEAN, B.STRATEGY_MAX):
+        got = B.adapt_pushup(div, res.best, st, 4)
+        for l in range(len(shapes)):
+            d = O.gradient_diversity(grads[l])[3]
+            want = O.pushup(d, ora[l]["best"][0], ora[l]["best"][1], st, 4)
+            assert list(got[l]) == list(want[:2]), (l, st)
