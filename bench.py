@@ -56,6 +56,11 @@ def parse_args():
                          "library's own choice; keyed serves round-to-nearest-even only)")
     ap.add_argument("--round-mode", default="workload", choices=["workload", "rne", "stochastic"],
                     help="profiling aid: override the workload's rounding mode")
+    ap.add_argument("--dist", default="",
+                    help="profiling aid: replace the (single-layer) workload's tensor by one of the "
+                         "value classes of the sweep (normal, uniform, half_zero_relu, zeros_90pct, "
+                         "on_grid_8_4, on_grid_16_12); use with --elements")
+    ap.add_argument("--bins", type=int, default=0, help="profiling aid: override the number of bins")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra", action="store_true",
@@ -546,6 +551,13 @@ def main():
     base = W.WORKLOADS[args.workload]
     if args.elements:
         base = W.scaled(base, args.elements)
+    if args.dist:
+        spec = dict(W.distribution_sweep(base.layers[0].numel))[args.dist]
+        base = W.Workload(f"{base.name}_{args.dist}", 11, (spec,), base.wl_values, base.n_bins,
+                          base.round_mode, f"{args.dist} values, {spec.numel} elements")
+    if args.bins:
+        base = W.Workload(base.name, base.seed, base.layers, base.wl_values, args.bins,
+                          base.round_mode, base.description)
     w = S.rank_workload(base, rank)
     round_mode = {"workload": w.round_mode, "rne": 0, "stochastic": 1}[args.round_mode]
     algorithm = {"auto": 0, "keyed": 1, "direct": 2}[args.algorithm]

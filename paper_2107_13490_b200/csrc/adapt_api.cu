@@ -168,7 +168,7 @@ struct Plan {
   int n_layers = 0, n_cand = 0, n_levels = 0, n_bins = 0;
   std::vector<int> slot, order, by_fl, fl_begin;
   // keyed-kernel shared-memory shape
-  int cell_cap = 0, d_levels = 0;
+  int cell_cap = 0, value_cap = 0, d_levels = 0;
   size_t keyed_smem = 0;
   // byte offsets inside the workspace -- descriptor block (uploaded)
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
@@ -227,8 +227,10 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
     p->cell_cap = 0;
   }
   p->keyed_smem = keyed_smem_bytes(p->cell_cap, n_bins, p->d_levels);
+  p->value_cap = p->cell_cap ? keyed_value_cap(p->cell_cap, n_bins, p->d_levels) : 0;
 
-  const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_levels, K = p->cell_cap;
+  // K: row length of the global cell arrays (the largest table a layer may use)
+  const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_levels, K = p->value_cap;
   size_t o = 0;
   p->off_layers = o;  o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
   p->off_keyed = o;   o = align_up(o + sizeof(LayerDesc) * (L + 1), 16);
@@ -375,7 +377,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   std::memcpy(h + plan.off_fl_begin, plan.fl_begin.data(), sizeof(int) * (plan.n_levels + 1));
   if (o.start_wl_fl) std::memcpy(h + plan.off_start, o.start_wl_fl, sizeof(int) * 2 * a.n_layers);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
-  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
 
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
@@ -416,6 +418,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     PlanParams pp;
     pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
     pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = bins_stride; pp.cell_cap = plan.cell_cap;
+    pp.value_cap = plan.value_cap; pp.cell_stride = plan.value_cap;
     pp.fine_ratio = ADAPT_FINE_RATIO;
     const int keyed_grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
     pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
@@ -428,11 +431,11 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     KeyedParams kp;
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
-    kp.qe_hist = d_qe; kp.u_hist = d_u; kp.zeros = d_zeros; kp.zero_class = d_zclass;
+    kp.qe_hist = d_qe; kp.u_hist = d_u; kp.q_hist = d_q; kp.zeros = d_zeros; kp.zero_class = d_zclass;
     kp.sub_count = d_sub;
     kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
     kp.n_bins = bins_stride; kp.n_levels = plan.n_levels;
-    kp.cell_cap = plan.cell_cap; kp.d_levels = plan.d_levels;
+    kp.cell_cap = plan.cell_cap; kp.cell_stride = plan.value_cap; kp.d_levels = plan.d_levels;
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(plan.keyed_smem)));
     {
@@ -447,7 +450,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ep.sub_count = d_sub; ep.edges = d_edges;
     ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
     ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
-    ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_cap = plan.cell_cap;
+    ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_stride = plan.value_cap;
     {
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
       const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / ((plan.n_levels + 1) * nk)));
@@ -1171,7 +1174,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   std::memcpy(h + plan.off_cands, plan.cands.data(), sizeof(FormatCand) * plan.n_cand);
   std::memcpy(h + plan.off_rules, plan.rules.data(), sizeof(FormatRule) * plan.n_rules);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
-  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
   ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
@@ -1422,7 +1425,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   for (int c = 0; c < C; ++c) h_fl_begin[grid->fl[c] + 1] += 1;
   for (int f = 0; f < n_levels; ++f) h_fl_begin[f + 1] += h_fl_begin[f];
   LayerState* hs = reinterpret_cast<LayerState*>(h + kStState);
-  for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
+  for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
 
   // the block is ordinary host memory: the copy is staged before the call returns
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, kStBlobEnd, cudaMemcpyHostToDevice, stream));

@@ -33,6 +33,10 @@ struct LayerState {
   float abs_sum;     // sum of |x| (any summation order; only steers table shapes, never results)
   unsigned zero_count;  // estimate of the exact zeros (the range scan samples one element in
                         // eight; steers the choice of loop form only, never results)
+  unsigned min_lsb;     // over the same sample of non-zero elements: the least (biased exponent +
+                        // trailing zero bits of the 24-bit significand), i.e. 150 + the binary
+                        // exponent of the coarsest grid 2^e all sampled elements lie on; 0xFFFFFFFF
+                        // if none was seen (steers the choice of loop form only, never results)
 };
 
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).

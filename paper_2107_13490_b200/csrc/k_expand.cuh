@@ -30,8 +30,8 @@ struct ExpandParams {
   int n_layers;
   const LayerState* state;
   const LayerPlan* plan;
-  const unsigned* cell_init;   // [layer][cell_cap]
-  const unsigned* cell_count;  // [layer][cell_cap]
+  const unsigned* cell_init;   // [layer][cell_stride]
+  const unsigned* cell_count;  // [layer][cell_stride]
   const unsigned* qe_hist;     // [layer][2][n_bins]
   const unsigned* sub_count;   // [layer][2][n_bins][kSubCells]  sub-cell counts of the edge cells
   const float* edges;          // [layer][n_bins + 1]  exact bin edges
@@ -40,7 +40,7 @@ struct ExpandParams {
   unsigned long long* zeros;   // [layer][n_levels]
   const unsigned long long* zero_class;  // [layer][kZeroClasses]
   const unsigned long long* cell_total;  // [layer] non-zero elements (sum of all cell counts)
-  int n_bins, n_levels, cell_cap;
+  int n_bins, n_levels, cell_stride;
 };
 
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandParams p) {
@@ -59,8 +59,8 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   if (threadIdx.x == 0) s_zero = 0;
   __syncthreads();
 
-  const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
-  const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
+  const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_stride;
+  const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
   unsigned long long zero = 0;
   // the cells are shared by the gridDim.z CTAs of this (level, layer), a contiguous slice each
   const int per_slice = ((P.total_cells + gridDim.z - 1) / gridDim.z + 3) & ~3;
@@ -83,7 +83,17 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
       const int s = (P.seg[1].cells > 0 && i >= P.seg[1].offset) ? 1 : 0;
       const SegPlan& sp = P.seg[s];
       const long long cc = sp.c0 + (i - sp.offset);
-      if (is_q || f >= sp.g) {
+      if (P.value) {
+        // value-keyed layer: the cell is the single value cc * 2^-g (exact: |cc| < 2^22)
+        const float x = __fmul_rn(__ll2float_rn(cc), pow2f(-sp.g));
+        float v = x;
+        if (!is_q) {
+          const float r = rintf(__fmul_rn(x, pow2f(f)));
+          v = __fmul_rn(r, pow2f(-f));
+          if (r == 0.0f) zero += m;
+        }
+        atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+      } else if (is_q || f >= sp.g) {
         if (!(ks[e] & kCellEdge)) {
           const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
           atomicAdd(&s_hist[bin_of(lf, S.lo, S.scale, S.bmax)], m);

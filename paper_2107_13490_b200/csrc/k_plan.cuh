@@ -26,7 +26,8 @@
 // This kernel chooses the segments, computes the exact bin edges (smallest
 // float of each bin, by bisection over the float order with the bin function
 // itself), and marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0 of
-// the main segment.
+// the main segment.  (Bit 29 is left to the counting kernel, which adds it to the word an
+// atomic returns when the element sits exactly on the cell grid.)
 #pragma once
 
 #include "common.cuh"
@@ -36,7 +37,8 @@ namespace adapt {
 
 constexpr unsigned kCellEdge = 0x80000000u;
 constexpr unsigned kCellNearZero = 0x40000000u;
-constexpr unsigned kCellCountMask = 0x3FFFFFFFu;
+constexpr unsigned kCellOnGrid = 0x20000000u;     // added to a returned word, never stored
+constexpr unsigned kCellCountMask = 0x1FFFFFFFu;
 constexpr int kPlanThreads = 256;
 
 // Second level under the edge cells.  An element of an edge cell is counted again in one of
@@ -94,6 +96,9 @@ struct LayerPlan {
                     // start in number more than kSubSharedIds (its sub-cell counts then go
                     // straight to global memory like the auxiliary segment's)
   unsigned grid_mul;   // 2^(32 - bits of grid_mask): x's bit pattern times this is 0 exactly when those bits are
+  int value;        // 1 if the table is keyed by the element's value itself: the layer (as sampled by
+                    // the range scan) lies on a grid 2^-g whose points between its extremes fit
+                    // the table, so seg[0] has one cell per grid point and no cell has marks
 };
 
 // A float x = M 2^(E-23) (M its 24-bit significand) lies on the grid of level G exactly when
@@ -117,9 +122,11 @@ struct PlanParams {
   const LayerState* state;   // indexed by LayerDesc::index
   LayerPlan* plan;           // indexed by LayerDesc::index
   float* edges;              // [all layers][n_bins + 1] (n_bins = the stride below)
-  unsigned* cell_init;       // [all layers][cell_cap]
+  unsigned* cell_init;       // [all layers][cell_stride]
   int n_bins;                // stride of the per-bin arrays (the largest layer's bins)
-  int cell_cap;              // table entries per layer (memory stride and upper limit)
+  int cell_cap;              // table entries a layer may use
+  int value_cap;             // ... when it is keyed by value (its table may run over the others)
+  int cell_stride;           // row length of cell_init
   int fine_ratio;            // stop refining once a bin holds this many cells
   long long elems_per_cta;   // elements one CTA of the keyed kernel processes
 };
@@ -226,10 +233,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
       const int biased = max(1, static_cast<int>((__float_as_uint(top) >> 23) & 0xFFu));
       zero_bits = min(zero_bits, 23 - (biased - 127) - P.seg[s].g);
     }
-    // sub-cells need every cell index exact as a float and 2^-(G + kSubBits) a normal float
     P.refined = (P.keyed && P.fast) ? 1 : 0;
-    for (int s = 0; s < 2; ++s)
-      if (P.seg[s].cells > 0 && (P.seg[s].g < -100 || P.seg[s].g > 100)) P.refined = 0;
     P.sub_base = -1;
     if (P.refined) {
       const SegPlan& m0 = P.seg[0];
@@ -244,6 +248,37 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     // zeros handled one by one cost about as much as edge elements: fine below one in 2048
     P.dense = (kDenseZeroRatio > 0 && P.masked && S.lo <= 0.0f && S.hi >= 0.0f &&
                static_cast<long long>(S.zero_count) * kDenseZeroRatio <= L.n) ? 1 : 0;
+    // A layer that already lies on a fixed-point grid (a layer after its re-quantisation: the
+    // float32 simulation of Sec. 4.1 keeps such tensors) is keyed by value when its grid points
+    // fit the table: cell i is the single value (c0 + i) 2^-g, every level's rounded value, bin
+    // and zero count is an exact function of the cell, and no element is ever on a boundary.
+    // The grid comes from a sample; the counting loop checks every element against it.
+    P.value = 0;
+    if (P.keyed && S.min_lsb != 0xFFFFFFFFu) {
+      const int g = 150 - static_cast<int>(S.min_lsb);
+      if (g >= -100 && g <= 100) {
+        const double span = ldexp(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
+        const double far = ldexp(static_cast<double>(amax), g);
+        if (span + 3.0 <= static_cast<double>(p.value_cap) && far < 4.0e6) {
+          SegPlan v;
+          v.g = g;
+          v.c0 = floor_scaled(S.lo, g) - 1;
+          v.cells = static_cast<int>(floor_scaled(S.hi, g) - v.c0 + 1);
+          v.fs = g > 0 ? g : 0;
+          v.offset = 0;
+          v.two_g = pow2f(g);
+          v.c0f = static_cast<float>(v.c0 + 1);
+          v.magic = 12582912.0f - static_cast<float>(v.c0);
+          v.pad_ = 0;
+          P.seg[0] = v;
+          P.seg[1].cells = 0; P.seg[1].offset = v.cells;
+          P.radius = __int_as_float(0x7f800000);
+          P.total_cells = v.cells;
+          P.fast = 1; P.masked = 0; P.dense = 0; P.refined = 0; P.sub_base = -1;
+          P.value = 1;
+        }
+      }
+    }
     s_plan = P;
     if (blockIdx.y == 0) p.plan[l] = P;   // every CTA of the layer derives the same plan
   }
@@ -273,7 +308,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   }
 
   // cell marks, both segments
-  unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
+  unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
   for (int i = first; i < P.total_cells; i += stride) {
     const int s = (i >= P.seg[1].offset && P.seg[1].cells > 0) ? 1 : 0;
     const SegPlan& sp = P.seg[s];
@@ -283,7 +318,7 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     unsigned mark = 0;
     if (bin_of(lf, S.lo, S.scale, S.bmax) != bin_of(rf, S.lo, S.scale, S.bmax)) mark |= kCellEdge;
     if (s == 0 && (cc == 0 || cc == -1)) mark |= kCellNearZero;
-    init[i] = mark;
+    init[i] = P.value ? 0u : mark;
   }
 }
 

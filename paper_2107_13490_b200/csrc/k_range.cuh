@@ -26,7 +26,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
 
   __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
   __shared__ float s_abs[kRangeThreads / 32];
-  __shared__ unsigned s_zero[kRangeThreads / 32];
+  __shared__ unsigned s_zero[kRangeThreads / 32], s_lsb[kRangeThreads / 32];
   int l = layer_of_tile(layers, n_layers, t);
 
   while (t < t_end) {
@@ -38,7 +38,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
     float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
     unsigned flags = 0;
     float asum = 0.0f;
-    unsigned nzero = 0;
+    unsigned nzero = 0, lsb = 0xFFFFFFFFu;
     for (; t < layer_tiles_end; ++t) {
       const long long j_tile = (t - L.tile_begin) * kTile;
       constexpr int kQ = kTile / 4 / kRangeThreads;
@@ -73,7 +73,13 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
             vmin = fminf(vmin, v[q][k]);
             vmax = fmaxf(vmax, v[q][k]);
             asum += a;
-            if (q == 0) nzero += (a == 0.0f) ? 1u : 0u;   // one quad in kQ: a sample is enough
+            if (q == 0) {                                  // one quad in kQ: a sample is enough
+              nzero += (a == 0.0f) ? 1u : 0u;
+              // position of the element's lowest set significand bit (hidden bit included)
+              const unsigned bits = __float_as_uint(v[q][k]);
+              const unsigned at = ((bits >> 23) & 0xFFu) + static_cast<unsigned>(__ffs(bits | 0x00800000u) - 1);
+              if (a != 0.0f) lsb = min(lsb, at);
+            }
           }
         }
       }
@@ -88,20 +94,22 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
       flags |= __shfl_xor_sync(0xffffffffu, flags, o);
       asum += __shfl_xor_sync(0xffffffffu, asum, o);
       nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
+      lsb = min(lsb, __shfl_xor_sync(0xffffffffu, lsb, o));
     }
     const int w = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; s_zero[w] = nzero; }
+    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; s_zero[w] = nzero; s_lsb[w] = lsb; }
     __syncthreads();
     if (threadIdx.x == 0) {
       for (int i = 1; i < kRangeThreads / 32; ++i) {
         kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
-        asum += s_abs[i]; nzero += s_zero[i];
+        asum += s_abs[i]; nzero += s_zero[i]; lsb = min(lsb, s_lsb[i]);
       }
       atomicMin(&state[L.index].min_key, kmin);
       atomicMax(&state[L.index].max_key, kmax);
       if (flags) atomicOr(&state[L.index].flags, flags);
       if (asum == asum && asum < 3.0e38f) atomicAdd(&state[L.index].abs_sum, asum);
       if (nzero) atomicAdd(&state[L.index].zero_count, nzero * static_cast<unsigned>(kTile / 4 / kRangeThreads));
+      if (lsb != 0xFFFFFFFFu) atomicMin(&state[L.index].min_lsb, lsb);
     }
     __syncthreads();
     ++l;

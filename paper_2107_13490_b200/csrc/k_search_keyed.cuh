@@ -3,33 +3,33 @@
 // common path.  See k_plan.cuh for the cell decomposition this relies on.
 //
 // Per element x != 0:   pos = table position of x's cell;  old = atomicAdd(cell[pos], 1)
-// An element that sits exactly on the cell grid is settled BEFORE its atomic: it is counted in
-// the cell to its left or right according to the parity rule of grid_point_goes_left, which
-// makes every coarse rounding tie come out even.  (Tensors that already lie on a fixed-point
-// grid - a layer after its re-quantisation - consist of such elements only.)
-// The returned word carries the cell's marks in its top bits:
-//   bit 30 (cell -1 / 0 of the main segment) or bit 31 (edge cell): the element goes to a
-//          per-warp queue that the warp drains 32 entries at a time:
+// The returned word carries the cell's marks in its top bits, and bit 29 is added to it when
+// the element sits exactly on the cell grid:
+//   bit 30 (cell -1 / 0 of the main segment), bit 31 (edge cell) or bit 29: the element goes
+//          to a per-warp queue that the warp drains 32 entries at a time:
 //            cell -1 / 0: the element is added to the class counter "highest level at
 //              which it still rounds to zero";
-//            edge cell: the element is counted once more in a sub-cell of its cell; only when
-//              the sub-cell itself holds a bin edge does it join a second per-warp queue, whose
-//              full groups of 32 run the level loop: b0 = bin(x) into the segment's
-//              edge-element histogram, then only the fine levels f whose half quantum can
-//              reach one of the bin's edges are evaluated; a level is recorded only if its
+//            edge entry: b0 = bin(x) into the segment's edge-element histogram,
+//              then only the fine levels f whose half quantum can reach one of
+//              the bin's edges are evaluated; a level is recorded only if its
 //              bin differs from b0 (-1 at b0, +1 at the new bin).
+// An element exactly on the cell grid is counted in the cell to its left or right according to
+// the parity rule of grid_point_goes_left (its handler moves the count when it belongs left),
+// which makes every coarse rounding tie come out even.
 // Exact zeros are sent to per-lane dummy slots (their number is the layer size
-// minus the sum of the cell counts).
+// minus the sum of the cell counts).  A dummy slot starts with all three top bits set; zero is
+// on every grid, so the added bit 29 wraps the returned word around to a plain small count.
 // Everything else about an element - the float histogram, all coarse levels, all fine levels
 // of interior cells - is derived from the cell counts by the expand kernel.
 //
 // Four forms of the counting loop, chosen per layer by the plan (same results, different cost):
 //   general  range far from zero (cell indices of 2^22 and more): difference to the first cell first;
 //   fast     magic-constant index, grid point = "round-down equals round-up" (two more FMAs);
-//   masked   magic-constant index, grid-point candidates = "the low significand bits that every
-//            grid point of the layer has zero are zero" (a superset, tested exactly only then);
-//   dense    as masked, for layers with (almost) no exact zeros: no zero test; a zero lands in
-//            the marked cell [0, 2^-G) and its handler takes it out again.
+//   masked   magic-constant index, grid-point flag = "the low significand bits that every grid
+//            point of the layer has zero are zero" (a superset, settled exactly by the handler);
+//   dense    as masked, for layers with (almost) no exact zeros: no zero test, no flag arithmetic
+//            on the returned word; a zero lands in the marked cell [0, 2^-G) and its handler
+//            takes it out again.
 //
 // One CTA of 1024 threads per SM owns (almost) all of the SM's shared memory
 // for its tables; each thread handles 16 elements (four 128-bit loads, issued
@@ -52,7 +52,6 @@ constexpr int kKeyedWarps = kKeyedThreads / 32;
 constexpr int kKeyedQuads = 4;                                  // 128-bit loads per thread per tile
 constexpr int kKeyedTile = kKeyedThreads * kKeyedQuads * 4;     // 16384 elements
 constexpr int kQueueCap = 160;      // per-warp queue entries: under 32 left over + at most 128 from one quad
-constexpr int kQueue2Cap = 64;      // second per-warp queue (level loop): under 32 left over + one group of 32
 constexpr int kZeroClasses = 34;    // class k+1, k = highest zero level in -1..32
 constexpr int kDummySlots = 32;     // where the atomics of exact zeros land (one per lane)
 constexpr int kKeyedPrefetchTiles = ADAPT_KEYED_PF_DIST;   // L2 prefetch distance in tiles (0: none)
@@ -64,17 +63,20 @@ struct KeyedParams {
   const LayerState* state;     // by LayerDesc::index
   const LayerPlan* plan;       // by LayerDesc::index
   const float* edges;          // [layer][n_bins + 1]
-  const unsigned* cell_init;   // [layer][cell_cap]
-  unsigned* cell_count;        // [layer][cell_cap]      global cell counts
+  const unsigned* cell_init;   // [layer][cell_stride]
+  unsigned* cell_count;        // [layer][cell_stride]   global cell counts
   unsigned* qe_hist;           // [layer][2][n_bins]     float histogram of the edge elements, per segment
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
+  unsigned* q_hist;            // [layer][n_bins]  float histogram (value-keyed layers: stray elements)
   unsigned* sub_count;         // [layer][2][n_bins][kSubCells]  sub-cell counts of the edge cells
   unsigned long long* zeros;   // [layer][n_levels]
   unsigned long long* zero_class;  // [layer][kZeroClasses]
   unsigned long long* cell_total;  // [layer] sum of all cell counts = non-zero elements
   int n_bins;
   int n_levels;                // levels 0..n_levels-1 are wanted
-  int cell_cap;
+  int cell_cap;                // table entries a layer may use (the other tables follow them)
+  int cell_stride;             // row length of the global cell arrays: the largest table any
+                               // layer may use, keyed_value_cap() of a value-keyed one
   int d_levels;                // fine levels of the main segment whose corrections stay in shared memory
 };
 
@@ -83,7 +85,16 @@ __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int
                              static_cast<size_t>(d_levels) * n_bins) +
          sizeof(float) * (static_cast<size_t>(n_bins) + 4) +      // the layer's bin edges
          sizeof(unsigned) * kSubSharedIds * kSubCells +          // main segment's sub-cell counts
-         sizeof(float) * kKeyedWarps * (kQueueCap + kQueue2Cap);
+         sizeof(float) * kKeyedWarps * kQueueCap;
+}
+
+// A value-keyed layer needs none of the other tables, so its cells may run over them, up to the
+// queues (its dummy slots come last).
+__host__ __device__ inline int keyed_value_cap(int cell_cap, int n_bins, int d_levels) {
+  const size_t words = static_cast<size_t>(cell_cap) + kDummySlots + n_bins +
+                       static_cast<size_t>(d_levels) * n_bins + (static_cast<size_t>(n_bins) + 4) +
+                       static_cast<size_t>(kSubSharedIds) * kSubCells;
+  return static_cast<int>((words - kDummySlots) & ~static_cast<size_t>(3));
 }
 
 // Everything the special-element handler needs about the current layer (in shared memory).
@@ -107,15 +118,16 @@ struct LayerCtx {
   unsigned grid_mask;
   int masked, dense;
   unsigned grid_mul;
-  int pbias[2];                // fast layers: cell index on the value axis = table position + pbias
   int zero_pos;                // table position of the main segment's cell [0, 2^-G)
   int refined;                 // edge cells have sub-cells
   int fs_edge[2];              // first level the level loop looks at: fs, or the sub-cells' level
-  float inv_two_g[2];          // 2^-G per segment (refined layers: a normal float)
-  float sub_w[2];              // 2^-(G + kSubBits) per segment: width of a sub-cell
+  float sub_two[2];            // 2^(G + kSubBits) per segment
   unsigned* sub;               // global, this layer's [2][n_bins][kSubCells]
   unsigned* sub_s;             // shared [kSubSharedIds][kSubCells]: main segment's, when sub_base >= 0
   int sub_base;
+  int value;                   // value-keyed layer
+  unsigned* q_hist;            // global, this layer's [n_bins]
+  unsigned* stray;             // shared: elements of a value-keyed layer that are off its grid
 };
 
 // An element that sits exactly on its segment's grid (x * 2^G = p, an integer) is a rounding
@@ -129,31 +141,27 @@ __device__ __forceinline__ int grid_point_goes_left(long long p) {
   const long long low = p & -p;
   return (p & (low << 1)) == 0 ? 1 : 0;
 }
-// The same rule on the low 32 bits of p (it looks at the lowest set bit and the bit above it;
-// callers keep |p| below 2^30).
-__device__ __forceinline__ int grid_point_goes_left32(int p) {
-  const int low = p & -p;
-  return (p & (low << 1)) == 0 ? 1 : 0;
-}
 
-// First stage for a queued element (its cell is marked): the zero class of an element next to
-// zero, and for an element of an edge cell its sub-cell count.  Returns whether the element
-// still has to run the level loop (its sub-cell holds a bin edge, or the layer has no
-// sub-cells).  No warp-level primitive inside: any subset of lanes may call it.
-__device__ __noinline__ bool handle_queued(const LayerCtx& c, float x) {
+// Handles one queued element (finite).  No warp-level primitive inside:
+// any subset of lanes may call it.
+__device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
+  const int B = c.n_bins;
   if (x == 0.0f) {
     // only the dense form lets an exact zero through: it was counted in the cell [0, 2^-G),
     // where no zero belongs (zeros are the layer size minus all cell counts)
     atomicSub(&c.cells[c.zero_pos], 1u);
-    return false;
+    return;
   }
   const int s = (fabsf(x) < c.radius) ? 0 : 1;
   const float z = __fmul_rn(x, c.two_g[s]);
   const float cf = floorf(z);
   int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s])) + 1;     // cell index inside the segment
-  // a point of the cell grid was counted in the cell the parity rule gives it
-  const bool moved = (z == cf) && grid_point_goes_left(c.c0[s] + ci);
-  if (moved) ci -= 1;
+  if (z == cf && grid_point_goes_left(c.c0[s] + ci)) {
+    // on the grid and belonging to the left cell: move its count there
+    atomicSub(&c.cells[c.offset[s] + ci], 1u);
+    ci -= 1;
+    atomicAdd(&c.cells[c.offset[s] + ci], 1u);
+  }
   const long long cc = c.c0[s] + ci;
   // ---- cells -1 / 0 of the main segment: the zero class of x --------------------------
   if (s == 0 && (cc == 0 || cc == -1)) {
@@ -163,40 +171,40 @@ __device__ __noinline__ bool handle_queued(const LayerCtx& c, float x) {
     kz = max(-1, min(kz, 32));
     atomicAdd(&c.zclass[kz + 1], 1u);
   }
-  if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return false;
-  if (!c.refined) return true;
-  // ---- edge cell: its sub-cell ----------------------------------------------------------
-  // Refined layers keep every cell index below 2^22 in magnitude, so the cell index is the
-  // float cf (less one if the point moved left), its left end cf * 2^-G is exact, and the
-  // position inside the cell, (z - cf) * 2^kSubBits, is exact too.  A point of the sub-grid goes
-  // left or right by the same parity rule as a point of the cell grid (for a point of both
-  // grids the two decisions agree: the rule does not depend on the scale).
-  const float cfl = moved ? __fsub_rn(cf, 1.0f) : cf;
-  int j = kSubCells - 1;                                    // a point that moved left: last sub-cell
-  if (!moved) {
-    const float fj = __fmul_rn(__fsub_rn(z, cf), static_cast<float>(kSubCells));
-    const float mj = floorf(fj);
-    j = __float2int_rz(mj);
-    if (fj == mj && j != 0) j -= grid_point_goes_left32(static_cast<int>(cc) * kSubCells + j);
+  // ---- edge cell: its sub-cell, float bin, then the fine levels that can still move ---------
+  if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
+  if (c.refined) {
+    // sub-cell index: x * 2^(G + kSubBits) is exact, the cell's first sub-cell index c * 2^kSubBits
+    // is a float (c < 2^22), and the two lie within 2^kSubBits of each other.  A point of the
+    // sub-grid goes left or right by the same parity rule as a point of the cell grid (for a
+    // point of both grids the two decisions agree: the rule does not depend on the scale).
+    const float zs = __fmul_rn(x, c.sub_two[s]);
+    const float cfs = floorf(zs);
+    int j = __float2int_rz(__fsub_rn(cfs, __ll2float_rn(cc * kSubCells)));
+    if (zs == cfs && grid_point_goes_left(cc * kSubCells + j)) j -= 1;
+    j = max(0, min(j, kSubCells - 1));      // always true by construction; keeps the address in the table
+    const long long jj = cc * kSubCells + j;
+    const int g = c.g[s];
+    // left end of the cell (exact: c < 2^22), then the ends of the sub-cell's closed interval,
+    // rounded outwards (c * 2^kSubBits + j can need 27 bits); in float when the powers of two
+    // involved are normal numbers - the same real numbers rounded the same way as in double
+    float lf, l2, r2;
+    if (g >= -120 && g + kSubBits <= 120) {
+      const float w2 = pow2f(-(g + kSubBits));
+      lf = __fmul_rn(__ll2float_rn(cc), pow2f(-g));
+      l2 = __fadd_rd(lf, __fmul_rn(__int2float_rn(j), w2));
+      r2 = __fadd_ru(lf, __fmul_rn(__int2float_rn(j + 1), w2));
+    } else {
+      lf = __double2float_rd(ldexp(static_cast<double>(cc), -g));
+      l2 = __double2float_rd(ldexp(static_cast<double>(jj), -(g + kSubBits)));
+      r2 = __double2float_ru(ldexp(static_cast<double>(jj + 1), -(g + kSubBits)));
+    }
+    const int id = bin_of(lf, c.lo, c.scale, c.bmax);
+    if (s == 0 && c.sub_base >= 0) atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
+    else atomicAdd(&c.sub[(static_cast<size_t>(s) * B + id) * kSubCells + j], 1u);
+    // an interior sub-cell (its closed interval in one bin) settles the element
+    if (bin_of(l2, c.lo, c.scale, c.bmax) == bin_of(r2, c.lo, c.scale, c.bmax)) return;
   }
-  j = max(0, min(j, kSubCells - 1));      // always true by construction; keeps the address in the table
-  const float lf = __fmul_rn(cfl, c.inv_two_g[s]);          // left end of the cell
-  const int id = bin_of(lf, c.lo, c.scale, c.bmax);
-  if (s == 0 && c.sub_base >= 0) atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
-  else atomicAdd(&c.sub[(static_cast<size_t>(s) * c.n_bins + id) * kSubCells + j], 1u);
-  // the ends of the sub-cell's closed interval, rounded outwards (cell index * 2^kSubBits + j can
-  // need 27 bits); an interior sub-cell (its closed interval in one bin) settles the element
-  const float w2 = c.sub_w[s];
-  const float l2 = __fadd_rd(lf, __fmul_rn(__int2float_rn(j), w2));
-  const float r2 = __fadd_ru(lf, __fmul_rn(__int2float_rn(j + 1), w2));
-  return bin_of(l2, c.lo, c.scale, c.bmax) != bin_of(r2, c.lo, c.scale, c.bmax);
-}
-
-// Second stage, for the few elements whose (sub-)cell holds a bin edge: the float bin, then the
-// fine levels that can still move the element across an edge.  No warp-level primitive inside.
-__device__ __noinline__ void level_loop(const LayerCtx& c, float x) {
-  const int B = c.n_bins;
-  const int s = (fabsf(x) < c.radius) ? 0 : 1;
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
   if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
   const float e_lo = c.E[b0], e_hi = c.E[b0 + 1];
@@ -223,6 +231,21 @@ __device__ __noinline__ void level_loop(const LayerCtx& c, float x) {
   }
 }
 
+// A value-keyed layer's element that is NOT on the layer's grid (the grid was taken from a
+// sample): evaluated by itself, every level, straight into the layer's global histograms and
+// zero counts, as the direct form of the kernel would.  No warp-level primitive inside.
+__device__ __noinline__ void handle_stray(const LayerCtx& c, float x) {
+  const int B = c.n_bins;
+  atomicAdd(c.stray, 1u);
+  atomicAdd(&c.q_hist[bin_of(x, c.lo, c.scale, c.bmax)], 1u);
+  for (int f = 0; f < c.n_levels; ++f) {
+    const float r = rintf(__fmul_rn(x, pow2f(f)));
+    const float v = __fmul_rn(r, pow2f(-f));
+    atomicAdd(&c.u_hist[static_cast<size_t>(f) * B + bin_of(v, c.lo, c.scale, c.bmax)], 1u);
+    if (r == 0.0f) atomicAdd(&c.zeros[f], 1ull);
+  }
+}
+
 // The constants one tile needs to place an element in the table.
 struct CellFn {
   float radius;
@@ -233,152 +256,126 @@ struct CellFn {
   unsigned cell_base;           // dense form: shared-memory byte address of position 0, minus 4 * 0x4B400000
 };
 
-// How the counting loop finds an element's table position and its grid points.
+// How the counting loop finds an element's table position and its grid-point flag.
 constexpr int kCellGeneral = 0;   // range far from zero: difference to the first cell formed first
 constexpr int kCellFast = 1;      // magic-constant index, grid point = round-down equals round-up
-constexpr int kCellMasked = 2;    // magic-constant index, grid-point candidates = low significand bits zero
+constexpr int kCellMasked = 2;    // magic-constant index, grid-point flag = low significand bits zero
 constexpr int kCellDense = 3;     // as masked, for layers with (almost) no exact zeros: a zero is
                                   // not steered to a dummy slot but counted in the cell [0, 2^-G),
                                   // which is marked, and taken out again by the element handler
+constexpr int kCellValue = 4;     // value-keyed layer: one cell per grid point, no marks; an element
+                                  // that is off the grid (round-down differs from round-up) is not
+                                  // counted in the table but handled by itself
 
-// Magic-constant forms (all cell indices below 2^22 in magnitude): adding the segment's constant
-// 1.5 * 2^23 - c0 + offset to x * 2^G with round-down leaves the table position in the low
-// mantissa bits of the sum; x is on the cell grid exactly when round-up gives the same sum.
-__device__ __forceinline__ float magic_sum_rd(float x, const CellFn& f) {
-  // both segments' products are written out and one is kept: measured faster than selecting
-  // the scale and the constant first, by compare-and-select or arithmetically
-  return fabsf(x) < f.radius ? __fmaf_rd(x, f.two_g0, f.magic0) : __fmaf_rd(x, f.two_g1, f.magic1);
-}
-__device__ __forceinline__ float magic_sum_ru(float x, const CellFn& f) {
-  return fabsf(x) < f.radius ? __fmaf_ru(x, f.two_g0, f.magic0) : __fmaf_ru(x, f.two_g1, f.magic1);
-}
-
-// Settles the grid points among four elements of a magic-constant form: rd[k] holds the
-// round-down sum of element k; an element exactly on its segment's grid whose parity rule sends
-// it left gets the sum of the cell before (one less in the last place).  Zeros are left alone:
-// they never count in a cell of their own.  c.c0 - c.offset turns a table position into the
-// cell's index on the value axis.
-__device__ __forceinline__ void settle_grid_points(const LayerCtx& c, const CellFn& fn,
-                                                   const float (&v)[4], float (&rd)[4]) {
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const float x = v[k];
-    if (x != 0.0f && magic_sum_ru(x, fn) == rd[k]) {
-      const int s = fabsf(x) < fn.radius ? 0 : 1;
-      const int p = (__float_as_int(rd[k]) - 0x4B400000) + c.pbias[s];
-      if (grid_point_goes_left32(p)) rd[k] = __int_as_float(__float_as_int(rd[k]) - 1);
-    }
-  }
-}
-
-// Phase A of one quad (four consecutive elements held by this thread): the four positions, the
-// rare settling of grid points, then the four atomics issued together.  Returns whether one of
-// the four must be looked at in phase B.
+// Table position of x, and in *grid_bit kCellOnGrid if x lies exactly on the cell grid, else 0.
+// Fast form (all cell indices below 2^22 in magnitude): adding the segment's magic constant
+// 1.5 * 2^23 - c0 + offset to x * 2^G with round-down leaves the position in the low mantissa
+// bits; x is on the grid exactly when round-up gives the same.  General form (range far from
+// zero, one segment): x * 2^G - c0 is formed first - exact, both are close - and the same
+// constant trick is applied to the difference.
+//
+// Masked form: the flag is a cheap superset instead - every grid point of the layer has its
+// low significand bits zero (LayerPlan::grid_mask), so those bits being zero sends the element
+// to its handler, which tests exactly; a zero passes the test too, as it must.
 template <int kMode>
-__device__ __forceinline__ bool keyed_count(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                            const CellFn& fn, const float (&v)[4],
-                                            unsigned (&old)[4]) {
-  unsigned any = 0;
-  if constexpr (kMode == kCellDense) {
-    // dense form: no zero test.  x's bit pattern times grid_mul is 0 exactly when the low
-    // significand bits that every grid point has zero are zero (a zero included, which lands
-    // in the marked cell [0, 2^-G) and is queued)
-    float rd[4];
-    unsigned tmin = 0xFFFFFFFFu;
+__device__ __forceinline__ int cell_position(float x, const CellFn& f, unsigned* grid_bit) {
+  constexpr bool kFast = kMode != kCellGeneral;
+  float rd, ru;
+  if (kMode == kCellMasked) {
+    const bool inner = fabsf(x) < f.radius;
+    rd = inner ? __fmaf_rd(x, f.two_g0, f.magic0) : __fmaf_rd(x, f.two_g1, f.magic1);
+    *grid_bit = (__float_as_uint(x) & f.grid_mask) == 0u ? kCellOnGrid : 0u;
+    return __float_as_int(rd) - 0x4B400000;
+  }
+  if (kFast) {
+    // both segments' products are written out and one is kept: measured faster than selecting
+    // the scale and the constant first, by compare-and-select or arithmetically
+    const bool inner = fabsf(x) < f.radius;
+    rd = inner ? __fmaf_rd(x, f.two_g0, f.magic0) : __fmaf_rd(x, f.two_g1, f.magic1);
+    ru = inner ? __fmaf_ru(x, f.two_g0, f.magic0) : __fmaf_ru(x, f.two_g1, f.magic1);
+  } else {
+    const float t = __fmaf_rn(x, f.two_g0, -f.c0f0);     // x * 2^G - (c0 + 1), exact
+    rd = __fadd_rd(t, 12582913.0f);
+    ru = __fadd_ru(t, 12582913.0f);
+  }
+  // A zero is on every grid: in the fast form rd == ru holds for it by itself; in the general
+  // form (where only padding can be zero) it lies far outside the table and is named here.
+  *grid_bit = (rd == ru || (!kFast && x == 0.0f)) ? kCellOnGrid : 0u;
+  return __float_as_int(rd) - 0x4B400000;
+}
+
+// Phase A of one quad (four consecutive elements held by this thread), no branches: the four
+// atomics are issued together.  Returns whether one of the four must be looked at in phase B.
+template <int kMode>
+__device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, const CellFn& fn,
+                                            const float (&v)[4], unsigned (&old)[4]) {
+  if (kMode == kCellValue) {
+    // x * 2^g is an integer for every element on the grid: round-down and round-up of the sum
+    // with the magic constant agree, and its low mantissa bits are the table position.  Zeros
+    // and stray elements go to the dummy slots; old[k] only says whether element k is a stray.
+    unsigned any = 0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      rd[k] = magic_sum_rd(v[k], fn);
-      tmin = min(tmin, __float_as_uint(v[k]) * fn.grid_mul);
+      const float x = v[k];
+      const float rd = __fmaf_rd(x, fn.two_g0, fn.magic0);
+      const bool stray = __fmaf_ru(x, fn.two_g0, fn.magic0) != rd;
+      const int pos = (x != 0.0f && !stray) ? __float_as_int(rd) - 0x4B400000 : dummy_pos;
+      atomicAdd(&cells[pos], 1u);
+      old[k] = stray ? kCellOnGrid : 0u;
+      any |= old[k];
     }
-    if (tmin == 0u) settle_grid_points(c, fn, v, rd);
+    return any != 0u;
+  }
+  if (kMode == kCellDense) {
+    // dense form: no zero test and no flag arithmetic.  The grid-point test is kept apart
+    // from the returned words: x's bit pattern times grid_mul is 0 exactly when the low
+    // significand bits that every grid point has zero are zero (a zero included, which lands
+    // in the marked cell [0, 2^-G) and is queued anyway).
+    unsigned any = 0, tmin = 0xFFFFFFFFu;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const unsigned addr = __float_as_uint(rd[k]) * 4u + fn.cell_base;
+      const float x = v[k];
+      const bool inner = fabsf(x) < fn.radius;
+      const float rd = inner ? __fmaf_rd(x, fn.two_g0, fn.magic0) : __fmaf_rd(x, fn.two_g1, fn.magic1);
+      const unsigned addr = __float_as_uint(rd) * 4u + fn.cell_base;
       unsigned o;
       asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(o) : "r"(addr) : "memory");
       old[k] = o;
       any |= o;
+      tmin = min(tmin, __float_as_uint(x) * fn.grid_mul);
     }
-    return any >= kCellNearZero;
-  } else if constexpr (kMode == kCellMasked) {
-    float rd[4];
-    bool cand = false;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      rd[k] = magic_sum_rd(v[k], fn);
-      cand = cand || (__float_as_uint(v[k]) & fn.grid_mask) == 0u;
-    }
-    if (cand) settle_grid_points(c, fn, v, rd);
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      // exact zeros go to a dummy slot (slots that are not loaded hold zeros)
-      const int pos = (v[k] != 0.0f) ? __float_as_int(rd[k]) - 0x4B400000 : dummy_pos;
-      const unsigned o = atomicAdd(&cells[pos], 1u);
-      old[k] = o;
-      any |= o;
-    }
-    return any >= kCellNearZero;
-  } else {
+    return any >= kCellOnGrid || tmin == 0u;
+  }
+  // exact zeros go to a dummy slot.  An element on the cell grid gets bit 29 added to its
+  // word and is queued too: its handler may move it one cell to the left.  (Slots that are
+  // not loaded hold zeros.)
+  unsigned any = 0;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const float x = v[k];
-    int pos;
-    if (kMode == kCellFast) {
-      const float rd = magic_sum_rd(x, fn);
-      pos = __float_as_int(rd) - 0x4B400000;
-      if (x != 0.0f && magic_sum_ru(x, fn) == rd)
-        pos -= grid_point_goes_left32(pos + c.pbias[fabsf(x) < fn.radius ? 0 : 1]);
-    } else {
-      // general form (range far from zero, one segment at offset 0): x * 2^G - (c0 + 1) is
-      // formed first - exact, both are close - and the constant trick applied to the difference
-      const float t = __fmaf_rn(x, fn.two_g0, -fn.c0f0);
-      const float rd = __fadd_rd(t, 12582913.0f);
-      pos = __float_as_int(rd) - 0x4B400000;
-      if (x != 0.0f && __fadd_ru(t, 12582913.0f) == rd) pos -= grid_point_goes_left(c.c0[0] + pos);
-    }
+    unsigned grid_bit;
+    int pos = cell_position<kMode>(x, fn, &grid_bit);
     pos = (x != 0.0f) ? pos : dummy_pos;
-    const unsigned o = atomicAdd(&cells[pos], 1u);
+    const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
     old[k] = o;
     any |= o;
   }
-  return any >= kCellNearZero;
-  }
+  return any >= kCellOnGrid;
 }
 
-// One group of the first queue: the first stage for every lane's entry, then the entries that
-// still need the level loop are compacted into the warp's second queue, whose full groups run it.
-// Called by the whole warp (lanes without an entry pass valid = false).
-__device__ __forceinline__ void keyed_drain(const LayerCtx& c, float x, bool valid, float* queue2,
-                                            unsigned* qn2_slot) {
-  const bool again = valid && handle_queued(c, x);
-  const unsigned pm = __ballot_sync(0xffffffffu, again);
-  if (pm) {
-    const unsigned lane = threadIdx.x & 31;
-    unsigned n2 = *qn2_slot;                   // the same in every lane
-    if (again) queue2[n2 + __popc(pm & ((1u << lane) - 1u))] = x;
-    n2 += __popc(pm);
-    __syncwarp();
-    if (n2 >= 32u) {
-      n2 -= 32u;
-      level_loop(c, queue2[n2 + lane]);
-      __syncwarp();
-    }
-    if (lane == 0) *qn2_slot = n2;
-    __syncwarp();
-  }
-}
-
-// Phase B of one quad (rare): elements of marked cells join the warp's queue, which is drained
-// when 32 entries have gathered; the whole warp enters so that the queue position can stay in
-// a register.
+// Phase B of one quad (rare): elements of marked cells and on-grid elements join the warp's
+// queue, which is drained when 32 entries have gathered; the whole warp enters so that the
+// queue position can stay in a register.
+template <int kMode>
 __device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, unsigned& qn,
-                                            float* queue2, unsigned* qn2_slot, const float (&v)[4],
+                                            const CellFn& fn, const float (&v)[4],
                                             const unsigned (&old)[4], bool enter) {
   if (__any_sync(0xffffffffu, enter)) {
     const unsigned lt = (1u << (threadIdx.x & 31)) - 1u;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const bool push = old[k] >= kCellNearZero;
+      bool push = old[k] >= kCellOnGrid;
+      if (kMode == kCellDense) push = push || __float_as_uint(v[k]) * fn.grid_mul == 0u;
       const unsigned pm = __ballot_sync(0xffffffffu, push);
       if (pm) {
         if (push) queue[qn + __popc(pm & lt)] = v[k];
@@ -389,7 +386,8 @@ __device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, uns
       __syncwarp();
       do {
         qn -= 32u;
-        keyed_drain(c, queue[qn + (threadIdx.x & 31)], true, queue2, qn2_slot);
+        if (kMode == kCellValue) handle_stray(c, queue[qn + (threadIdx.x & 31)]);
+        else handle_special(c, queue[qn + (threadIdx.x & 31)]);
       } while (qn >= 32u);
       __syncwarp();
     }
@@ -398,19 +396,18 @@ __device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, uns
 
 template <int kMode>
 __device__ __forceinline__ void keyed_quad(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                           float* queue, unsigned& qn, float* queue2,
-                                           unsigned* qn2_slot, const CellFn& fn, const float (&v)[4]) {
+                                           float* queue, unsigned& qn, const CellFn& fn,
+                                           const float (&v)[4]) {
   unsigned old[4];
-  const bool enter = keyed_count<kMode>(c, cells, dummy_pos, fn, v, old);
-  keyed_queue(c, queue, qn, queue2, qn2_slot, v, old, enter);
+  const bool enter = keyed_count<kMode>(cells, dummy_pos, fn, v, old);
+  keyed_queue<kMode>(c, queue, qn, fn, v, old, enter);
 }
 
 // A ragged tile (the layer's first one when the tensor does not start on a 16-byte boundary, or
 // its last): guarded loads, slots outside the layer hold zeros.
 template <int kMode>
 __device__ __forceinline__ void keyed_tile_ragged(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                                  float* queue, unsigned& qn, float* queue2,
-                                                  unsigned* qn2_slot, const CellFn& fn,
+                                                  float* queue, unsigned& qn, const CellFn& fn,
                                                   const float* base, long long j_tile,
                                                   long long jbeg, long long jend) {
   float v[kKeyedQuads][4];
@@ -421,8 +418,7 @@ __device__ __forceinline__ void keyed_tile_ragged(const LayerCtx& c, unsigned* c
     if (j0 < jend) load_quad(base, j0, jbeg, jend, v[q]);
   }
 #pragma unroll
-  for (int q = 0; q < kKeyedQuads; ++q)
-    keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, queue2, qn2_slot, fn, v[q]);
+  for (int q = 0; q < kKeyedQuads; ++q) keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, fn, v[q]);
 }
 
 __device__ __forceinline__ void load_full_quad(const float4* src, float (&v)[4]) {
@@ -437,8 +433,7 @@ __device__ __forceinline__ void load_full_quad(const float4* src, float (&v)[4])
 // (inlined side by side the four forms spill inside their loops).
 template <int kMode>
 __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, int dummy_pos,
-                                           float* queue, float* queue2, unsigned* qn2_slot,
-                                           const float* base, long long jbeg,
+                                           float* queue, const float* base, long long jbeg,
                                            long long jend, int k0, int k1) {
   // only the constants this form uses are taken into registers
   CellFn fn;
@@ -449,14 +444,12 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
   fn.grid_mul = c.grid_mul;
   fn.cell_base = static_cast<unsigned>(__cvta_generic_to_shared(cells)) - 4u * 0x4B400000u;
   unsigned qn = 0;             // entries in this warp's queue (same in every lane)
-  if ((threadIdx.x & 31) == 0) *qn2_slot = 0;
-  __syncwarp();
   // a ragged tile pads with zeros, which the dense form must not see
   constexpr int kRagged = kMode == kCellDense ? kCellMasked : kMode;
   const int kf0 = max(k0, jbeg > 0 ? 1 : 0);
   const int kf1 = min(k1, static_cast<int>(jend / kKeyedTile));
   if (k0 < kf0)
-    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, queue2, qn2_slot, fn, base,
+    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, fn, base,
                                static_cast<long long>(k0) * kKeyedTile, jbeg, jend);
   if (kf0 < kf1) {
     const float4* src = reinterpret_cast<const float4*>(base + static_cast<long long>(kf0) * kKeyedTile) +
@@ -475,27 +468,24 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
 #pragma unroll
       for (int q = 0; q < kKeyedQuads; ++q) load_full_quad(src + q * kKeyedThreads, v[q]);
 #pragma unroll
-      for (int q = 0; q < kKeyedQuads; ++q)
-        keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, queue2, qn2_slot, fn, v[q]);
+      for (int q = 0; q < kKeyedQuads; ++q) keyed_quad<kMode>(c, cells, dummy_pos, queue, qn, fn, v[q]);
     }
   }
   for (int k = max(kf1, kf0); k < k1; ++k)
-    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, queue2, qn2_slot, fn, base,
+    keyed_tile_ragged<kRagged>(c, cells, dummy_pos, queue, qn, fn, base,
                                static_cast<long long>(k) * kKeyedTile, jbeg, jend);
-  // what is left in the two queues
+  // what is left in the queue
   __syncwarp();
-  const unsigned lane = threadIdx.x & 31;
-  keyed_drain(c, queue[lane], lane < qn, queue2, qn2_slot);
-  __syncwarp();
-  if (lane < *qn2_slot) level_loop(c, queue2[lane]);
-  __syncwarp();
-  if (lane == 0) *qn2_slot = 0;
+  if ((threadIdx.x & 31) < qn) {
+    if (kMode == kCellValue) handle_stray(c, queue[threadIdx.x & 31]);
+    else handle_special(c, queue[threadIdx.x & 31]);
+  }
 }
 
 __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const KeyedParams p) {
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ unsigned s_zclass[kZeroClasses];
-  __shared__ unsigned s_qn2[kKeyedWarps];      // entries in each warp's second queue
+  __shared__ unsigned s_stray;
   __shared__ LayerCtx s_ctx;
 
   unsigned* cells = reinterpret_cast<unsigned*>(s_raw);          // [cell_cap + kDummySlots]
@@ -507,8 +497,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   float* queue = queues + warp * kQueueCap;
-  float* queue2 = queues + kKeyedWarps * kQueueCap + warp * kQueue2Cap;
-  const int dummy_pos = p.cell_cap + lane;
+  const int value_cap = keyed_value_cap(p.cell_cap, p.n_bins, p.d_levels);
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
@@ -537,13 +526,14 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       for (int sg = 0; sg < 2; ++sg) {
         const int gs = P->seg[sg].g + kSubBits;
         c.fs_edge[sg] = P->refined ? max(gs, 0) : P->seg[sg].fs;
-        c.inv_two_g[sg] = P->refined ? pow2f(-P->seg[sg].g) : 1.0f;
-        c.sub_w[sg] = P->refined ? pow2f(-gs) : 1.0f;
-        c.pbias[sg] = static_cast<int>(P->seg[sg].c0) - P->seg[sg].offset;   // used by fast layers only
+        c.sub_two[sg] = P->refined ? pow2f(max(-126, min(gs, 127))) : 1.0f;
       }
       c.sub = p.sub_count + static_cast<size_t>(l) * 2 * p.n_bins * kSubCells;
       c.sub_s = sub_s; c.sub_base = P->refined ? P->sub_base : -1;
       c.grid_mul = P->grid_mul;
+      c.value = P->value;
+      c.q_hist = p.q_hist + static_cast<size_t>(l) * p.n_bins;
+      c.stray = &s_stray;
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
       c.E = edges;
       c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
@@ -563,39 +553,50 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     const int total_cells = c.total_cells;
     const bool masked = c.masked != 0;
     const bool dense = c.dense != 0;
+    const bool by_value = c.value != 0;
+    // where the atomics of exact zeros (and of a value-keyed layer's strays) land: one slot per lane
+    const int dummy_pos = (by_value ? value_cap : p.cell_cap) + lane;
 
     // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
-      const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_cap;
+      const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
       // 128-bit copies, several in flight per thread (the table and its rows are 16-byte aligned,
       // the row has room for the last quad: the table size is a multiple of four)
       const uint4* init4 = reinterpret_cast<const uint4*>(init);
       uint4* cells4 = reinterpret_cast<uint4*>(cells);
       const int n4 = (total_cells + 3) >> 2;
+      if (by_value) {
+        // no marks, and the cells may run over the other tables, which this layer does not use
+        for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = make_uint4(0u, 0u, 0u, 0u);
+      } else {
 #pragma unroll 4
-      for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = __ldg(init4 + i);
-      for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
-      const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
-      for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
+        for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = __ldg(init4 + i);
+        for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
+        const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
+        for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
+        for (int i = threadIdx.x; i < kSubSharedIds * kSubCells; i += kKeyedThreads) sub_s[i] = 0;
+      }
       if (threadIdx.x < kZeroClasses) s_zclass[threadIdx.x] = 0;
-      for (int i = threadIdx.x; i < kSubSharedIds * kSubCells; i += kKeyedThreads) sub_s[i] = 0;
-      if (threadIdx.x < kDummySlots) cells[p.cell_cap + threadIdx.x] = 0;
+      if (threadIdx.x == 0) s_stray = 0;
+      if (threadIdx.x < kDummySlots)
+        cells[dummy_pos - lane + threadIdx.x] = kCellEdge | kCellNearZero | kCellOnGrid;
     }
     __syncthreads();
 
     if (ok) {
       const int k0 = static_cast<int>(t - L.tile_begin), k1 = static_cast<int>(layer_tiles_end - L.tile_begin);
-      if (dense) keyed_segment<kCellDense>(c, cells, dummy_pos, queue, queue2, &s_qn2[warp], base, jbeg, jend, k0, k1);
-      else if (masked) keyed_segment<kCellMasked>(c, cells, dummy_pos, queue, queue2, &s_qn2[warp], base, jbeg, jend, k0, k1);
-      else if (fast) keyed_segment<kCellFast>(c, cells, dummy_pos, queue, queue2, &s_qn2[warp], base, jbeg, jend, k0, k1);
-      else keyed_segment<kCellGeneral>(c, cells, dummy_pos, queue, queue2, &s_qn2[warp], base, jbeg, jend, k0, k1);
+      if (by_value) keyed_segment<kCellValue>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else if (dense) keyed_segment<kCellDense>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else if (masked) keyed_segment<kCellMasked>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else if (fast) keyed_segment<kCellFast>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
+      else keyed_segment<kCellGeneral>(c, cells, dummy_pos, queue, base, jbeg, jend, k0, k1);
     }
     t = layer_tiles_end;
     __syncthreads();
 
     // ---- flush the private tables into the layer's global ones -----------------------
     if (ok) {
-      unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_cap;
+      unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_stride;
       unsigned long long counted = 0;
       for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) {
         const unsigned n = cells[i] & kCellCountMask;
@@ -605,12 +606,13 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) counted += __shfl_xor_sync(0xffffffffu, counted, o);
       if (lane == 0 && counted) atomicAdd(&p.cell_total[l], counted);
+      if (threadIdx.x == 0 && s_stray) atomicAdd(&p.cell_total[l], static_cast<unsigned long long>(s_stray));
       unsigned* gq = p.qe_hist + static_cast<size_t>(l) * 2 * p.n_bins;
-      for (int i = threadIdx.x; i < p.n_bins; i += kKeyedThreads) {
+      for (int i = threadIdx.x; i < (by_value ? 0 : p.n_bins); i += kKeyedThreads) {
         const unsigned n = qe[i];
         if (n) atomicAdd(&gq[i], n);
       }
-      if (c.sub_base >= 0) {
+      if (c.sub_base >= 0 && !by_value) {
         unsigned* gs = c.sub + static_cast<size_t>(c.sub_base) * kSubCells;     // segment 0, id sub_base
         const int room = (p.n_bins - c.sub_base) * kSubCells;
         for (int i = threadIdx.x; i < min(kSubSharedIds * kSubCells, room); i += kKeyedThreads) {
@@ -618,7 +620,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
           if (n) atomicAdd(&gs[i], n);
         }
       }
-      for (int i = threadIdx.x; i < p.n_bins * p.d_levels; i += kKeyedThreads) {
+      for (int i = threadIdx.x; i < (by_value ? 0 : p.n_bins * p.d_levels); i += kKeyedThreads) {
         const int dv = dtab[i];
         if (dv) {
           const int j = i / p.n_bins, b = i - j * p.n_bins;

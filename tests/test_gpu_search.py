@@ -187,6 +187,18 @@ def test_adversarial_value_patterns(B):
     cases["fine_grid_15"] = (fine * 2.0 ** -15 + 2.0 ** -16).astype(np.float32)
     cases["fine_grid_mixed"] = np.where(rng.random(n) < 0.5, fine * 2.0 ** -15,
                                         rng.integers(-(1 << 15), 1 << 15, n) * 2.0 ** -17).astype(np.float32)
+    # tensors on a fixed-point grid (the table is keyed by value), and such tensors with a few
+    # elements off the grid at places the range scan's sample does not look at
+    for name, spec in W.distribution_sweep(n):
+        if name.startswith("on_grid"):
+            cases[name] = W.generate_layer(spec, 5, 0)
+    stray = (rng.integers(-2000, 2000, n) * 2.0 ** -6).astype(np.float32)
+    for at in (700, 1000, 4095, 5000, 20000, n - 1):
+        stray[at] = np.float32(rng.standard_normal() * 3.0)
+    stray[30000] = 0.0
+    cases["on_grid_with_strays"] = stray
+    cases["on_grid_far_from_zero"] = (300.0 + rng.integers(0, 3000, n) * 2.0 ** -3).astype(np.float32)
+    cases["on_grid_negative_powers"] = (rng.integers(-9, 9, n) * 2.0 ** -20).astype(np.float32)
     wl, fl = W.candidate_grid(range(2, 33))
     for name, x in cases.items():
         for n_bins in (100, 2048):
