@@ -16,7 +16,8 @@
  *    pointers, sizes or formats out of range, workspace too small) return
  *    before anything is launched and write nothing.  Errors in the data
  *    (NaN/Inf elements, |x| >= 2^64) cannot be seen by the host without a
- *    device round trip: they are reported per layer in best_out's flag word,
+ *    device round trip: they are reported per layer in best_out's flag word
+ *    (and, when asked for, as a status word per layer in opts->status_out);
  *    the other outputs of that layer are then unspecified (but in bounds).
  *    Nothing traps on the device and no C++ exception crosses this boundary.
  *  - Formats: 2 <= WL <= 32, 0 <= FL <= WL-1 (Sec. 2.1: a WL-bit signed word
@@ -102,6 +103,11 @@ typedef struct adapt_search_opts {
                              -1 if the start is not in the grid).  When NULL,
                              best_out is the lowest admissible format of the
                              whole grid                                          */
+  int32_t* status_out;    /* DEVICE, optional: int32[n_layers], the adapt_status of
+                             each layer's data - ADAPT_OK, ADAPT_ERR_NONFINITE
+                             (NaN/Inf in the layer) or ADAPT_ERR_RANGE
+                             (|x| >= 2^64) - the same facts as the flag bits of
+                             best_out, as one status word per layer              */
 } adapt_search_opts;
 
 /* Forms of the fused quantize / zero-count / histogram kernel.  Both give the
@@ -449,7 +455,7 @@ size_t adapt_format_search_workspace_bytes(const int64_t* lens, int n_layers,
  *   best_out     DEVICE int32[n_layers * 4] = {a, b as used, index in formats, flags}
  *   opts         HOST, may be NULL (round to nearest even, eps 0, bits).  Used:
  *                round_mode, layer_base, seed, eps, pseudo_count, log_base, stream,
- *                workspace, workspace_bytes, range_out, hist_out (DEVICE, optional:
+ *                workspace, workspace_bytes, range_out, status_out, hist_out (DEVICE, optional:
  *                uint32[n_layers][n_formats+1][n_bins], slot 0 = histogram of the float
  *                tensor, slot c+1 = histogram of format c's values).  n_bins_per_layer
  *                and start_wl_fl must be NULL and algorithm 0: ADAPT_ERR_INVALID_ARG

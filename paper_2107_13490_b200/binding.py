@@ -53,7 +53,8 @@ class AdaptSearchOpts(C.Structure):
                 ("eps", C.c_double), ("pseudo_count", C.c_double), ("log_base", C.c_double),
                 ("stream", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
                 ("hist_out", C.c_void_p), ("range_out", C.c_void_p), ("algorithm", C.c_int32),
-                ("n_bins_per_layer", C.c_void_p), ("start_wl_fl", C.c_void_p)]
+                ("n_bins_per_layer", C.c_void_p), ("start_wl_fl", C.c_void_p),
+                ("status_out", C.c_void_p)]
 
 
 class AdaptFormat(C.Structure):
@@ -373,8 +374,9 @@ def adapt_search_workspace_bytes(lens: Sequence[int], grid: Grid, n_bins: int) -
 class SearchResult:
     """Device outputs of one search call (torch tensors on the input device)."""
 
-    def __init__(self, kld, zeros, best, hist=None, value_range=None):
+    def __init__(self, kld, zeros, best, hist=None, value_range=None, status=None):
         self.kld, self.zeros, self.best, self.hist, self.range = kld, zeros, best, hist, value_range
+        self.status = status
 
 
 def _marshal_tensors(tensors):
@@ -432,7 +434,8 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
                               out: Optional[SearchResult] = None,
                               algorithm: int = ALGO_AUTO,
                               n_bins_per_layer: Optional[Sequence[int]] = None,
-                              start_wl_fl: Optional[Sequence[Sequence[int]]] = None) -> SearchResult:
+                              start_wl_fl: Optional[Sequence[Sequence[int]]] = None,
+                              want_status: bool = False) -> SearchResult:
     dev = tensors[0].device
     assert all(t.is_cuda for t in tensors)
     ptrs, lens = _marshal_tensors(tensors)
@@ -462,6 +465,9 @@ def adapt_precision_search_ex(tensors: Sequence[torch.Tensor], grid: Grid, n_bin
     o.algorithm = algorithm
     o.n_bins_per_layer = per_layer.ctypes.data if per_layer is not None else None
     o.start_wl_fl = start.ctypes.data if start is not None else None
+    if want_status and out.status is None:
+        out.status = torch.full((L,), -1, dtype=torch.int32, device=dev)
+    o.status_out = out.status.data_ptr() if want_status else None
     _check(lib().adapt_precision_search_ex(ptrs.ctypes.data, lens.ctypes.data, L, C.byref(grid.c),
                                            n_bins, out.kld.data_ptr(), out.zeros.data_ptr(),
                                            out.best.data_ptr(), C.byref(o)),

@@ -174,12 +174,14 @@ struct Plan {
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
          off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_start = 0, off_state = 0, blob_bytes = 0;
   // written by kernels, not cleared
-  size_t off_plan = 0, off_edges = 0, off_cell_init = 0;
+  size_t off_plan = 0, off_edges = 0;
   // accumulators (cleared every call)
   size_t off_sub = 0, off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
          off_zclass = 0, off_nzero = 0, accum_begin = 0, accum_bytes = 0;
   size_t total = 0;
 };
+
+static_assert(ADAPT_ERR_NONFINITE == 2 && ADAPT_ERR_RANGE == 3, "the kernels write these codes into status_out");
 
 bool valid_format(int wl, int fl) { return wl >= 2 && wl <= 32 && fl >= 0 && fl < wl; }
 
@@ -246,7 +248,6 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->blob_bytes = o;
   p->off_plan = o;      o = align_up(o + sizeof(LayerPlan) * L, 256);
   p->off_edges = o;     o = align_up(o + sizeof(float) * L * (B + 1), 256);
-  p->off_cell_init = o; o = align_up(o + sizeof(unsigned) * L * K, 256);
   p->accum_begin = o;
   p->off_zeros = o;   o = align_up(o + sizeof(unsigned long long) * L * F, 256);
   p->off_zclass = o;  o = align_up(o + sizeof(unsigned long long) * L * kZeroClasses, 256);
@@ -266,6 +267,19 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
 // ---- search driver ----------------------------------------------------------------
 
 namespace {
+
+// Grid of the range scan, and for every layer of its list the number of CTAs that hold tiles of
+// the layer (each CTA walks a contiguous slice of `per` tiles; the last CTA of a layer to finish
+// settles it).  list: n_layers descriptors + sentinel, tile_begin filled in.
+int plan_range_grid(LayerDesc* list, int n_layers, long long tiles, int sm_count) {
+  const int grid = static_cast<int>(std::max<long long>(1, std::min<long long>(tiles, 16ll * sm_count)));
+  const long long per = (tiles + grid - 1) / grid;
+  for (int k = 0; k < n_layers; ++k) {
+    const long long b = list[k].tile_begin, e = list[k + 1].tile_begin;
+    list[k].range_ctas = (e > b && per > 0) ? static_cast<int>((e - 1) / per - b / per + 1) : 0;
+  }
+  return grid;
+}
 
 struct SearchArgs {
   const float* const* tensors;  // host array of device pointers
@@ -300,10 +314,12 @@ long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchAr
     d.layer_id = a.opts.layer_base + l;
     d.index = l;
     d.n_bins = a.opts.n_bins_per_layer ? a.opts.n_bins_per_layer[l] : a.n_bins;
+    d.range_ctas = 0;
     if (a.lens[l] > 0) tiles += (a.lens[l] + mis + tile - 1) / tile;
   }
   LayerDesc& s = out[k];
   s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.n_bins = 1;
+  s.range_ctas = 0;
   return tiles;
 }
 
@@ -367,6 +383,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   char* h = static_cast<char*>(slot->host);
   std::memset(h, 0, plan.blob_bytes);
   const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, a, kTile);
+  const int range_grid = plan_range_grid(reinterpret_cast<LayerDesc*>(h + plan.off_layers), a.n_layers, tiles, dc.sm_count);
   const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a, kKeyedTile);
   const long long direct_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_direct), direct, a, kTile);
   std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
@@ -377,11 +394,10 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   std::memcpy(h + plan.off_fl_begin, plan.fl_begin.data(), sizeof(int) * (plan.n_levels + 1));
   if (o.start_wl_fl) std::memcpy(h + plan.off_start, o.start_wl_fl, sizeof(int) * 2 * a.n_layers);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
-  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
-  ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
 
   const LayerDesc* d_layers = reinterpret_cast<const LayerDesc*>(ws + plan.off_layers);
   const LayerDesc* d_keyed = reinterpret_cast<const LayerDesc*>(ws + plan.off_keyed);
@@ -389,7 +405,6 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   LayerState* d_state = reinterpret_cast<LayerState*>(ws + plan.off_state);
   LayerPlan* d_plan = reinterpret_cast<LayerPlan*>(ws + plan.off_plan);
   float* d_edges = reinterpret_cast<float*>(ws + plan.off_edges);
-  unsigned* d_cell_init = reinterpret_cast<unsigned*>(ws + plan.off_cell_init);
   unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + plan.off_zeros);
   unsigned long long* d_zclass = reinterpret_cast<unsigned long long*>(ws + plan.off_zclass);
   unsigned* d_q = reinterpret_cast<unsigned*>(ws + plan.off_q);
@@ -398,39 +413,36 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   unsigned* d_sub = reinterpret_cast<unsigned*>(ws + plan.off_sub);
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + plan.off_u);
 
-  // K1: range scan over every layer, then bin origin / scale per layer
-  if (tiles > 0) {
-    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc.sm_count));
-    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
-    range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(d_layers, a.n_layers, tiles, d_state);
-    ADAPT_CUDA(cudaGetLastError());
-  }
+  ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
+
+  // K1: range scan over every layer; its last CTA per layer derives the bin origin and scale
+  const int keyed_grid = static_cast<int>(std::max<long long>(1, std::min<long long>(keyed_tiles, 1ll * dc.sm_count)));
   {
-    LaunchScope ls(ADAPT_KERNEL_RANGE_FINALIZE, stream);
-    range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
-        d_layers, a.n_layers, d_state, o.range_out);
+    RangeParams rp;
+    rp.layers = d_layers; rp.n_layers = a.n_layers; rp.n_tiles = tiles; rp.state = d_state;
+    rp.range_out = o.range_out;
+    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
+    range_scan_kernel<<<range_grid, kRangeThreads, 0, stream>>>(rp);
     ADAPT_CUDA(cudaGetLastError());
   }
 
   // K2, keyed form: plan -> cell counting -> expansion
   if (!keyed.empty() && keyed_tiles > 0) {
     const int nk = static_cast<int>(keyed.size());
-    PlanParams pp;
-    pp.layers = d_keyed; pp.n_layers = nk; pp.state = d_state; pp.plan = d_plan;
-    pp.edges = d_edges; pp.cell_init = d_cell_init; pp.n_bins = bins_stride; pp.cell_cap = plan.cell_cap;
-    pp.value_cap = plan.value_cap; pp.cell_stride = plan.value_cap;
-    pp.fine_ratio = ADAPT_FINE_RATIO;
-    const int keyed_grid = static_cast<int>(std::min<long long>(keyed_tiles, 1ll * dc.sm_count));
-    pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
     {
+      PlanParams pp;
+      pp.layers = d_keyed; pp.state = d_state; pp.plan = d_plan; pp.edges = d_edges;
+      pp.n_bins = bins_stride; pp.cell_cap = plan.cell_cap; pp.value_cap = plan.value_cap;
+      pp.fine_ratio = ADAPT_FINE_RATIO;
+      pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
-      const int plan_slices = std::max(1, std::min(16, (2 * dc.sm_count) / nk));
+      const int plan_slices = std::max(1, std::min(8, (bins_stride + kPlanThreads - 1) / kPlanThreads));
       plan_kernel<<<dim3(nk, plan_slices), kPlanThreads, 0, stream>>>(pp);
       ADAPT_CUDA(cudaGetLastError());
     }
     KeyedParams kp;
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
-    kp.plan = d_plan; kp.edges = d_edges; kp.cell_init = d_cell_init; kp.cell_count = d_cells;
+    kp.plan = d_plan; kp.edges = d_edges; kp.cell_count = d_cells;
     kp.qe_hist = d_qe; kp.u_hist = d_u; kp.q_hist = d_q; kp.zeros = d_zeros; kp.zero_class = d_zclass;
     kp.sub_count = d_sub;
     kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
@@ -446,7 +458,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     }
     ExpandParams ep;
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
-    ep.cell_init = d_cell_init; ep.cell_count = d_cells; ep.qe_hist = d_qe;
+    ep.cell_count = d_cells; ep.qe_hist = d_qe;
     ep.sub_count = d_sub; ep.edges = d_edges;
     ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros; ep.zero_class = d_zclass;
     ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
@@ -497,7 +509,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ADAPT_CUDA(cudaGetLastError());
   }
 
-  // K3: divergence per (layer, candidate), then selection per layer
+  // K3: divergence per (layer, candidate); the last CTA of a layer selects its format
   KldParams kp;
   kp.layers = d_layers; kp.state = d_state;
   kp.cand_wl = reinterpret_cast<const int*>(ws + plan.off_wl);
@@ -512,16 +524,12 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   kp.kld_out = a.kld_out; kp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
   kp.best_out = a.best_out; kp.hist_out = o.hist_out;
   kp.start = o.start_wl_fl ? reinterpret_cast<const int*>(ws + plan.off_start) : nullptr;
+  kp.status_out = o.status_out;
   {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
     // enough CTAs to fill the GPU when there are few (FL, layer) pairs
     const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / std::max(1, plan.n_levels * a.n_layers)));
     kld_kernel<<<dim3(plan.n_levels, a.n_layers, slices), kKldThreads, 0, stream>>>(kp);
-    ADAPT_CUDA(cudaGetLastError());
-  }
-  {
-    LaunchScope ls(ADAPT_KERNEL_SELECT, stream);
-    select_kernel<<<a.n_layers, 32, 0, stream>>>(kp);
     ADAPT_CUDA(cudaGetLastError());
   }
   return ADAPT_OK;
@@ -933,7 +941,7 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
   int rc = current_cache(&dc);
   if (rc != ADAPT_OK) return rc;
   adapt_search_opts o = opts ? *opts : default_opts();
-  if (o.workspace || o.workspace_bytes || o.hist_out || o.range_out) return ADAPT_ERR_INVALID_ARG;
+  if (o.workspace || o.workspace_bytes || o.hist_out || o.range_out || o.status_out) return ADAPT_ERR_INVALID_ARG;
   if (!tensors || !kld_out || !zeros_out || !best_out) return ADAPT_ERR_INVALID_ARG;
   Plan plan;
   if (!make_plan(lens, n_layers, grid, n_bins, &plan)) return ADAPT_ERR_INVALID_ARG;
@@ -1171,10 +1179,11 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   std::iota(all.begin(), all.end(), 0);
   SearchArgs la{a.tensors, a.lens, a.n_layers, nullptr, a.n_bins, nullptr, nullptr, nullptr, o};
   const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, la, kTile);
+  const int range_grid = plan_range_grid(reinterpret_cast<LayerDesc*>(h + plan.off_layers), a.n_layers, tiles, dc.sm_count);
   std::memcpy(h + plan.off_cands, plan.cands.data(), sizeof(FormatCand) * plan.n_cand);
   std::memcpy(h + plan.off_rules, plan.rules.data(), sizeof(FormatRule) * plan.n_rules);
   LayerState* hs = reinterpret_cast<LayerState*>(h + plan.off_state);
-  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
+  for (int l = 0; l < a.n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, plan.blob_bytes, cudaMemcpyHostToDevice, stream));
   ADAPT_CUDA(cudaEventRecord(slot->done, stream));
   ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
@@ -1195,7 +1204,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   fp.seed = o.seed;
   fp.alpha = o.pseudo_count; fp.inv_ln_base = 1.0 / std::log(base); fp.eps = o.eps;
   fp.kld_out = a.kld_out; fp.zeros_out = reinterpret_cast<long long*>(a.zeros_out);
-  fp.b_out = a.b_out; fp.best_out = a.best_out; fp.hist_out = o.hist_out;
+  fp.b_out = a.b_out; fp.best_out = a.best_out; fp.hist_out = o.hist_out; fp.status_out = o.status_out;
 
   // rule groups: few tiles spread the rules over more CTAs, many tiles fill shared memory
   int rpg = static_cast<int>(std::min<size_t>(kMaxRulesPerGroup, budget / per_hist));
@@ -1207,16 +1216,12 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   const int groups = (plan.n_rules + rpg - 1) / rpg;
   const size_t smem = per_hist * rpg;
 
-  if (tiles > 0) {
-    const int grid = static_cast<int>(std::min<long long>(tiles, 16ll * dc.sm_count));
-    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
-    range_scan_kernel<<<grid, kRangeThreads, 0, stream>>>(fp.layers, a.n_layers, tiles, d_state);
-    ADAPT_CUDA(cudaGetLastError());
-  }
   {
-    LaunchScope ls(ADAPT_KERNEL_RANGE_FINALIZE, stream);
-    range_finalize_kernel<<<(a.n_layers + 127) / 128, 128, 0, stream>>>(
-        fp.layers, a.n_layers, d_state, o.range_out);
+    RangeParams rp;
+    rp.layers = fp.layers; rp.n_layers = a.n_layers; rp.n_tiles = tiles; rp.state = d_state;
+    rp.range_out = o.range_out;
+    LaunchScope ls(ADAPT_KERNEL_RANGE, stream);
+    range_scan_kernel<<<range_grid, kRangeThreads, 0, stream>>>(rp);
     ADAPT_CUDA(cudaGetLastError());
   }
   {
@@ -1326,6 +1331,7 @@ constexpr size_t kStZeros = (kStBlobEnd + 255) / 256 * 256;                     
 constexpr size_t kStQ = kStZeros + 8 * kStaticMaxLayers * kMaxFl;                 // u32[L][B]
 constexpr size_t kStU = kStQ + 4 * static_cast<size_t>(kStaticMaxLayers) * kStaticMaxBins;
 constexpr size_t kStEnd = kStU + 4 * static_cast<size_t>(kStaticMaxLayers) * kMaxFl * kStaticMaxBins;
+static_assert((kStEnd - kStZeros) % 16 == 0, "the accumulators are cleared in 16-byte units");
 static_assert(sizeof(LayerDesc) <= 64 && sizeof(LayerState) <= 64, "descriptor slots too small");
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStEnd];
@@ -1409,6 +1415,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
     if (lens[l] > 0) tiles += (lens[l] + mis + kTile - 1) / kTile;
   }
   hl[n_layers].tile_begin = tiles;
+  const int range_grid = plan_range_grid(hl, n_layers, tiles, dc->sm_count);
   int* h_wl = reinterpret_cast<int*>(h + kStWl);
   int* h_fl = reinterpret_cast<int*>(h + kStFl);
   int* h_slot = reinterpret_cast<int*>(h + kStSlot);
@@ -1425,28 +1432,26 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   for (int c = 0; c < C; ++c) h_fl_begin[grid->fl[c] + 1] += 1;
   for (int f = 0; f < n_levels; ++f) h_fl_begin[f + 1] += h_fl_begin[f];
   LayerState* hs = reinterpret_cast<LayerState*>(h + kStState);
-  for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; hs[l].min_lsb = 0xFFFFFFFFu; }
+  for (int l = 0; l < n_layers; ++l) { hs[l].min_key = 0xFFFFFFFFu; hs[l].max_key = 0u; }
 
   // the block is ordinary host memory: the copy is staged before the call returns
   ADAPT_CUDA(cudaMemcpyAsync(ws, h, kStBlobEnd, cudaMemcpyHostToDevice, stream));
   // the scratch keeps the previous call's counts: clear every accumulator
   ADAPT_CUDA(cudaMemsetAsync(ws + kStZeros, 0, kStEnd - kStZeros, stream));
-
   const LayerDesc* d_layers = reinterpret_cast<const LayerDesc*>(ws + kStLayers);
   LayerState* d_state = reinterpret_cast<LayerState*>(ws + kStState);
   unsigned long long* d_zeros = reinterpret_cast<unsigned long long*>(ws + kStZeros);
   unsigned* d_q = reinterpret_cast<unsigned*>(ws + kStQ);
   unsigned* d_u = reinterpret_cast<unsigned*>(ws + kStU);
 
-  if (tiles > 0) {
-    const int g = static_cast<int>(std::min<long long>(tiles, 16ll * dc->sm_count));
-    range_scan_kernel<<<g, kRangeThreads, 0, stream>>>(d_layers, n_layers, tiles, d_state);
+  {
+    RangeParams rp;
+    rp.layers = d_layers; rp.n_layers = n_layers; rp.n_tiles = tiles; rp.state = d_state;
+    rp.range_out = nullptr;
+    range_scan_kernel<<<range_grid, kRangeThreads, 0, stream>>>(rp);
     ADAPT_LAUNCH_OK("range scan launch");
     ++g_launches;
   }
-  range_finalize_kernel<<<1, 128, 0, stream>>>(d_layers, n_layers, d_state, nullptr);
-  ADAPT_LAUNCH_OK("range finalize launch");
-  ++g_launches;
   if (tiles > 0) {
     SearchParams sp;
     sp.layers = d_layers; sp.state = d_state; sp.n_layers = n_layers; sp.n_fl = n_levels;
@@ -1480,12 +1485,9 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   kp.q_hist = d_q; kp.u_hist = d_u; kp.zeros = d_zeros;
   kp.alpha = 0.0; kp.inv_ln_base = 1.0 / std::log(2.0); kp.eps = 0.0;
   kp.kld_out = kld_out; kp.zeros_out = reinterpret_cast<long long*>(zeros_out);
-  kp.best_out = best_out; kp.hist_out = nullptr; kp.start = nullptr;
+  kp.best_out = best_out; kp.hist_out = nullptr; kp.start = nullptr; kp.status_out = nullptr;
   kld_kernel<<<dim3(n_levels, n_layers), kKldThreads, 0, stream>>>(kp);
   ADAPT_LAUNCH_OK("kld launch");
-  ++g_launches;
-  select_kernel<<<n_layers, 32, 0, stream>>>(kp);
-  ADAPT_LAUNCH_OK("select launch");
   ++g_launches;
   return ADAPT_OK;
 }

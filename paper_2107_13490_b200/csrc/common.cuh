@@ -12,6 +12,12 @@
 namespace adapt {
 
 constexpr int kMaxFl = 32;  // FL in 0..31
+constexpr int kTile = 4096; // elements per tile of the range scan and the direct kernels (in aligned indexing)
+
+// LayerState::flags (the same bits as ADAPT_FLAG_* of the C interface)
+constexpr unsigned kFlagDegenerate = 2u;
+constexpr unsigned kFlagNonfinite = 4u;
+constexpr unsigned kFlagRange = 8u;
 
 // Per-layer descriptor, written by the host into the workspace.
 struct LayerDesc {
@@ -22,6 +28,8 @@ struct LayerDesc {
   int layer_id;          // hash layer id
   int index;             // position in the caller's tensor list (addresses state and outputs)
   int n_bins;            // bins of this layer's histograms (<= the stride the arrays use)
+  int range_ctas;        // CTAs of the range scan that hold tiles of this layer (set by the host for
+                         // the list that kernel walks; the last of them to finish settles the layer)
 };
 
 // Per-layer state produced on the device by the range scan.
@@ -33,10 +41,10 @@ struct LayerState {
   float abs_sum;     // sum of |x| (any summation order; only steers table shapes, never results)
   unsigned zero_count;  // estimate of the exact zeros (the range scan samples one element in
                         // eight; steers the choice of loop form only, never results)
-  unsigned min_lsb;     // over the same sample of non-zero elements: the least (biased exponent +
-                        // trailing zero bits of the 24-bit significand), i.e. 150 + the binary
-                        // exponent of the coarsest grid 2^e all sampled elements lie on; 0xFFFFFFFF
-                        // if none was seen (steers the choice of loop form only, never results)
+  unsigned ticket;      // range scan: CTAs that have added their part of this layer (the last one
+                        // turns the extremes into the bin origin and scale)
+  unsigned kld_ticket;  // divergence kernel: CTAs that have written their candidates of this layer
+                        // (the last one selects the layer's format)
 };
 
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).

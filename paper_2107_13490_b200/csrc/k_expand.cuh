@@ -30,7 +30,6 @@ struct ExpandParams {
   int n_layers;
   const LayerState* state;
   const LayerPlan* plan;
-  const unsigned* cell_init;   // [layer][cell_stride]
   const unsigned* cell_count;  // [layer][cell_stride]
   const unsigned* qe_hist;     // [layer][2][n_bins]
   const unsigned* sub_count;   // [layer][2][n_bins][kSubCells]  sub-cell counts of the edge cells
@@ -60,7 +59,6 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   __syncthreads();
 
   const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_stride;
-  const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
   unsigned long long zero = 0;
   // the cells are shared by the gridDim.z CTAs of this (level, layer), a contiguous slice each
   const int per_slice = ((P.total_cells + gridDim.z - 1) / gridDim.z + 3) & ~3;
@@ -68,13 +66,10 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
   // four cells per thread and trip, counts and marks fetched as 128-bit words (slices start on
   // multiples of four cells; the rows are 16-byte aligned and a multiple of four cells long)
   const uint4* count4 = reinterpret_cast<const uint4*>(count);
-  const uint4* init4 = reinterpret_cast<const uint4*>(init);
 #pragma unroll 2
   for (int i0 = blockIdx.z * per_slice + 4 * threadIdx.x; i0 < i_end; i0 += 4 * kExpandThreads) {
     const uint4 m4 = __ldg(count4 + (i0 >> 2));
-    const uint4 k4 = __ldg(init4 + (i0 >> 2));
     const unsigned ms[4] = {m4.x, m4.y, m4.z, m4.w};
-    const unsigned ks[4] = {k4.x, k4.y, k4.z, k4.w};
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
       const int i = i0 + e;
@@ -94,10 +89,11 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
         }
         atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
       } else if (is_q || f >= sp.g) {
-        if (!(ks[e] & kCellEdge)) {
-          const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
-          atomicAdd(&s_hist[bin_of(lf, S.lo, S.scale, S.bmax)], m);
-        }
+        // interior cells only (the marks are recomputed: a cell whose closed interval meets two bins)
+        float lf, rf;
+        cell_ends(cc, sp.g, P.fast != 0, &lf, &rf);
+        const int bl = bin_of(lf, S.lo, S.scale, S.bmax);
+        if (bl == bin_of(rf, S.lo, S.scale, S.bmax)) atomicAdd(&s_hist[bl], m);
       } else {
         const int d = sp.g - f;                      // 1..32
         const long long a = cc >> d;                 // floor(c / 2^d)

@@ -46,6 +46,7 @@ struct FormatParams {
   int* b_out;                   // optional [n_layers][n_cand]
   int* best_out;                // [n_layers][4]
   unsigned* hist_out;           // optional [n_layers][n_cand + 1][n_bins]; slot 0 = float tensor
+  int* status_out;              // optional [n_layers]: 0, or the status code of the layer's data error
 };
 
 // x * 2^k for -149 <= k <= 149 in two exact steps (a single 2^k may not be a normal float).
@@ -421,6 +422,7 @@ __global__ void format_select_kernel(const FormatParams p) {
   }
   if (lane == 0) {
     unsigned flags = p.state[l].flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
+    if (p.status_out) p.status_out[l] = (flags & kFlagNonfinite) ? 2 : ((flags & kFlagRange) ? 3 : 0);
     int c;
     if (first_ok != 0x7fffffff) { c = first_ok; flags |= 1u; }
     else if (min_pos >= 0) c = min_pos;

@@ -1,4 +1,4 @@
-// K3: batched divergence and selection over all (layer, candidate) pairs.
+// K3: batched divergence and selection over all (layer, candidate) pairs, one launch.
 //
 // kld_kernel: one CTA per (fraction length, layer).  Folds the layer's unsaturated
 // per-FL histogram into each candidate's histogram (both tails collapse into
@@ -8,8 +8,11 @@
 // N, the term (p/N) log((p/N)/(q/N)) is evaluated as p * log1p((p - q)/q) / N:
 // the difference is exact in integers, so histograms that differ by a few
 // counts in well-filled bins do not lose their divergence to cancellation.
+// The unsaturated divergence is summed by the whole CTA; the candidates that
+// saturate inside the range are dealt to the CTA's warps, one warp each.
 //
-// select_kernel: one warp per layer; the lowest <WL,FL> (WL first, then FL)
+// The CTA that writes the last divergences of a layer (a ticket per layer, no
+// waiting) selects the layer's format: the lowest <WL,FL> (WL first, then FL)
 // with KLD <= eps, else the candidate of least divergence (Algorithm 3).
 #pragma once
 
@@ -24,7 +27,7 @@ constexpr int kKldThreads = 256;
 
 struct KldParams {
   const LayerDesc* layers;
-  const LayerState* state;
+  LayerState* state;           // read, and its kld_ticket counted up
   const int* cand_wl;          // [n_cand]
   const int* cand_fl;          // [n_cand]
   const int* cand_slot;        // [n_cand] index of the candidate's FL in the distinct-FL list
@@ -43,6 +46,7 @@ struct KldParams {
   int* best_out;               // [n_layers][4]
   unsigned* hist_out;          // optional [n_layers][n_cand + 1][n_bins]
   const int* start;            // optional [n_layers][2]: descent from this <WL,FL> per layer
+  int* status_out;             // optional [n_layers]: 0, or the status code of the layer's data error
 };
 
 __device__ __forceinline__ double block_sum(double v, double* s_buf) {
@@ -66,103 +70,151 @@ __device__ __forceinline__ double kld_term(long long pc, long long qc, double al
   return pa * log1p(static_cast<double>(pc - qc) / qa);
 }
 
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 // One CTA per (fraction length, layer).  The candidates of one FL differ only in where they
 // saturate; those whose two saturation values fall in the first and the last bin have exactly
 // the unsaturated histogram U[FL], so their divergence is computed once.  The others fold the
 // two tails of U[FL] into the bins of their saturation values and are summed one by one.
+__device__ void select_layer(const KldParams& p, int l, int lane);
+
 __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   __shared__ double s_buf[kKldThreads / 32];
-  __shared__ int s_inf;
+  __shared__ int s_inf, s_last;
   const int f = blockIdx.x, l = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c_begin = p.fl_begin[f], c_end = p.fl_begin[f + 1];
-  if (c_begin == c_end) return;
   const int stride = p.n_bins;
   const LayerState S = p.state[l];
   const int B = p.layers[l].n_bins;        // this layer's bins; arrays are laid out with `stride`
   const long long n = p.layers[l].n;
 
-  if (S.flags & (kFlagNonfinite | kFlagRange)) {
+  if (c_begin == c_end) {
+    // no candidate has this fraction length: nothing to write
+  } else if (S.flags & (kFlagNonfinite | kFlagRange)) {
     for (int i = c_begin + blockIdx.z * kKldThreads + threadIdx.x; i < c_end;
          i += kKldThreads * gridDim.z) {
       const size_t out = static_cast<size_t>(l) * p.n_cand + p.cand_by_fl[i];
       p.kld_out[out] = __longlong_as_double(0x7ff8000000000000ll);  // NaN: unspecified output
       p.zeros_out[out] = 0;
     }
-    return;
+  } else {
+    const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + f) * stride;
+    const unsigned* Q = p.q_hist + static_cast<size_t>(l) * stride;
+    const double n_eff = static_cast<double>(n) + p.alpha * B;
+    const double inf_value = __longlong_as_double(0x7ff0000000000000ll);
+    const long long zero_count = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + f]);
+
+    // divergence of the unsaturated histogram, by the whole CTA
+    if (threadIdx.x == 0) s_inf = 0;
+    __syncthreads();
+    double sum = 0.0;
+    bool inf = false;
+    for (int b = threadIdx.x; b < B; b += kKldThreads) sum += kld_term(U[b], Q[b], p.alpha, &inf);
+    if (inf) s_inf = 1;
+    sum = block_sum(sum, s_buf);
+    double unsat;
+    if (n_eff <= 0.0) unsat = 0.0;
+    else if (s_inf) unsat = inf_value;
+    else { unsat = sum * p.inv_ln_base / n_eff; if (!(unsat > 0.0)) unsat = 0.0; }
+
+    // A candidate whose saturation values fall inside the range folds the tails of U[FL] and is
+    // summed by itself: by one warp when the histogram is short (the FL's candidates are then
+    // dealt to the warps of the gridDim.z CTAs that share this (FL, layer)), by the whole CTA
+    // when it is long (candidates dealt to the CTAs).
+    constexpr int kWarps = kKldThreads / 32;
+    const bool by_warp = B <= 512;
+    const int first = by_warp ? blockIdx.z * kWarps + warp : blockIdx.z;
+    const int step = by_warp ? kWarps * gridDim.z : gridDim.z;
+    const int me = by_warp ? lane : threadIdx.x, team = by_warp ? 32 : kKldThreads;
+    for (int i = c_begin + first; i < c_end; i += step) {
+      const int c = p.cand_by_fl[i];
+      const int wl = p.cand_wl[c];
+      const size_t out = static_cast<size_t>(l) * p.n_cand + c;
+      // bins of the two saturation values of <WL,FL>
+      const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
+      const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
+      const int bh = bin_of(dequantize(hi_code, f), S.lo, S.scale, S.bmax);
+      const int bl = bin_of(dequantize(lo_code, f), S.lo, S.scale, S.bmax);
+      unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * stride
+                               : nullptr;
+      unsigned* H0 = (p.hist_out && c == 0)
+                         ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * stride : nullptr;
+      double k;
+      if (bl == 0 && bh == B - 1 && B > 1 && !H) {
+        k = unsat;                     // nothing folds: the candidate's histogram is U[FL] itself
+      } else {
+        // tail masses that fold into bl and bh (exact: sums of counts)
+        unsigned long long lo_mass = 0, hi_mass = 0;
+        for (int b = me; b < B; b += team) {
+          const unsigned u = U[b];
+          if (b <= bl) lo_mass += u;
+          if (b >= bh) hi_mass += u;
+        }
+        if (by_warp) {
+          lo_mass = warp_sum(lo_mass);
+          hi_mass = warp_sum(hi_mass);
+        } else {
+          lo_mass = static_cast<unsigned long long>(block_sum(static_cast<double>(lo_mass), s_buf));
+          hi_mass = static_cast<unsigned long long>(block_sum(static_cast<double>(hi_mass), s_buf));
+          if (threadIdx.x == 0) s_inf = 0;
+          __syncthreads();
+        }
+        double part = 0.0;
+        bool part_inf = false;
+        for (int b = me; b < B; b += team) {
+          long long pc;
+          if (bl == bh) pc = (b == bl) ? n : 0;
+          else if (b < bl || b > bh) pc = 0;
+          else if (b == bl) pc = static_cast<long long>(lo_mass);
+          else if (b == bh) pc = static_cast<long long>(hi_mass);
+          else pc = U[b];
+          const long long qc = Q[b];
+          if (H) H[b] = static_cast<unsigned>(pc);
+          if (H0) H0[b] = static_cast<unsigned>(qc);
+          part += kld_term(pc, qc, p.alpha, &part_inf);
+        }
+        bool any_inf;
+        if (by_warp) {
+          part = warp_sum(part);
+          any_inf = __any_sync(0xffffffffu, part_inf);
+        } else {
+          if (part_inf) s_inf = 1;
+          part = block_sum(part, s_buf);
+          any_inf = s_inf != 0;
+          __syncthreads();             // s_inf is rewritten by the next candidate
+        }
+        if (n_eff <= 0.0) k = 0.0;
+        else if (any_inf) k = inf_value;
+        else { k = part * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
+      }
+      if (me == 0) {
+        p.kld_out[out] = k;
+        p.zeros_out[out] = zero_count;
+      }
+    }
   }
-  const unsigned* U = p.u_hist + (static_cast<size_t>(l) * p.n_fl + f) * stride;
-  const unsigned* Q = p.q_hist + static_cast<size_t>(l) * stride;
-  const double n_eff = static_cast<double>(n) + p.alpha * B;
-  const double inf_value = __longlong_as_double(0x7ff0000000000000ll);
-  const long long zero_count = static_cast<long long>(p.zeros[static_cast<size_t>(l) * p.n_fl + f]);
 
-  // divergence of the unsaturated histogram
-  if (threadIdx.x == 0) s_inf = 0;
+  // the CTA that completes the layer's divergences selects its format
   __syncthreads();
-  double sum = 0.0;
-  bool inf = false;
-  for (int b = threadIdx.x; b < B; b += kKldThreads) sum += kld_term(U[b], Q[b], p.alpha, &inf);
-  if (inf) s_inf = 1;
-  sum = block_sum(sum, s_buf);
-  double unsat;
-  if (n_eff <= 0.0) unsat = 0.0;
-  else if (s_inf) unsat = inf_value;
-  else { unsat = sum * p.inv_ln_base / n_eff; if (!(unsat > 0.0)) unsat = 0.0; }
-
-  // the FL's candidates are dealt round-robin to the gridDim.z CTAs that share this (FL, layer)
-  for (int i = c_begin + blockIdx.z; i < c_end; i += gridDim.z) {
-    const int c = p.cand_by_fl[i];
-    const int wl = p.cand_wl[c];
-    const size_t out = static_cast<size_t>(l) * p.n_cand + c;
-    // bins of the two saturation values of <WL,FL>
-    const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
-    const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
-    const int bh = bin_of(dequantize(hi_code, f), S.lo, S.scale, S.bmax);
-    const int bl = bin_of(dequantize(lo_code, f), S.lo, S.scale, S.bmax);
-    unsigned* H = p.hist_out ? p.hist_out + (static_cast<size_t>(l) * (p.n_cand + 1) + c + 1) * stride
-                             : nullptr;
-    unsigned* H0 = (p.hist_out && c == 0)
-                       ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * stride : nullptr;
-    double k;
-    if (bl == 0 && bh == B - 1 && B > 1 && !H) {
-      k = unsat;                     // nothing folds: the candidate's histogram is U[FL] itself
-    } else {
-      // tail masses that fold into bl and bh
-      double lo_mass = 0.0, hi_mass = 0.0;
-      for (int b = threadIdx.x; b < B; b += kKldThreads) {
-        const unsigned u = U[b];
-        if (b <= bl) lo_mass += u;
-        if (b >= bh) hi_mass += u;
-      }
-      lo_mass = block_sum(lo_mass, s_buf);
-      hi_mass = block_sum(hi_mass, s_buf);
-      if (threadIdx.x == 0) s_inf = 0;
-      __syncthreads();
-      sum = 0.0;
-      inf = false;
-      for (int b = threadIdx.x; b < B; b += kKldThreads) {
-        long long pc;
-        if (bl == bh) pc = (b == bl) ? n : 0;
-        else if (b < bl || b > bh) pc = 0;
-        else if (b == bl) pc = static_cast<long long>(lo_mass);
-        else if (b == bh) pc = static_cast<long long>(hi_mass);
-        else pc = U[b];
-        const long long qc = Q[b];
-        if (H) H[b] = static_cast<unsigned>(pc);
-        if (H0) H0[b] = static_cast<unsigned>(qc);
-        sum += kld_term(pc, qc, p.alpha, &inf);
-      }
-      if (inf) s_inf = 1;
-      sum = block_sum(sum, s_buf);
-      if (n_eff <= 0.0) k = 0.0;
-      else if (s_inf) k = inf_value;
-      else { k = sum * p.inv_ln_base / n_eff; if (!(k > 0.0)) k = 0.0; }
-      __syncthreads();               // s_inf is rewritten by the next candidate
-    }
-    if (threadIdx.x == 0) {
-      p.kld_out[out] = k;
-      p.zeros_out[out] = zero_count;
-    }
+  if (threadIdx.x == 0) {
+    __threadfence();
+    const unsigned done = atomicAdd(&p.state[l].kld_ticket, 1u);
+    s_last = (done == gridDim.x * gridDim.z - 1u) ? 1 : 0;
+  }
+  __syncthreads();
+  if (s_last && warp == 0) {
+    __threadfence();
+    select_layer(p, l, lane);
   }
 }
 
@@ -171,17 +223,19 @@ __device__ __forceinline__ void arg_min_merge(double& k, int& pos, double k2, in
   if (pos2 >= 0 && (pos < 0 || k2 < k || (k2 == k && pos2 < pos))) { k = k2; pos = pos2; }
 }
 
-__global__ void select_kernel(const KldParams p) {
-  const int l = blockIdx.x;
-  const int lane = threadIdx.x;  // one warp
+// One warp: the layer's choice from its divergences (written by other CTAs of this launch:
+// read past the L1 cache).
+__device__ void select_layer(const KldParams& p, int l, int lane) {
   const LayerState S = p.state[l];
+  if (p.status_out && lane == 0)       // 2 / 3: the interface's codes for NaN/Inf and |x| >= 2^64
+    p.status_out[l] = (S.flags & kFlagNonfinite) ? 2 : ((S.flags & kFlagRange) ? 3 : 0);
   const double* kld = p.kld_out + static_cast<size_t>(l) * p.n_cand;
 
   int first_ok = 0x7fffffff;  // position (in candidate order) of the first KLD <= eps
   double min_k = 0.0;
   int min_pos = -1;           // position of the least finite divergence
   for (int pos = lane; pos < p.n_cand; pos += 32) {
-    const double k = kld[p.cand_order[pos]];
+    const double k = __ldcg(kld + p.cand_order[pos]);
     if (k <= p.eps) first_ok = min(first_ok, pos);
     if (k < __longlong_as_double(0x7ff0000000000000ll)) arg_min_merge(min_k, min_pos, k, pos);
   }
@@ -209,14 +263,14 @@ __global__ void select_kernel(const KldParams p) {
     int last_bad = -1;   // highest position below the start whose divergence exceeds eps
     if (spos >= 0)
       for (int pos = lane; pos < spos; pos += 32)
-        if (!(kld[p.cand_order[pos]] <= p.eps)) last_bad = max(last_bad, pos);
+        if (!(__ldcg(kld + p.cand_order[pos]) <= p.eps)) last_bad = max(last_bad, pos);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) last_bad = max(last_bad, __shfl_xor_sync(0xffffffffu, last_bad, o));
     if (lane == 0) {
       unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
       int* o = p.best_out + 4 * l;
       if (spos < 0) { o[0] = swl; o[1] = sfl; o[2] = -1; o[3] = static_cast<int>(flags); return; }
-      const bool ok = kld[p.cand_order[spos]] <= p.eps;
+      const bool ok = __ldcg(kld + p.cand_order[spos]) <= p.eps;
       const int pos = ok ? last_bad + 1 : spos;
       const int c = p.cand_order[pos];
       if (ok) flags |= 1u;

@@ -23,15 +23,13 @@
 // cells over the whole range for the few elements outside.  R only steers
 // speed: any R gives the same results.
 //
-// This kernel chooses the segments, computes the exact bin edges (smallest
-// float of each bin, by bisection over the float order with the bin function
-// itself), and marks each cell: bit 31 = edge cell, bit 30 = cell -1 or 0 of
-// the main segment.  (Bit 29 is left to the counting kernel, which adds it to the word an
+// plan_kernel: make_layer_plan chooses the segments; bin_lower_edge gives the exact bin edges (smallest float of each bin, found with
+// the bin function itself); cell_mark gives each cell its marks: bit 31 = edge cell,
+// bit 30 = cell -1 or 0 of the main segment.  (Bit 29 is left to the counting kernel, which adds it to the word an
 // atomic returns when the element sits exactly on the cell grid.)
 #pragma once
 
 #include "common.cuh"
-#include "k_range.cuh"
 
 namespace adapt {
 
@@ -39,7 +37,6 @@ constexpr unsigned kCellEdge = 0x80000000u;
 constexpr unsigned kCellNearZero = 0x40000000u;
 constexpr unsigned kCellOnGrid = 0x20000000u;     // added to a returned word, never stored
 constexpr unsigned kCellCountMask = 0x1FFFFFFFu;
-constexpr int kPlanThreads = 256;
 
 // Second level under the edge cells.  An element of an edge cell is counted again in one of
 // kSubCells sub-cells (2^-(G + kSubBits) wide) of a table in global memory, indexed by segment,
@@ -118,15 +115,12 @@ constexpr long long kDenseZeroRatio = ADAPT_DENSE_ZERO_RATIO;   // <= 0 switches
 
 struct PlanParams {
   const LayerDesc* layers;   // keyed layer list
-  int n_layers;              // entries in that list
   const LayerState* state;   // indexed by LayerDesc::index
   LayerPlan* plan;           // indexed by LayerDesc::index
   float* edges;              // [all layers][n_bins + 1] (n_bins = the stride below)
-  unsigned* cell_init;       // [all layers][cell_stride]
   int n_bins;                // stride of the per-bin arrays (the largest layer's bins)
   int cell_cap;              // table entries a layer may use
   int value_cap;             // ... when it is keyed by value (its table may run over the others)
-  int cell_stride;           // row length of cell_init
   int fine_ratio;            // stop refining once a bin holds this many cells
   long long elems_per_cta;   // elements one CTA of the keyed kernel processes
 };
@@ -138,7 +132,12 @@ __device__ __forceinline__ long long floor_scaled(float v, int g) {
 
 // Largest level G <= g_max such that the cells covering [lo, hi] number at most max_cells.
 __device__ inline void fit_segment(float lo, float hi, int max_cells, int g_max, SegPlan* s) {
+  // the answer is near log2(max_cells / (hi - lo)): start just above it instead of at g_max
   int g = g_max;
+  {
+    const double span0 = static_cast<double>(hi) - static_cast<double>(lo);
+    if (span0 > 0.0) g = min(g_max, ilogb(static_cast<double>(max_cells)) - ilogb(span0) + 2);
+  }
   long long c0 = 0, c1 = 0;
   for (; g > -100; --g) {
     const double span = ldexp(static_cast<double>(hi) - static_cast<double>(lo), g);
@@ -163,14 +162,39 @@ __device__ inline int level_for_ratio(float lo, float hi, int n_bins, int ratio)
   return max(-100, min(g, 32));
 }
 
-__global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) {
-  const LayerDesc L = p.layers[blockIdx.x];
-  const int l = L.index;
-  const LayerState S = p.state[l];
-  __shared__ LayerPlan s_plan;
-  const int B = L.n_bins;      // this layer's own number of bins
+// The two ends of cell cc of level g as floats, rounded outwards.  Magic-constant layers keep
+// |cc| below 2^22 and g within the normal exponents, so both products are exact in float.
+__device__ __forceinline__ void cell_ends(long long cc, int g, bool exact_in_float, float* lf, float* rf) {
+  if (exact_in_float && g >= -100 && g <= 100) {
+    const float w = pow2f(-g);
+    *lf = __fmul_rn(__ll2float_rn(cc), w);
+    *rf = __fmul_rn(__ll2float_rn(cc + 1), w);
+  } else {
+    *lf = __double2float_rd(ldexp(static_cast<double>(cc), -g));
+    *rf = __double2float_ru(ldexp(static_cast<double>(cc + 1), -g));
+  }
+}
 
-  if (threadIdx.x == 0) {
+// Marks of table position i of a layer: edge cell (its closed interval meets two bins), cell -1
+// or 0 of the main segment.  A value-keyed layer has no marks.
+__device__ __forceinline__ unsigned cell_mark(const LayerPlan& P, const LayerState& S, int i) {
+  if (P.value) return 0u;
+  const int s = (i >= P.seg[1].offset && P.seg[1].cells > 0) ? 1 : 0;
+  const SegPlan& sp = P.seg[s];
+  const long long cc = sp.c0 + (i - sp.offset);
+  float lf, rf;
+  cell_ends(cc, sp.g, P.fast != 0, &lf, &rf);
+  unsigned mark = 0;
+  if (bin_of(lf, S.lo, S.scale, S.bmax) != bin_of(rf, S.lo, S.scale, S.bmax)) mark |= kCellEdge;
+  if (s == 0 && (cc == 0 || cc == -1)) mark |= kCellNearZero;
+  return mark;
+}
+
+// The plan of one layer from its final state: called by one thread.
+__device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, const LayerState& S,
+                                       unsigned min_lsb, LayerPlan* out) {
+  const int B = L.n_bins;      // this layer's own number of bins
+  {
     LayerPlan P;
     P.keyed = !(S.flags & (kFlagNonfinite | kFlagRange)) && L.n > 0;
     P.radius = __int_as_float(0x7f800000);
@@ -254,8 +278,8 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
     // and zero count is an exact function of the cell, and no element is ever on a boundary.
     // The grid comes from a sample; the counting loop checks every element against it.
     P.value = 0;
-    if (P.keyed && S.min_lsb != 0xFFFFFFFFu) {
-      const int g = 150 - static_cast<int>(S.min_lsb);
+    if (P.keyed && min_lsb != 0xFFFFFFFFu) {
+      const int g = 150 - static_cast<int>(min_lsb);
       if (g >= -100 && g <= 100) {
         const double span = ldexp(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
         const double far = ldexp(static_cast<double>(amax), g);
@@ -279,46 +303,83 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
         }
       }
     }
-    s_plan = P;
-    if (blockIdx.y == 0) p.plan[l] = P;   // every CTA of the layer derives the same plan
+    *out = P;
+  }
+}
+
+// Exact lower edge of bin b (1 <= b < n_bins) of a layer: the smallest float v with
+// bin_of(v) >= b, or +inf if no value up to the layer's maximum reaches the bin.  The bin
+// function is monotone, so the edge is found by walking the float order from an estimate
+// (lo + b / scale is within a few floats of it), with a bisection over [lo, hi] as the fallback.
+__device__ inline float bin_lower_edge(int b, const LayerState& S) {
+  if (bin_of(S.hi, S.lo, S.scale, S.bmax) < b) return __int_as_float(0x7f800000);
+  const unsigned klo = float_key(S.lo), khi = float_key(S.hi);   // bin(lo) = 0 < b <= bin(hi)
+  const float guess = __fadd_rn(S.lo, __fdiv_rn(static_cast<float>(b), S.scale));
+  unsigned k = float_key(guess);
+  if (guess == guess && k > klo && k <= khi) {
+    // walk down while the float below still reaches the bin, up while this one does not
+    int steps = 0;
+    if (bin_of(key_float(k), S.lo, S.scale, S.bmax) >= b) {
+      while (steps < 48 && k - 1u > klo && bin_of(key_float(k - 1u), S.lo, S.scale, S.bmax) >= b) { --k; ++steps; }
+      if (steps < 48 && bin_of(key_float(k - 1u), S.lo, S.scale, S.bmax) < b) return key_float(k);
+    } else {
+      while (steps < 48 && k < khi && bin_of(key_float(k), S.lo, S.scale, S.bmax) < b) { ++k; ++steps; }
+      if (steps < 48 && bin_of(key_float(k), S.lo, S.scale, S.bmax) >= b) return key_float(k);
+    }
+  }
+  unsigned a = klo, z = khi;   // bin(a) < b, bin(z) >= b
+  while (z - a > 1) {
+    const unsigned m = a + ((z - a) >> 1);
+    if (bin_of(key_float(m), S.lo, S.scale, S.bmax) >= b) z = m; else a = m;
+  }
+  return key_float(z);
+}
+
+constexpr int kPlanThreads = 256;
+constexpr int kPlanSamples = 1024;   // elements of a layer looked at for the grid it lies on
+
+// One layer per blockIdx.x; the gridDim.y CTAs of a layer all derive its plan (one thread each)
+// and share its bin edges.
+__global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) {
+  __shared__ LayerPlan s_plan;
+  __shared__ unsigned s_lsb;
+  const LayerDesc L = p.layers[blockIdx.x];
+  const int l = L.index;
+  const LayerState S = p.state[l];
+  // The grid the layer lies on, from a sample of kPlanSamples elements spread over the layer:
+  // 150 + the binary exponent of the coarsest grid 2^e that all sampled non-zero elements lie on
+  // (biased exponent + trailing zero bits of the 24-bit significand).  It only decides whether
+  // the layer is keyed by value; the counting loop checks every element against the grid.
+  if (threadIdx.x == 0) s_lsb = 0xFFFFFFFFu;
+  __syncthreads();
+  {
+    const long long n_s = min(L.n, static_cast<long long>(kPlanSamples));
+    const long long step = n_s > 0 ? L.n / n_s : 1;
+    unsigned lsb = 0xFFFFFFFFu;
+    for (long long i = threadIdx.x; i < n_s; i += kPlanThreads) {
+      const unsigned bits = __float_as_uint(__ldg(L.ptr + i * step));
+      const unsigned at = ((bits >> 23) & 0xFFu) + static_cast<unsigned>(__ffs(bits | 0x00800000u) - 1);
+      if ((bits & 0x7FFFFFFFu) != 0u) lsb = min(lsb, at);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) lsb = min(lsb, __shfl_xor_sync(0xffffffffu, lsb, o));
+    if ((threadIdx.x & 31) == 0 && lsb != 0xFFFFFFFFu) atomicMin(&s_lsb, lsb);
   }
   __syncthreads();
-  const LayerPlan P = s_plan;
-  if (!P.keyed) return;
-
-  // exact lower edge of every bin: smallest float v with bin_of(v) >= b
-  float* E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
-  const unsigned klo = float_key(S.lo), khi = float_key(S.hi);
-  // the layer's CTAs (gridDim.y of them) share the edges and the cells
-  const int first = blockIdx.y * kPlanThreads + threadIdx.x, stride = kPlanThreads * gridDim.y;
-  for (int b = first; b <= B; b += stride) {
-    float e;
-    if (b == 0) e = __int_as_float(0xff800000);          // -inf: bin 0 takes everything below
-    else if (b == B) e = __int_as_float(0x7f800000);     // +inf
-    else if (bin_of(S.hi, S.lo, S.scale, S.bmax) < b) e = __int_as_float(0x7f800000);
-    else {
-      unsigned a = klo, z = khi;   // bin(a) < b (bin(lo) = 0), bin(z) >= b
-      while (z - a > 1) {
-        unsigned m = a + ((z - a) >> 1);
-        if (bin_of(key_float(m), S.lo, S.scale, S.bmax) >= b) z = m; else a = m;
-      }
-      e = key_float(z);
-    }
-    E[b] = e;
+  if (threadIdx.x == 0) {
+    make_layer_plan(p, L, S, s_lsb, &s_plan);
+    if (blockIdx.y == 0) p.plan[l] = s_plan;
   }
-
-  // cell marks, both segments
-  unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
-  for (int i = first; i < P.total_cells; i += stride) {
-    const int s = (i >= P.seg[1].offset && P.seg[1].cells > 0) ? 1 : 0;
-    const SegPlan& sp = P.seg[s];
-    const long long cc = sp.c0 + (i - sp.offset);
-    const float lf = __double2float_rd(ldexp(static_cast<double>(cc), -sp.g));
-    const float rf = __double2float_ru(ldexp(static_cast<double>(cc + 1), -sp.g));
-    unsigned mark = 0;
-    if (bin_of(lf, S.lo, S.scale, S.bmax) != bin_of(rf, S.lo, S.scale, S.bmax)) mark |= kCellEdge;
-    if (s == 0 && (cc == 0 || cc == -1)) mark |= kCellNearZero;
-    init[i] = P.value ? 0u : mark;
+  __syncthreads();
+  if (!s_plan.keyed || s_plan.value) return;     // a value-keyed layer needs no bin edges
+  // exact lower edge of every bin (bin 0 takes everything below, nothing lies above the last)
+  float* E = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
+  for (int b = blockIdx.y * kPlanThreads + threadIdx.x; b <= L.n_bins; b += kPlanThreads * gridDim.y) {
+    float e;
+    if (b == 0) e = __int_as_float(0xff800000);
+    else if (b == L.n_bins) e = __int_as_float(0x7f800000);
+    else e = bin_lower_edge(b, S);
+    E[b] = e;
   }
 }
 

@@ -1,32 +1,115 @@
 // K1: per-layer range scan (min, max, non-finite / out-of-range flags) over all
-// layers in one launch, and the small finalisation kernel that turns the
-// result into the bin origin and scale shared by all histograms of the layer
-// (Sec. 3.3: binning at resolution r on the float tensor's own range).
+// layers in one launch.  The CTA that adds the last part of a layer (a ticket per
+// layer, no waiting) turns the result into the bin origin and scale shared by all
+// histograms of the layer (Sec. 3.3: binning at resolution r on the float tensor's
+// own range).
 #pragma once
 
 #include "common.cuh"
 
 namespace adapt {
 
-constexpr int kTile = 4096;          // elements per tile (in aligned indexing)
 constexpr int kRangeThreads = 128;   // 8 quads per thread per tile: loads first, then arithmetic
 
-constexpr unsigned kFlagDegenerate = 2u;
-constexpr unsigned kFlagNonfinite = 4u;
-constexpr unsigned kFlagRange = 8u;
+struct RangeParams {
+  const LayerDesc* layers;   // all layers (+ sentinel), tiles of kTile elements
+  int n_layers;
+  long long n_tiles;
+  LayerState* state;         // by LayerDesc::index; keys, flags and tickets start as the host set them
+  float* range_out;          // optional [n_layers][2] = {min, max}
+};
 
-__global__ void __launch_bounds__(kRangeThreads)
-range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long n_tiles,
-                  LayerState* __restrict__ state) {
+// Decodes the extremes of layer l into the bin origin, scale and flags.
+__device__ __forceinline__ void range_finalize_layer(const RangeParams& p, const LayerDesc* layer) {
+  const LayerDesc L = *layer;
+  LayerState* st = p.state + L.index;
+  const unsigned min_key = *reinterpret_cast<volatile unsigned*>(&st->min_key);
+  const unsigned max_key = *reinterpret_cast<volatile unsigned*>(&st->max_key);
+  unsigned flags = *reinterpret_cast<volatile unsigned*>(&st->flags);
+  float lo = 0.0f, hi = 0.0f;
+  if (L.n > 0 && !(flags & kFlagNonfinite)) {
+    lo = key_float(min_key);
+    hi = key_float(max_key);
+  }
+  const float w = __fsub_rn(hi, lo);
+  const float scale = (w == 0.0f) ? 0.0f : __fdiv_rn(static_cast<float>(L.n_bins), w);
+  if (L.n == 0 || hi == lo) flags |= kFlagDegenerate;
+  st->flags = flags; st->lo = lo; st->hi = hi; st->scale = scale;
+  st->bmax = static_cast<float>(L.n_bins - 1);
+  if (p.range_out) { p.range_out[2 * L.index] = lo; p.range_out[2 * L.index + 1] = hi; }
+}
+
+// One CTA's part of a layer (already reduced over the CTA) is added to the layer's state; returns
+// whether it was the last part, in which case the layer's bin origin and scale have been derived.
+__device__ __forceinline__ bool range_layer_commit(const RangeParams& p, const LayerDesc* layer,
+                                                unsigned kmin, unsigned kmax, unsigned flags, float asum,
+                                                unsigned nzero) {
+  LayerState* st = p.state + layer->index;
+  atomicMin(&st->min_key, kmin);
+  atomicMax(&st->max_key, kmax);
+  if (flags) atomicOr(&st->flags, flags);
+  if (asum == asum && asum < 3.0e38f) atomicAdd(&st->abs_sum, asum);
+  if (nzero) atomicAdd(&st->zero_count, nzero * static_cast<unsigned>(kTile / 4 / kRangeThreads));
+  __threadfence();
+  const unsigned done = atomicAdd(&st->ticket, 1u);
+  if (done + 1u != static_cast<unsigned>(layer->range_ctas)) return false;
+  __threadfence();
+  range_finalize_layer(p, layer);
+  return true;
+}
+
+// What a CTA does with its part of a layer once its tiles are read: reduce the threads' values
+// and add them to the layer's state.  Called by the whole CTA.
+__device__ __forceinline__ void range_layer_tail(const RangeParams& p, const LayerDesc* layer,
+                                                 float vmin, float vmax, unsigned flags, float asum,
+                                                 unsigned nzero) {
+  __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
+  __shared__ float s_abs[kRangeThreads / 32];
+  __shared__ unsigned s_zero[kRangeThreads / 32];
+  // -0.0 and +0.0 are the same value: canonicalise before taking keys
+  unsigned kmin = float_key(__fadd_rn(vmin, 0.0f));
+  unsigned kmax = float_key(__fadd_rn(vmax, 0.0f));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+    kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    flags |= __shfl_xor_sync(0xffffffffu, flags, o);
+    asum += __shfl_xor_sync(0xffffffffu, asum, o);
+    nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
+  }
+  const int w = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; s_zero[w] = nzero; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 1; i < kRangeThreads / 32; ++i) {
+      kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
+      asum += s_abs[i]; nzero += s_zero[i];
+    }
+    // the CTA that brings the last part of the layer finishes it
+    range_layer_commit(p, layer, kmin, kmax, flags, asum, nzero);
+  }
+  __syncthreads();
+}
+
+// Layers without elements have no tile and no last CTA: the first CTA settles them.
+__device__ __forceinline__ void range_prologue(const RangeParams& p) {
+  if (blockIdx.x == 0)
+    for (int l = threadIdx.x; l < p.n_layers; l += kRangeThreads)
+      if (p.layers[l].n == 0) range_finalize_layer(p, p.layers + l);
+}
+
+__global__ void __launch_bounds__(kRangeThreads, 8) range_scan_kernel(const __grid_constant__ RangeParams p) {
+  const LayerDesc* __restrict__ layers = p.layers;
+  const int n_layers = p.n_layers;
+  const long long n_tiles = p.n_tiles;
+  range_prologue(p);
+
   // contiguous slice of the global tile list for this CTA
   const long long per = (n_tiles + gridDim.x - 1) / gridDim.x;
   long long t = per * blockIdx.x;
   const long long t_end = min(n_tiles, t + per);
   if (t >= t_end) return;
 
-  __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
-  __shared__ float s_abs[kRangeThreads / 32];
-  __shared__ unsigned s_zero[kRangeThreads / 32], s_lsb[kRangeThreads / 32];
   int l = layer_of_tile(layers, n_layers, t);
 
   while (t < t_end) {
@@ -38,7 +121,7 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
     float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
     unsigned flags = 0;
     float asum = 0.0f;
-    unsigned nzero = 0, lsb = 0xFFFFFFFFu;
+    unsigned nzero = 0;
     for (; t < layer_tiles_end; ++t) {
       const long long j_tile = (t - L.tile_begin) * kTile;
       constexpr int kQ = kTile / 4 / kRangeThreads;
@@ -73,69 +156,15 @@ range_scan_kernel(const LayerDesc* __restrict__ layers, int n_layers, long long 
             vmin = fminf(vmin, v[q][k]);
             vmax = fmaxf(vmax, v[q][k]);
             asum += a;
-            if (q == 0) {                                  // one quad in kQ: a sample is enough
-              nzero += (a == 0.0f) ? 1u : 0u;
-              // position of the element's lowest set significand bit (hidden bit included)
-              const unsigned bits = __float_as_uint(v[q][k]);
-              const unsigned at = ((bits >> 23) & 0xFFu) + static_cast<unsigned>(__ffs(bits | 0x00800000u) - 1);
-              if (a != 0.0f) lsb = min(lsb, at);
-            }
+            if (q == 0) nzero += (a == 0.0f) ? 1u : 0u;   // one quad in kQ: a sample is enough
           }
         }
       }
     }
-    // -0.0 and +0.0 are the same value: canonicalise before taking keys
-    unsigned kmin = float_key(__fadd_rn(vmin, 0.0f));
-    unsigned kmax = float_key(__fadd_rn(vmax, 0.0f));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
-      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-      flags |= __shfl_xor_sync(0xffffffffu, flags, o);
-      asum += __shfl_xor_sync(0xffffffffu, asum, o);
-      nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
-      lsb = min(lsb, __shfl_xor_sync(0xffffffffu, lsb, o));
-    }
-    const int w = threadIdx.x >> 5;
-    if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; s_zero[w] = nzero; s_lsb[w] = lsb; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      for (int i = 1; i < kRangeThreads / 32; ++i) {
-        kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
-        asum += s_abs[i]; nzero += s_zero[i]; lsb = min(lsb, s_lsb[i]);
-      }
-      atomicMin(&state[L.index].min_key, kmin);
-      atomicMax(&state[L.index].max_key, kmax);
-      if (flags) atomicOr(&state[L.index].flags, flags);
-      if (asum == asum && asum < 3.0e38f) atomicAdd(&state[L.index].abs_sum, asum);
-      if (nzero) atomicAdd(&state[L.index].zero_count, nzero * static_cast<unsigned>(kTile / 4 / kRangeThreads));
-      if (lsb != 0xFFFFFFFFu) atomicMin(&state[L.index].min_lsb, lsb);
-    }
-    __syncthreads();
+    range_layer_tail(p, layers + l, vmin, vmax, flags, asum, nzero);
     ++l;
     while (l < n_layers && layers[l + 1].tile_begin <= t) ++l;  // skip empty layers
   }
-}
-
-// One thread per layer: decode min/max, derive the bin scale and flags.
-__global__ void range_finalize_kernel(const LayerDesc* __restrict__ layers, int n_layers,
-                                      LayerState* __restrict__ state,
-                                      float* __restrict__ range_out) {
-  int l = blockIdx.x * blockDim.x + threadIdx.x;
-  if (l >= n_layers) return;
-  LayerState s = state[l];
-  const int n_bins = layers[l].n_bins;
-  float lo = 0.0f, hi = 0.0f;
-  if (layers[l].n > 0 && !(s.flags & kFlagNonfinite)) {
-    lo = key_float(s.min_key);
-    hi = key_float(s.max_key);
-  }
-  float w = __fsub_rn(hi, lo);
-  float scale = (w == 0.0f) ? 0.0f : __fdiv_rn(static_cast<float>(n_bins), w);
-  if (layers[l].n == 0 || hi == lo) s.flags |= kFlagDegenerate;
-  s.lo = lo; s.hi = hi; s.scale = scale; s.bmax = static_cast<float>(n_bins - 1);
-  state[l] = s;
-  if (range_out) { range_out[2 * l] = lo; range_out[2 * l + 1] = hi; }
 }
 
 }  // namespace adapt

@@ -39,7 +39,6 @@
 
 #include "common.cuh"
 #include "k_plan.cuh"
-#include "k_range.cuh"
 
 namespace adapt {
 
@@ -63,7 +62,6 @@ struct KeyedParams {
   const LayerState* state;     // by LayerDesc::index
   const LayerPlan* plan;       // by LayerDesc::index
   const float* edges;          // [layer][n_bins + 1]
-  const unsigned* cell_init;   // [layer][cell_stride]
   unsigned* cell_count;        // [layer][cell_stride]   global cell counts
   unsigned* qe_hist;           // [layer][2][n_bins]     float histogram of the edge elements, per segment
   unsigned* u_hist;            // [layer][n_levels][n_bins]  receives the per-level corrections
@@ -559,18 +557,22 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
 
     // ---- per-layer set-up of the private tables ----------------------------------
     if (ok) {
-      const unsigned* init = p.cell_init + static_cast<size_t>(l) * p.cell_stride;
-      // 128-bit copies, several in flight per thread (the table and its rows are 16-byte aligned,
-      // the row has room for the last quad: the table size is a multiple of four)
-      const uint4* init4 = reinterpret_cast<const uint4*>(init);
-      uint4* cells4 = reinterpret_cast<uint4*>(cells);
-      const int n4 = (total_cells + 3) >> 2;
       if (by_value) {
         // no marks, and the cells may run over the other tables, which this layer does not use
+        uint4* cells4 = reinterpret_cast<uint4*>(cells);
+        const int n4 = (total_cells + 3) >> 2;
         for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = make_uint4(0u, 0u, 0u, 0u);
       } else {
-#pragma unroll 4
-        for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = __ldg(init4 + i);
+        // every count starts at zero; the marks follow below
+        if (fast) {
+          uint4* cells4 = reinterpret_cast<uint4*>(cells);
+          const int n4 = (total_cells + 3) >> 2;
+          for (int i = threadIdx.x; i < n4; i += kKeyedThreads) cells4[i] = make_uint4(0u, 0u, 0u, 0u);
+        } else {
+          const LayerState S = p.state[l];
+          const LayerPlan P = p.plan[l];
+          for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) cells[i] = cell_mark(P, S, i);
+        }
         for (int i = threadIdx.x; i < p.n_bins * (1 + p.d_levels); i += kKeyedThreads) qe[i] = 0;
         const float* layer_edges = p.edges + static_cast<size_t>(l) * (p.n_bins + 1);
         for (int i = threadIdx.x; i <= L.n_bins; i += kKeyedThreads) edges[i] = __ldg(layer_edges + i);
@@ -582,6 +584,29 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
         cells[dummy_pos - lane + threadIdx.x] = kCellEdge | kCellNearZero | kCellOnGrid;
     }
     __syncthreads();
+    if (ok && fast && !by_value) {
+      // Marks of a magic-constant layer, from the bin edges instead of cell by cell: the cell
+      // whose closed interval holds the exact edge E[b] (lf < E[b] <= rf, both ends exact here)
+      // is cell ceil(E[b] 2^G) - 1 - the same cells the cell-by-cell test marks.
+      for (int b = 1 + threadIdx.x; b < L.n_bins; b += kKeyedThreads) {
+        const float e = edges[b];
+        if (!(fabsf(e) <= 3.402823466e38f)) continue;
+#pragma unroll
+        for (int sg = 0; sg < 2; ++sg) {
+          if (sg == 1 && c.offset[1] >= total_cells) break;      // no auxiliary segment
+          const float t = ceilf(__fmul_rn(e, c.two_g[sg]));      // exact product
+          if (!(fabsf(t) < 8388608.0f)) continue;
+          const int n_seg = (sg == 0) ? (c.offset[1] - c.offset[0]) : (total_cells - c.offset[1]);
+          const int ci = __float2int_rz(t) - 1 - static_cast<int>(c.c0[sg]);
+          if (ci >= 0 && ci < n_seg) atomicOr(&cells[c.offset[sg] + ci], kCellEdge);
+        }
+      }
+      if (threadIdx.x < 2) {
+        const int ci = -static_cast<int>(threadIdx.x) - static_cast<int>(c.c0[0]);   // cells 0 and -1
+        if (ci >= 0 && ci < c.offset[1] - c.offset[0]) atomicOr(&cells[c.offset[0] + ci], kCellNearZero);
+      }
+      __syncthreads();
+    }
 
     if (ok) {
       const int k0 = static_cast<int>(t - L.tile_begin), k1 = static_cast<int>(layer_tiles_end - L.tile_begin);

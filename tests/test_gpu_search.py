@@ -281,8 +281,9 @@ def test_nonfinite_and_out_of_range_layers_are_flagged(B):
     wl, fl = W.candidate_grid([4, 8])
     grid = B.Grid(wl, fl)
     dev = G.to_device([good, bad_nan, bad_inf, bad_big, good])
-    res = B.adapt_precision_search_ex(dev, grid, 64, want_hist=True)
+    res = B.adapt_precision_search_ex(dev, grid, 64, want_hist=True, want_status=True)
     torch.cuda.synchronize()
+    assert list(res.status.cpu().numpy()) == [B.OK, B.ERR_NONFINITE, B.ERR_NONFINITE, B.ERR_RANGE, B.OK]
     flags = res.best.cpu().numpy()[:, 3]
     assert not flags[0] & (B.FLAG_NONFINITE | B.FLAG_RANGE)
     assert flags[1] & B.FLAG_NONFINITE and flags[2] & B.FLAG_NONFINITE
