@@ -476,6 +476,19 @@ int adapt_format_search(const float* const* tensors, const int64_t* lens, int n_
 int adapt_format_quantize(const float* x, int64_t n, int kind, int a, int b, int round_mode,
                           uint64_t seed, int layer, float* values_out, void* stream);
 
+/* The bounds-checking build of the library (libadapt_b200_check.so, made by
+ * `python -m paper_2107_13490_b200.build --check`; the stand-in for a memory checker
+ * where none can be run).  In it every table index that the kernels form from
+ * the data - cell positions taken from float bit patterns, bins, sub-cells, queue
+ * slots - is tested against its table's size; an index outside is skipped (never
+ * dereferenced, nothing traps) and the first such event is kept in a device word.
+ *   out  HOST uint32[4] or NULL: {events since the library was loaded or the word
+ *        was last cleared, site number of the first event, its index, its limit}
+ *   clear non-zero resets the word after reading
+ * Returns 1 in the bounds-checking build, 0 in the normal build (out is then all
+ * zero), a negative adapt_status on a CUDA error.  Synchronises the device. */
+int adapt_bounds_check_status(uint32_t* out, int clear);
+
 /* Frees every library-owned device and pinned buffer of the current device's
  * caches.  Safe to call at any time no library work is in flight. */
 int adapt_release(void);

@@ -15,7 +15,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libadapt_b200.so")
+# ADAPT_B200_LIBRARY names another build of the same library (the bounds-checking one)
+LIB_PATH = os.environ.get("ADAPT_B200_LIBRARY") or os.path.join(_HERE, "libadapt_b200.so")
 
 ROUND_RNE = 0
 ROUND_STOCHASTIC = 1
@@ -32,7 +33,7 @@ EXPORTS = (
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
     "adapt_format_search_workspace_bytes", "adapt_format_search", "adapt_format_quantize",
-    "adapt_pushup",
+    "adapt_pushup", "adapt_bounds_check_status",
 )
 STRATEGY_MIN, STRATEGY_MEAN, STRATEGY_MAX = 0, 1, 2
 FMT_FIXED, FMT_BFP, FMT_FLOAT = 0, 1, 2
@@ -111,6 +112,8 @@ def lib():
         L.adapt_gradient_diversity.restype = C.c_int
         L.adapt_gradient_diversity.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                C.c_void_p]
+        L.adapt_bounds_check_status.restype = C.c_int
+        L.adapt_bounds_check_status.argtypes = [C.c_void_p, C.c_int]
         L.adapt_pushup.restype = C.c_int
         L.adapt_pushup.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                    C.c_void_p]
@@ -198,6 +201,15 @@ def adapt_kernel_times(reset: bool = False):
     _check(lib().adapt_kernel_times(ms.ctypes.data, cnt.ctypes.data, 1 if reset else 0),
            "adapt_kernel_times")
     return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def adapt_bounds_check_status(clear: bool = False):
+    """adapt_bounds_check_status of adapt.h: (checking build?, uint32[4] = {events, site, index, limit})."""
+    word = np.zeros(4, dtype=np.uint32)
+    rc = lib().adapt_bounds_check_status(word.ctypes.data, 1 if clear else 0)
+    if rc < 0:
+        raise AdaptError(-rc, "adapt_bounds_check_status")
+    return bool(rc), word
 
 
 def adapt_release() -> None:

@@ -1492,6 +1492,25 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
   return ADAPT_OK;
 }
 
+int adapt_bounds_check_status(uint32_t* out, int clear) {
+  if (out) out[0] = out[1] = out[2] = out[3] = 0;
+#ifdef ADAPT_CHECK_BOUNDS
+  unsigned word[4] = {0, 0, 0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpyFromSymbol(word, adapt::g_bounds_error, sizeof(word)) != cudaSuccess)
+    return -ADAPT_ERR_CUDA;
+  if (out) for (int i = 0; i < 4; ++i) out[i] = word[i];
+  if (clear) {
+    const unsigned zero[4] = {0, 0, 0, 0};
+    if (cudaMemcpyToSymbol(adapt::g_bounds_error, zero, sizeof(zero)) != cudaSuccess) return -ADAPT_ERR_CUDA;
+  }
+  return 1;
+#else
+  (void)clear;
+  return 0;
+#endif
+}
+
 int adapt_release(void) {
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceCache* dc = nullptr;

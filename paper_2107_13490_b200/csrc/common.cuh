@@ -47,6 +47,29 @@ struct LayerState {
                         // (the last one selects the layer's format)
 };
 
+// Index checks of the bounds-checking build (-DADAPT_CHECK_BOUNDS; the stand-in for a memory
+// checker): every table index that is formed from the data - a cell position from a float's
+// bit pattern, a bin, a sub-cell, a queue slot - goes through ADAPT_IN_BOUNDS, which in that
+// build skips an access outside [0, limit) and records the first such event in a device word
+// that adapt_bounds_check_status returns; nothing traps.  In the normal build the macro is
+// `true` and the checks cost nothing.
+#ifdef ADAPT_CHECK_BOUNDS
+__device__ unsigned g_bounds_error[4];   // {events, site of the first, its index, its limit}
+__device__ __forceinline__ bool index_in_bounds(long long idx, long long limit, int site) {
+  if (idx >= 0 && idx < limit) return true;
+  if (atomicAdd(&g_bounds_error[0], 1u) == 0u) {
+    g_bounds_error[1] = static_cast<unsigned>(site);
+    g_bounds_error[2] = static_cast<unsigned>(idx);
+    g_bounds_error[3] = static_cast<unsigned>(limit);
+  }
+  return false;
+}
+#define ADAPT_IN_BOUNDS(idx, limit, site) \
+  ::adapt::index_in_bounds(static_cast<long long>(idx), static_cast<long long>(limit), (site))
+#else
+#define ADAPT_IN_BOUNDS(idx, limit, site) true
+#endif
+
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).
 __device__ __forceinline__ unsigned float_key(float v) {
   unsigned b = __float_as_uint(v);

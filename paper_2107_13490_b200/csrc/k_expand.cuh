@@ -87,20 +87,20 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
           v = __fmul_rn(r, pow2f(-f));
           if (r == 0.0f) zero += m;
         }
-        atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+        if (ADAPT_IN_BOUNDS(bin_of(v, S.lo, S.scale, S.bmax), B, 30)) atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
       } else if (is_q || f >= sp.g) {
         // interior cells only (the marks are recomputed: a cell whose closed interval meets two bins)
         float lf, rf;
         cell_ends(cc, sp.g, P.fast != 0, &lf, &rf);
         const int bl = bin_of(lf, S.lo, S.scale, S.bmax);
-        if (bl == bin_of(rf, S.lo, S.scale, S.bmax)) atomicAdd(&s_hist[bl], m);
+        if (bl == bin_of(rf, S.lo, S.scale, S.bmax) && ADAPT_IN_BOUNDS(bl, B, 31)) atomicAdd(&s_hist[bl], m);
       } else {
         const int d = sp.g - f;                      // 1..32
         const long long a = cc >> d;                 // floor(c / 2^d)
         const long long rem = cc - (a << d);
         const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
         const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
-        atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+        if (ADAPT_IN_BOUNDS(bin_of(v, S.lo, S.scale, S.bmax), B, 32)) atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
         if (r == 0) zero += m;
       }
     }
@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
         const unsigned ms[4] = {m4.x, m4.y, m4.z, m4.w};
         if ((m4.x | m4.y | m4.z | m4.w) == 0u) continue;
         const int id = k0 / kSubCells;                      // the four share their edge cell
+        if (!ADAPT_IN_BOUNDS(id + 1, B + 1, 35)) continue;
         const long long cc = static_cast<long long>(ceil(ldexp(static_cast<double>(E[id + 1]), sp.g))) - 1;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -142,14 +143,14 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
             const float l2 = __double2float_rd(ldexp(static_cast<double>(jj), -gs));
             const float r2 = __double2float_ru(ldexp(static_cast<double>(jj + 1), -gs));
             const int bl = bin_of(l2, S.lo, S.scale, S.bmax);
-            if (bl == bin_of(r2, S.lo, S.scale, S.bmax)) atomicAdd(&s_hist[bl], m);
+            if (bl == bin_of(r2, S.lo, S.scale, S.bmax) && ADAPT_IN_BOUNDS(bl, B, 33)) atomicAdd(&s_hist[bl], m);
           } else {
             const int d = gs - f;                        // 1..kSubBits
             const long long a = jj >> d;
             const long long rem = jj - (a << d);
             const long long r = a + ((rem >= (1ll << (d - 1))) ? 1 : 0);
             const float v = __fmul_rn(__ll2float_rn(r), pow2f(-f));
-            atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
+            if (ADAPT_IN_BOUNDS(bin_of(v, S.lo, S.scale, S.bmax), B, 34)) atomicAdd(&s_hist[bin_of(v, S.lo, S.scale, S.bmax)], m);
           }
         }
       }

@@ -193,8 +193,10 @@ __device__ __forceinline__ void format_quad(const float (&v)[4], unsigned m, lon
         cls = eb ? static_cast<int>(eb) + 23 : 32 - __clz(mant);   // e + 150
         p2 = eb ? (mant == 0u) : ((mant & (mant - 1u)) == 0u);
       }
-      atomicAdd(&s_cls[0][cls], 1u);
-      if (p2) atomicAdd(&s_cls[1][cls], 1u);
+      if (ADAPT_IN_BOUNDS(cls, kExpClasses, 40)) {
+        atomicAdd(&s_cls[0][cls], 1u);
+        if (p2) atomicAdd(&s_cls[1][cls], 1u);
+      }
     }
   }
   unsigned hb = hist_base;
@@ -203,7 +205,9 @@ __device__ __forceinline__ void format_quad(const float (&v)[4], unsigned m, lon
     if (kind == kRuleIdentity) {
 #pragma unroll
       for (int k = 0; k < 4; ++k)
-        if (!kMasked || ((m >> k) & 1u)) format_shared_inc(hb + format_bin_offset(v[k], lo, scale, top));
+        if ((!kMasked || ((m >> k) & 1u)) &&
+            ADAPT_IN_BOUNDS(static_cast<int>(format_bin_offset(v[k], lo, scale, top) >> 2) - 0x0B400000, hist_stride >> 2, 41))
+          format_shared_inc(hb + format_bin_offset(v[k], lo, scale, top));
       continue;
     }
     float xq[4];
@@ -218,7 +222,9 @@ __device__ __forceinline__ void format_quad(const float (&v)[4], unsigned m, lon
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k)
-      if (!kMasked || ((m >> k) & 1u)) format_shared_inc(hb + format_bin_offset(xq[k], lo, scale, top));
+      if ((!kMasked || ((m >> k) & 1u)) &&
+          ADAPT_IN_BOUNDS(static_cast<int>(format_bin_offset(xq[k], lo, scale, top) >> 2) - 0x0B400000, hist_stride >> 2, 42))
+        format_shared_inc(hb + format_bin_offset(xq[k], lo, scale, top));
     if (kStochastic) {
       // zero count by a warp reduction (the stochastic threshold is per element)
       unsigned nz = 0;

@@ -82,13 +82,17 @@ __device__ __forceinline__ void direct_quad(const float (&v)[4], unsigned m, lon
   for (int k = 0; k < 4; ++k) {
     const bool valid = !kMasked || ((m >> k) & 1u);
     pr[k] = 0.0f;
-    if (valid && do_q) shared_inc(hist_base + bin_offset_magic(v[k], lo, scale, top));
+    if (valid && do_q) {
+      const unsigned off = bin_offset_magic(v[k], lo, scale, top);
+      if (ADAPT_IN_BOUNDS(static_cast<int>(off >> 2) - 0x0B400000, hist_stride >> 2, 20)) shared_inc(hist_base + off);
+    }
     if (kStochastic) {
       const unsigned h = hash24(p.seed, static_cast<unsigned long long>(layer_id),
                                 static_cast<unsigned long long>(index0 + k));
       pr[k] = __fmul_rn(__uint2float_rn(h), 5.9604644775390625e-8f);  // k * 2^-24, exact
     } else if (valid) {
-      atomicAdd(&s_zlevel[highest_zero_level(v[k]) + 1], 1u);
+      if (ADAPT_IN_BOUNDS(highest_zero_level(v[k]) + 1, kMaxFl + 2, 21))
+        atomicAdd(&s_zlevel[highest_zero_level(v[k]) + 1], 1u);
     }
   }
   // the thread walks the fraction lengths with its four elements in registers
@@ -100,7 +104,7 @@ __device__ __forceinline__ void direct_quad(const float (&v)[4], unsigned m, lon
     for (int k = 0; k < 4; ++k) {
       const float r = round_scaled<kStochastic>(v[k], two_f, pr[k]);
       const unsigned off = bin_offset_magic(__fmul_rn(r, inv_f), lo, scale, top);
-      if (!kMasked || ((m >> k) & 1u)) {
+      if ((!kMasked || ((m >> k) & 1u)) && ADAPT_IN_BOUNDS(static_cast<int>(off >> 2) - 0x0B400000, hist_stride >> 2, 22)) {
         shared_inc(hb + off);
         if (kStochastic) nz += (r == 0.0f) ? 1u : 0u;
       }

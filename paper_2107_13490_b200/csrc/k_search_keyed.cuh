@@ -123,6 +123,7 @@ struct LayerCtx {
   unsigned* sub;               // global, this layer's [2][n_bins][kSubCells]
   unsigned* sub_s;             // shared [kSubSharedIds][kSubCells]: main segment's, when sub_base >= 0
   int sub_base;
+  int table_words;             // words of the cell table this layer may touch (cells + dummy slots)
   int value;                   // value-keyed layer
   unsigned* q_hist;            // global, this layer's [n_bins]
   unsigned* stray;             // shared: elements of a value-keyed layer that are off its grid
@@ -147,13 +148,15 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   if (x == 0.0f) {
     // only the dense form lets an exact zero through: it was counted in the cell [0, 2^-G),
     // where no zero belongs (zeros are the layer size minus all cell counts)
-    atomicSub(&c.cells[c.zero_pos], 1u);
+    if (ADAPT_IN_BOUNDS(c.zero_pos, c.table_words, 10)) atomicSub(&c.cells[c.zero_pos], 1u);
     return;
   }
   const int s = (fabsf(x) < c.radius) ? 0 : 1;
   const float z = __fmul_rn(x, c.two_g[s]);
   const float cf = floorf(z);
   int ci = __float2int_rz(__fsub_rn(cf, c.c0f[s])) + 1;     // cell index inside the segment
+  if (!ADAPT_IN_BOUNDS(c.offset[s] + ci - 1, c.total_cells, 11) ||
+      !ADAPT_IN_BOUNDS(c.offset[s] + ci, c.total_cells, 12)) return;
   if (z == cf && grid_point_goes_left(c.c0[s] + ci)) {
     // on the grid and belonging to the left cell: move its count there
     atomicSub(&c.cells[c.offset[s] + ci], 1u);
@@ -198,12 +201,17 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
       r2 = __double2float_ru(ldexp(static_cast<double>(jj + 1), -(g + kSubBits)));
     }
     const int id = bin_of(lf, c.lo, c.scale, c.bmax);
-    if (s == 0 && c.sub_base >= 0) atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
-    else atomicAdd(&c.sub[(static_cast<size_t>(s) * B + id) * kSubCells + j], 1u);
+    if (s == 0 && c.sub_base >= 0) {
+      if (ADAPT_IN_BOUNDS((id - c.sub_base) * kSubCells + j, kSubSharedIds * kSubCells, 13))
+        atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
+    } else if (ADAPT_IN_BOUNDS(id, B, 14)) {
+      atomicAdd(&c.sub[(static_cast<size_t>(s) * B + id) * kSubCells + j], 1u);
+    }
     // an interior sub-cell (its closed interval in one bin) settles the element
     if (bin_of(l2, c.lo, c.scale, c.bmax) == bin_of(r2, c.lo, c.scale, c.bmax)) return;
   }
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
+  if (!ADAPT_IN_BOUNDS(b0, B, 15)) return;
   if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
   const float e_lo = c.E[b0], e_hi = c.E[b0 + 1];
   // distance to the bin's two edges, rounded down: a level is safe once 2^-(f+1) < margin
@@ -217,6 +225,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     const float v = __fmul_rn(r, pow2f(-f));
     if (v >= e_lo && v < e_hi) continue;       // still in b0 (edges are exact)
     const int b = bin_of(v, c.lo, c.scale, c.bmax);
+    if (!ADAPT_IN_BOUNDS(b, B, 16)) continue;
     const int j = f - fs;
     if (s == 0 && j < c.d_levels) {
       atomicAdd(&c.d[j * B + b], 1);
@@ -235,11 +244,12 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
 __device__ __noinline__ void handle_stray(const LayerCtx& c, float x) {
   const int B = c.n_bins;
   atomicAdd(c.stray, 1u);
-  atomicAdd(&c.q_hist[bin_of(x, c.lo, c.scale, c.bmax)], 1u);
+  if (ADAPT_IN_BOUNDS(bin_of(x, c.lo, c.scale, c.bmax), B, 17)) atomicAdd(&c.q_hist[bin_of(x, c.lo, c.scale, c.bmax)], 1u);
   for (int f = 0; f < c.n_levels; ++f) {
     const float r = rintf(__fmul_rn(x, pow2f(f)));
     const float v = __fmul_rn(r, pow2f(-f));
-    atomicAdd(&c.u_hist[static_cast<size_t>(f) * B + bin_of(v, c.lo, c.scale, c.bmax)], 1u);
+    if (ADAPT_IN_BOUNDS(bin_of(v, c.lo, c.scale, c.bmax), B, 18))
+      atomicAdd(&c.u_hist[static_cast<size_t>(f) * B + bin_of(v, c.lo, c.scale, c.bmax)], 1u);
     if (r == 0.0f) atomicAdd(&c.zeros[f], 1ull);
   }
 }
@@ -252,6 +262,9 @@ struct CellFn {
   unsigned grid_mask;           // masked form: low significand bits every grid point has zero
   unsigned grid_mul;            // dense form: 2^(32 - those bits)
   unsigned cell_base;           // dense form: shared-memory byte address of position 0, minus 4 * 0x4B400000
+#ifdef ADAPT_CHECK_BOUNDS
+  int table_words;              // words of the cell table this layer may touch
+#endif
 };
 
 // How the counting loop finds an element's table position and its grid-point flag.
@@ -318,7 +331,7 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
       const float rd = __fmaf_rd(x, fn.two_g0, fn.magic0);
       const bool stray = __fmaf_ru(x, fn.two_g0, fn.magic0) != rd;
       const int pos = (x != 0.0f && !stray) ? __float_as_int(rd) - 0x4B400000 : dummy_pos;
-      atomicAdd(&cells[pos], 1u);
+      if (ADAPT_IN_BOUNDS(pos, fn.table_words, 1)) atomicAdd(&cells[pos], 1u);
       old[k] = stray ? kCellOnGrid : 0u;
       any |= old[k];
     }
@@ -336,8 +349,9 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
       const bool inner = fabsf(x) < fn.radius;
       const float rd = inner ? __fmaf_rd(x, fn.two_g0, fn.magic0) : __fmaf_rd(x, fn.two_g1, fn.magic1);
       const unsigned addr = __float_as_uint(rd) * 4u + fn.cell_base;
-      unsigned o;
-      asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(o) : "r"(addr) : "memory");
+      unsigned o = 0u;
+      if (ADAPT_IN_BOUNDS(static_cast<int>(__float_as_uint(rd)) - 0x4B400000, fn.table_words, 2))
+        asm volatile("atom.shared.add.u32 %0, [%1], 1;" : "=r"(o) : "r"(addr) : "memory");
       old[k] = o;
       any |= o;
       tmin = min(tmin, __float_as_uint(x) * fn.grid_mul);
@@ -354,7 +368,7 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
     unsigned grid_bit;
     int pos = cell_position<kMode>(x, fn, &grid_bit);
     pos = (x != 0.0f) ? pos : dummy_pos;
-    const unsigned o = atomicAdd(&cells[pos], 1u) + grid_bit;
+    const unsigned o = (ADAPT_IN_BOUNDS(pos, fn.table_words, 3) ? atomicAdd(&cells[pos], 1u) : 0u) + grid_bit;
     old[k] = o;
     any |= o;
   }
@@ -376,7 +390,7 @@ __device__ __forceinline__ void keyed_queue(const LayerCtx& c, float* queue, uns
       if (kMode == kCellDense) push = push || __float_as_uint(v[k]) * fn.grid_mul == 0u;
       const unsigned pm = __ballot_sync(0xffffffffu, push);
       if (pm) {
-        if (push) queue[qn + __popc(pm & lt)] = v[k];
+        if (push && ADAPT_IN_BOUNDS(qn + __popc(pm & lt), kQueueCap, 4)) queue[qn + __popc(pm & lt)] = v[k];
         qn += __popc(pm);
       }
     }
@@ -441,6 +455,9 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
   fn.grid_mask = c.grid_mask;
   fn.grid_mul = c.grid_mul;
   fn.cell_base = static_cast<unsigned>(__cvta_generic_to_shared(cells)) - 4u * 0x4B400000u;
+#ifdef ADAPT_CHECK_BOUNDS
+  fn.table_words = c.table_words;
+#endif
   unsigned qn = 0;             // entries in this warp's queue (same in every lane)
   // a ragged tile pads with zeros, which the dense form must not see
   constexpr int kRagged = kMode == kCellDense ? kCellMasked : kMode;
@@ -530,6 +547,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.sub_s = sub_s; c.sub_base = P->refined ? P->sub_base : -1;
       c.grid_mul = P->grid_mul;
       c.value = P->value;
+      c.table_words = (P->value ? keyed_value_cap(p.cell_cap, p.n_bins, p.d_levels) : p.cell_cap) + kDummySlots;
       c.q_hist = p.q_hist + static_cast<size_t>(l) * p.n_bins;
       c.stray = &s_stray;
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
