@@ -667,11 +667,18 @@ def main():
         host_out = B.SearchResult(torch.empty((len(xs), n_cand), dtype=torch.float64).pin_memory(),
                                   torch.empty((len(xs), n_cand), dtype=torch.int64).pin_memory(),
                                   torch.empty((len(xs), 4), dtype=torch.int32).pin_memory())
-        host_codes = [torch.empty(n, dtype=torch.int32).pin_memory() for n in lens]
+        # the narrowest code type that holds every layer's selected word length (known from the
+        # device-resident steps above): the download is that many bytes per element
+        wl_max = int(out.best[:, 0].max().item())
+        code_bits = 8 if wl_max <= 8 else (16 if wl_max <= 16 else 32)
+        code_dtype = {8: torch.int8, 16: torch.int16, 32: torch.int32}[code_bits]
+        host_codes = [torch.empty(n, dtype=code_dtype).pin_memory() for n in lens]
 
         def e2e_step():
-            B.adapt_precision_switch_host(pinned, grid, w.n_bins, round_mode=round_mode,
-                                          seed=w.seed, out=host_out, codes_out=host_codes)
+            _, _, unfit = B.adapt_precision_switch_host_packed(pinned, grid, w.n_bins, code_bits,
+                                                               round_mode=round_mode, seed=w.seed,
+                                                               out=host_out, codes_out=host_codes)
+            assert not unfit.any()
 
         e2e_step()
         S.barrier()
@@ -683,11 +690,14 @@ def main():
         dt = time.perf_counter() - t0
         S.barrier()
         e2e_value, _ = S.job_throughput(float(total) * n_cand * args.e2e_steps, dt, dev)
-        res_bytes = len(xs) * (n_cand * 16 + 16)
+        res_bytes = len(xs) * (n_cand * 16 + 16 + 4)
         e2e = {"value": e2e_value, "unit": UNIT, "steps": args.e2e_steps,
                "ms_per_step": dt / args.e2e_steps * 1e3,
-               "h2d_bytes_per_step": 4 * total, "d2h_bytes_per_step": res_bytes + 4 * total,
-               "api": "adapt_precision_switch_host (pinned host buffers in, results and codes out)"}
+               "h2d_bytes_per_step": 4 * total, "d2h_bytes_per_step": res_bytes + code_bits // 8 * total,
+               "code_bits": code_bits, "largest_selected_wl": wl_max,
+               "api": "adapt_precision_switch_host_packed (pinned host buffers in; results and codes of "
+                      "the narrowest type that holds every selected word length out, downloaded slice "
+                      "by slice behind the quantize kernel)"}
         del host_codes
 
     # ---- the other configs and other value classes (single GPU, default workload only) -----

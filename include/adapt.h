@@ -304,7 +304,7 @@ int adapt_precision_search_ex(const float* const* tensors, const int64_t* lens,
  * copies the layers to a library-owned device buffer, runs the search,
  * copies the results back and synchronises the stream before returning, so
  * data errors are returned as ADAPT_ERR_NONFINITE / ADAPT_ERR_RANGE.
- * opts->workspace, hist_out and range_out must be NULL/0 here. */
+ * opts->workspace, hist_out, range_out and status_out must be NULL/0 here. */
 int adapt_precision_search_host(const float* const* tensors, const int64_t* lens,
                                 int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
                                 double* kld_out, int64_t* zeros_out, int32_t* best_out,
@@ -320,6 +320,19 @@ int adapt_precision_switch_host(const float* const* tensors, const int64_t* lens
                                 int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
                                 double* kld_out, int64_t* zeros_out, int32_t* best_out,
                                 int32_t* const* codes_out, const adapt_search_opts* opts);
+
+/* adapt_precision_switch_host with packed codes: codes_out[l] is HOST int8[lens[l]]
+ * (code_bits 8), int16[...] (16) or int32[...] (32).  The codes leave the device slice
+ * by slice (about 64 MB of input each), every slice's download overlapping the next
+ * slice's kernel, so the narrower the codes the shorter the call.  A layer whose
+ * selected WL exceeds code_bits gets no codes (its buffer is left as it was) and, when
+ * unfit_out is given (HOST int32[n_layers]), unfit_out[l] = WL; the other entries are 0.
+ * (Algorithm 1: the Quantize of every layer after the switch.)  Synchronous. */
+int adapt_precision_switch_host_packed(const float* const* tensors, const int64_t* lens,
+                                       int n_layers, const adapt_grid* wl_fl_grid, int n_bins,
+                                       double* kld_out, int64_t* zeros_out, int32_t* best_out,
+                                       int code_bits, void* const* codes_out, int32_t* unfit_out,
+                                       const adapt_search_opts* opts);
 
 /* Host-buffer form of adapt_quantize_ex: x and codes_out are HOST memory;
  * synchronous. */

@@ -29,7 +29,7 @@ EXPORTS = (
     "adapt_requantize_selected_batch", "adapt_quantize_selected_batch_packed",
     "adapt_search_workspace_bytes", "adapt_gradient_diversity", "adapt_normalize_gradients",
     "adapt_precision_search", "adapt_precision_search_ex", "adapt_precision_search_host",
-    "adapt_precision_switch_host",
+    "adapt_precision_switch_host", "adapt_precision_switch_host_packed",
     "adapt_quantize_host", "adapt_kernel_launch_count", "adapt_kernel_timing",
     "adapt_kernel_times", "adapt_precision_search_static", "adapt_release",
     "adapt_format_search_workspace_bytes", "adapt_format_search", "adapt_format_quantize",
@@ -129,6 +129,9 @@ def lib():
         L.adapt_precision_search_host.argtypes = search_args + [C.POINTER(AdaptSearchOpts)]
         L.adapt_precision_switch_host.restype = C.c_int
         L.adapt_precision_switch_host.argtypes = search_args + [C.c_void_p, C.POINTER(AdaptSearchOpts)]
+        L.adapt_precision_switch_host_packed.restype = C.c_int
+        L.adapt_precision_switch_host_packed.argtypes = search_args + [C.c_int, C.c_void_p, C.c_void_p,
+                                                                       C.POINTER(AdaptSearchOpts)]
         L.adapt_precision_search_static.restype = C.c_int
         L.adapt_precision_search_static.argtypes = search_args + [C.c_void_p]
         L.adapt_quantize_host.restype = C.c_int
@@ -537,6 +540,38 @@ def adapt_precision_switch_host(tensors: Sequence[torch.Tensor], grid: Grid, n_b
                                              cptr.ctypes.data, C.byref(o)),
            "adapt_precision_switch_host")
     return out, codes_out
+
+
+def adapt_precision_switch_host_packed(tensors: Sequence[torch.Tensor], grid: Grid, n_bins: int,
+                                       code_bits: int, round_mode: int = ROUND_RNE, seed: int = 0,
+                                       layer_base: int = 0, eps: float = 0.0,
+                                       out: Optional[SearchResult] = None,
+                                       codes_out: Optional[Sequence[torch.Tensor]] = None):
+    """adapt_precision_switch_host_packed of adapt.h.  Returns (SearchResult, list of CPU code
+    tensors of code_bits width, int32[L] numpy array of the word lengths that did not fit)."""
+    assert all(not t.is_cuda for t in tensors)
+    ptrs, lens = _marshal_tensors(tensors)
+    L, Cn = len(tensors), len(grid)
+    dt = {8: torch.int8, 16: torch.int16, 32: torch.int32}[code_bits]
+    if out is None:
+        out = SearchResult(torch.empty((L, Cn), dtype=torch.float64),
+                           torch.empty((L, Cn), dtype=torch.int64),
+                           torch.empty((L, 4), dtype=torch.int32))
+    if codes_out is None:
+        codes_out = [torch.empty(t.numel(), dtype=dt) for t in tensors]
+    assert all(c.dtype == dt for c in codes_out)
+    cptr = np.array([c.data_ptr() for c in codes_out], dtype=np.uint64)
+    unfit = np.zeros(L, dtype=np.int32)
+    o = AdaptSearchOpts()
+    o.round_mode, o.layer_base, o.seed, o.eps = round_mode, layer_base, seed, eps
+    o.stream = _stream_handle(None)
+    _check(lib().adapt_precision_switch_host_packed(ptrs.ctypes.data, lens.ctypes.data, L,
+                                                    C.byref(grid.c), n_bins, out.kld.data_ptr(),
+                                                    out.zeros.data_ptr(), out.best.data_ptr(),
+                                                    code_bits, cptr.ctypes.data, unfit.ctypes.data,
+                                                    C.byref(o)),
+           "adapt_precision_switch_host_packed")
+    return out, codes_out, unfit
 
 
 def adapt_quantize_host(x: torch.Tensor, wl: int, fl: int, round_mode: int = ROUND_RNE,

@@ -109,6 +109,9 @@ struct DeviceCache {
   void* div_buf = nullptr;     size_t div_buf_bytes = 0;     // gradient diversity: tables + sums
   PinnedSlot ring[kRingSlots];
   int ring_next = 0;
+  cudaStream_t copy_stream = nullptr;   // host-form calls: downloads that overlap the kernels
+  cudaEvent_t slice_done[2] = {nullptr, nullptr};
+  cudaEvent_t copies_done = nullptr;
 };
 
 DeviceCache g_cache[kMaxDevices];
@@ -680,7 +683,7 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
   long long tiles = 0;
   for (int l = 0; l < n_layers; ++l) {
     h[l].x = tensors[l]; h[l].out = codes_out[l]; h[l].n = lens[l]; h[l].tile_begin = tiles;
-    h[l].layer_id = layer_base + l;
+    h[l].layer_id = layer_base + l; h[l].select = l; h[l].pad_ = 0; h[l].index_base = 0;
     h[l].vec = !(reinterpret_cast<uintptr_t>(tensors[l]) & 15u) &&
                !(reinterpret_cast<uintptr_t>(codes_out[l]) & (4u * elem - 1u));
     tiles += (lens[l] + kQuantTile - 1) / kQuantTile;
@@ -931,11 +934,36 @@ int adapt_precision_search(const float* const* tensors, const int64_t* lens, int
 }  // extern "C"
 
 namespace {
+
+// Launches the batched quantize kernel over table entries [first, first + count) of a device
+// table whose tile numbering restarts at `first`.  Caller holds g_mutex.
+int launch_quantize_entries(const QuantLayer* d_table, int count, long long tiles, const int32_t* best,
+                            int round_mode, uint64_t seed, int out_bits, int32_t* unfit, int sm_count,
+                            cudaStream_t stream) {
+  if (tiles == 0) return ADAPT_OK;
+  const int grid = static_cast<int>(std::min<long long>(tiles, 32ll * sm_count));
+  LaunchScope ls(ADAPT_KERNEL_QUANTIZE, stream);
+  const bool sr = round_mode == ADAPT_ROUND_STOCHASTIC;
+  void (*kern)(const QuantLayer*, int, long long, const int*, unsigned long long, int*) = nullptr;
+  switch (out_bits) {
+    case 8:  kern = sr ? quantize_batch_kernel<true, int8_t>  : quantize_batch_kernel<false, int8_t>;  break;
+    case 16: kern = sr ? quantize_batch_kernel<true, int16_t> : quantize_batch_kernel<false, int16_t>; break;
+    default: kern = sr ? quantize_batch_kernel<true, int32_t> : quantize_batch_kernel<false, int32_t>; break;
+  }
+  kern<<<grid, kQuantThreads, 0, stream>>>(d_table, count, tiles, best, seed, unfit);
+  ADAPT_CUDA(cudaGetLastError());
+  return ADAPT_OK;
+}
+
 // Host-buffer search, optionally followed by the quantization of every layer at its selected
-// format from the same device copy (codes_out: HOST array of HOST int32 buffers, or null).
+// format from the same device copy (codes_out: HOST array of HOST buffers of code_bits-wide codes,
+// or null).  The codes are produced slice by slice (a slice is a run of whole small layers or a
+// piece of a large one, about 64 MB of input) and each slice's download runs on a second stream
+// while the next slice is quantized.
 int run_search_host(const float* const* tensors, const int64_t* lens, int n_layers,
                     const adapt_grid* grid, int n_bins, double* kld_out, int64_t* zeros_out,
-                    int32_t* best_out, int32_t* const* codes_out, const adapt_search_opts* opts) {
+                    int32_t* best_out, void* const* codes_out, int code_bits, int32_t* unfit_out,
+                    const adapt_search_opts* opts) {
   std::lock_guard<std::mutex> lock(g_mutex);
   DeviceCache* dc = nullptr;
   int rc = current_cache(&dc);
@@ -943,10 +971,13 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
   adapt_search_opts o = opts ? *opts : default_opts();
   if (o.workspace || o.workspace_bytes || o.hist_out || o.range_out || o.status_out) return ADAPT_ERR_INVALID_ARG;
   if (!tensors || !kld_out || !zeros_out || !best_out) return ADAPT_ERR_INVALID_ARG;
+  if (codes_out && code_bits != 8 && code_bits != 16 && code_bits != 32) return ADAPT_ERR_INVALID_ARG;
   Plan plan;
   if (!make_plan(lens, n_layers, grid, n_bins, &plan)) return ADAPT_ERR_INVALID_ARG;
-  for (int l = 0; l < n_layers; ++l)
+  for (int l = 0; l < n_layers; ++l) {
     if (lens[l] > 0 && !tensors[l]) return ADAPT_ERR_INVALID_ARG;
+    if (codes_out && lens[l] > 0 && !codes_out[l]) return ADAPT_ERR_INVALID_ARG;
+  }
 
   // device copies of the layers, 256-byte aligned each
   std::vector<size_t> off(n_layers);
@@ -959,9 +990,10 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
   const size_t kld_bytes = align_up(sizeof(double) * L * C, 256);
   const size_t zeros_bytes = align_up(sizeof(int64_t) * L * C, 256);
   const size_t best_bytes = align_up(sizeof(int32_t) * 4 * L, 256);
+  const size_t unfit_bytes = align_up(sizeof(int32_t) * L, 256);
   rc = grow_device(&dc->stage_in, &dc->stage_in_bytes, std::max<size_t>(in_bytes, 256));
   if (rc != ADAPT_OK) return rc;
-  rc = grow_device(&dc->stage_out, &dc->stage_out_bytes, kld_bytes + zeros_bytes + best_bytes);
+  rc = grow_device(&dc->stage_out, &dc->stage_out_bytes, kld_bytes + zeros_bytes + best_bytes + unfit_bytes);
   if (rc != ADAPT_OK) return rc;
 
   cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
@@ -977,25 +1009,78 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
   SearchArgs a{dptr.data(), lens, n_layers, grid, n_bins, reinterpret_cast<double*>(so),
                reinterpret_cast<int64_t*>(so + kld_bytes),
                reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes), o};
+  int32_t* d_unfit = reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes + best_bytes);
   rc = run_search(*dc, a);
   if (rc != ADAPT_OK) return rc;
   if (codes_out) {
-    // codes of all layers in one more library-owned buffer, same offsets as the inputs
-    rc = grow_device(&dc->stage_codes, &dc->stage_codes_bytes, std::max<size_t>(in_bytes, 256));
+    const size_t cb = static_cast<size_t>(code_bits / 8);
+    // codes of all layers in one more library-owned buffer: layer l at off[l] / 4 * cb
+    rc = grow_device(&dc->stage_codes, &dc->stage_codes_bytes, std::max<size_t>(in_bytes / 4 * cb, 256));
     if (rc != ADAPT_OK) return rc;
-    std::vector<int32_t*> dcodes(n_layers);
-    for (int l = 0; l < n_layers; ++l) {
-      if (lens[l] > 0 && !codes_out[l]) return ADAPT_ERR_INVALID_ARG;
-      dcodes[l] = reinterpret_cast<int32_t*>(static_cast<char*>(dc->stage_codes) + off[l]);
+    if (!dc->copy_stream) {
+      ADAPT_CUDA(cudaStreamCreateWithFlags(&dc->copy_stream, cudaStreamNonBlocking));
+      for (cudaEvent_t& e : dc->slice_done) ADAPT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+      ADAPT_CUDA(cudaEventCreateWithFlags(&dc->copies_done, cudaEventDisableTiming));
     }
-    rc = run_quantize_batch(dptr.data(), lens, n_layers, a.best_out, o.round_mode, o.seed,
-                            o.layer_base, reinterpret_cast<void* const*>(dcodes.data()), 32, nullptr,
-                            o.stream);
-    if (rc != ADAPT_OK) return rc;
-    for (int l = 0; l < n_layers; ++l)
-      if (lens[l] > 0)
-        ADAPT_CUDA(cudaMemcpyAsync(codes_out[l], dcodes[l], sizeof(int32_t) * static_cast<size_t>(lens[l]),
-                                   cudaMemcpyDeviceToHost, stream));
+    ADAPT_CUDA(cudaMemsetAsync(d_unfit, 0, sizeof(int32_t) * L, stream));
+    // table entries: pieces of at most kSliceElems elements, in layer order
+    constexpr long long kSliceElems = 16ll << 20;
+    std::vector<QuantLayer> table;
+    std::vector<int> group_first;           // first entry of every launch group
+    std::vector<long long> group_tiles;
+    long long in_group = 0, tiles = 0;
+    for (int l = 0; l < n_layers; ++l) {
+      for (long long at = 0; at < lens[l]; at += kSliceElems) {
+        const long long n = std::min<long long>(kSliceElems, lens[l] - at);
+        if (group_first.empty() || in_group + n > kSliceElems) {
+          if (!group_first.empty()) group_tiles.push_back(tiles);
+          group_first.push_back(static_cast<int>(table.size()));
+          in_group = 0; tiles = 0;
+        }
+        QuantLayer q;
+        q.x = dptr[l] + at;
+        q.out = static_cast<char*>(dc->stage_codes) + off[l] / 4 * cb + static_cast<size_t>(at) * cb;
+        q.n = n; q.tile_begin = tiles; q.layer_id = o.layer_base + l; q.vec = 1;   // 256-byte aligned pieces
+        q.select = l; q.pad_ = 0; q.index_base = at;
+        table.push_back(q);
+        tiles += (n + kQuantTile - 1) / kQuantTile;
+        in_group += n;
+      }
+    }
+    if (!group_first.empty()) group_tiles.push_back(tiles);
+    if (!table.empty()) {
+      const size_t bytes = sizeof(QuantLayer) * table.size();
+      rc = grow_device(&dc->batch_tab, &dc->batch_tab_bytes, align_up(bytes, 4096));
+      if (rc != ADAPT_OK) return rc;
+      PinnedSlot* slot = nullptr;
+      rc = acquire_slot(*dc, bytes, &slot);
+      if (rc != ADAPT_OK) return rc;
+      std::memcpy(slot->host, table.data(), bytes);
+      ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, slot->host, bytes, cudaMemcpyHostToDevice, stream));
+      ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+      const QuantLayer* d_table = static_cast<const QuantLayer*>(dc->batch_tab);
+      for (size_t g = 0; g < group_first.size(); ++g) {
+        const int first = group_first[g];
+        const int count = (g + 1 < group_first.size() ? group_first[g + 1] : static_cast<int>(table.size())) - first;
+        rc = launch_quantize_entries(d_table + first, count, group_tiles[g], a.best_out, o.round_mode, o.seed,
+                                     code_bits, d_unfit, dc->sm_count, stream);
+        if (rc != ADAPT_OK) return rc;
+        // the group's download starts when its kernel is done and overlaps the next group's kernel
+        cudaEvent_t ev = dc->slice_done[g & 1];
+        ADAPT_CUDA(cudaEventRecord(ev, stream));
+        ADAPT_CUDA(cudaStreamWaitEvent(dc->copy_stream, ev, 0));
+        for (int e = first; e < first + count; ++e) {
+          const QuantLayer& q = table[e];
+          char* host_at = static_cast<char*>(codes_out[q.select]) + static_cast<size_t>(q.index_base) * cb;
+          ADAPT_CUDA(cudaMemcpyAsync(host_at, q.out, static_cast<size_t>(q.n) * cb, cudaMemcpyDeviceToHost,
+                                     dc->copy_stream));
+        }
+      }
+      ADAPT_CUDA(cudaEventRecord(dc->copies_done, dc->copy_stream));
+      ADAPT_CUDA(cudaStreamWaitEvent(stream, dc->copies_done, 0));
+    }
+    if (unfit_out)
+      ADAPT_CUDA(cudaMemcpyAsync(unfit_out, d_unfit, sizeof(int32_t) * L, cudaMemcpyDeviceToHost, stream));
   }
   ADAPT_CUDA(cudaMemcpyAsync(kld_out, a.kld_out, sizeof(double) * L * C, cudaMemcpyDeviceToHost, stream));
   ADAPT_CUDA(cudaMemcpyAsync(zeros_out, a.zeros_out, sizeof(int64_t) * L * C, cudaMemcpyDeviceToHost, stream));
@@ -1017,7 +1102,7 @@ int adapt_precision_search_host(const float* const* tensors, const int64_t* lens
                                 int64_t* zeros_out, int32_t* best_out,
                                 const adapt_search_opts* opts) {
   return run_search_host(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
-                         nullptr, opts);
+                         nullptr, 32, nullptr, opts);
 }
 
 int adapt_precision_switch_host(const float* const* tensors, const int64_t* lens, int n_layers,
@@ -1026,7 +1111,17 @@ int adapt_precision_switch_host(const float* const* tensors, const int64_t* lens
                                 const adapt_search_opts* opts) {
   if (!codes_out) return ADAPT_ERR_INVALID_ARG;
   return run_search_host(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
-                         codes_out, opts);
+                         reinterpret_cast<void* const*>(codes_out), 32, nullptr, opts);
+}
+
+int adapt_precision_switch_host_packed(const float* const* tensors, const int64_t* lens, int n_layers,
+                                       const adapt_grid* grid, int n_bins, double* kld_out,
+                                       int64_t* zeros_out, int32_t* best_out, int code_bits,
+                                       void* const* codes_out, int32_t* unfit_out,
+                                       const adapt_search_opts* opts) {
+  if (!codes_out) return ADAPT_ERR_INVALID_ARG;
+  return run_search_host(tensors, lens, n_layers, grid, n_bins, kld_out, zeros_out, best_out,
+                         codes_out, code_bits, unfit_out, opts);
 }
 
 int adapt_quantize_host(const float* x, int64_t n, int wl, int fl, int round_mode, uint64_t seed,
@@ -1523,6 +1618,11 @@ int adapt_release(void) {
   if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
   if (dc->div_buf) { ADAPT_CUDA(cudaFree(dc->div_buf)); dc->div_buf = nullptr; dc->div_buf_bytes = 0; }
   if (dc->stage_codes) { ADAPT_CUDA(cudaFree(dc->stage_codes)); dc->stage_codes = nullptr; dc->stage_codes_bytes = 0; }
+  if (dc->copy_stream) {
+    ADAPT_CUDA(cudaStreamDestroy(dc->copy_stream)); dc->copy_stream = nullptr;
+    for (cudaEvent_t& e : dc->slice_done) { ADAPT_CUDA(cudaEventDestroy(e)); e = nullptr; }
+    ADAPT_CUDA(cudaEventDestroy(dc->copies_done)); dc->copies_done = nullptr;
+  }
   for (PinnedSlot& s : dc->ring) {
     if (s.host) { ADAPT_CUDA(cudaFreeHost(s.host)); s.host = nullptr; s.bytes = 0; }
     if (s.done) { ADAPT_CUDA(cudaEventDestroy(s.done)); s.done = nullptr; }

@@ -80,6 +80,9 @@ struct QuantLayer {
   long long tile_begin;   // first tile of the layer in the launch's tile list (4096 elements each)
   int layer_id;           // hash layer id
   int vec;                // x is 16-byte aligned and out aligned for a 4-element store
+  int select;             // row of `best` (and of `unfit`) that holds this entry's <WL,FL>
+  int pad_;
+  long long index_base;   // element index of x[0] inside its layer (an entry may be a slice of one)
 };
 
 constexpr int kQuantTile = 4096;
@@ -109,10 +112,10 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
       if (layers[mid].tile_begin <= t) lo = mid; else hi = mid - 1;
     }
     const QuantLayer L = layers[lo];
-    const int wl = best[4 * lo], fl = best[4 * lo + 1];
+    const int wl = best[4 * L.select], fl = best[4 * L.select + 1];
     if (wl < 2 || wl > 32 || fl < 0 || fl >= wl) continue;   // layer without a valid selection
     if (wl > kBits) {
-      if (unfit && t == L.tile_begin && threadIdx.x == 0) unfit[lo] = wl;
+      if (unfit && t == L.tile_begin && threadIdx.x == 0) unfit[L.select] = wl;
       continue;
     }
     const float two_fl = pow2f(fl);
@@ -125,7 +128,7 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
       P4* o4 = reinterpret_cast<P4*>(out + i0);
       for (int q = threadIdx.x; q < kQuantTile / 4; q += kQuantThreads) {
         const float4 v = __ldcs(x4 + q);
-        const long long i = i0 + 4ll * q;
+        const long long i = L.index_base + i0 + 4ll * q;
         P4 c;
         c.x = quant_out<T>(quantize_one<kStochastic>(v.x, two_fl, wl, seed, L.layer_id, i + 0), fl);
         c.y = quant_out<T>(quantize_one<kStochastic>(v.y, two_fl, wl, seed, L.layer_id, i + 1), fl);
@@ -135,7 +138,8 @@ quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long 
       }
     } else {
       for (long long i = i0 + threadIdx.x; i < i1; i += kQuantThreads)
-        out[i] = quant_out<T>(quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id, i), fl);
+        out[i] = quant_out<T>(quantize_one<kStochastic>(__ldcs(L.x + i), two_fl, wl, seed, L.layer_id,
+                                                        L.index_base + i), fl);
     }
   }
 }

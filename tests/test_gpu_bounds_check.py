@@ -36,7 +36,7 @@ cases = {
     "on_grid_strays": np.where(rng.random(n) < 0.001, base, np.round(base * 64) / 64).astype(np.float32),
     "ties": (rng.integers(-4000, 4000, n) * 2.0 ** -9 + 2.0 ** -10).astype(np.float32),
     "subnormals": np.float32([1e-40, -1e-41, 3e-39, 0.0, 5e-45] * 50),
-    "extremes": np.float32([-3e38, 3e38, 0.0, 1.0]),
+    "extremes": np.float32([-1e19, 1e19, 0.0, 1.0, -1e-30]),
 }
 wl, fl = W.candidate_grid(range(2, 33))
 for name, x in cases.items():

@@ -352,3 +352,33 @@ def test_host_buffer_form_matches(B):
     for l, x in enumerate(xs):
         want, _ = O.quantize(x, int(ora[l]["best"][0]), int(ora[l]["best"][1]), w.round_mode, w.seed, l)
         assert np.array_equal(codes[l].numpy(), want), l
+
+
+def test_host_switch_with_packed_codes_in_slices(B):
+    """Packed codes through the host-buffer switch: layers larger than a download slice, many
+    small ones, both rounding modes; a word length that does not fit is reported, not written."""
+    import torch
+    rng = np.random.default_rng(31)
+    xs = [(rng.standard_normal((1 << 24) + 12345) * 0.05).astype(np.float32),      # two slices
+          (rng.integers(-100, 100, 70000) * 2.0 ** -3).astype(np.float32),          # fits 8 bits
+          np.zeros(0, np.float32),
+          (rng.standard_normal(5000) * 0.3).astype(np.float32),
+          (rng.integers(-20000, 20000, 40000) * 2.0 ** -2).astype(np.float32)]      # needs 17 bits
+    wl, fl = W.candidate_grid(range(2, 21))
+    host = [torch.from_numpy(x).pin_memory() for x in xs]
+    for mode in (O.ROUND_RNE, O.ROUND_STOCHASTIC):
+        ora = O.precision_search(xs, wl, fl, 64, mode, 9, threads=G.host_threads())
+        for bits, dt in ((8, np.int8), (16, np.int16), (32, np.int32)):
+            sentinel = [torch.full((x.size,), -77, dtype={8: torch.int8, 16: torch.int16, 32: torch.int32}[bits])
+                        for x in xs]
+            res, codes, unfit = B.adapt_precision_switch_host_packed(host, B.Grid(wl, fl), 64, bits,
+                                                                    round_mode=mode, seed=9, codes_out=sentinel)
+            G.compare_search(res, ora, len(xs), f"packed switch {bits} bits mode {mode}")
+            for l, x in enumerate(xs):
+                w_sel, f_sel = int(ora[l]["best"][0]), int(ora[l]["best"][1])
+                if w_sel > bits:
+                    assert unfit[l] == w_sel and (codes[l].numpy() == -77).all(), (l, bits)
+                    continue
+                assert unfit[l] == 0
+                want, _ = O.quantize(x, w_sel, f_sel, mode, 9, l)
+                assert np.array_equal(codes[l].numpy(), want.astype(dt)), (l, bits, mode)
