@@ -22,6 +22,7 @@
 #include "k_range.cuh"
 #include "k_search_direct.cuh"
 #include "k_search_keyed.cuh"
+#include "k_search_sr.cuh"
 
 namespace {
 
@@ -173,13 +174,16 @@ struct Plan {
   // keyed-kernel shared-memory shape
   int cell_cap = 0, value_cap = 0, d_levels = 0;
   size_t keyed_smem = 0;
+  // stochastic-rounding kernel's shared-memory shape
+  int sr_cap = 0, sr_d_levels = 0;
+  size_t sr_smem = 0;
   // byte offsets inside the workspace -- descriptor block (uploaded)
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
          off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_start = 0, off_state = 0, blob_bytes = 0;
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0;
   // accumulators (cleared every call)
-  size_t off_sub = 0, off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
+  size_t off_coarse = 0, off_sub = 0, off_zeros = 0, off_q = 0, off_u = 0, off_cells = 0, off_qe = 0,
          off_zclass = 0, off_nzero = 0, accum_begin = 0, accum_bytes = 0;
   size_t total = 0;
 };
@@ -233,6 +237,14 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   }
   p->keyed_smem = keyed_smem_bytes(p->cell_cap, n_bins, p->d_levels);
   p->value_cap = p->cell_cap ? keyed_value_cap(p->cell_cap, n_bins, p->d_levels) : 0;
+  if (n_bins <= kKeyedMaxBins) {
+    p->sr_d_levels = std::min(static_cast<int>(std::min<size_t>(4, (16 * 1024) / hist)), p->n_levels);
+    const size_t fixed = sr_smem_bytes(0, n_bins, p->sr_d_levels);
+    // (the kernel's static tables - lane-private counters of the central values - take 13 KB more)
+    p->sr_cap = static_cast<int>((kKeyedSmemBudget - 14 * 1024 - fixed) / 8) & ~3;
+    p->sr_cap = std::min(p->sr_cap, p->value_cap);      // rows of the global tables are value_cap long
+    p->sr_smem = sr_smem_bytes(p->sr_cap, n_bins, p->sr_d_levels);
+  }
 
   // K: row length of the global cell arrays (the largest table a layer may use)
   const size_t C = grid->n_cand, L = n_layers, B = n_bins, F = p->n_levels, K = p->value_cap;
@@ -258,6 +270,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_q = o;       o = align_up(o + sizeof(unsigned) * L * B, 256);
   p->off_qe = o;      o = align_up(o + sizeof(unsigned) * L * B * 2, 256);
   p->off_cells = o;   o = align_up(o + sizeof(unsigned) * L * K, 256);
+  p->off_coarse = o;  o = align_up(o + sizeof(unsigned) * L * K, 256);
   p->off_sub = o;     o = align_up(o + sizeof(unsigned) * (K ? L * 2 * B * kSubCells : 0), 256);
   p->off_u = o;       o = align_up(o + sizeof(unsigned) * L * F * B, 256);
   p->accum_bytes = o - p->accum_begin;
@@ -317,12 +330,12 @@ long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchAr
     d.layer_id = a.opts.layer_base + l;
     d.index = l;
     d.n_bins = a.opts.n_bins_per_layer ? a.opts.n_bins_per_layer[l] : a.n_bins;
-    d.range_ctas = 0;
+    d.range_ctas = 0; d.via_plan = 0; d.pad_ = 0;
     if (a.lens[l] > 0) tiles += (a.lens[l] + mis + tile - 1) / tile;
   }
   LayerDesc& s = out[k];
   s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.n_bins = 1;
-  s.range_ctas = 0;
+  s.range_ctas = 0; s.via_plan = 0; s.pad_ = 0;
   return tiles;
 }
 
@@ -366,17 +379,23 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   cudaStream_t stream = static_cast<cudaStream_t>(o.stream);
 
   // which kernel serves which layer
-  const bool keyed_possible = o.round_mode == ADAPT_ROUND_RNE && plan.cell_cap >= 1024 &&
-                              plan.keyed_smem + 2048 <= static_cast<size_t>(dc.max_smem_optin) &&
-                              (o.algorithm == ADAPT_ALGO_AUTO || o.algorithm == ADAPT_ALGO_KEYED);
   if (o.algorithm != ADAPT_ALGO_AUTO && o.algorithm != ADAPT_ALGO_KEYED &&
       o.algorithm != ADAPT_ALGO_DIRECT) return ADAPT_ERR_INVALID_ARG;
+  const bool stochastic = o.round_mode == ADAPT_ROUND_STOCHASTIC;
+  const bool keyed_possible =
+      (o.algorithm == ADAPT_ALGO_AUTO || o.algorithm == ADAPT_ALGO_KEYED) &&
+      (stochastic ? (plan.sr_cap >= 2048 && plan.sr_smem + 15 * 1024 <= static_cast<size_t>(dc.max_smem_optin))
+                  : (plan.cell_cap >= 1024 && plan.keyed_smem + 2048 <= static_cast<size_t>(dc.max_smem_optin)));
   const long long keyed_min = (o.algorithm == ADAPT_ALGO_KEYED) ? 1 : kKeyedMinElements;
   std::vector<int> all(a.n_layers), keyed, direct;
   std::iota(all.begin(), all.end(), 0);
   for (int l = 0; l < a.n_layers; ++l) {
-    if (keyed_possible && a.lens[l] >= keyed_min) keyed.push_back(l);
-    else direct.push_back(l);
+    const bool k = keyed_possible && a.lens[l] >= keyed_min;
+    if (k) keyed.push_back(l);
+    // Stochastic rounding: whether the keyed kernel can serve a layer is only known on the
+    // device (its cell indices must be exact in a float), so its layers also stand in the
+    // direct kernel's list, which skips those whose plan says "keyed"
+    if (!k || stochastic) direct.push_back(l);
   }
 
   // host image of the descriptor block
@@ -387,8 +406,17 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   std::memset(h, 0, plan.blob_bytes);
   const long long tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_layers), all, a, kTile);
   const int range_grid = plan_range_grid(reinterpret_cast<LayerDesc*>(h + plan.off_layers), a.n_layers, tiles, dc.sm_count);
-  const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a, kKeyedTile);
+  const long long keyed_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_keyed), keyed, a,
+                                          stochastic ? kSrTile : kKeyedTile);
   const long long direct_tiles = fill_list(reinterpret_cast<LayerDesc*>(h + plan.off_direct), direct, a, kTile);
+  if (stochastic && !keyed.empty()) {
+    LayerDesc* dl = reinterpret_cast<LayerDesc*>(h + plan.off_direct);
+    size_t k = 0;
+    for (size_t i = 0; i < direct.size(); ++i) {
+      while (k < keyed.size() && keyed[k] < direct[i]) ++k;
+      if (k < keyed.size() && keyed[k] == direct[i]) dl[i].via_plan = 1;
+    }
+  }
   std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
@@ -435,7 +463,11 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     {
       PlanParams pp;
       pp.layers = d_keyed; pp.state = d_state; pp.plan = d_plan; pp.edges = d_edges;
-      pp.n_bins = bins_stride; pp.cell_cap = plan.cell_cap; pp.value_cap = plan.value_cap;
+      pp.n_bins = bins_stride; pp.value_cap = plan.value_cap;
+      // stochastic rounding: cells and coarse tables share the limit; a little room for the
+      // three spare entries of every coarse level
+      pp.stochastic = stochastic ? 1 : 0;
+      pp.cell_cap = stochastic ? plan.sr_cap - 128 : plan.cell_cap;
       pp.fine_ratio = ADAPT_FINE_RATIO;
       pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
@@ -443,6 +475,34 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       plan_kernel<<<dim3(nk, plan_slices), kPlanThreads, 0, stream>>>(pp);
       ADAPT_CUDA(cudaGetLastError());
     }
+    if (stochastic) {
+      SrParams sp;
+      sp.layers = d_keyed; sp.n_layers = nk; sp.n_tiles = keyed_tiles; sp.state = d_state;
+      sp.plan = d_plan; sp.edges = d_edges; sp.cell_count = d_cells;
+      sp.coarse_count = reinterpret_cast<unsigned*>(ws + plan.off_coarse);
+      sp.qe_hist = d_qe; sp.u_hist = d_u; sp.zeros = d_zeros;
+      sp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
+      sp.seed = o.seed; sp.n_bins = bins_stride; sp.n_levels = plan.n_levels;
+      sp.table_cap = plan.sr_cap; sp.cell_stride = plan.value_cap; sp.d_levels = plan.sr_d_levels;
+      ADAPT_CUDA(cudaFuncSetAttribute(search_sr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(plan.sr_smem)));
+      {
+        LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
+        search_sr_kernel<<<keyed_grid, kSrThreads, plan.sr_smem, stream>>>(sp);
+        ADAPT_CUDA(cudaGetLastError());
+      }
+      SrExpandParams ep;
+      ep.layers = d_keyed; ep.state = d_state; ep.plan = d_plan; ep.cell_count = d_cells;
+      ep.coarse_count = sp.coarse_count; ep.qe_hist = d_qe; ep.cell_total = sp.cell_total;
+      ep.q_hist = d_q; ep.u_hist = d_u; ep.zeros = d_zeros;
+      ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_stride = plan.value_cap;
+      {
+        LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
+        expand_sr_kernel<<<dim3(plan.n_levels + 1, nk), kSrExpandThreads,
+                           sizeof(unsigned) * bins_stride, stream>>>(ep);
+        ADAPT_CUDA(cudaGetLastError());
+      }
+    } else {
     KeyedParams kp;
     kp.layers = d_keyed; kp.n_layers = nk; kp.n_tiles = keyed_tiles; kp.state = d_state;
     kp.plan = d_plan; kp.edges = d_edges; kp.cell_count = d_cells;
@@ -473,6 +533,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
                       sizeof(unsigned) * bins_stride, stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
+    }
   }
 
   // K2, direct form: stochastic rounding, small layers, very large bin counts
@@ -481,7 +542,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     sp.layers = d_direct; sp.state = d_state;
     sp.n_layers = static_cast<int>(direct.size()); sp.n_fl = plan.n_levels; sp.n_bins = bins_stride;
     sp.n_tiles = direct_tiles;
-    sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed;
+    sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros; sp.seed = o.seed; sp.plan = d_plan;
     const size_t per_hist = sizeof(unsigned) * bins_stride;
     // When the histograms of all fraction lengths overflow half an SM's shared memory and there
     // is work for every SM, one CTA of 1024 threads takes the whole of it: fewer FL groups (each
@@ -1009,11 +1070,21 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
   SearchArgs a{dptr.data(), lens, n_layers, grid, n_bins, reinterpret_cast<double*>(so),
                reinterpret_cast<int64_t*>(so + kld_bytes),
                reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes), o};
-  int32_t* d_unfit = reinterpret_cast<int32_t*>(so + kld_bytes + zeros_bytes + best_bytes);
   rc = run_search(*dc, a);
   if (rc != ADAPT_OK) return rc;
+  std::vector<int32_t> fits(n_layers, 0);       // 1: the layer's codes are produced and downloaded
   if (codes_out) {
     const size_t cb = static_cast<size_t>(code_bits / 8);
+    // the selected word lengths decide which layers get codes: fetch them (16 bytes per layer)
+    ADAPT_CUDA(cudaMemcpyAsync(best_out, a.best_out, sizeof(int32_t) * 4 * L, cudaMemcpyDeviceToHost, stream));
+    ADAPT_CUDA(cudaStreamSynchronize(stream));
+    for (int l = 0; l < n_layers; ++l) {
+      const int wl_sel = best_out[4 * l], fl_sel = best_out[4 * l + 1];
+      const bool valid_sel = valid_format(wl_sel, fl_sel) &&
+                             !(best_out[4 * l + 3] & (ADAPT_FLAG_NONFINITE | ADAPT_FLAG_RANGE));
+      fits[l] = (valid_sel && wl_sel <= code_bits) ? 1 : 0;
+      if (unfit_out) unfit_out[l] = (valid_sel && wl_sel > code_bits) ? wl_sel : 0;
+    }
     // codes of all layers in one more library-owned buffer: layer l at off[l] / 4 * cb
     rc = grow_device(&dc->stage_codes, &dc->stage_codes_bytes, std::max<size_t>(in_bytes / 4 * cb, 256));
     if (rc != ADAPT_OK) return rc;
@@ -1022,7 +1093,6 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
       for (cudaEvent_t& e : dc->slice_done) ADAPT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
       ADAPT_CUDA(cudaEventCreateWithFlags(&dc->copies_done, cudaEventDisableTiming));
     }
-    ADAPT_CUDA(cudaMemsetAsync(d_unfit, 0, sizeof(int32_t) * L, stream));
     // table entries: pieces of at most kSliceElems elements, in layer order
     constexpr long long kSliceElems = 16ll << 20;
     std::vector<QuantLayer> table;
@@ -1030,6 +1100,7 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
     std::vector<long long> group_tiles;
     long long in_group = 0, tiles = 0;
     for (int l = 0; l < n_layers; ++l) {
+      if (!fits[l]) continue;
       for (long long at = 0; at < lens[l]; at += kSliceElems) {
         const long long n = std::min<long long>(kSliceElems, lens[l] - at);
         if (group_first.empty() || in_group + n > kSliceElems) {
@@ -1063,7 +1134,7 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
         const int first = group_first[g];
         const int count = (g + 1 < group_first.size() ? group_first[g + 1] : static_cast<int>(table.size())) - first;
         rc = launch_quantize_entries(d_table + first, count, group_tiles[g], a.best_out, o.round_mode, o.seed,
-                                     code_bits, d_unfit, dc->sm_count, stream);
+                                     code_bits, nullptr, dc->sm_count, stream);
         if (rc != ADAPT_OK) return rc;
         // the group's download starts when its kernel is done and overlaps the next group's kernel
         cudaEvent_t ev = dc->slice_done[g & 1];
@@ -1079,8 +1150,6 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
       ADAPT_CUDA(cudaEventRecord(dc->copies_done, dc->copy_stream));
       ADAPT_CUDA(cudaStreamWaitEvent(stream, dc->copies_done, 0));
     }
-    if (unfit_out)
-      ADAPT_CUDA(cudaMemcpyAsync(unfit_out, d_unfit, sizeof(int32_t) * L, cudaMemcpyDeviceToHost, stream));
   }
   ADAPT_CUDA(cudaMemcpyAsync(kld_out, a.kld_out, sizeof(double) * L * C, cudaMemcpyDeviceToHost, stream));
   ADAPT_CUDA(cudaMemcpyAsync(zeros_out, a.zeros_out, sizeof(int64_t) * L * C, cudaMemcpyDeviceToHost, stream));
@@ -1507,6 +1576,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
     const int mis = static_cast<int>((reinterpret_cast<uintptr_t>(tensors[l]) >> 2) & 3u);
     hl[l].ptr = tensors[l]; hl[l].n = lens[l]; hl[l].tile_begin = tiles;
     hl[l].mis = lens[l] > 0 ? mis : 0; hl[l].layer_id = l; hl[l].index = l; hl[l].n_bins = n_bins;
+    hl[l].via_plan = 0; hl[l].pad_ = 0;
     if (lens[l] > 0) tiles += (lens[l] + mis + kTile - 1) / kTile;
   }
   hl[n_layers].tile_begin = tiles;
@@ -1551,7 +1621,7 @@ int adapt_precision_search_static(const float* const* tensors, const int64_t* le
     SearchParams sp;
     sp.layers = d_layers; sp.state = d_state; sp.n_layers = n_layers; sp.n_fl = n_levels;
     sp.n_bins = n_bins; sp.n_tiles = tiles; sp.q_hist = d_q; sp.u_hist = d_u; sp.zeros = d_zeros;
-    sp.seed = 0;
+    sp.seed = 0; sp.plan = nullptr;
     const size_t per_hist = sizeof(unsigned) * n_bins;
     int fg = static_cast<int>((40 * 1024) / per_hist) - 1;   // stays under the 48 KB default limit
     fg = std::max(1, std::min(fg, n_levels));

@@ -30,6 +30,9 @@ struct LayerDesc {
   int n_bins;            // bins of this layer's histograms (<= the stride the arrays use)
   int range_ctas;        // CTAs of the range scan that hold tiles of this layer (set by the host for
                          // the list that kernel walks; the last of them to finish settles the layer)
+  int via_plan;          // direct kernel's list: 1 = the layer also stands in the stochastic-rounding
+                         // kernel's list and is served here only if its plan says "not keyed"
+  int pad_;
 };
 
 // Per-layer state produced on the device by the range scan.
@@ -69,6 +72,22 @@ __device__ __forceinline__ bool index_in_bounds(long long idx, long long limit, 
 #else
 #define ADAPT_IN_BOUNDS(idx, limit, site) true
 #endif
+
+// Shared-memory atomics by 32-bit shared address.  A table pointer that a kernel keeps in a
+// context structure is a generic pointer to the compiler, and atomics through generic pointers
+// are far slower than the shared-memory forms; kernels therefore keep shared addresses
+// (smem_addr of the table's first word) and add byte offsets.
+__device__ __forceinline__ unsigned smem_addr(const void* p) {
+  return static_cast<unsigned>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned smem_atom_add(unsigned addr, unsigned v) {
+  unsigned o;
+  asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(o) : "r"(addr), "r"(v) : "memory");
+  return o;
+}
+__device__ __forceinline__ void smem_red_add(unsigned addr, unsigned v) {
+  asm volatile("red.shared.add.u32 [%0], %1;" :: "r"(addr), "r"(v) : "memory");
+}
 
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).
 __device__ __forceinline__ unsigned float_key(float v) {

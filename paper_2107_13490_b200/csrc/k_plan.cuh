@@ -121,6 +121,8 @@ struct PlanParams {
   int n_bins;                // stride of the per-bin arrays (the largest layer's bins)
   int cell_cap;              // table entries a layer may use
   int value_cap;             // ... when it is keyed by value (its table may run over the others)
+  int stochastic;            // 1: plans for the stochastic-rounding kernel (one segment, cell indices
+                             // exact in float, room for the coarse levels' tables)
   int fine_ratio;            // stop refining once a bin holds this many cells
   long long elems_per_cta;   // elements one CTA of the keyed kernel processes
 };
@@ -201,6 +203,33 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
     P.seg[1].c0 = 0; P.seg[1].g = 0; P.seg[1].cells = 0; P.seg[1].fs = 0; P.seg[1].offset = 0;
     P.seg[1].two_g = 1.0f; P.seg[1].c0f = 0.0f; P.seg[1].magic = 0.0f; P.seg[1].pad_ = 0;
     P.seg[0].pad_ = 0;
+    if (p.stochastic) {
+      // Stochastic rounding: every level below the cells' costs each element an evaluation, every
+      // element of an edge cell a walk over the levels above; about 16 cells per bin balances
+      // the two.  The tables of the coarse levels (about as many words as there are cells) must
+      // fit beside the cells, and every cell index must be exact in a float.
+      const int want_g = level_for_ratio(S.lo, S.hi, B, 16);
+      fit_segment(S.lo, S.hi, p.cell_cap, want_g, &P.seg[0]);
+      for (;;) {
+        long long words = 0;
+        for (int f = 0; f < P.seg[0].g && f < kMaxFl; ++f)
+          words += floor_scaled(S.hi, f) - floor_scaled(S.lo, f) + 3;
+        if (words <= p.cell_cap || P.seg[0].g <= -100) break;
+        fit_segment(S.lo, S.hi, p.cell_cap, P.seg[0].g - 1, &P.seg[0]);
+      }
+      P.seg[0].offset = 0;
+      P.seg[1].offset = P.seg[0].cells;
+      P.total_cells = P.seg[0].cells;
+      const float top = fmaxf(fabsf(S.lo), fabsf(S.hi));
+      P.fast = (ldexp(static_cast<double>(top), max(P.seg[0].g, 0)) < 4.0e6 && P.seg[0].g >= -100 &&
+                P.seg[0].g <= 100) ? 1 : 0;
+      if (!P.fast) P.keyed = 0;           // left to the direct kernel
+      P.seg[0].magic = 0.0f;
+      P.grid_mask = 0u; P.grid_mul = 0u; P.masked = 0; P.dense = 0; P.refined = 0; P.sub_base = -1;
+      P.value = 0;
+      *out = P;
+      return;
+    }
     const int g_want = level_for_ratio(S.lo, S.hi, B, p.fine_ratio);
     // every CTA that meets the layer sets up and flushes its private table once (cost ~ cells),
     // while the share of elements that need the slow path falls as n_bins / cells: the sum is

@@ -16,6 +16,7 @@
 #pragma once
 
 #include "common.cuh"
+#include "k_plan.cuh"
 #include "k_range.cuh"
 
 namespace adapt {
@@ -35,6 +36,7 @@ struct SearchParams {
   unsigned* u_hist;            // [n_layers][n_fl][n_bins]
   unsigned long long* zeros;   // [n_layers][n_fl]
   unsigned long long seed;
+  const LayerPlan* plan;       // by LayerDesc::index; read only for layers with via_plan set
 };
 
 // Bin index by one convert-with-floor and two integer clamps; equal to bin_of for every input
@@ -157,7 +159,9 @@ search_direct_kernel(const SearchParams p) {
     const long long layer_tiles_end = min(t_end, p.layers[l + 1].tile_begin);
     const float* base = L.ptr - L.mis;
     const long long jbeg = L.mis, jend = L.mis + L.n;
-    const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange));
+    // (a layer that the stochastic-rounding kernel serves is skipped here)
+    const bool layer_ok = !(S.flags & (kFlagNonfinite | kFlagRange)) &&
+                          !(L.via_plan && p.plan[gl].keyed);
     // largest float below the number of bins: floor of anything clamped to it is the last bin
     const float top = __uint_as_float(__float_as_uint(__fadd_rn(S.bmax, 1.0f)) - 1u);
 

@@ -382,3 +382,38 @@ def test_host_switch_with_packed_codes_in_slices(B):
                 assert unfit[l] == 0
                 want, _ = O.quantize(x, w_sel, f_sel, mode, 9, l)
                 assert np.array_equal(codes[l].numpy(), want.astype(dt)), (l, bits, mode)
+
+
+def test_stochastic_rounding_large_layers_keyed_and_direct(B):
+    """Stochastic rounding on layers large enough for its keyed kernel (cells for the fine
+    levels, tables of rounded values for the coarse ones), against the oracle, next to the
+    direct form: smooth data, many exact zeros, values on grids, ranges far from zero (left to
+    the direct kernel by the plan), tiny and wide ranges, several layers in one call."""
+    rng = np.random.default_rng(777)
+    n = 50000
+    base = (rng.standard_normal(n) * 0.25).astype(np.float32)
+    cases = {
+        "normal": base,
+        "laplace_outliers": W.generate_layer(W.LayerSpec("t", (n,), "laplace_outliers", 0.02,
+                                                         outlier_frac=0.01, outlier_gain=50.0), 3, 0),
+        "half_zero": np.maximum(base, 0),
+        "on_grid": (rng.integers(-2000, 2000, n) * 2.0 ** -6).astype(np.float32),
+        "ties": (rng.integers(-4000, 4000, n) * 2.0 ** -9 + 2.0 ** -10).astype(np.float32),
+        "far_from_zero": (1000.0 + rng.random(n) * 0.01).astype(np.float32),
+        "far_negative": (-123456.0 - rng.random(n) * 64).astype(np.float32),
+        "wide": (rng.standard_normal(n) * 1e6).astype(np.float32),
+        "tiny": (rng.standard_normal(n) * 1e-9).astype(np.float32),
+        "tiny_negative_fractions": (-np.abs(rng.standard_normal(n)) * 2.0 ** -30).astype(np.float32),
+        "integers": rng.integers(-300, 300, n).astype(np.float32),
+        "positive_only": (0.5 + 0.5 * rng.random(n)).astype(np.float32),
+    }
+    wl, fl = W.candidate_grid(range(2, 33))
+    for name, x in cases.items():
+        for n_bins in (100, 2048):
+            G.run_and_compare(B, [x], wl, fl, n_bins, round_mode=O.ROUND_STOCHASTIC, seed=13, layer_base=2,
+                              where=f"SR {name} B={n_bins}", algorithms=(0, 1, 2))
+    # several layers, large and small, ragged and misaligned, in one call
+    xs = [base[1:40001], cases["half_zero"][:33000], base[:100], np.zeros(0, np.float32),
+          cases["far_from_zero"], cases["on_grid"][3:45000], np.full(40000, 0.37, np.float32)]
+    G.run_and_compare(B, [np.ascontiguousarray(x) for x in xs], wl, fl, 128, round_mode=O.ROUND_STOCHASTIC,
+                      seed=7, where="SR layers", algorithms=(0, 1, 2))
