@@ -123,6 +123,7 @@ struct LayerCtx {
   unsigned* sub;               // global, this layer's [2][n_bins][kSubCells]
   unsigned* sub_s;             // shared [kSubSharedIds][kSubCells]: main segment's, when sub_base >= 0
   int sub_base;
+  unsigned cells_at, zclass_at, sub_s_at, qe_at, d_at;   // shared addresses of the tables the handler adds to
   int table_words;             // words of the cell table this layer may touch (cells + dummy slots)
   int value;                   // value-keyed layer
   unsigned* q_hist;            // global, this layer's [n_bins]
@@ -148,7 +149,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   if (x == 0.0f) {
     // only the dense form lets an exact zero through: it was counted in the cell [0, 2^-G),
     // where no zero belongs (zeros are the layer size minus all cell counts)
-    if (ADAPT_IN_BOUNDS(c.zero_pos, c.table_words, 10)) atomicSub(&c.cells[c.zero_pos], 1u);
+    if (ADAPT_IN_BOUNDS(c.zero_pos, c.table_words, 10)) smem_red_add(c.cells_at + 4u * c.zero_pos, 0xFFFFFFFFu);
     return;
   }
   const int s = (fabsf(x) < c.radius) ? 0 : 1;
@@ -159,9 +160,9 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
       !ADAPT_IN_BOUNDS(c.offset[s] + ci, c.total_cells, 12)) return;
   if (z == cf && grid_point_goes_left(c.c0[s] + ci)) {
     // on the grid and belonging to the left cell: move its count there
-    atomicSub(&c.cells[c.offset[s] + ci], 1u);
+    smem_red_add(c.cells_at + 4u * (c.offset[s] + ci), 0xFFFFFFFFu);
     ci -= 1;
-    atomicAdd(&c.cells[c.offset[s] + ci], 1u);
+    smem_red_add(c.cells_at + 4u * (c.offset[s] + ci), 1u);
   }
   const long long cc = c.c0[s] + ci;
   // ---- cells -1 / 0 of the main segment: the zero class of x --------------------------
@@ -170,7 +171,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     const unsigned ax = __float_as_uint(x) & 0x7FFFFFFFu;
     int kz = 125 - static_cast<int>((ax - 1u) >> 23);
     kz = max(-1, min(kz, 32));
-    atomicAdd(&c.zclass[kz + 1], 1u);
+    smem_red_add(c.zclass_at + 4u * (kz + 1), 1u);
   }
   // ---- edge cell: its sub-cell, float bin, then the fine levels that can still move ---------
   if (!(c.cells[c.offset[s] + ci] & kCellEdge)) return;
@@ -203,7 +204,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     const int id = bin_of(lf, c.lo, c.scale, c.bmax);
     if (s == 0 && c.sub_base >= 0) {
       if (ADAPT_IN_BOUNDS((id - c.sub_base) * kSubCells + j, kSubSharedIds * kSubCells, 13))
-        atomicAdd(&c.sub_s[(id - c.sub_base) * kSubCells + j], 1u);
+        smem_red_add(c.sub_s_at + 4u * ((id - c.sub_base) * kSubCells + j), 1u);
     } else if (ADAPT_IN_BOUNDS(id, B, 14)) {
       atomicAdd(&c.sub[(static_cast<size_t>(s) * B + id) * kSubCells + j], 1u);
     }
@@ -212,7 +213,7 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
   }
   const int b0 = bin_of(x, c.lo, c.scale, c.bmax);
   if (!ADAPT_IN_BOUNDS(b0, B, 15)) return;
-  if (s == 0) atomicAdd(&c.qe[b0], 1u); else atomicAdd(&c.qe_aux[b0], 1u);
+  if (s == 0) smem_red_add(c.qe_at + 4u * b0, 1u); else atomicAdd(&c.qe_aux[b0], 1u);
   const float e_lo = c.E[b0], e_hi = c.E[b0 + 1];
   // distance to the bin's two edges, rounded down: a level is safe once 2^-(f+1) < margin
   const float m = fminf(__fsub_rd(x, e_lo), __fsub_rd(e_hi, x));
@@ -228,8 +229,8 @@ __device__ __noinline__ void handle_special(const LayerCtx& c, float x) {
     if (!ADAPT_IN_BOUNDS(b, B, 16)) continue;
     const int j = f - fs;
     if (s == 0 && j < c.d_levels) {
-      atomicAdd(&c.d[j * B + b], 1);
-      atomicAdd(&c.d[j * B + b0], -1);
+      smem_red_add(c.d_at + 4u * (j * B + b), 1u);
+      smem_red_add(c.d_at + 4u * (j * B + b0), 0xFFFFFFFFu);
     } else {
       unsigned* U = c.u_hist + static_cast<size_t>(f) * B;
       atomicAdd(&U[b], 1u);
@@ -262,6 +263,7 @@ struct CellFn {
   unsigned grid_mask;           // masked form: low significand bits every grid point has zero
   unsigned grid_mul;            // dense form: 2^(32 - those bits)
   unsigned cell_base;           // dense form: shared-memory byte address of position 0, minus 4 * 0x4B400000
+  unsigned cells_at;            // shared-memory byte address of position 0
 #ifdef ADAPT_CHECK_BOUNDS
   int table_words;              // words of the cell table this layer may touch
 #endif
@@ -331,7 +333,7 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
       const float rd = __fmaf_rd(x, fn.two_g0, fn.magic0);
       const bool stray = __fmaf_ru(x, fn.two_g0, fn.magic0) != rd;
       const int pos = (x != 0.0f && !stray) ? __float_as_int(rd) - 0x4B400000 : dummy_pos;
-      if (ADAPT_IN_BOUNDS(pos, fn.table_words, 1)) atomicAdd(&cells[pos], 1u);
+      if (ADAPT_IN_BOUNDS(pos, fn.table_words, 1)) smem_red_add(fn.cells_at + 4u * pos, 1u);
       old[k] = stray ? kCellOnGrid : 0u;
       any |= old[k];
     }
@@ -368,7 +370,7 @@ __device__ __forceinline__ bool keyed_count(unsigned* cells, int dummy_pos, cons
     unsigned grid_bit;
     int pos = cell_position<kMode>(x, fn, &grid_bit);
     pos = (x != 0.0f) ? pos : dummy_pos;
-    const unsigned o = (ADAPT_IN_BOUNDS(pos, fn.table_words, 3) ? atomicAdd(&cells[pos], 1u) : 0u) + grid_bit;
+    const unsigned o = (ADAPT_IN_BOUNDS(pos, fn.table_words, 3) ? smem_atom_add(fn.cells_at + 4u * pos, 1u) : 0u) + grid_bit;
     old[k] = o;
     any |= o;
   }
@@ -454,7 +456,8 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
   fn.two_g1 = c.two_g[1]; fn.magic1 = c.magic[1];
   fn.grid_mask = c.grid_mask;
   fn.grid_mul = c.grid_mul;
-  fn.cell_base = static_cast<unsigned>(__cvta_generic_to_shared(cells)) - 4u * 0x4B400000u;
+  fn.cells_at = smem_addr(cells);
+  fn.cell_base = fn.cells_at - 4u * 0x4B400000u;
 #ifdef ADAPT_CHECK_BOUNDS
   fn.table_words = c.table_words;
 #endif
@@ -553,6 +556,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
       c.zero_pos = P->seg[0].offset + static_cast<int>(-P->seg[0].c0);
       c.E = edges;
       c.cells = cells; c.qe = qe; c.d = dtab; c.zclass = s_zclass;
+      c.cells_at = smem_addr(cells); c.qe_at = smem_addr(qe); c.d_at = smem_addr(dtab);
+      c.zclass_at = smem_addr(s_zclass); c.sub_s_at = smem_addr(sub_s);
       c.qe_aux = p.qe_hist + (static_cast<size_t>(l) * 2 + 1) * p.n_bins;
       c.u_hist = layer_u;
       c.zeros = p.zeros + static_cast<size_t>(l) * p.n_levels;
