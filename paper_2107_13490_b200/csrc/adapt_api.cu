@@ -165,6 +165,10 @@ constexpr int kMaxBins = 16384;
 #define ADAPT_D_LEVELS_MAX 6   // fine levels of the main segment whose corrections stay in shared memory
 #endif
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
+// Stochastic rounding: the keyed route saves about 10 us per 2^20 elements over the direct kernel and
+// costs three more launches, so it takes layers of 2^20 elements up, and only 2^22 of them together.
+constexpr long long kSrKeyedMinElements = 1ll << 20;
+constexpr long long kSrKeyedMinTotal = 1ll << 22;
 constexpr int kKeyedMaxBins = 8192;
 constexpr size_t kKeyedSmemBudget = 224 * 1024; // one CTA per SM owns its shared memory
 
@@ -386,11 +390,18 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       (o.algorithm == ADAPT_ALGO_AUTO || o.algorithm == ADAPT_ALGO_KEYED) &&
       (stochastic ? (plan.sr_cap >= 2048 && plan.sr_smem + 15 * 1024 <= static_cast<size_t>(dc.max_smem_optin))
                   : (plan.cell_cap >= 1024 && plan.keyed_smem + 2048 <= static_cast<size_t>(dc.max_smem_optin)));
-  const long long keyed_min = (o.algorithm == ADAPT_ALGO_KEYED) ? 1 : kKeyedMinElements;
+  const long long keyed_min = (o.algorithm == ADAPT_ALGO_KEYED) ? 1
+                              : stochastic ? kSrKeyedMinElements : kKeyedMinElements;
   std::vector<int> all(a.n_layers), keyed, direct;
   std::iota(all.begin(), all.end(), 0);
+  bool keyed_pays = keyed_possible;
+  if (stochastic && o.algorithm == ADAPT_ALGO_AUTO) {
+    long long total = 0;
+    for (int l = 0; l < a.n_layers; ++l) total += a.lens[l] >= keyed_min ? a.lens[l] : 0;
+    keyed_pays = keyed_pays && total >= kSrKeyedMinTotal;
+  }
   for (int l = 0; l < a.n_layers; ++l) {
-    const bool k = keyed_possible && a.lens[l] >= keyed_min;
+    const bool k = keyed_pays && a.lens[l] >= keyed_min;
     if (k) keyed.push_back(l);
     // Stochastic rounding: whether the keyed kernel can serve a layer is only known on the
     // device (its cell indices must be exact in a float), so its layers also stand in the

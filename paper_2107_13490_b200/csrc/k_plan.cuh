@@ -59,8 +59,8 @@ constexpr int kSubSharedIds = 128;
 #ifndef ADAPT_CELL_BALANCE
 #define ADAPT_CELL_BALANCE 4    // cells ~ sqrt(balance * n_bins * elements one CTA sees of the layer)
 #endif
-#ifndef ADAPT_RADIUS_FACTOR
-#define ADAPT_RADIUS_FACTOR 8.0   // main segment reaches to the power of two above this many mean magnitudes
+#ifndef ADAPT_TWO_SEGMENT_GAIN
+#define ADAPT_TWO_SEGMENT_GAIN 0.8   // two segments must promise this much of one segment's edge-cell share, or less
 #endif
 #ifndef ADAPT_FINE_RATIO
 #define ADAPT_FINE_RATIO 512    // stop refining once a bin holds this many cells
@@ -127,9 +127,21 @@ struct PlanParams {
   long long elems_per_cta;   // elements one CTA of the keyed kernel processes
 };
 
+// v * 2^g by one multiplication with a constructed power of two: exact while |g| <= 1000 and the
+// product is a normal double (floats times 2^g with |g| <= 200 always are), and far cheaper
+// than the library's ldexp for the single thread that plans a layer.
+__device__ __forceinline__ double scale_pow2(double v, int g) {
+  return v * __hiloint2double((1023 + g) << 20, 0);
+}
+
+// Binary exponent of a positive normal double (floor of its base-2 logarithm); 1024 for +inf.
+__device__ __forceinline__ int exponent_of(double v) {
+  return ((__double2hiint(v) >> 20) & 0x7FF) - 1023;
+}
+
 __device__ __forceinline__ long long floor_scaled(float v, int g) {
   // floor(v * 2^g) exactly: the product stays inside double
-  return static_cast<long long>(floor(ldexp(static_cast<double>(v), g)));
+  return static_cast<long long>(floor(scale_pow2(static_cast<double>(v), g)));
 }
 
 // Largest level G <= g_max such that the cells covering [lo, hi] number at most max_cells.
@@ -138,14 +150,14 @@ __device__ inline void fit_segment(float lo, float hi, int max_cells, int g_max,
   int g = g_max;
   {
     const double span0 = static_cast<double>(hi) - static_cast<double>(lo);
-    if (span0 > 0.0) g = min(g_max, ilogb(static_cast<double>(max_cells)) - ilogb(span0) + 2);
+    if (span0 > 1.0e-300 && span0 < 1.0e300) g = min(g_max, exponent_of(static_cast<double>(max_cells)) - exponent_of(span0) + 2);
   }
   long long c0 = 0, c1 = 0;
   for (; g > -100; --g) {
-    const double span = ldexp(static_cast<double>(hi) - static_cast<double>(lo), g);
+    const double span = scale_pow2(static_cast<double>(hi) - static_cast<double>(lo), g);
     if (span + 1.0 >= static_cast<double>(max_cells)) continue;
-    if (fabs(ldexp(static_cast<double>(hi), g)) > 9.0e18 ||
-        fabs(ldexp(static_cast<double>(lo), g)) > 9.0e18) continue;
+    if (fabs(scale_pow2(static_cast<double>(hi), g)) > 9.0e18 ||
+        fabs(scale_pow2(static_cast<double>(lo), g)) > 9.0e18) continue;
     c0 = floor_scaled(lo, g) - 1;   // one spare cell on the left (grid points that go left)
     c1 = floor_scaled(hi, g);
     if (c1 - c0 + 1 <= max_cells) break;
@@ -160,7 +172,12 @@ __device__ inline void fit_segment(float lo, float hi, int max_cells, int g_max,
 __device__ inline int level_for_ratio(float lo, float hi, int n_bins, int ratio) {
   const double bw = (static_cast<double>(hi) - static_cast<double>(lo)) / n_bins;
   if (!(bw > 0.0)) return 32;
-  int g = static_cast<int>(ceil(log2(static_cast<double>(ratio) / bw)));
+  const double y = static_cast<double>(ratio) / bw;
+  if (!(y < 1.0e300)) return 32;
+  if (!(y > 1.0e-300)) return -100;
+  // ceil(log2(y)): the exponent, one more unless y is a power of two
+  const bool pow2 = (__double2hiint(y) & 0xFFFFF) == 0 && __double2loint(y) == 0;
+  const int g = exponent_of(y) + (pow2 ? 0 : 1);
   return max(-100, min(g, 32));
 }
 
@@ -172,8 +189,8 @@ __device__ __forceinline__ void cell_ends(long long cc, int g, bool exact_in_flo
     *lf = __fmul_rn(__ll2float_rn(cc), w);
     *rf = __fmul_rn(__ll2float_rn(cc + 1), w);
   } else {
-    *lf = __double2float_rd(ldexp(static_cast<double>(cc), -g));
-    *rf = __double2float_ru(ldexp(static_cast<double>(cc + 1), -g));
+    *lf = __double2float_rd(scale_pow2(static_cast<double>(cc), -g));
+    *rf = __double2float_ru(scale_pow2(static_cast<double>(cc + 1), -g));
   }
 }
 
@@ -192,9 +209,11 @@ __device__ __forceinline__ unsigned cell_mark(const LayerPlan& P, const LayerSta
   return mark;
 }
 
-// The plan of one layer from its final state: called by one thread.
+// The plan of one layer from its final state: called by all 32 lanes of one warp together (they
+// compute the same plan; the candidate radii of the two-segment choice are dealt to the lanes).
 __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, const LayerState& S,
-                                       unsigned min_lsb, LayerPlan* out) {
+                                       unsigned min_lsb, const int* exp_below, int n_samples,
+                                       LayerPlan* out) {
   const int B = L.n_bins;      // this layer's own number of bins
   {
     LayerPlan P;
@@ -221,7 +240,7 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
       P.seg[1].offset = P.seg[0].cells;
       P.total_cells = P.seg[0].cells;
       const float top = fmaxf(fabsf(S.lo), fabsf(S.hi));
-      P.fast = (ldexp(static_cast<double>(top), max(P.seg[0].g, 0)) < 4.0e6 && P.seg[0].g >= -100 &&
+      P.fast = (scale_pow2(static_cast<double>(top), max(P.seg[0].g, 0)) < 4.0e6 && P.seg[0].g >= -100 &&
                 P.seg[0].g <= 100) ? 1 : 0;
       if (!P.fast) P.keyed = 0;           // left to the direct kernel
       P.seg[0].magic = 0.0f;
@@ -238,23 +257,57 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
     const long long want = static_cast<long long>(sqrt(ADAPT_CELL_BALANCE * static_cast<double>(B) * seen));
     const int cap = static_cast<int>(min(static_cast<long long>(p.cell_cap), max(2048ll, want)));
     fit_segment(S.lo, S.hi, cap, g_want, &P.seg[0]);
-    // two segments pay off when zero is inside the range, the single segment cannot reach
-    // the wanted fineness, and the mass sits within a small radius
+    // Two segments pay off when zero is inside the range, the single segment cannot reach the
+    // wanted fineness, and the mass sits within a small radius.  The radius is the power of two
+    // for which the sampled magnitudes promise the fewest elements in edge cells: a segment whose
+    // bins hold k cells each leaves about 1/k of its elements there.  (Exact zeros are left out
+    // of the estimate: they never sit in an edge cell.)
     const float amax = fmaxf(fabsf(S.lo), fabsf(S.hi));
-    const float mean = S.abs_sum / static_cast<float>(L.n > 0 ? L.n : 1);
-    if (P.keyed && S.lo <= 0.0f && S.hi >= 0.0f && P.seg[0].g < g_want && mean > 0.0f &&
-        mean < 3.0e38f) {
-      const int rexp = static_cast<int>(ceil(log2(static_cast<double>(mean) * ADAPT_RADIUS_FACTOR)));
-      if (rexp > -100 && rexp < 100) {
-        const float r = pow2f(rexp);
-        if (r < 0.25f * amax) {
+    if (P.keyed && S.lo <= 0.0f && S.hi >= 0.0f && P.seg[0].g < g_want && n_samples > 0 &&
+        amax > 0.0f && amax < 3.0e38f) {
+      const double span = static_cast<double>(S.hi) - static_cast<double>(S.lo);
+      const double bw = span / B;
+      const double share_one = fmin(1.0, scale_pow2(1.0, -P.seg[0].g) / bw);
+      const int top_e = static_cast<int>((__float_as_uint(amax) >> 23) & 0xFFu) - 127;   // 2^top_e <= amax
+      const int main_cap = cap - cap / 4;
+      // one candidate radius 2^e per lane, the largest first
+      const int lane = threadIdx.x & 31;
+      const int e = top_e - lane;
+      double share = 2.0;                           // "not a candidate"
+      if (e > -100) {
+        const double r = scale_pow2(1.0, e);
+        const double span_m = fmin(static_cast<double>(S.hi), r) - fmax(static_cast<double>(S.lo), -r);
+        const int g_m = min(g_want, exponent_of((main_cap - 3) / span_m));
+        const double cells_m = scale_pow2(span_m, g_m) + 3.0;
+        const int g_a = min(g_want, exponent_of((cap - cells_m - 3.0) / span));
+        // finer main cells than one segment's, and the auxiliary cells next to zero stay empty
+        if (g_m > P.seg[0].g && r > scale_pow2(1.0, -g_a)) {
+          // sampled share of the elements below 2^e in magnitude (biased exponent below e + 127)
+          const int below = exp_below[max(0, min(e + 127, 255))];
+          const double in = static_cast<double>(below) / n_samples;
+          share = in * fmin(1.0, scale_pow2(1.0, -g_m) / bw) +
+                  (1.0 - in) * fmin(1.0, scale_pow2(1.0, -g_a) / bw);
+        }
+      }
+      // the smallest share wins, the larger radius among equals
+      int best_e = e;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const double s2 = __shfl_xor_sync(0xffffffffu, share, o);
+        const int e2 = __shfl_xor_sync(0xffffffffu, best_e, o);
+        if (s2 < share || (s2 == share && e2 > best_e)) { share = s2; best_e = e2; }
+      }
+      if (!(share < share_one * ADAPT_TWO_SEGMENT_GAIN)) best_e = -1000;
+      if (best_e > -1000) {
+        const float r = pow2f(best_e);
+        {
           SegPlan aux, main;
           // the main segment takes what it needs (up to three quarters), the rest is auxiliary
           const float mlo = fmaxf(S.lo, -r), mhi = fminf(S.hi, r);
-          fit_segment(mlo, mhi, cap - cap / 4, g_want, &main);
+          fit_segment(mlo, mhi, main_cap, g_want, &main);
           fit_segment(S.lo, S.hi, cap - main.cells, g_want, &aux);
           // the auxiliary cells next to zero must stay empty: R at least two of them wide
-          if (main.g > P.seg[0].g + 1 && r > pow2f(-aux.g)) {
+          if (main.g > P.seg[0].g && r > pow2f(-aux.g)) {
             P.seg[0] = main; P.seg[1] = aux; P.radius = r;
             P.seg[0].pad_ = 0; P.seg[1].pad_ = 0;
           }
@@ -290,8 +343,8 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
     P.sub_base = -1;
     if (P.refined) {
       const SegPlan& m0 = P.seg[0];
-      const float first = __double2float_rd(ldexp(static_cast<double>(m0.c0), -m0.g));
-      const float last = __double2float_rd(ldexp(static_cast<double>(m0.c0 + m0.cells - 1), -m0.g));
+      const float first = __double2float_rd(scale_pow2(static_cast<double>(m0.c0), -m0.g));
+      const float last = __double2float_rd(scale_pow2(static_cast<double>(m0.c0 + m0.cells - 1), -m0.g));
       const int b_first = bin_of(first, S.lo, S.scale, S.bmax);
       if (bin_of(last, S.lo, S.scale, S.bmax) - b_first < kSubSharedIds) P.sub_base = b_first;
     }
@@ -310,8 +363,8 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
     if (P.keyed && min_lsb != 0xFFFFFFFFu) {
       const int g = 150 - static_cast<int>(min_lsb);
       if (g >= -100 && g <= 100) {
-        const double span = ldexp(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
-        const double far = ldexp(static_cast<double>(amax), g);
+        const double span = scale_pow2(static_cast<double>(S.hi) - static_cast<double>(S.lo), g);
+        const double far = scale_pow2(static_cast<double>(amax), g);
         if (span + 3.0 <= static_cast<double>(p.value_cap) && far < 4.0e6) {
           SegPlan v;
           v.g = g;
@@ -338,25 +391,22 @@ __device__ inline void make_layer_plan(const PlanParams& p, const LayerDesc& L, 
 
 // Exact lower edge of bin b (1 <= b < n_bins) of a layer: the smallest float v with
 // bin_of(v) >= b, or +inf if no value up to the layer's maximum reaches the bin.  The bin
-// function is monotone, so the edge is found by walking the float order from an estimate
-// (lo + b / scale is within a few floats of it), with a bisection over [lo, hi] as the fallback.
+// function is monotone, so the edge is found by bisection over the float order.  The bracket
+// starts around the estimate lo + b / scale: the bin function rounds v - lo and its product with
+// the scale, so the edge lies within a few units in the last place OF THAT DIFFERENCE from the
+// estimate (which near zero can be thousands of floats); [lo, hi] is the fallback bracket.
 __device__ inline float bin_lower_edge(int b, const LayerState& S) {
   if (bin_of(S.hi, S.lo, S.scale, S.bmax) < b) return __int_as_float(0x7f800000);
-  const unsigned klo = float_key(S.lo), khi = float_key(S.hi);   // bin(lo) = 0 < b <= bin(hi)
-  const float guess = __fadd_rn(S.lo, __fdiv_rn(static_cast<float>(b), S.scale));
-  unsigned k = float_key(guess);
-  if (guess == guess && k > klo && k <= khi) {
-    // walk down while the float below still reaches the bin, up while this one does not
-    int steps = 0;
-    if (bin_of(key_float(k), S.lo, S.scale, S.bmax) >= b) {
-      while (steps < 48 && k - 1u > klo && bin_of(key_float(k - 1u), S.lo, S.scale, S.bmax) >= b) { --k; ++steps; }
-      if (steps < 48 && bin_of(key_float(k - 1u), S.lo, S.scale, S.bmax) < b) return key_float(k);
-    } else {
-      while (steps < 48 && k < khi && bin_of(key_float(k), S.lo, S.scale, S.bmax) < b) { ++k; ++steps; }
-      if (steps < 48 && bin_of(key_float(k), S.lo, S.scale, S.bmax) >= b) return key_float(k);
-    }
+  unsigned a = float_key(S.lo), z = float_key(S.hi);   // bin(a) = 0 < b <= bin(z)
+  const float t = __fdiv_rn(static_cast<float>(b), S.scale);
+  const float guess = __fadd_rn(S.lo, t);
+  const float d = __fmul_rn(fmaxf(t, fabsf(guess)), 4.76837158203125e-7f);   // 2^-21 of the larger
+  const float ga = __fsub_rn(guess, d), gz = __fadd_rn(guess, d);
+  if (ga == ga && gz == gz && d > 0.0f && fabsf(gz) < 3.0e38f && fabsf(ga) < 3.0e38f) {
+    const unsigned ka = float_key(ga), kz = float_key(gz);
+    if (ka > a && ka < z && bin_of(ga, S.lo, S.scale, S.bmax) < b) a = ka;
+    if (kz < z && kz > a && bin_of(gz, S.lo, S.scale, S.bmax) >= b) z = kz;
   }
-  unsigned a = klo, z = khi;   // bin(a) < b, bin(z) >= b
   while (z - a > 1) {
     const unsigned m = a + ((z - a) >> 1);
     if (bin_of(key_float(m), S.lo, S.scale, S.bmax) >= b) z = m; else a = m;
@@ -366,12 +416,16 @@ __device__ inline float bin_lower_edge(int b, const LayerState& S) {
 
 constexpr int kPlanThreads = 256;
 constexpr int kPlanSamples = 1024;   // elements of a layer looked at for the grid it lies on
+static_assert(kPlanThreads == 256, "the exponent classes are scanned one per thread");
 
 // One layer per blockIdx.x; the gridDim.y CTAs of a layer all derive its plan (one thread each)
 // and share its bin edges.
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) {
   __shared__ LayerPlan s_plan;
   __shared__ unsigned s_lsb;
+  __shared__ int s_exp[256];     // sampled elements by biased exponent, then "below this exponent"
+  __shared__ int s_warp[kPlanThreads / 32];
+  __shared__ int s_total;
   const LayerDesc L = p.layers[blockIdx.x];
   const int l = L.index;
   const LayerState S = p.state[l];
@@ -380,24 +434,48 @@ __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) 
   // (biased exponent + trailing zero bits of the 24-bit significand).  It only decides whether
   // the layer is keyed by value; the counting loop checks every element against the grid.
   if (threadIdx.x == 0) s_lsb = 0xFFFFFFFFu;
+  for (int i = threadIdx.x; i < 256; i += kPlanThreads) s_exp[i] = 0;
   __syncthreads();
+  const long long n_s = min(L.n, static_cast<long long>(kPlanSamples));
   {
-    const long long n_s = min(L.n, static_cast<long long>(kPlanSamples));
     const long long step = n_s > 0 ? L.n / n_s : 1;
     unsigned lsb = 0xFFFFFFFFu;
     for (long long i = threadIdx.x; i < n_s; i += kPlanThreads) {
       const unsigned bits = __float_as_uint(__ldg(L.ptr + i * step));
       const unsigned at = ((bits >> 23) & 0xFFu) + static_cast<unsigned>(__ffs(bits | 0x00800000u) - 1);
       if ((bits & 0x7FFFFFFFu) != 0u) lsb = min(lsb, at);
+      if ((bits & 0x7FFFFFFFu) != 0u) atomicAdd(&s_exp[(bits >> 23) & 0xFFu], 1);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) lsb = min(lsb, __shfl_xor_sync(0xffffffffu, lsb, o));
     if ((threadIdx.x & 31) == 0 && lsb != 0xFFFFFFFFu) atomicMin(&s_lsb, lsb);
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    make_layer_plan(p, L, S, s_lsb, &s_plan);
-    if (blockIdx.y == 0) p.plan[l] = s_plan;
+  // the same sample by magnitude: s_exp[k] becomes the number of sampled non-zero elements whose
+  // biased exponent is below k (it steers the choice of segments only); kPlanThreads == 256
+  {
+    const int own = s_exp[threadIdx.x];
+    int incl = own;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(0xffffffffu, incl, o);
+      if ((threadIdx.x & 31) >= o) incl += up;
+    }
+    if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < (threadIdx.x >> 5); ++w) before += s_warp[w];
+    s_exp[threadIdx.x] = before + incl - own;
+    if (threadIdx.x == kPlanThreads - 1) s_total = before + incl;
+  }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    LayerPlan P;
+    make_layer_plan(p, L, S, s_lsb, s_exp, s_total, &P);
+    if (threadIdx.x == 0) {
+      s_plan = P;
+      if (blockIdx.y == 0) p.plan[l] = P;
+    }
   }
   __syncthreads();
   if (!s_plan.keyed || s_plan.value) return;     // a value-keyed layer needs no bin edges

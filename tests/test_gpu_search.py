@@ -417,3 +417,9 @@ def test_stochastic_rounding_large_layers_keyed_and_direct(B):
           cases["far_from_zero"], cases["on_grid"][3:45000], np.full(40000, 0.37, np.float32)]
     G.run_and_compare(B, [np.ascontiguousarray(x) for x in xs], wl, fl, 128, round_mode=O.ROUND_STOCHASTIC,
                       seed=7, where="SR layers", algorithms=(0, 1, 2))
+    # a layer large enough for the automatic choice to take the keyed route by itself
+    big = W.generate_layer(W.LayerSpec("t", ((1 << 22) + 777,), "laplace_outliers", 0.02,
+                                       outlier_frac=0.01, outlier_gain=50.0), 5, 0)
+    wl2, fl2 = W.candidate_grid((6, 12, 20, 32))
+    G.run_and_compare(B, [big, base], wl2, fl2, 256, round_mode=O.ROUND_STOCHASTIC, seed=21,
+                      where="SR automatic route", algorithms=(0,))
