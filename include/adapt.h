@@ -57,7 +57,7 @@ enum {
   ADAPT_FLAG_MET_EPS = 1,    /* the returned candidate has KLD <= eps           */
   ADAPT_FLAG_DEGENERATE = 2, /* max == min (or empty layer): one bin, KLD == 0  */
   ADAPT_FLAG_NONFINITE = 4,  /* layer holds NaN/Inf: its outputs are unspecified */
-  ADAPT_FLAG_RANGE = 8       /* layer holds |x| >= 2^64: outputs unspecified     */
+  ADAPT_FLAG_RANGE = 8       /* layer holds |x| >= 2^64 (and no NaN/Inf): outputs unspecified */
 };
 
 /* Candidate formats. HOST arrays of n_cand entries each, in any order. */
@@ -111,10 +111,13 @@ typedef struct adapt_search_opts {
 } adapt_search_opts;
 
 /* Forms of the fused quantize / zero-count / histogram kernel.  Both give the
- * same results bit for bit.  AUTO: the keyed form for round-to-nearest-even
- * layers of at least 32768 elements with n_bins <= 8192, the direct form for
- * the rest.  KEYED: the keyed form for every layer it can serve (RNE,
- * n_bins <= 8192).  DIRECT: the direct form everywhere. */
+ * same results bit for bit.  AUTO: the keyed form for layers of at least 32768
+ * elements under round-to-nearest-even, and under stochastic rounding for
+ * layers of at least 2^20 elements when the call holds 2^22 of them, in both
+ * cases with n_bins <= 8192; the direct form for the rest.  KEYED: the keyed
+ * form for every layer it can serve (n_bins <= 8192; under stochastic rounding
+ * a layer whose range lies too far from zero for exact cell indices stays with
+ * the direct form).  DIRECT: the direct form everywhere. */
 enum { ADAPT_ALGO_AUTO = 0, ADAPT_ALGO_KEYED = 1, ADAPT_ALGO_DIRECT = 2 };
 
 /* Library version string: "adapt-b200 <major>.<minor>". Never NULL. */

@@ -662,7 +662,7 @@ int run_quantize(const float* x, int64_t n, int wl, int fl, const int32_t* selec
 
 extern "C" {
 
-const char* adapt_version(void) { return "adapt-b200 0.8"; }
+const char* adapt_version(void) { return "adapt-b200 0.9"; }
 
 const char* adapt_status_string(int status) {
   switch (status) {

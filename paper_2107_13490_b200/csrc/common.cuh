@@ -41,7 +41,7 @@ struct LayerState {
   unsigned max_key;  // ... of the maximum
   unsigned flags;    // ADAPT_FLAG_NONFINITE / ADAPT_FLAG_RANGE / ADAPT_FLAG_DEGENERATE
   float lo, hi, scale, bmax;
-  float abs_sum;     // sum of |x| (any summation order; only steers table shapes, never results)
+  unsigned pad_;
   unsigned zero_count;  // estimate of the exact zeros (the range scan samples one element in
                         // eight; steers the choice of loop form only, never results)
   unsigned ticket;      // range scan: CTAs that have added their part of this layer (the last one

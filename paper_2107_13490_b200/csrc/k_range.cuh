@@ -42,13 +42,12 @@ __device__ __forceinline__ void range_finalize_layer(const RangeParams& p, const
 // One CTA's part of a layer (already reduced over the CTA) is added to the layer's state; returns
 // whether it was the last part, in which case the layer's bin origin and scale have been derived.
 __device__ __forceinline__ bool range_layer_commit(const RangeParams& p, const LayerDesc* layer,
-                                                unsigned kmin, unsigned kmax, unsigned flags, float asum,
+                                                unsigned kmin, unsigned kmax, unsigned flags,
                                                 unsigned nzero) {
   LayerState* st = p.state + layer->index;
   atomicMin(&st->min_key, kmin);
   atomicMax(&st->max_key, kmax);
   if (flags) atomicOr(&st->flags, flags);
-  if (asum == asum && asum < 3.0e38f) atomicAdd(&st->abs_sum, asum);
   if (nzero) atomicAdd(&st->zero_count, nzero * static_cast<unsigned>(kTile / 4 / kRangeThreads));
   __threadfence();
   const unsigned done = atomicAdd(&st->ticket, 1u);
@@ -61,10 +60,9 @@ __device__ __forceinline__ bool range_layer_commit(const RangeParams& p, const L
 // What a CTA does with its part of a layer once its tiles are read: reduce the threads' values
 // and add them to the layer's state.  Called by the whole CTA.
 __device__ __forceinline__ void range_layer_tail(const RangeParams& p, const LayerDesc* layer,
-                                                 float vmin, float vmax, unsigned flags, float asum,
+                                                 float vmin, float vmax, unsigned amax,
                                                  unsigned nzero) {
   __shared__ unsigned s_min[kRangeThreads / 32], s_max[kRangeThreads / 32], s_flag[kRangeThreads / 32];
-  __shared__ float s_abs[kRangeThreads / 32];
   __shared__ unsigned s_zero[kRangeThreads / 32];
   // -0.0 and +0.0 are the same value: canonicalise before taking keys
   unsigned kmin = float_key(__fadd_rn(vmin, 0.0f));
@@ -73,20 +71,23 @@ __device__ __forceinline__ void range_layer_tail(const RangeParams& p, const Lay
   for (int o = 16; o > 0; o >>= 1) {
     kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
     kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-    flags |= __shfl_xor_sync(0xffffffffu, flags, o);
-    asum += __shfl_xor_sync(0xffffffffu, asum, o);
+    amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, o));
     nzero += __shfl_xor_sync(0xffffffffu, nzero, o);
   }
+  // amax = the largest magnitude as a bit pattern (sign cleared): NaN and Inf are the patterns
+  // from 0x7F800000 up, 2^64 is 0x5F800000.  (An out-of-range magnitude is reported only for
+  // layers without NaN/Inf.)
+  unsigned flags = amax >= 0x7F800000u ? kFlagNonfinite : (amax >= 0x5F800000u ? kFlagRange : 0u);
   const int w = threadIdx.x >> 5;
-  if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_abs[w] = asum; s_zero[w] = nzero; }
+  if ((threadIdx.x & 31) == 0) { s_min[w] = kmin; s_max[w] = kmax; s_flag[w] = flags; s_zero[w] = nzero; }
   __syncthreads();
   if (threadIdx.x == 0) {
     for (int i = 1; i < kRangeThreads / 32; ++i) {
       kmin = min(kmin, s_min[i]); kmax = max(kmax, s_max[i]); flags |= s_flag[i];
-      asum += s_abs[i]; nzero += s_zero[i];
+      nzero += s_zero[i];
     }
     // the CTA that brings the last part of the layer finishes it
-    range_layer_commit(p, layer, kmin, kmax, flags, asum, nzero);
+    range_layer_commit(p, layer, kmin, kmax, flags, nzero);
   }
   __syncthreads();
 }
@@ -119,8 +120,7 @@ __global__ void __launch_bounds__(kRangeThreads, 8) range_scan_kernel(const __gr
     const long long jbeg = L.mis, jend = L.mis + L.n;
 
     float vmin = __int_as_float(0x7f800000), vmax = __int_as_float(0xff800000);
-    unsigned flags = 0;
-    float asum = 0.0f;
+    unsigned amax = 0;
     unsigned nzero = 0;
     for (; t < layer_tiles_end; ++t) {
       const long long j_tile = (t - L.tile_begin) * kTile;
@@ -149,19 +149,16 @@ __global__ void __launch_bounds__(kRangeThreads, 8) range_scan_kernel(const __gr
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           if (m[q] & (1u << k)) {
-            float a = fabsf(v[q][k]);
-            // NaN fails both compares; Inf is caught by the first
-            if (!(a <= 3.402823466e38f)) flags |= kFlagNonfinite;
-            else if (a >= 18446744073709551616.0f) flags |= kFlagRange;
-            vmin = fminf(vmin, v[q][k]);
+            const unsigned a = __float_as_uint(v[q][k]) & 0x7FFFFFFFu;
+            amax = max(amax, a);                  // NaN, Inf and |x| >= 2^64 show in the pattern
+            vmin = fminf(vmin, v[q][k]);          // (a NaN operand is ignored)
             vmax = fmaxf(vmax, v[q][k]);
-            asum += a;
-            if (q == 0) nzero += (a == 0.0f) ? 1u : 0u;   // one quad in kQ: a sample is enough
+            if (q == 0) nzero += (a == 0u) ? 1u : 0u;   // one quad in kQ: a sample is enough
           }
         }
       }
     }
-    range_layer_tail(p, layers + l, vmin, vmax, flags, asum, nzero);
+    range_layer_tail(p, layers + l, vmin, vmax, amax, nzero);
     ++l;
     while (l < n_layers && layers[l + 1].tile_begin <= t) ++l;  // skip empty layers
   }
