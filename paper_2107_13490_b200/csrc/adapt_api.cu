@@ -538,10 +538,20 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ep.cell_total = reinterpret_cast<const unsigned long long*>(ws + plan.off_nzero);
     ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_stride = plan.value_cap;
     {
+      // pyramid form: enough slices (times six roles) per layer to fill the GPU, and at least as many as keep
+      // a slice's cells (1.5 words each) and the fine histogram inside one CTA's shared memory
+      const size_t room = static_cast<size_t>(dc.max_smem_optin) - 2048 - sizeof(unsigned) * bins_stride;
+      const int cap_max = static_cast<int>(std::min<size_t>(room / 6, 1u << 20)) & ~3;
+      int slices = std::max(1, std::min(32, (3 * dc.sm_count + nk * kExpandRoles - 1) / (nk * kExpandRoles)));
+      slices = std::max(slices, (plan.value_cap + cap_max - 1) / std::max(cap_max, 4));
+      ep.slices = slices;
+      ep.slice_cap = ((plan.value_cap + slices - 1) / slices + 3) & ~3;
+      const size_t smem = sizeof(unsigned) * (static_cast<size_t>(bins_stride) + ep.slice_cap + ep.slice_cap / 2 + 2);
+      if (smem + 1024 > static_cast<size_t>(dc.max_smem_optin)) return ADAPT_ERR_INVALID_ARG;
+      ADAPT_CUDA(cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(smem)));
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / ((plan.n_levels + 1) * nk)));
-      expand_kernel<<<dim3(plan.n_levels + 1, nk, slices), kExpandThreads,
-                      sizeof(unsigned) * bins_stride, stream>>>(ep);
+      expand_kernel<<<dim3(std::max(slices * kExpandRoles, plan.n_levels + 1), nk), kExpandThreads, smem, stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
     }
