@@ -165,6 +165,10 @@ constexpr int kMaxBins = 16384;
 #define ADAPT_D_LEVELS_MAX 6   // fine levels of the main segment whose corrections stay in shared memory
 #endif
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
+constexpr int kMaxKeyedGrid = 1023;             // CTAs of the keyed kernel (one per SM) whose tile ranges fit the descriptor block
+// What it costs a CTA of the keyed kernel to take up one more layer (context, table set-up, flush),
+// in tiles' worth of counting: the tile ranges of the CTAs are balanced with it.
+constexpr double kLayerCostTiles = 4.0;
 // Stochastic rounding: the keyed route saves about 10 us per 2^20 elements over the direct kernel and
 // costs three more launches, so it takes layers of 2^20 elements up, and only 2^22 of them together.
 constexpr long long kSrKeyedMinElements = 1ll << 20;
@@ -183,7 +187,7 @@ struct Plan {
   size_t sr_smem = 0;
   // byte offsets inside the workspace -- descriptor block (uploaded)
   size_t off_layers = 0, off_keyed = 0, off_direct = 0, off_wl = 0, off_fl = 0, off_slot = 0,
-         off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_start = 0, off_state = 0, blob_bytes = 0;
+         off_order = 0, off_by_fl = 0, off_fl_begin = 0, off_start = 0, off_cta = 0, off_state = 0, blob_bytes = 0;
   // written by kernels, not cleared
   size_t off_plan = 0, off_edges = 0;
   // accumulators (cleared every call)
@@ -263,6 +267,7 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
   p->off_by_fl = o;   o = align_up(o + sizeof(int) * C, 16);
   p->off_fl_begin = o; o = align_up(o + sizeof(int) * (F + 1), 16);
   p->off_start = o;   o = align_up(o + sizeof(int) * 2 * L, 16);
+  p->off_cta = o;     o = align_up(o + sizeof(long long) * (kMaxKeyedGrid + 1), 16);
   p->off_state = o;   o = align_up(o + sizeof(LayerState) * L, 256);
   p->blob_bytes = o;
   p->off_plan = o;      o = align_up(o + sizeof(LayerPlan) * L, 256);
@@ -341,6 +346,39 @@ long long fill_list(LayerDesc* out, const std::vector<int>& pick, const SearchAr
   s.ptr = nullptr; s.n = 0; s.tile_begin = tiles; s.mis = 0; s.layer_id = 0; s.index = 0; s.n_bins = 1;
   s.range_ctas = 0; s.via_plan = 0; s.pad_ = 0;
   return tiles;
+}
+
+// Contiguous tile ranges for the CTAs of the keyed kernel, balanced by cost: a tile costs 1, and
+// every layer a CTA touches costs kLayerCostTiles more (so CTAs in a stretch of small layers get
+// fewer tiles).  list: the keyed layer list with its sentinel; out: grid + 1 first tiles.  The
+// smallest per-CTA budget under which a greedy walk places all tiles is found by bisection.
+void balance_keyed_ctas(const LayerDesc* list, int n_layers, long long tiles, int grid, long long* out) {
+  auto walk = [&](double budget, long long* begin) {
+    int k = 0;
+    long long t = 0;
+    for (int cta = 0; cta < grid; ++cta) {
+      if (begin) begin[cta] = t;
+      double load = 0.0;
+      while (t < tiles) {
+        while (k < n_layers && list[k + 1].tile_begin <= t) ++k;
+        if (load > 0.0 && load + kLayerCostTiles + 1.0 > budget) break;
+        load += kLayerCostTiles;
+        const long long left = list[k + 1].tile_begin - t;
+        const long long take = std::max<long long>(1, std::min<long long>(left, static_cast<long long>(budget - load)));
+        t += take;
+        load += static_cast<double>(take);
+        if (take < left) break;
+      }
+    }
+    if (begin) begin[grid] = tiles;
+    return t >= tiles;
+  };
+  double lo = static_cast<double>(tiles) / grid, hi = static_cast<double>(tiles) + kLayerCostTiles * (n_layers + 1) + 1.0;
+  for (int it = 0; it < 40 && hi - lo > 0.25; ++it) {
+    const double mid = 0.5 * (lo + hi);
+    if (walk(mid, nullptr)) hi = mid; else lo = mid;
+  }
+  walk(hi, out);
 }
 
 // Enqueues the whole search on opts.stream.  Caller holds g_mutex.
@@ -428,6 +466,11 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       if (k < keyed.size() && keyed[k] == direct[i]) dl[i].via_plan = 1;
     }
   }
+  const int keyed_grid = static_cast<int>(std::max<long long>(
+      1, std::min<long long>(keyed_tiles, std::min(dc.sm_count, kMaxKeyedGrid))));
+  if (!stochastic && keyed_tiles > 0)
+    balance_keyed_ctas(reinterpret_cast<const LayerDesc*>(h + plan.off_keyed), static_cast<int>(keyed.size()),
+                       keyed_tiles, keyed_grid, reinterpret_cast<long long*>(h + plan.off_cta));
   std::memcpy(h + plan.off_wl, a.grid->wl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_fl, a.grid->fl, sizeof(int) * plan.n_cand);
   std::memcpy(h + plan.off_slot, plan.slot.data(), sizeof(int) * plan.n_cand);
@@ -458,7 +501,6 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   ADAPT_CUDA(cudaMemsetAsync(ws + plan.accum_begin, 0, plan.accum_bytes, stream));
 
   // K1: range scan over every layer; its last CTA per layer derives the bin origin and scale
-  const int keyed_grid = static_cast<int>(std::max<long long>(1, std::min<long long>(keyed_tiles, 1ll * dc.sm_count)));
   {
     RangeParams rp;
     rp.layers = d_layers; rp.n_layers = a.n_layers; rp.n_tiles = tiles; rp.state = d_state;
@@ -522,6 +564,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     kp.cell_total = reinterpret_cast<unsigned long long*>(ws + plan.off_nzero);
     kp.n_bins = bins_stride; kp.n_levels = plan.n_levels;
     kp.cell_cap = plan.cell_cap; kp.cell_stride = plan.value_cap; kp.d_levels = plan.d_levels;
+    kp.cta_begin = reinterpret_cast<const long long*>(ws + plan.off_cta);
     ADAPT_CUDA(cudaFuncSetAttribute(search_keyed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     static_cast<int>(plan.keyed_smem)));
     {

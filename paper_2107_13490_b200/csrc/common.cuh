@@ -89,6 +89,33 @@ __device__ __forceinline__ void smem_red_add(unsigned addr, unsigned v) {
   asm volatile("red.shared.add.u32 [%0], %1;" :: "r"(addr), "r"(v) : "memory");
 }
 
+// Adds the u32 words of a shared-memory array to a global array through the bulk-copy engine
+// (cp.reduce.async.bulk: the addition happens at the L2, no thread touches the words).  Both
+// addresses are 16-byte aligned and n_bytes is a multiple of 16.  Called by one thread, after a
+// barrier behind the last ordinary write to the array; the caller commits the group and waits for
+// it (bulk_reduce_wait_read) before the array is written again.
+__device__ __forceinline__ void bulk_reduce_add_u32(unsigned* dst, unsigned smem_src, unsigned n_bytes) {
+  const unsigned long long gdst = static_cast<unsigned long long>(__cvta_generic_to_global(dst));
+  constexpr unsigned kPiece = 32768u;
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  for (unsigned at = 0; at < n_bytes; at += kPiece) {
+    const unsigned len = min(kPiece, n_bytes - at);
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.u32 [%0], [%1], %2;"
+                 :: "l"(gdst + at), "r"(smem_src + at), "r"(len) : "memory");
+  }
+}
+__device__ __forceinline__ void bulk_reduce_commit() {
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// The engine has read the shared-memory sources of every committed group (they may be reused).
+__device__ __forceinline__ void bulk_reduce_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// Every committed group is complete.
+__device__ __forceinline__ void bulk_reduce_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 // Monotone map float -> uint32 (a < b  <=>  key(a) < key(b) for non-NaN a, b).
 __device__ __forceinline__ unsigned float_key(float v) {
   unsigned b = __float_as_uint(v);

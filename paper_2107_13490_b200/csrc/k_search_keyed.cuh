@@ -76,6 +76,8 @@ struct KeyedParams {
   int cell_stride;             // row length of the global cell arrays: the largest table any
                                // layer may use, keyed_value_cap() of a value-keyed one
   int d_levels;                // fine levels of the main segment whose corrections stay in shared memory
+  const long long* cta_begin;  // [gridDim.x + 1] first tile of every CTA (a CTA's tiles are contiguous);
+                               // NULL: equal shares
 };
 
 __host__ __device__ inline size_t keyed_smem_bytes(int cell_cap, int n_bins, int d_levels) {
@@ -518,8 +520,8 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
   const int value_cap = keyed_value_cap(p.cell_cap, p.n_bins, p.d_levels);
 
   const long long per = (p.n_tiles + gridDim.x - 1) / gridDim.x;
-  long long t = per * blockIdx.x;
-  const long long t_end = min(p.n_tiles, t + per);
+  long long t = p.cta_begin ? p.cta_begin[blockIdx.x] : per * blockIdx.x;
+  const long long t_end = p.cta_begin ? min(p.n_tiles, p.cta_begin[blockIdx.x + 1]) : min(p.n_tiles, t + per);
   if (t >= t_end) return;
   int li = layer_of_tile(p.layers, p.n_layers, t);
 
@@ -646,10 +648,38 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
     if (ok) {
       unsigned* gc = p.cell_count + static_cast<size_t>(l) * p.cell_stride;
       unsigned long long counted = 0;
-      for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) {
-        const unsigned n = cells[i] & kCellCountMask;
-        if (n) atomicAdd(&gc[i], n);
-        counted += n;
+      // Cell counts (and the main segment's sub-cell counts below) go through the bulk-copy
+      // engine as whole arrays: the marks are taken out of the words first.  Tables of the
+      // magic-constant and value-keyed forms are zero-filled in whole quads, so the last quad's
+      // spare words add nothing.  (The general form's table is flushed word by word.)
+      const bool bulk = fast || by_value;
+      // (the sub-cell table follows arrays of n_bins words: 16-byte aligned only for some n_bins)
+      const bool bulk_sub = bulk && (smem_addr(sub_s) & 15u) == 0u;
+      if (bulk) {
+        uint4* cells4 = reinterpret_cast<uint4*>(cells);
+        const int n4 = (total_cells + 3) >> 2;
+        for (int i = threadIdx.x; i < n4; i += kKeyedThreads) {
+          uint4 w = cells4[i];
+          w.x &= kCellCountMask; w.y &= kCellCountMask; w.z &= kCellCountMask; w.w &= kCellCountMask;
+          cells4[i] = w;
+          counted += static_cast<unsigned long long>(w.x) + w.y + w.z + w.w;
+        }
+      } else {
+        for (int i = threadIdx.x; i < total_cells; i += kKeyedThreads) {
+          const unsigned n = cells[i] & kCellCountMask;
+          if (n) atomicAdd(&gc[i], n);
+          counted += n;
+        }
+      }
+      __syncthreads();
+      if (threadIdx.x == 0 && bulk) {
+        bulk_reduce_add_u32(gc, smem_addr(cells), 16u * static_cast<unsigned>((total_cells + 3) >> 2));
+        if (c.sub_base >= 0 && !by_value && bulk_sub) {
+          const int room = (p.n_bins - c.sub_base) * kSubCells;
+          bulk_reduce_add_u32(c.sub + static_cast<size_t>(c.sub_base) * kSubCells, smem_addr(sub_s),
+                              4u * static_cast<unsigned>(min(kSubSharedIds * kSubCells, room)));
+        }
+        bulk_reduce_commit();
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) counted += __shfl_xor_sync(0xffffffffu, counted, o);
@@ -660,7 +690,7 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
         const unsigned n = qe[i];
         if (n) atomicAdd(&gq[i], n);
       }
-      if (c.sub_base >= 0 && !by_value) {
+      if (c.sub_base >= 0 && !by_value && !bulk_sub) {
         unsigned* gs = c.sub + static_cast<size_t>(c.sub_base) * kSubCells;     // segment 0, id sub_base
         const int room = (p.n_bins - c.sub_base) * kSubCells;
         for (int i = threadIdx.x; i < min(kSubSharedIds * kSubCells, room); i += kKeyedThreads) {
@@ -682,11 +712,14 @@ __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const Ke
         if (n) atomicAdd(&p.zero_class[static_cast<size_t>(l) * kZeroClasses + threadIdx.x],
                          static_cast<unsigned long long>(n));
       }
+      // the engine must have read the tables before the next layer's set-up writes them
+      if (threadIdx.x == 0 && bulk) bulk_reduce_wait_read();
     }
     __syncthreads();
     ++li;
     while (li < p.n_layers && p.layers[li + 1].tile_begin <= t) ++li;
   }
+  if (threadIdx.x == 0) bulk_reduce_wait_all();
 }
 
 }  // namespace adapt
