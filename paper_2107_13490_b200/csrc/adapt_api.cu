@@ -168,7 +168,10 @@ constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direc
 constexpr int kMaxKeyedGrid = 1023;             // CTAs of the keyed kernel (one per SM) whose tile ranges fit the descriptor block
 // What it costs a CTA of the keyed kernel to take up one more layer (context, table set-up, flush),
 // in tiles' worth of counting: the tile ranges of the CTAs are balanced with it.
-constexpr double kLayerCostTiles = 4.0;
+#ifndef ADAPT_LAYER_COST_TILES
+#define ADAPT_LAYER_COST_TILES 6.0
+#endif
+constexpr double kLayerCostTiles = ADAPT_LAYER_COST_TILES;
 // Stochastic rounding: the keyed route saves about 10 us per 2^20 elements over the direct kernel and
 // costs three more launches, so it takes layers of 2^20 elements up, and only 2^22 of them together.
 constexpr long long kSrKeyedMinElements = 1ll << 20;
