@@ -165,6 +165,9 @@ constexpr int kMaxBins = 16384;
 #define ADAPT_D_LEVELS_MAX 6   // fine levels of the main segment whose corrections stay in shared memory
 #endif
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
+#ifndef ADAPT_EXPAND_FILL
+#define ADAPT_EXPAND_FILL 3    // CTAs of the expand kernel per SM, over all layers, slices and roles
+#endif
 constexpr int kMaxKeyedGrid = 1023;             // CTAs of the keyed kernel (one per SM) whose tile ranges fit the descriptor block
 // What it costs a CTA of the keyed kernel to take up one more layer (context, table set-up, flush),
 // in tiles' worth of counting: the tile ranges of the CTAs are balanced with it.
@@ -588,7 +591,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       // a slice's cells (1.5 words each) and the fine histogram inside one CTA's shared memory
       const size_t room = static_cast<size_t>(dc.max_smem_optin) - 2048 - sizeof(unsigned) * bins_stride;
       const int cap_max = static_cast<int>(std::min<size_t>(room / 6, 1u << 20)) & ~3;
-      int slices = std::max(1, std::min(32, (3 * dc.sm_count + nk * kExpandRoles - 1) / (nk * kExpandRoles)));
+      int slices = std::max(1, std::min(32, (ADAPT_EXPAND_FILL * dc.sm_count + nk * kExpandRoles - 1) / (nk * kExpandRoles)));
       slices = std::max(slices, (plan.value_cap + cap_max - 1) / std::max(cap_max, 4));
       ep.slices = slices;
       ep.slice_cap = ((plan.value_cap + slices - 1) / slices + 3) & ~3;
