@@ -121,6 +121,29 @@ def test_thousands_of_small_layers_share_ctas(B):
                           algorithms=(0, 2))
 
 
+def test_hundreds_of_keyed_layers_of_uneven_size(B):
+    """More keyed layers than the counting kernel has CTAs, sizes from just above the keyed
+    threshold to a few hundred thousand elements, several value classes: the CTAs' tile ranges
+    (balanced by cost, several layers per CTA, large layers cut over many CTAs) must cover every
+    tile once, and the slices and roles of the expand kernel must add up."""
+    rng = np.random.default_rng(909)
+    xs = []
+    for l in range(220):
+        n = int(rng.choice([32768, 33001, 40000, 65537, 131072, 300000], p=[.3, .3, .2, .1, .07, .03]))
+        kind = l % 4
+        if kind == 0:
+            x = rng.standard_normal(n) * 2.0 ** rng.integers(-8, 3)
+        elif kind == 1:
+            x = np.maximum(rng.standard_normal(n), 0) * 0.7
+        elif kind == 2:
+            x = rng.laplace(0, 0.02, n) * np.where(rng.random(n) < 0.01, 50.0, 1.0)
+        else:
+            x = rng.integers(-100, 100, n) * 2.0 ** -5          # on a grid: keyed by value
+        xs.append(x.astype(np.float32))
+    wl, fl = W.candidate_grid([5, 11, 18])
+    G.run_and_compare(B, xs, wl, fl, 96, where="220 keyed layers", algorithms=(0,))
+
+
 def test_options_eps_pseudocount_base_and_grid_order(B):
     rng = np.random.default_rng(3)
     xs = [(rng.laplace(0, 0.02, 20000)).astype(np.float32),
