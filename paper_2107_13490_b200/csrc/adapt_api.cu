@@ -517,6 +517,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   }
 
   // K2, keyed form: plan -> cell counting -> expansion
+  const long long elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
   if (!keyed.empty() && keyed_tiles > 0) {
     const int nk = static_cast<int>(keyed.size());
     {
@@ -528,7 +529,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       pp.stochastic = stochastic ? 1 : 0;
       pp.cell_cap = stochastic ? plan.sr_cap - 128 : plan.cell_cap;
       pp.fine_ratio = ADAPT_FINE_RATIO;
-      pp.elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
+      pp.elems_per_cta = elems_per_cta;
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
       const int plan_slices = std::max(1, std::min(8, (bins_stride + kPlanThreads - 1) / kPlanThreads));
       plan_kernel<<<dim3(nk, plan_slices), kPlanThreads, 0, stream>>>(pp);
@@ -592,15 +593,24 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       const size_t room = static_cast<size_t>(dc.max_smem_optin) - 2048 - sizeof(unsigned) * bins_stride;
       const int cap_max = static_cast<int>(std::min<size_t>(room / 6, 1u << 20)) & ~3;
       int slices = std::max(1, std::min(32, (ADAPT_EXPAND_FILL * dc.sm_count + nk * kExpandRoles - 1) / (nk * kExpandRoles)));
-      slices = std::max(slices, (plan.value_cap + cap_max - 1) / std::max(cap_max, 4));
+      slices = std::max(slices, (plan.cell_cap + cap_max - 1) / std::max(cap_max, 4));
       ep.slices = slices;
-      ep.slice_cap = ((plan.value_cap + slices - 1) / slices + 3) & ~3;
+      // the largest table a layer of the pyramid form can have: the cap its plan works with
+      // (make_layer_plan: cells ~ sqrt(balance * bins * elements one CTA sees), at most cell_cap)
+      long long cells_bound = 2048;
+      for (int l : keyed) {
+        const int bins_l = o.n_bins_per_layer ? o.n_bins_per_layer[l] : a.n_bins;
+        const double seen = static_cast<double>(std::min<long long>(a.lens[l], elems_per_cta));
+        const long long want = static_cast<long long>(std::sqrt(ADAPT_CELL_BALANCE * static_cast<double>(bins_l) * seen)) + 16;
+        cells_bound = std::max(cells_bound, std::min<long long>(plan.cell_cap, std::max<long long>(2048, want)));
+      }
+      ep.slice_cap = (static_cast<int>((cells_bound + slices - 1) / slices) + 3) & ~3;
       const size_t smem = sizeof(unsigned) * (static_cast<size_t>(bins_stride) + ep.slice_cap + ep.slice_cap / 2 + 2);
       if (smem + 1024 > static_cast<size_t>(dc.max_smem_optin)) return ADAPT_ERR_INVALID_ARG;
       ADAPT_CUDA(cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(smem)));
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      expand_kernel<<<dim3(std::max(slices * kExpandRoles, plan.n_levels + 1), nk), kExpandThreads, smem, stream>>>(ep);
+      expand_kernel<<<dim3(slices * kExpandRoles, nk), kExpandThreads, smem, stream>>>(ep);
       ADAPT_CUDA(cudaGetLastError());
     }
     }

@@ -54,14 +54,15 @@ struct ExpandParams {
   int slice_cap;               // ... and the cells one of them may hold (a multiple of 4)
 };
 
-// Level form: this CTA serves level f (n_levels: the float histogram) of the layer.
+// Level form: this CTA serves slice `slice` of n_slices of the cells at level f (n_levels: the
+// float histogram) of the layer.
 __device__ __forceinline__ void expand_by_level(const ExpandParams& p, const LayerDesc& L, const LayerPlan& P,
-                                                const LayerState& S, int f, unsigned* s_hist) {
+                                                const LayerState& S, int f, int slice, int n_slices,
+                                                unsigned* s_hist) {
   __shared__ unsigned long long s_zero;
   const int l = L.index;
   const int B = p.n_bins;
   const bool is_q = (f == p.n_levels);
-  const int slice = 0, n_slices = 1;
   // From level f_same on, what the cells and sub-cells add is the same at every level and in the
   // float histogram (interior cells and interior sub-cells, each into its own bin): the float
   // histogram's CTAs compute it once and add it to all of those levels, whose own CTAs only add
@@ -80,7 +81,7 @@ __device__ __forceinline__ void expand_by_level(const ExpandParams& p, const Lay
 
   const unsigned* count = p.cell_count + static_cast<size_t>(l) * p.cell_stride;
   unsigned long long zero = 0;
-  // the cells are shared by the gridDim.z CTAs of this (level, layer), a contiguous slice each
+  // the cells are shared by the n_slices CTAs of this (level, layer), a contiguous slice each
   const int per_slice = ((P.total_cells + n_slices - 1) / n_slices + 3) & ~3;
   const int i_end = min(P.total_cells, (slice + 1) * per_slice);
   // four cells per thread and trip, counts and marks fetched as 128-bit words (slices start on
@@ -194,6 +195,7 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
 
   // the layer's table is cut into equal slices (multiples of four cells)
   const int per_slice = ((P.total_cells + p.slices - 1) / p.slices + 3) & ~3;
+  if (per_slice > p.slice_cap) return;   // cannot happen: the host sized the buffers from the plan's own cap
   const int t_lo = min(P.total_cells, slice * per_slice);
   const int t_hi = min(P.total_cells, t_lo + per_slice);
 
@@ -242,11 +244,23 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
       const int my_lo = id_lo + slice * per_ids, my_hi = min(id_hi, my_lo + per_ids);
       const unsigned* sub = p.sub_count + (static_cast<size_t>(l) * 2 + s) * B * kSubCells;
       const int gs = g + kSubBits;
-      for (int id = my_lo + warp; id < my_hi; id += kWarps) {
-        unsigned m = __ldg(sub + static_cast<size_t>(id) * kSubCells + lane);
+      // (the counts and edges of four of the warp's cells are fetched together: the loads are
+      // what a warp would otherwise wait for, cell after cell)
+      constexpr int kAhead = 4;
+      for (int id0 = my_lo + warp; id0 < my_hi; id0 += kWarps * kAhead) {
+        unsigned m_in[kAhead];
+        float e_in[kAhead];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+          const int idu = id0 + u * kWarps;
+          m_in[u] = idu < my_hi ? __ldg(sub + static_cast<size_t>(idu) * kSubCells + lane) : 0u;
+          e_in[u] = (idu < my_hi && ADAPT_IN_BOUNDS(idu + 1, B + 1, 35)) ? __ldg(E + idu + 1) : 0.0f;
+        }
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+        const unsigned m = m_in[u];
         if (__ballot_sync(0xffffffffu, m != 0u) == 0u) continue;
-        if (!ADAPT_IN_BOUNDS(id + 1, B + 1, 35)) continue;
-        const int cc = static_cast<int>(ceil(scale_pow2(static_cast<double>(E[id + 1]), g))) - 1;
+        const int cc = static_cast<int>(ceil(scale_pow2(static_cast<double>(e_in[u]), g))) - 1;
         const int jj = cc * kSubCells + lane;           // sub-cell index, below 2^27 in magnitude
         // interior sub-cells serve the levels from fe on and the float histogram.  The two ends
         // of the sub-cell, rounded outwards: the cell's left end and the offsets are exact floats
@@ -286,6 +300,7 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
             if (ADAPT_IN_BOUNDS(bv, B, 34)) atomicAdd(&U[static_cast<size_t>(f) * B + bv], mm);
           }
         }
+        }
       }
     }
     if (part == kRoleSub) {
@@ -316,26 +331,31 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
     int cur_first = c_first, cur_n = n;
     int f = g - 1;
     auto level = [&](int tid, int stride) {
-      if (f < F) {
-        const float w = pow2f(-f);
-        for (int j = tid; j < cur_n; j += stride) {
-          const unsigned m = cur[j];
-          if (m == 0u) continue;
-          const int r = (cur_first + j + 1) >> 1;
-          const float v = __fmul_rn(__int2float_rn(r), w);
-          const int bv = bin_of(v, S.lo, S.scale, S.bmax);
-          if (ADAPT_IN_BOUNDS(bv, B, 32)) atomicAdd(&U[static_cast<size_t>(f) * B + bv], m);
-          if (r == 0) atomicAdd(&Z[f], static_cast<unsigned long long>(m));
-        }
-      }
+      // one pass: entries 2q and 2q + 1 (by absolute index) of the level above are binned at
+      // level f and summed into entry q of the next level
+      const bool wanted = f < F;
+      const float w = pow2f(-f);
       const int nxt_first = cur_first >> 1;
       const int nxt_n = ((cur_first + cur_n - 1) >> 1) - nxt_first + 1;
       for (int j = tid; j < nxt_n; j += stride) {
-        const int i0 = 2 * (nxt_first + j) - cur_first;       // entries i0 and i0 + 1 of the level above
-        unsigned m = 0;
-        if (i0 >= 0 && i0 < cur_n) m += cur[i0];
-        if (i0 + 1 >= 0 && i0 + 1 < cur_n) m += cur[i0 + 1];
-        if (ADAPT_IN_BOUNDS(j, p.slice_cap / 2 + 2, 37)) nxt[j] = m;
+        const int i0 = 2 * (nxt_first + j) - cur_first;
+        unsigned sum = 0;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int i = i0 + e;
+          if (i < 0 || i >= cur_n) continue;
+          const unsigned m = cur[i];
+          if (m == 0u) continue;
+          sum += m;
+          if (wanted) {
+            const int r = (cur_first + i + 1) >> 1;
+            const float v = __fmul_rn(__int2float_rn(r), w);
+            const int bv = bin_of(v, S.lo, S.scale, S.bmax);
+            if (ADAPT_IN_BOUNDS(bv, B, 32)) atomicAdd(&U[static_cast<size_t>(f) * B + bv], m);
+            if (r == 0) atomicAdd(&Z[f], static_cast<unsigned long long>(m));
+          }
+        }
+        if (ADAPT_IN_BOUNDS(j, p.slice_cap / 2 + 2, 37)) nxt[j] = sum;
       }
       unsigned* sw = cur; cur = nxt; nxt = sw;
       cur_first = nxt_first; cur_n = nxt_n;
@@ -374,7 +394,7 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
 }
 
 // blockIdx.y: the layer.  Pyramid form: blockIdx.x = slice and role (the first 6 p.slices CTAs work);
-// level form: blockIdx.x = level (the first n_levels + 1 CTAs work).
+// level form: the levels (and the float histogram) are dealt to the gridDim.x CTAs of the layer.
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandParams p) {
   extern __shared__ unsigned s_expand[];
   const LayerDesc L = p.layers[blockIdx.y];
@@ -385,7 +405,17 @@ __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandPara
     if (static_cast<int>(blockIdx.x) < p.slices * kExpandRoles)
       expand_pyramid(p, L, P, S, blockIdx.x / kExpandRoles, blockIdx.x % kExpandRoles, s_expand);
   } else {
-    if (static_cast<int>(blockIdx.x) <= p.n_levels) expand_by_level(p, L, P, S, blockIdx.x, s_expand);
+    // enough CTAs: each level's cells are cut into slices; too few: a CTA takes several levels
+    const int per_level = static_cast<int>(gridDim.x) / (p.n_levels + 1);
+    if (per_level >= 1) {
+      const int slice = blockIdx.x / (p.n_levels + 1);
+      if (slice < per_level) expand_by_level(p, L, P, S, blockIdx.x % (p.n_levels + 1), slice, per_level, s_expand);
+    } else {
+      for (int f = blockIdx.x; f <= p.n_levels; f += gridDim.x) {
+        expand_by_level(p, L, P, S, f, 0, 1, s_expand);
+        __syncthreads();
+      }
+    }
   }
 }
 
