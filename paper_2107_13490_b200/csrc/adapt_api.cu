@@ -672,7 +672,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
     // enough CTAs to fill the GPU when there are few (FL, layer) pairs
-    const int slices = std::max(1, std::min(8, (2 * dc.sm_count) / std::max(1, plan.n_levels * a.n_layers)));
+    const int slices = std::max(1, std::min(16, (4 * dc.sm_count) / std::max(1, plan.n_levels * a.n_layers)));
     kld_kernel<<<dim3(plan.n_levels, a.n_layers, slices), kKldThreads, 0, stream>>>(kp);
     ADAPT_CUDA(cudaGetLastError());
   }

@@ -23,7 +23,13 @@
 
 namespace adapt {
 
-constexpr int kKldThreads = 256;
+#ifndef ADAPT_KLD_THREADS
+#define ADAPT_KLD_THREADS 256
+#endif
+#ifndef ADAPT_KLD_WARP_BINS
+#define ADAPT_KLD_WARP_BINS 128
+#endif
+constexpr int kKldThreads = ADAPT_KLD_THREADS;
 
 struct KldParams {
   const LayerDesc* layers;
@@ -63,6 +69,7 @@ __device__ __forceinline__ double block_sum(double v, double* s_buf) {
 
 // One term of the divergence sum and whether it is infinite (a filled P bin over an empty Q bin).
 __device__ __forceinline__ double kld_term(long long pc, long long qc, double alpha, bool* inf) {
+  if (pc == qc) return 0.0;      // log1p(0) = 0 exactly: the term vanishes whatever the pseudo-count
   const double pa = static_cast<double>(pc) + alpha;
   const double qa = static_cast<double>(qc) + alpha;
   if (!(pa > 0.0)) return 0.0;
@@ -85,11 +92,14 @@ __device__ __forceinline__ unsigned long long warp_sum(unsigned long long v) {
 // saturate; those whose two saturation values fall in the first and the last bin have exactly
 // the unsaturated histogram U[FL], so their divergence is computed once.  The others fold the
 // two tails of U[FL] into the bins of their saturation values and are summed one by one.
-__device__ void select_layer(const KldParams& p, int l, int lane);
+struct SelectScratch;
+__device__ void select_layer(const KldParams& p, int l, SelectScratch* sh);
 
 __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
   __shared__ double s_buf[kKldThreads / 32];
-  __shared__ int s_inf, s_last;
+  __shared__ int s_inf, s_last, s_nfold;
+  __shared__ int s_fold[kKldThreads];       // positions (in FL order) of the candidates that fold
+  __shared__ double s_select[(kKldThreads / 32) * 2 + 2];   // a SelectScratch
   const int f = blockIdx.x, l = blockIdx.y;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int c_begin = p.fl_begin[f], c_end = p.fl_begin[f + 1];
@@ -127,16 +137,43 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
     else if (s_inf) unsat = inf_value;
     else { unsat = sum * p.inv_ln_base / n_eff; if (!(unsat > 0.0)) unsat = 0.0; }
 
-    // A candidate whose saturation values fall inside the range folds the tails of U[FL] and is
-    // summed by itself: by one warp when the histogram is short (the FL's candidates are then
-    // dealt to the warps of the gridDim.z CTAs that share this (FL, layer)), by the whole CTA
-    // when it is long (candidates dealt to the CTAs).
+    // The candidates of this FL are dealt to the gridDim.z CTAs that share this (FL, layer).  A
+    // candidate whose two saturation values fall in the first and the last bin has the
+    // unsaturated histogram itself: those are settled one per thread.  The others fold the tails
+    // of U[FL] into the bins of their saturation values and are summed one by one: by the whole
+    // CTA (by one warp each when the histogram is short), in rounds of kKldThreads candidates.
     constexpr int kWarps = kKldThreads / 32;
-    const bool by_warp = B <= 512;
-    const int first = by_warp ? blockIdx.z * kWarps + warp : blockIdx.z;
-    const int step = by_warp ? kWarps * gridDim.z : gridDim.z;
+    const bool by_warp = B <= ADAPT_KLD_WARP_BINS;
     const int me = by_warp ? lane : threadIdx.x, team = by_warp ? 32 : kKldThreads;
-    for (int i = c_begin + first; i < c_end; i += step) {
+    const int n_mine = (c_end - c_begin - static_cast<int>(blockIdx.z) + static_cast<int>(gridDim.z) - 1) /
+                       static_cast<int>(gridDim.z);          // candidates c_begin + z, + gridDim.z, ...
+    for (int round0 = 0; round0 < n_mine; round0 += kKldThreads) {
+      if (threadIdx.x == 0) s_nfold = 0;
+      __syncthreads();
+      {
+        const int kk = round0 + threadIdx.x;
+        if (kk < n_mine) {
+          const int i = c_begin + blockIdx.z + kk * gridDim.z;
+          const int c = p.cand_by_fl[i];
+          const int wl = p.cand_wl[c];
+          const int hi_code = static_cast<int>((1ll << (wl - 1)) - 1);
+          const int lo_code = static_cast<int>(-(1ll << (wl - 1)));
+          const int bh = bin_of(dequantize(hi_code, f), S.lo, S.scale, S.bmax);
+          const int bl = bin_of(dequantize(lo_code, f), S.lo, S.scale, S.bmax);
+          if (bl == 0 && bh == B - 1 && B > 1 && !p.hist_out) {
+            // nothing folds: the candidate's histogram is U[FL] itself
+            const size_t out = static_cast<size_t>(l) * p.n_cand + c;
+            p.kld_out[out] = unsat;
+            p.zeros_out[out] = zero_count;
+          } else {
+            s_fold[atomicAdd(&s_nfold, 1)] = i;
+          }
+        }
+      }
+      __syncthreads();
+      const int n_fold = s_nfold;
+      for (int j = by_warp ? warp : 0; j < n_fold; j += by_warp ? kWarps : 1) {
+      const int i = s_fold[j];
       const int c = p.cand_by_fl[i];
       const int wl = p.cand_wl[c];
       const size_t out = static_cast<size_t>(l) * p.n_cand + c;
@@ -150,9 +187,7 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
       unsigned* H0 = (p.hist_out && c == 0)
                          ? p.hist_out + static_cast<size_t>(l) * (p.n_cand + 1) * stride : nullptr;
       double k;
-      if (bl == 0 && bh == B - 1 && B > 1 && !H) {
-        k = unsat;                     // nothing folds: the candidate's histogram is U[FL] itself
-      } else {
+      {
         // tail masses that fold into bl and bh (exact: sums of counts)
         unsigned long long lo_mass = 0, hi_mass = 0;
         for (int b = me; b < B; b += team) {
@@ -201,6 +236,8 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
         p.kld_out[out] = k;
         p.zeros_out[out] = zero_count;
       }
+      }
+      __syncthreads();                 // the list is rewritten by the next round
     }
   }
 
@@ -212,9 +249,9 @@ __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
     s_last = (done == gridDim.x * gridDim.z - 1u) ? 1 : 0;
   }
   __syncthreads();
-  if (s_last && warp == 0) {
+  if (s_last) {
     __threadfence();
-    select_layer(p, l, lane);
+    select_layer(p, l, reinterpret_cast<SelectScratch*>(s_select));
   }
 }
 
@@ -223,18 +260,66 @@ __device__ __forceinline__ void arg_min_merge(double& k, int& pos, double k2, in
   if (pos2 >= 0 && (pos < 0 || k2 < k || (k2 == k && pos2 < pos))) { k = k2; pos = pos2; }
 }
 
-// One warp: the layer's choice from its divergences (written by other CTAs of this launch:
-// read past the L1 cache).
-__device__ void select_layer(const KldParams& p, int l, int lane) {
+// The whole CTA: the layer's choice from its divergences (written by other CTAs of this
+// launch: read past the L1 cache).  Every thread looks at the candidates tid, tid + 256, ...;
+// warps reduce by shuffles, the CTA through a few words of shared memory.
+struct SelectScratch {
+  int first[kKldThreads / 32];
+  int pos[kKldThreads / 32];
+  double key[kKldThreads / 32];
+  int spos, last_bad;
+};
+
+__device__ void select_layer(const KldParams& p, int l, SelectScratch* sh) {
+  constexpr int kWarps = kKldThreads / 32;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const LayerState S = p.state[l];
-  if (p.status_out && lane == 0)       // 2 / 3: the interface's codes for NaN/Inf and |x| >= 2^64
+  if (p.status_out && tid == 0)        // 2 / 3: the interface's codes for NaN/Inf and |x| >= 2^64
     p.status_out[l] = (S.flags & kFlagNonfinite) ? 2 : ((S.flags & kFlagRange) ? 3 : 0);
   const double* kld = p.kld_out + static_cast<size_t>(l) * p.n_cand;
+
+  if (p.start) {
+    // PushDown as a descent (Algorithm 3): from the layer's current format walk down the
+    // (WL, FL) order while the divergence stays <= eps; stop before the first violation
+    const int swl = p.start[2 * l], sfl = p.start[2 * l + 1];
+    if (tid == 0) { sh->spos = 0x7fffffff; sh->last_bad = -1; }
+    __syncthreads();
+    int spos = 0x7fffffff;     // position of the start format in candidate order
+    for (int pos = tid; pos < p.n_cand; pos += kKldThreads) {
+      const int c = p.cand_order[pos];
+      if (p.cand_wl[c] == swl && p.cand_fl[c] == sfl) spos = min(spos, pos);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) spos = min(spos, __shfl_xor_sync(0xffffffffu, spos, o));
+    if (lane == 0 && spos != 0x7fffffff) atomicMin(&sh->spos, spos);
+    __syncthreads();
+    spos = sh->spos;
+    int last_bad = -1;         // highest position below the start whose divergence exceeds eps
+    if (spos != 0x7fffffff)
+      for (int pos = tid; pos < spos; pos += kKldThreads)
+        if (!(__ldcg(kld + p.cand_order[pos]) <= p.eps)) last_bad = max(last_bad, pos);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) last_bad = max(last_bad, __shfl_xor_sync(0xffffffffu, last_bad, o));
+    if (lane == 0 && last_bad >= 0) atomicMax(&sh->last_bad, last_bad);
+    __syncthreads();
+    if (tid == 0) {
+      last_bad = sh->last_bad;
+      unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
+      int* o = p.best_out + 4 * l;
+      if (spos == 0x7fffffff) { o[0] = swl; o[1] = sfl; o[2] = -1; o[3] = static_cast<int>(flags); return; }
+      const bool ok = __ldcg(kld + p.cand_order[spos]) <= p.eps;
+      const int pos = ok ? last_bad + 1 : spos;
+      const int c = p.cand_order[pos];
+      if (ok) flags |= 1u;
+      o[0] = p.cand_wl[c]; o[1] = p.cand_fl[c]; o[2] = c; o[3] = static_cast<int>(flags);
+    }
+    return;
+  }
 
   int first_ok = 0x7fffffff;  // position (in candidate order) of the first KLD <= eps
   double min_k = 0.0;
   int min_pos = -1;           // position of the least finite divergence
-  for (int pos = lane; pos < p.n_cand; pos += 32) {
+  for (int pos = tid; pos < p.n_cand; pos += kKldThreads) {
     const double k = __ldcg(kld + p.cand_order[pos]);
     if (k <= p.eps) first_ok = min(first_ok, pos);
     if (k < __longlong_as_double(0x7ff0000000000000ll)) arg_min_merge(min_k, min_pos, k, pos);
@@ -246,39 +331,13 @@ __device__ void select_layer(const KldParams& p, int l, int lane) {
     int pos2 = __shfl_xor_sync(0xffffffffu, min_pos, o);
     arg_min_merge(min_k, min_pos, k2, pos2);
   }
-  if (p.start) {
-    // PushDown as a descent (Algorithm 3): from the layer's current format walk down the
-    // (WL, FL) order while the divergence stays <= eps; stop before the first violation
-    const int swl = p.start[2 * l], sfl = p.start[2 * l + 1];
-    int spos = -1;
-    for (int pos = lane; pos < p.n_cand; pos += 32) {
-      const int c = p.cand_order[pos];
-      if (p.cand_wl[c] == swl && p.cand_fl[c] == sfl) spos = (spos < 0) ? pos : min(spos, pos);
+  if (lane == 0) { sh->first[warp] = first_ok; sh->pos[warp] = min_pos; sh->key[warp] = min_k; }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kWarps; ++w) {
+      first_ok = min(first_ok, sh->first[w]);
+      arg_min_merge(min_k, min_pos, sh->key[w], sh->pos[w]);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const int other = __shfl_xor_sync(0xffffffffu, spos, o);
-      spos = (spos < 0) ? other : (other < 0 ? spos : min(spos, other));
-    }
-    int last_bad = -1;   // highest position below the start whose divergence exceeds eps
-    if (spos >= 0)
-      for (int pos = lane; pos < spos; pos += 32)
-        if (!(__ldcg(kld + p.cand_order[pos]) <= p.eps)) last_bad = max(last_bad, pos);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) last_bad = max(last_bad, __shfl_xor_sync(0xffffffffu, last_bad, o));
-    if (lane == 0) {
-      unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
-      int* o = p.best_out + 4 * l;
-      if (spos < 0) { o[0] = swl; o[1] = sfl; o[2] = -1; o[3] = static_cast<int>(flags); return; }
-      const bool ok = __ldcg(kld + p.cand_order[spos]) <= p.eps;
-      const int pos = ok ? last_bad + 1 : spos;
-      const int c = p.cand_order[pos];
-      if (ok) flags |= 1u;
-      o[0] = p.cand_wl[c]; o[1] = p.cand_fl[c]; o[2] = c; o[3] = static_cast<int>(flags);
-    }
-    return;
-  }
-  if (lane == 0) {
     unsigned flags = S.flags & (kFlagDegenerate | kFlagNonfinite | kFlagRange);
     int pos;
     if (first_ok != 0x7fffffff) { pos = first_ok; flags |= 1u; }
