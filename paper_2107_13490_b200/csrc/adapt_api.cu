@@ -113,6 +113,8 @@ struct DeviceCache {
   cudaStream_t copy_stream = nullptr;   // host-form calls: downloads that overlap the kernels
   cudaEvent_t slice_done[2] = {nullptr, nullptr};
   cudaEvent_t copies_done = nullptr;
+  cudaStream_t side_stream = nullptr;   // search: the direct kernel runs beside the keyed kernels
+  cudaEvent_t side_fork = nullptr, side_join = nullptr;
 };
 
 DeviceCache g_cache[kMaxDevices];
@@ -516,6 +518,22 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     ADAPT_CUDA(cudaGetLastError());
   }
 
+  // Layers of both forms in one call (round-to-nearest-even): the direct kernel needs only the
+  // ranges, so it runs on a stream of the library's own beside plan -> counting -> expansion and
+  // joins before the divergences.  (Under stochastic rounding it reads the plans: no overlap.)
+  const bool beside = !stochastic && !keyed.empty() && keyed_tiles > 0 && !direct.empty() && direct_tiles > 0;
+  cudaStream_t direct_stream = stream;
+  if (beside) {
+    if (!dc.side_stream) {
+      ADAPT_CUDA(cudaStreamCreateWithFlags(&dc.side_stream, cudaStreamNonBlocking));
+      ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_fork, cudaEventDisableTiming));
+      ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_join, cudaEventDisableTiming));
+    }
+    ADAPT_CUDA(cudaEventRecord(dc.side_fork, stream));
+    ADAPT_CUDA(cudaStreamWaitEvent(dc.side_stream, dc.side_fork, 0));
+    direct_stream = dc.side_stream;
+  }
+
   // K2, keyed form: plan -> cell counting -> expansion
   const long long elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
   if (!keyed.empty() && keyed_tiles > 0) {
@@ -648,9 +666,15 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     const int ctas_per_sm = wide ? 1 : std::max<int>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
     dim3 grid(static_cast<unsigned>(std::min<long long>(direct_tiles, 1ll * ctas_per_sm * dc.sm_count)),
               groups);
-    LaunchScope ls(ADAPT_KERNEL_SEARCH_DIRECT, stream);
-    kern<<<grid, threads, smem, stream>>>(sp);
-    ADAPT_CUDA(cudaGetLastError());
+    {
+      LaunchScope ls(ADAPT_KERNEL_SEARCH_DIRECT, direct_stream);
+      kern<<<grid, threads, smem, direct_stream>>>(sp);
+      ADAPT_CUDA(cudaGetLastError());
+    }
+    if (beside) {
+      ADAPT_CUDA(cudaEventRecord(dc.side_join, dc.side_stream));
+      ADAPT_CUDA(cudaStreamWaitEvent(stream, dc.side_join, 0));
+    }
   }
 
   // K3: divergence per (layer, candidate); the last CTA of a layer selects its format
@@ -1768,6 +1792,11 @@ int adapt_release(void) {
   if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
   if (dc->div_buf) { ADAPT_CUDA(cudaFree(dc->div_buf)); dc->div_buf = nullptr; dc->div_buf_bytes = 0; }
   if (dc->stage_codes) { ADAPT_CUDA(cudaFree(dc->stage_codes)); dc->stage_codes = nullptr; dc->stage_codes_bytes = 0; }
+  if (dc->side_stream) {
+    ADAPT_CUDA(cudaStreamDestroy(dc->side_stream)); dc->side_stream = nullptr;
+    ADAPT_CUDA(cudaEventDestroy(dc->side_fork)); dc->side_fork = nullptr;
+    ADAPT_CUDA(cudaEventDestroy(dc->side_join)); dc->side_join = nullptr;
+  }
   if (dc->copy_stream) {
     ADAPT_CUDA(cudaStreamDestroy(dc->copy_stream)); dc->copy_stream = nullptr;
     for (cudaEvent_t& e : dc->slice_done) { ADAPT_CUDA(cudaEventDestroy(e)); e = nullptr; }
