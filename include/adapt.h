@@ -11,7 +11,11 @@
  *    read (or written) before the call returns.
  *  - Calls enqueue their kernels on a CUDA stream (the legacy default stream
  *    for the entry points without a stream argument) and return without
- *    waiting; outputs are valid once that stream has been synchronised.
+ *    waiting; outputs are valid once that stream has been synchronised.  A
+ *    search may run one of its kernels on a stream of the library's own; that
+ *    stream branches off the caller's stream and joins it again inside the
+ *    call (events), so to the caller the call still is work on one stream,
+ *    and it may be captured into a CUDA graph.
  *  - The return value is an adapt_status.  Errors that the host can see (null
  *    pointers, sizes or formats out of range, workspace too small) return
  *    before anything is launched and write nothing.  Errors in the data
