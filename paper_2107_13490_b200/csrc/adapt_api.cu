@@ -164,7 +164,8 @@ int acquire_slot(DeviceCache& c, size_t bytes, PinnedSlot** out) {
 
 constexpr int kMaxBins = 16384;
 #ifndef ADAPT_D_LEVELS_MAX
-#define ADAPT_D_LEVELS_MAX 6   // fine levels of the main segment whose corrections stay in shared memory
+#define ADAPT_D_LEVELS_MAX 0   // fine levels of the main segment whose corrections stay in shared memory
+                               // (none: the table is worth more as cells; the corrections are few)
 #endif
 constexpr long long kKeyedMinElements = 32768;  // smaller layers take the direct kernel
 #ifndef ADAPT_EXPAND_FILL
