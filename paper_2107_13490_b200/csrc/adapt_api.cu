@@ -298,6 +298,23 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
 
 }  // namespace
 
+// Launch of a kernel that follows another kernel of this library in the stream and begins with
+// grid_dependency_wait(): with programmatic stream serialization its CTAs may be scheduled while
+// the earlier kernel's last CTAs are still running, which hides the launch latency between the
+// dependent kernels of a search.  (Not while per-kernel events are recorded between them.)
+template <typename Params>
+cudaError_t launch_dependent(void (*kern)(Params), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                             const Params& params) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_timing.load() ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kern, params);
+}
+
 // ---- search driver ----------------------------------------------------------------
 
 namespace {
@@ -524,16 +541,6 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
   // joins before the divergences.  (Under stochastic rounding it reads the plans: no overlap.)
   const bool beside = !stochastic && !keyed.empty() && keyed_tiles > 0 && !direct.empty() && direct_tiles > 0;
   cudaStream_t direct_stream = stream;
-  if (beside) {
-    if (!dc.side_stream) {
-      ADAPT_CUDA(cudaStreamCreateWithFlags(&dc.side_stream, cudaStreamNonBlocking));
-      ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_fork, cudaEventDisableTiming));
-      ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_join, cudaEventDisableTiming));
-    }
-    ADAPT_CUDA(cudaEventRecord(dc.side_fork, stream));
-    ADAPT_CUDA(cudaStreamWaitEvent(dc.side_stream, dc.side_fork, 0));
-    direct_stream = dc.side_stream;
-  }
 
   // K2, keyed form: plan -> cell counting -> expansion
   const long long elems_per_cta = (keyed_tiles + keyed_grid - 1) / keyed_grid * kKeyedTile;
@@ -551,8 +558,18 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       pp.elems_per_cta = elems_per_cta;
       LaunchScope ls(ADAPT_KERNEL_PLAN, stream);
       const int plan_slices = std::max(1, std::min(8, (bins_stride + kPlanThreads - 1) / kPlanThreads));
-      plan_kernel<<<dim3(nk, plan_slices), kPlanThreads, 0, stream>>>(pp);
-      ADAPT_CUDA(cudaGetLastError());
+      ADAPT_CUDA(launch_dependent(plan_kernel, dim3(nk, plan_slices), dim3(kPlanThreads), 0, stream, pp));
+    }
+    // (the branch comes after the plan kernel so that nothing stands between the range scan and it)
+    if (beside) {
+      if (!dc.side_stream) {
+        ADAPT_CUDA(cudaStreamCreateWithFlags(&dc.side_stream, cudaStreamNonBlocking));
+        ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_fork, cudaEventDisableTiming));
+        ADAPT_CUDA(cudaEventCreateWithFlags(&dc.side_join, cudaEventDisableTiming));
+      }
+      ADAPT_CUDA(cudaEventRecord(dc.side_fork, stream));
+      ADAPT_CUDA(cudaStreamWaitEvent(dc.side_stream, dc.side_fork, 0));
+      direct_stream = dc.side_stream;
     }
     if (stochastic) {
       SrParams sp;
@@ -567,8 +584,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
                                       static_cast<int>(plan.sr_smem)));
       {
         LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
-        search_sr_kernel<<<keyed_grid, kSrThreads, plan.sr_smem, stream>>>(sp);
-        ADAPT_CUDA(cudaGetLastError());
+        ADAPT_CUDA(launch_dependent(search_sr_kernel, dim3(keyed_grid), dim3(kSrThreads), plan.sr_smem, stream, sp));
       }
       SrExpandParams ep;
       ep.layers = d_keyed; ep.state = d_state; ep.plan = d_plan; ep.cell_count = d_cells;
@@ -577,9 +593,8 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       ep.n_bins = bins_stride; ep.n_levels = plan.n_levels; ep.cell_stride = plan.value_cap;
       {
         LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-        expand_sr_kernel<<<dim3(plan.n_levels + 1, nk), kSrExpandThreads,
-                           sizeof(unsigned) * bins_stride, stream>>>(ep);
-        ADAPT_CUDA(cudaGetLastError());
+        ADAPT_CUDA(launch_dependent(expand_sr_kernel, dim3(plan.n_levels + 1, nk), dim3(kSrExpandThreads),
+                                    sizeof(unsigned) * bins_stride, stream, ep));
       }
     } else {
     KeyedParams kp;
@@ -596,8 +611,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     {
       const int grid = keyed_grid;
       LaunchScope ls(ADAPT_KERNEL_SEARCH, stream);
-      search_keyed_kernel<<<grid, kKeyedThreads, plan.keyed_smem, stream>>>(kp);
-      ADAPT_CUDA(cudaGetLastError());
+      ADAPT_CUDA(launch_dependent(search_keyed_kernel, dim3(grid), dim3(kKeyedThreads), plan.keyed_smem, stream, kp));
     }
     ExpandParams ep;
     ep.layers = d_keyed; ep.n_layers = nk; ep.state = d_state; ep.plan = d_plan;
@@ -629,8 +643,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
       ADAPT_CUDA(cudaFuncSetAttribute(expand_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(smem)));
       LaunchScope ls(ADAPT_KERNEL_EXPAND, stream);
-      expand_kernel<<<dim3(slices * kExpandRoles, nk), kExpandThreads, smem, stream>>>(ep);
-      ADAPT_CUDA(cudaGetLastError());
+      ADAPT_CUDA(launch_dependent(expand_kernel, dim3(slices * kExpandRoles, nk), dim3(kExpandThreads), smem, stream, ep));
     }
     }
   }
@@ -669,8 +682,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
               groups);
     {
       LaunchScope ls(ADAPT_KERNEL_SEARCH_DIRECT, direct_stream);
-      kern<<<grid, threads, smem, direct_stream>>>(sp);
-      ADAPT_CUDA(cudaGetLastError());
+      ADAPT_CUDA(launch_dependent(kern, grid, dim3(threads), smem, direct_stream, sp));
     }
     if (beside) {
       ADAPT_CUDA(cudaEventRecord(dc.side_join, dc.side_stream));
@@ -698,8 +710,7 @@ int run_search(DeviceCache& dc, const SearchArgs& a) {
     LaunchScope ls(ADAPT_KERNEL_KLD, stream);
     // enough CTAs to fill the GPU when there are few (FL, layer) pairs
     const int slices = std::max(1, std::min(16, (4 * dc.sm_count) / std::max(1, plan.n_levels * a.n_layers)));
-    kld_kernel<<<dim3(plan.n_levels, a.n_layers, slices), kKldThreads, 0, stream>>>(kp);
-    ADAPT_CUDA(cudaGetLastError());
+    ADAPT_CUDA(launch_dependent(kld_kernel, dim3(plan.n_levels, a.n_layers, slices), dim3(kKldThreads), 0, stream, kp));
   }
   return ADAPT_OK;
 }

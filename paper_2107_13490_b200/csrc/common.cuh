@@ -89,6 +89,14 @@ __device__ __forceinline__ void smem_red_add(unsigned addr, unsigned v) {
   asm volatile("red.shared.add.u32 [%0], %1;" :: "r"(addr), "r"(v) : "memory");
 }
 
+// A kernel that may be launched with programmatic stream serialization (its CTAs may become
+// resident while the kernel before it in the stream is still draining) calls this before it
+// touches anything that kernel wrote: it returns once the earlier grid has completed and its
+// writes are visible.  Without the launch attribute it returns at once.
+__device__ __forceinline__ void grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Adds the u32 words of a shared-memory array to a global array through the bulk-copy engine
 // (cp.reduce.async.bulk: the addition happens at the L2, no thread touches the words).  Both
 // addresses are 16-byte aligned and n_bytes is a multiple of 16.  Called by one thread, after a

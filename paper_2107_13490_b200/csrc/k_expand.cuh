@@ -396,6 +396,7 @@ __device__ __forceinline__ void expand_pyramid(const ExpandParams& p, const Laye
 // blockIdx.y: the layer.  Pyramid form: blockIdx.x = slice and role (the first 6 p.slices CTAs work);
 // level form: the levels (and the float histogram) are dealt to the gridDim.x CTAs of the layer.
 __global__ void __launch_bounds__(kExpandThreads) expand_kernel(const ExpandParams p) {
+  grid_dependency_wait();
   extern __shared__ unsigned s_expand[];
   const LayerDesc L = p.layers[blockIdx.y];
   const LayerPlan P = p.plan[L.index];

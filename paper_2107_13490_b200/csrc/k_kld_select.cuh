@@ -96,6 +96,7 @@ struct SelectScratch;
 __device__ void select_layer(const KldParams& p, int l, SelectScratch* sh);
 
 __global__ void __launch_bounds__(kKldThreads) kld_kernel(const KldParams p) {
+  grid_dependency_wait();
   __shared__ double s_buf[kKldThreads / 32];
   __shared__ int s_inf, s_last, s_nfold;
   __shared__ int s_fold[kKldThreads];       // positions (in FL order) of the candidates that fold

@@ -421,6 +421,7 @@ static_assert(kPlanThreads == 256, "the exponent classes are scanned one per thr
 // One layer per blockIdx.x; the gridDim.y CTAs of a layer all derive its plan (one thread each)
 // and share its bin edges.
 __global__ void __launch_bounds__(kPlanThreads) plan_kernel(const PlanParams p) {
+  grid_dependency_wait();
   __shared__ LayerPlan s_plan;
   __shared__ unsigned s_lsb;
   __shared__ int s_exp[256];     // sampled elements by biased exponent, then "below this exponent"

@@ -121,6 +121,7 @@ __device__ __forceinline__ void direct_quad(const float (&v)[4], unsigned m, lon
 template <bool kStochastic>
 __global__ void __launch_bounds__(kSearchThreadsWide)
 search_direct_kernel(const SearchParams p) {
+  grid_dependency_wait();
   extern __shared__ unsigned s_hist[];  // [(fl_per_group + 1)][n_bins]
   __shared__ float s_two[kMaxFl], s_inv[kMaxFl];
   __shared__ unsigned s_zero[kMaxFl];

@@ -503,6 +503,7 @@ __device__ __noinline__ void keyed_segment(const LayerCtx& c, unsigned* cells, i
 }
 
 __global__ void __launch_bounds__(kKeyedThreads, 1) search_keyed_kernel(const KeyedParams p) {
+  grid_dependency_wait();
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ unsigned s_zclass[kZeroClasses];
   __shared__ unsigned s_stray;

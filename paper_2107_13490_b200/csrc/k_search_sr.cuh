@@ -224,6 +224,7 @@ __device__ __forceinline__ void sr_quad(const SrCtx& c, const SrParams& p, int l
 }
 
 __global__ void __launch_bounds__(kSrThreads, 1) search_sr_kernel(const SrParams p) {
+  grid_dependency_wait();
   extern __shared__ __align__(16) unsigned char s_raw[];
   __shared__ SrCtx s_ctx;
   __shared__ SrLevels s_lv;
@@ -400,6 +401,7 @@ struct SrExpandParams {
 constexpr int kSrExpandThreads = 512;
 
 __global__ void __launch_bounds__(kSrExpandThreads) expand_sr_kernel(const SrExpandParams p) {
+  grid_dependency_wait();
   extern __shared__ unsigned s_hist[];          // [n_bins]
   __shared__ SrLevels s_lv;
   __shared__ unsigned long long s_zero;
