@@ -106,6 +106,8 @@ struct DeviceCache {
   void* stage_in = nullptr;    size_t stage_in_bytes = 0;    // host-form calls: inputs
   void* stage_out = nullptr;   size_t stage_out_bytes = 0;   // host-form calls: outputs
   void* batch_tab = nullptr;   size_t batch_tab_bytes = 0;   // batched quantize: layer table
+  std::vector<unsigned char> batch_tab_image;   // host copy of what batch_tab holds (empty: unknown)
+  cudaStream_t batch_tab_stream = nullptr;      // the stream that uploaded it
   void* stage_codes = nullptr; size_t stage_codes_bytes = 0; // host-form calls: codes
   void* div_buf = nullptr;     size_t div_buf_bytes = 0;     // gradient diversity: tables + sums
   PinnedSlot ring[kRingSlots];
@@ -302,9 +304,9 @@ bool make_plan(const int64_t* lens, int n_layers, const adapt_grid* grid, int n_
 // grid_dependency_wait(): with programmatic stream serialization its CTAs may be scheduled while
 // the earlier kernel's last CTAs are still running, which hides the launch latency between the
 // dependent kernels of a search.  (Not while per-kernel events are recorded between them.)
-template <typename Params>
-cudaError_t launch_dependent(void (*kern)(Params), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                             const Params& params) {
+template <typename... Params, typename... Args>
+cudaError_t launch_dependent(void (*kern)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                             Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
   cudaLaunchAttribute attr[1];
@@ -312,7 +314,7 @@ cudaError_t launch_dependent(void (*kern)(Params), dim3 grid, dim3 block, size_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = g_timing.load() ? 0 : 1;
-  return cudaLaunchKernelEx(&cfg, kern, params);
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
 // ---- search driver ----------------------------------------------------------------
@@ -851,12 +853,12 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
   int rc = current_cache(&dc);
   if (rc != ADAPT_OK) return rc;
   const size_t bytes = sizeof(QuantLayer) * static_cast<size_t>(n_layers);
+  void* const tab_before = dc->batch_tab;
   rc = grow_device(&dc->batch_tab, &dc->batch_tab_bytes, align_up(bytes, 4096));
   if (rc != ADAPT_OK) return rc;
-  PinnedSlot* slot = nullptr;
-  rc = acquire_slot(*dc, bytes, &slot);
-  if (rc != ADAPT_OK) return rc;
-  QuantLayer* h = static_cast<QuantLayer*>(slot->host);
+  if (dc->batch_tab != tab_before) dc->batch_tab_image.clear();
+  std::vector<unsigned char> image(bytes);
+  QuantLayer* h = reinterpret_cast<QuantLayer*>(image.data());
   long long tiles = 0;
   for (int l = 0; l < n_layers; ++l) {
     h[l].x = tensors[l]; h[l].out = codes_out[l]; h[l].n = lens[l]; h[l].tile_begin = tiles;
@@ -868,8 +870,22 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
   cudaStream_t stream = static_cast<cudaStream_t>(stream_handle);
   if (unfit) ADAPT_CUDA(cudaMemsetAsync(unfit, 0, sizeof(int32_t) * static_cast<size_t>(n_layers), stream));
   if (tiles == 0) return ADAPT_OK;
-  ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, h, bytes, cudaMemcpyHostToDevice, stream));
-  ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+  // The same layer list as in the call before, on the same stream (a training loop's case): the
+  // table on the device is still the right one, and with no copy in between the kernel can follow
+  // the search's last kernel as a dependent launch.
+  const bool same = dc->batch_tab_stream == stream && dc->batch_tab_image.size() == bytes &&
+                    std::memcmp(dc->batch_tab_image.data(), image.data(), bytes) == 0;
+  if (!same) {
+    PinnedSlot* slot = nullptr;
+    rc = acquire_slot(*dc, bytes, &slot);
+    if (rc != ADAPT_OK) return rc;
+    std::memcpy(slot->host, image.data(), bytes);
+    dc->batch_tab_image.clear();
+    ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, slot->host, bytes, cudaMemcpyHostToDevice, stream));
+    ADAPT_CUDA(cudaEventRecord(slot->done, stream));
+    dc->batch_tab_image.swap(image);
+    dc->batch_tab_stream = stream;
+  }
   const int grid = static_cast<int>(std::min<long long>(tiles, 32ll * dc->sm_count));
   const QuantLayer* d = static_cast<const QuantLayer*>(dc->batch_tab);
   LaunchScope ls(ADAPT_KERNEL_QUANTIZE, stream);
@@ -881,8 +897,8 @@ int run_quantize_batch(const float* const* tensors, const int64_t* lens, int n_l
     case 16: kern = sr ? quantize_batch_kernel<true, int16_t> : quantize_batch_kernel<false, int16_t>; break;
     default: kern = sr ? quantize_batch_kernel<true, int32_t> : quantize_batch_kernel<false, int32_t>; break;
   }
-  kern<<<grid, kQuantThreads, 0, stream>>>(d, n_layers, tiles, best, seed, unfit);
-  ADAPT_CUDA(cudaGetLastError());
+  ADAPT_CUDA(launch_dependent(kern, dim3(grid), dim3(kQuantThreads), 0, stream, d, n_layers, tiles, best,
+                              static_cast<unsigned long long>(seed), unfit));
   return ADAPT_OK;
 }
 }  // namespace
@@ -1243,6 +1259,7 @@ int run_search_host(const float* const* tensors, const int64_t* lens, int n_laye
       rc = acquire_slot(*dc, bytes, &slot);
       if (rc != ADAPT_OK) return rc;
       std::memcpy(slot->host, table.data(), bytes);
+      dc->batch_tab_image.clear();
       ADAPT_CUDA(cudaMemcpyAsync(dc->batch_tab, slot->host, bytes, cudaMemcpyHostToDevice, stream));
       ADAPT_CUDA(cudaEventRecord(slot->done, stream));
       const QuantLayer* d_table = static_cast<const QuantLayer*>(dc->batch_tab);
@@ -1802,6 +1819,7 @@ int adapt_release(void) {
   if (dc->stage_in) { ADAPT_CUDA(cudaFree(dc->stage_in)); dc->stage_in = nullptr; dc->stage_in_bytes = 0; }
   if (dc->stage_out) { ADAPT_CUDA(cudaFree(dc->stage_out)); dc->stage_out = nullptr; dc->stage_out_bytes = 0; }
   if (dc->batch_tab) { ADAPT_CUDA(cudaFree(dc->batch_tab)); dc->batch_tab = nullptr; dc->batch_tab_bytes = 0; }
+  dc->batch_tab_image.clear();
   if (dc->div_buf) { ADAPT_CUDA(cudaFree(dc->div_buf)); dc->div_buf = nullptr; dc->div_buf_bytes = 0; }
   if (dc->stage_codes) { ADAPT_CUDA(cudaFree(dc->stage_codes)); dc->stage_codes = nullptr; dc->stage_codes_bytes = 0; }
   if (dc->side_stream) {

@@ -104,6 +104,7 @@ template <bool kStochastic, typename T>
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_batch_kernel(const QuantLayer* __restrict__ layers, int n_layers, long long n_tiles,
                       const int* __restrict__ best, unsigned long long seed, int* __restrict__ unfit) {
+  grid_dependency_wait();
   constexpr int kBits = sizeof(T) == 1 ? 8 : (sizeof(T) == 2 ? 16 : 32);   // float carries any code
   for (long long t = blockIdx.x; t < n_tiles; t += gridDim.x) {
     int lo = 0, hi = n_layers - 1;                 // layer that owns tile t
