@@ -135,6 +135,43 @@ def test_batched_quantize_at_device_resident_selections(B):
             assert torch.equal(bufs[j], vals[j]), (mode, j)
 
 
+def test_batched_quantize_repeats_and_changes_its_layer_list(B):
+    """The library keeps the layer table of the call before: the same list again (no upload), a
+    different list, the first list once more, and the same tensors with new formats must each
+    give the oracle's codes."""
+    import torch
+    rng = np.random.default_rng(31)
+    xs = [(rng.standard_normal(n) * 0.3).astype(np.float32) for n in (5000, 70001, 333)]
+    dev = [torch.from_numpy(x).cuda() for x in xs]
+    fmt_a = np.array([[8, 4, 0, 1], [12, 9, 0, 1], [5, 2, 0, 1]], dtype=np.int32)
+    fmt_b = np.array([[16, 12, 0, 1], [4, 1, 0, 1], [9, 8, 0, 1]], dtype=np.int32)
+
+    def check(tensors, hosts, fmt):
+        best = torch.from_numpy(fmt[:len(tensors)].copy()).cuda()
+        codes = B.adapt_quantize_selected_batch(tensors, best, O.ROUND_RNE, seed=0, layer_base=0)
+        torch.cuda.synchronize()
+        for j, x in enumerate(hosts):
+            want, _ = O.quantize(x, int(fmt[j][0]), int(fmt[j][1]), O.ROUND_RNE, 0, j)
+            assert np.array_equal(codes[j].cpu().numpy(), want), j
+        return codes
+
+    outs = [torch.empty(x.size, dtype=torch.int32, device="cuda") for x in xs]
+
+    def check_into(fmt):
+        best = torch.from_numpy(fmt.copy()).cuda()
+        B.adapt_quantize_selected_batch(dev, best, O.ROUND_RNE, seed=0, layer_base=0, codes_out=outs)
+        torch.cuda.synchronize()
+        for j, x in enumerate(xs):
+            want, _ = O.quantize(x, int(fmt[j][0]), int(fmt[j][1]), O.ROUND_RNE, 0, j)
+            assert np.array_equal(outs[j].cpu().numpy(), want), j
+
+    check_into(fmt_a)            # uploads the table
+    check_into(fmt_a)            # same tensors, same outputs: the table is reused
+    check_into(fmt_b)            # same table, other formats on the device
+    check(dev[:2], xs[:2], fmt_b)    # a different list (new output tensors)
+    check_into(fmt_a)            # the first list again
+
+
 def test_quantize_argument_errors_and_host_form(B):
     import torch
     x = torch.zeros(16, dtype=torch.float32, device="cuda")
