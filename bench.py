@@ -31,7 +31,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the search kernel from an ncu capture (bytes per element per launch),
 # valid only for the library version it was taken on; see profiles/.
-TRAFFIC_CAPTURE = {"version": "adapt-b200 0.9", "bytes_per_element": 4.075}
+TRAFFIC_CAPTURE = {"version": "adapt-b200 0.9", "bytes_per_element": 4.074}
 
 
 def parse_args():
