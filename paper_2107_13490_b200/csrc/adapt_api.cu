@@ -1523,8 +1523,7 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
   }
   {
     LaunchScope ls(ADAPT_KERNEL_FORMAT_RESOLVE, stream);
-    format_resolve_kernel<<<a.n_layers, 128, 0, stream>>>(fp);
-    ADAPT_CUDA(cudaGetLastError());
+    ADAPT_CUDA(launch_dependent(format_resolve_kernel, dim3(a.n_layers), dim3(128), 0, stream, fp));
   }
   if (tiles > 0) {
     auto kern = (o.round_mode == ADAPT_ROUND_STOCHASTIC) ? format_search_kernel<true>
@@ -1534,18 +1533,15 @@ int run_format_search(DeviceCache& dc, const FormatArgs& a) {
     const int ctas_per_sm = std::max<int>(1, std::min<size_t>(2, (200 * 1024) / (smem + 2048)));
     dim3 grid(static_cast<unsigned>(std::min<long long>(tiles, 1ll * ctas_per_sm * dc.sm_count)), groups);
     LaunchScope ls(ADAPT_KERNEL_FORMAT_SEARCH, stream);
-    kern<<<grid, kFormatThreads, smem, stream>>>(fp);
-    ADAPT_CUDA(cudaGetLastError());
+    ADAPT_CUDA(launch_dependent(kern, grid, dim3(kFormatThreads), smem, stream, fp));
   }
   {
     LaunchScope ls(ADAPT_KERNEL_FORMAT_KLD, stream);
-    format_kld_kernel<<<dim3(plan.n_cand, a.n_layers), kKldThreads, 0, stream>>>(fp);
-    ADAPT_CUDA(cudaGetLastError());
+    ADAPT_CUDA(launch_dependent(format_kld_kernel, dim3(plan.n_cand, a.n_layers), dim3(kKldThreads), 0, stream, fp));
   }
   {
     LaunchScope ls(ADAPT_KERNEL_SELECT, stream);
-    format_select_kernel<<<a.n_layers, 32, 0, stream>>>(fp);
-    ADAPT_CUDA(cudaGetLastError());
+    ADAPT_CUDA(launch_dependent(format_select_kernel, dim3(a.n_layers), dim3(32), 0, stream, fp));
   }
   return ADAPT_OK;
 }

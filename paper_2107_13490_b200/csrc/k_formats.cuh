@@ -103,6 +103,7 @@ __device__ __forceinline__ float float_value(float x, int emin, int m_bits, floa
 
 // One CTA per layer: grid level of every rule, clamp values and b-as-used of every candidate.
 __global__ void format_resolve_kernel(const FormatParams p) {
+  grid_dependency_wait();
   const int l = blockIdx.x;
   const LayerState S = p.state[l];
   for (int r = threadIdx.x; r < p.n_rules; r += blockDim.x) {
@@ -242,6 +243,7 @@ __device__ __forceinline__ void format_quad(const float (&v)[4], unsigned m, lon
 // group's rules with them, so a rule's constants are fetched once per four evaluations.
 template <bool kStochastic>
 __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const FormatParams p) {
+  grid_dependency_wait();
   extern __shared__ unsigned s_fhist[];   // [rules in the group][n_bins]
   __shared__ int s_kind[kMaxRulesPerGroup], s_i0[kMaxRulesPerGroup], s_i1[kMaxRulesPerGroup];
   __shared__ float s_f0[kMaxRulesPerGroup], s_f1[kMaxRulesPerGroup];
@@ -348,6 +350,7 @@ __global__ void __launch_bounds__(kFormatThreads) format_search_kernel(const For
 // One CTA per (candidate, layer): the rule's histogram with both tails folded into the bins
 // of the candidate's clamp values, then KL(P||Q) against the identity rule's histogram.
 __global__ void __launch_bounds__(kKldThreads) format_kld_kernel(const FormatParams p) {
+  grid_dependency_wait();
   __shared__ double s_buf[kKldThreads / 32];
   __shared__ int s_inf;
   const int c = blockIdx.x, l = blockIdx.y;
@@ -410,6 +413,7 @@ __global__ void __launch_bounds__(kKldThreads) format_kld_kernel(const FormatPar
 // One warp per layer: the first format of the caller's list with KLD <= eps, else the one of
 // least divergence (first among ties; the last one if every divergence is +inf).
 __global__ void format_select_kernel(const FormatParams p) {
+  grid_dependency_wait();
   const int l = blockIdx.x, lane = threadIdx.x;
   const double* kld = p.kld_out + static_cast<size_t>(l) * p.n_cand;
   int first_ok = 0x7fffffff, min_pos = -1;
